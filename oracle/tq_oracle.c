@@ -1,0 +1,344 @@
+/*
+ * Tiny-QMoE CPU oracle -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+ *
+ * A plain, slow, single-threaded, obviously-correct restatement of what the
+ * paper's pipeline computes: the naive min-max quantizer (Listing 1), the
+ * 4-gram dictionary (Listing 2), the uint16 token stream encoder (Listing 3),
+ * the decoder (Listing 4) and the dense layer product that consumes the
+ * decoded weights (Section 2.3, Section 5 "Model Loading").  It shares no code,
+ * header, table or helper with the CUDA library; only tests, the smoke check
+ * and the benchmark's CPU-baseline leg may call it.
+ *
+ * No blocking, fusion, SIMD or threading: each function follows the listing it
+ * cites step by step so that it can be checked against the paper by eye.
+ *
+ * Pins (see tests/test_oracle_pins.py): round trip exactness, the stream-size
+ * identity, closed forms (constant input, empty table, all-hit), brute-force
+ * window counting on tiny inputs, hand-worked fixtures, quantizer end points
+ * and error bound, and a library fp64 GEMV.  The one thing with no pin is the
+ * paper's Table 1 (model sizes): it cannot be derived from the listings and is
+ * "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define TQO_ESCAPE 0xFFFFu      /* Listing 3: marker that precedes raw values   */
+#define TQO_SEQ 4               /* Listing 2: sequence_length default            */
+#define TQO_MAX_ENTRIES 65534u  /* codes 1..65534; 65535 would collide with the
+                                   escape marker that the decoder tests first   */
+
+/* ------------------------------------------------------------------------ */
+/* Listing 1: naive min-max quantizer, per tensor, bits = 8 (maxq = 255).    */
+/* All arithmetic in fp32 with round-half-to-even, as the listing's tensor   */
+/* ops do.  Writes the integer level q (0..255); returns scale and zero.     */
+/* Returns -1 when the range is empty (scale would be 0).                    */
+/* ------------------------------------------------------------------------ */
+int tqo_quantize_paper(const float *x, uint64_t n, uint8_t *q, float *scale_out,
+                       float *zero_out) {
+  if (n == 0) return -1;
+  const float maxq = 255.0f;
+  float xmin = x[0], xmax = x[0];
+  for (uint64_t i = 1; i < n; ++i) {
+    if (x[i] < xmin) xmin = x[i];
+    if (x[i] > xmax) xmax = x[i];
+  }
+  float scale = (xmax - xmin) / maxq;
+  if (!(scale > 0.0f)) return -1;
+  float zero = nearbyintf(-xmin / scale);
+  for (uint64_t i = 0; i < n; ++i) {
+    float v = nearbyintf(x[i] / scale) + zero;
+    if (v < 0.0f) v = 0.0f;
+    if (v > maxq) v = maxq;
+    q[i] = (uint8_t)v;
+  }
+  *scale_out = scale;
+  *zero_out = zero;
+  return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* The benchmark configurations' quantizer (not in the paper): per output    */
+/* row, symmetric, s_r = max|w| / 127, q = clamp(round(w / s_r), -127, 127). */
+/* An all-zero row gets s_r = 1.  The byte that is dictionary coded is the   */
+/* two's-complement pattern of q (Listing 2's astype(uint8)).                */
+/* ------------------------------------------------------------------------ */
+void tqo_quantize_rows(const float *w, uint32_t rows, uint32_t cols, int8_t *q,
+                       float *scale) {
+  for (uint32_t r = 0; r < rows; ++r) {
+    const float *wr = w + (uint64_t)r * cols;
+    float amax = 0.0f;
+    for (uint32_t c = 0; c < cols; ++c) {
+      float a = fabsf(wr[c]);
+      if (a > amax) amax = a;
+    }
+    float s = amax > 0.0f ? amax / 127.0f : 1.0f;
+    scale[r] = s;
+    for (uint32_t c = 0; c < cols; ++c) {
+      float v = nearbyintf(wr[c] / s);
+      if (v < -127.0f) v = -127.0f;
+      if (v > 127.0f) v = 127.0f;
+      q[(uint64_t)r * cols + c] = (int8_t)v;
+    }
+  }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Listing 2: count every stride-1 window of 4 bytes over each flattened     */
+/* matrix (windows never span two matrices), keep the top_k most frequent,   */
+/* code = rank + 1.  Ties keep first-insertion order, which is what a stable */
+/* descending sort of an insertion-ordered counter gives.                    */
+/* ------------------------------------------------------------------------ */
+typedef struct {
+  uint32_t key;    /* the 4 bytes, byte i of the window in bits 8i..8i+7 */
+  uint32_t used;
+  uint64_t count;
+  uint64_t first;  /* insertion order */
+} tqo_slot;
+
+typedef struct {
+  uint32_t n_entries;             /* K                                    */
+  uint8_t *entries;               /* K x 4, rank order                    */
+  uint64_t *counts;               /* K, occurrence count of each entry    */
+  uint64_t n_distinct;            /* distinct windows seen                */
+  uint64_t n_windows;             /* total windows counted                */
+  /* lookup map for the encoder: key -> code */
+  uint32_t map_cap;
+  uint32_t *map_key;
+  uint16_t *map_code;             /* 0 = empty */
+} tqo_dict;
+
+static uint32_t tqo_hash(uint32_t k) {
+  k ^= k >> 16;
+  k *= 0x7feb352du;
+  k ^= k >> 15;
+  k *= 0x846ca68bu;
+  k ^= k >> 16;
+  return k;
+}
+
+static int tqo_cmp_rank(const void *a, const void *b) {
+  const tqo_slot *x = (const tqo_slot *)a, *y = (const tqo_slot *)b;
+  if (x->count != y->count) return x->count > y->count ? -1 : 1;
+  if (x->first != y->first) return x->first < y->first ? -1 : 1;
+  return 0;
+}
+
+static void tqo_map_insert(tqo_dict *d, uint32_t key, uint16_t code) {
+  uint32_t m = d->map_cap - 1, h = tqo_hash(key) & m;
+  while (d->map_code[h] != 0) h = (h + 1) & m;
+  d->map_key[h] = key;
+  d->map_code[h] = code;
+}
+
+/* code of a 4-byte window, 0 if it is not in the table */
+static uint16_t tqo_map_find(const tqo_dict *d, uint32_t key) {
+  uint32_t m = d->map_cap - 1, h = tqo_hash(key) & m;
+  while (d->map_code[h] != 0) {
+    if (d->map_key[h] == key) return d->map_code[h];
+    h = (h + 1) & m;
+  }
+  return 0;
+}
+
+void tqo_dict_free(tqo_dict *d) {
+  if (!d) return;
+  free(d->entries);
+  free(d->counts);
+  free(d->map_key);
+  free(d->map_code);
+  free(d);
+}
+
+tqo_dict *tqo_build_dictionary(const uint8_t *const *mats, const uint64_t *n_elems,
+                               int n_mats, uint32_t top_k) {
+  uint64_t cap = 1024;
+  uint64_t used = 0, windows = 0;
+  tqo_slot *tab = (tqo_slot *)calloc(cap, sizeof(tqo_slot));
+  if (!tab) return NULL;
+  for (int m = 0; m < n_mats; ++m) {
+    const uint8_t *w = mats[m];
+    uint64_t n = n_elems[m];
+    for (uint64_t i = 0; i + TQO_SEQ <= n; ++i) {
+      uint32_t key = (uint32_t)w[i] | ((uint32_t)w[i + 1] << 8) |
+                     ((uint32_t)w[i + 2] << 16) | ((uint32_t)w[i + 3] << 24);
+      if ((used + 1) * 10 > cap * 6) { /* grow at 60 % load */
+        uint64_t ncap = cap * 2;
+        tqo_slot *nt = (tqo_slot *)calloc(ncap, sizeof(tqo_slot));
+        if (!nt) { free(tab); return NULL; }
+        for (uint64_t s = 0; s < cap; ++s)
+          if (tab[s].used) {
+            uint64_t h = tqo_hash(tab[s].key) & (ncap - 1);
+            while (nt[h].used) h = (h + 1) & (ncap - 1);
+            nt[h] = tab[s];
+          }
+        free(tab);
+        tab = nt;
+        cap = ncap;
+      }
+      uint64_t h = tqo_hash(key) & (cap - 1);
+      while (tab[h].used && tab[h].key != key) h = (h + 1) & (cap - 1);
+      if (!tab[h].used) {
+        tab[h].used = 1;
+        tab[h].key = key;
+        tab[h].count = 0;
+        tab[h].first = used++;
+      }
+      tab[h].count++;
+      windows++;
+    }
+  }
+  /* compact, rank */
+  tqo_slot *all = (tqo_slot *)malloc((used ? used : 1) * sizeof(tqo_slot));
+  uint64_t k = 0;
+  for (uint64_t s = 0; s < cap; ++s)
+    if (tab[s].used) all[k++] = tab[s];
+  free(tab);
+  qsort(all, used, sizeof(tqo_slot), tqo_cmp_rank);
+
+  uint64_t K = used;
+  if (K > top_k) K = top_k;
+  if (K > TQO_MAX_ENTRIES) K = TQO_MAX_ENTRIES;
+
+  tqo_dict *d = (tqo_dict *)calloc(1, sizeof(tqo_dict));
+  d->n_entries = (uint32_t)K;
+  d->n_distinct = used;
+  d->n_windows = windows;
+  d->entries = (uint8_t *)malloc(K ? K * 4 : 4);
+  d->counts = (uint64_t *)malloc(K ? K * 8 : 8);
+  d->map_cap = 1u << 18; /* > 2 x 65534 */
+  d->map_key = (uint32_t *)calloc(d->map_cap, sizeof(uint32_t));
+  d->map_code = (uint16_t *)calloc(d->map_cap, sizeof(uint16_t));
+  for (uint64_t r = 0; r < K; ++r) {
+    uint32_t key = all[r].key;
+    d->entries[4 * r + 0] = (uint8_t)(key);
+    d->entries[4 * r + 1] = (uint8_t)(key >> 8);
+    d->entries[4 * r + 2] = (uint8_t)(key >> 16);
+    d->entries[4 * r + 3] = (uint8_t)(key >> 24);
+    d->counts[r] = all[r].count;
+    tqo_map_insert(d, key, (uint16_t)(r + 1)); /* code = rank + 1 */
+  }
+  free(all);
+  return d;
+}
+
+/* Build a dictionary object from an explicit entry list (rank order), so the
+ * encoder/decoder can be exercised with hand-made tables. */
+tqo_dict *tqo_dict_from_entries(const uint8_t *entries, uint32_t K) {
+  if (K > TQO_MAX_ENTRIES) return NULL;
+  tqo_dict *d = (tqo_dict *)calloc(1, sizeof(tqo_dict));
+  d->n_entries = K;
+  d->entries = (uint8_t *)malloc(K ? (size_t)K * 4 : 4);
+  d->counts = (uint64_t *)calloc(K ? K : 1, 8);
+  memcpy(d->entries, entries, (size_t)K * 4);
+  d->map_cap = 1u << 18;
+  d->map_key = (uint32_t *)calloc(d->map_cap, sizeof(uint32_t));
+  d->map_code = (uint16_t *)calloc(d->map_cap, sizeof(uint16_t));
+  for (uint32_t r = 0; r < K; ++r) {
+    uint32_t key = (uint32_t)entries[4 * r] | ((uint32_t)entries[4 * r + 1] << 8) |
+                   ((uint32_t)entries[4 * r + 2] << 16) |
+                   ((uint32_t)entries[4 * r + 3] << 24);
+    if (tqo_map_find(d, key) == 0) tqo_map_insert(d, key, (uint16_t)(r + 1));
+  }
+  return d;
+}
+
+uint32_t tqo_dict_size(const tqo_dict *d) { return d->n_entries; }
+const uint8_t *tqo_dict_entries(const tqo_dict *d) { return d->entries; }
+const uint64_t *tqo_dict_counts(const tqo_dict *d) { return d->counts; }
+uint64_t tqo_dict_distinct(const tqo_dict *d) { return d->n_distinct; }
+uint64_t tqo_dict_windows(const tqo_dict *d) { return d->n_windows; }
+
+/* ------------------------------------------------------------------------ */
+/* Listing 3: aligned scan in steps of 4.  Known window -> its code; unknown */
+/* -> escape marker then the 4 bytes, each widened to uint16; a tail of 1..3 */
+/* bytes -> escape marker then those bytes.  out == NULL: size query.        */
+/* Returns the stream length in uint16 units, or (uint64_t)-1 if cap is too  */
+/* small.  n_hits / n_miss may be NULL.                                      */
+/* ------------------------------------------------------------------------ */
+uint64_t tqo_encode(const tqo_dict *d, const uint8_t *w, uint64_t n, uint16_t *out,
+                    uint64_t cap, uint64_t *n_hits, uint64_t *n_miss) {
+  uint64_t len = 0, hits = 0, miss = 0, i = 0;
+  while (i + TQO_SEQ <= n) {
+    uint32_t key = (uint32_t)w[i] | ((uint32_t)w[i + 1] << 8) |
+                   ((uint32_t)w[i + 2] << 16) | ((uint32_t)w[i + 3] << 24);
+    uint16_t code = tqo_map_find(d, key);
+    if (code != 0) {
+      if (out) { if (len + 1 > cap) return (uint64_t)-1; out[len] = code; }
+      len += 1;
+      hits++;
+    } else {
+      if (out) {
+        if (len + 5 > cap) return (uint64_t)-1;
+        out[len] = TQO_ESCAPE;
+        for (int j = 0; j < TQO_SEQ; ++j) out[len + 1 + j] = w[i + j];
+      }
+      len += 5;
+      miss++;
+    }
+    i += TQO_SEQ;
+  }
+  if (i < n) {
+    uint64_t r = n - i;
+    if (out) {
+      if (len + 1 + r > cap) return (uint64_t)-1;
+      out[len] = TQO_ESCAPE;
+      for (uint64_t j = 0; j < r; ++j) out[len + 1 + j] = w[i + j];
+    }
+    len += 1 + r;
+  }
+  if (n_hits) *n_hits = hits;
+  if (n_miss) *n_miss = miss;
+  return len;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Listing 4: walk the tokens; the escape marker means "the next up to 4     */
+/* slots are raw bytes" (a slice, so fewer at the very end), anything else   */
+/* is looked up in the table.  Returns the number of bytes produced, -1 for  */
+/* an unknown code (the listing raises), -2 if out is too small.             */
+/* ------------------------------------------------------------------------ */
+int64_t tqo_decode(const tqo_dict *d, const uint16_t *s, uint64_t len, uint8_t *out,
+                   uint64_t cap) {
+  uint64_t i = 0, o = 0;
+  while (i < len) {
+    uint16_t code = s[i];
+    i += 1;
+    if (code == TQO_ESCAPE) {
+      uint64_t take = len - i < TQO_SEQ ? len - i : TQO_SEQ;
+      if (o + take > cap) return -2;
+      for (uint64_t j = 0; j < take; ++j) out[o + j] = (uint8_t)s[i + j];
+      o += take;
+      i += TQO_SEQ;
+    } else {
+      if (code == 0 || code > d->n_entries) return -1;
+      if (o + TQO_SEQ > cap) return -2;
+      memcpy(out + o, d->entries + 4 * (uint64_t)(code - 1), TQO_SEQ);
+      o += TQO_SEQ;
+    }
+  }
+  return (int64_t)o;
+}
+
+/* ------------------------------------------------------------------------ */
+/* The layer that consumes the decoded weights (Section 2.3; Listing 1's     */
+/* dequantisation scale * (q - zero)): y[b][r] = s_r * sum_c (q[r][c]-z_r) * */
+/* x[b][c], everything in fp64.  is_signed: the byte is an int8 pattern.     */
+/* zero may be NULL (all zero).  No bias (LLaMA linears have none).          */
+/* ------------------------------------------------------------------------ */
+void tqo_layer_forward(const uint8_t *q, int is_signed, uint32_t rows, uint32_t cols,
+                       const float *scale, const float *zero, const double *x,
+                       uint32_t batch, double *y) {
+  for (uint32_t b = 0; b < batch; ++b)
+    for (uint32_t r = 0; r < rows; ++r) {
+      double z = zero ? (double)zero[r] : 0.0;
+      double acc = 0.0;
+      for (uint32_t c = 0; c < cols; ++c) {
+        uint8_t byte = q[(uint64_t)r * cols + c];
+        double v = is_signed ? (double)(int8_t)byte : (double)byte;
+        acc += (v - z) * x[(uint64_t)b * cols + c];
+      }
+      y[(uint64_t)b * rows + r] = (double)scale[r] * acc;
+    }
+}
