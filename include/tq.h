@@ -1,0 +1,175 @@
+/*
+ * tq -- fused dictionary-decode + GEMV/GEMM for Tiny-QMoE-format weights on B200 (sm_100a).
+ *
+ * C ABI.  Every call returns an int status (TQ_OK = 0, negative = error); nothing throws or
+ * aborts across this boundary.  Pointers are marked HOST or DEVICE.  The library never calls
+ * cudaMalloc on behalf of the caller: all device memory is caller-owned (a tq_ddict / tq_dmat
+ * only remembers addresses inside the caller's buffer, so the buffer must outlive the handle).
+ * Streams are passed as void* (a cudaStream_t); device calls are asynchronous on that stream
+ * unless stated otherwise.  Handles are opaque, library-owned host objects released with the
+ * matching *_free call.
+ *
+ * The data format is the paper's (Section 4, Listings 2-4): 8-bit weight levels, a table of the
+ * K <= 65534 most frequent windows of 4 consecutive levels (code = rank + 1), and per matrix a
+ * uint16 token stream in which every aligned group of 4 levels is either its code or the marker
+ * 0xFFFF followed by the 4 levels, each widened to 16 bits.
+ */
+#ifndef TQ_H_
+#define TQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TQ_OK 0
+#define TQ_ERR_INVALID_ARG (-1)
+#define TQ_ERR_CORRUPT_STREAM (-2)
+#define TQ_ERR_BUFFER_TOO_SMALL (-3)
+#define TQ_ERR_UNSUPPORTED_SHAPE (-4)
+#define TQ_ERR_CUDA (-5)
+#define TQ_ERR_TIMEOUT (-6)
+#define TQ_ERR_NOMEM (-7)
+
+#define TQ_ESCAPE 0xFFFFu
+#define TQ_MAX_ENTRIES 65534u
+
+/* Device status bits (tq_device_status). */
+#define TQ_STATUS_BAD_CODE 1u      /* a code of 0 or > K was met; it decoded as four zero bytes */
+#define TQ_STATUS_BAD_ROW 2u       /* a row segment did not hold exactly cols/4 groups          */
+#define TQ_STATUS_WAIT_EXPIRED 4u  /* a bounded wait inside a kernel ran out                    */
+
+typedef struct tq_dict tq_dict;   /* HOST: the compression table                                */
+typedef struct tq_ddict tq_ddict; /* handle of a table resident in DEVICE memory                */
+typedef struct tq_dmat tq_dmat;   /* handle of one compressed matrix resident in DEVICE memory  */
+
+/* Human-readable text for a status code (static storage). */
+const char* tq_strerror(int status);
+
+/* Worker threads used by the host calls below (0 = hardware concurrency).  Returns the value in
+ * effect. */
+int tq_set_num_threads(int n);
+
+/* ------------------------------------------------------------------------------------------
+ * Host side: quantize, build the table, encode.
+ * ---------------------------------------------------------------------------------------- */
+
+/* Per-tensor min-max quantizer at 8 bits (Listing 1): scale = (max-min)/255,
+ * zero = round(-min/scale), q = clamp(round(x/scale) + zero, 0, 255); fp32, round half to even.
+ * x, q: HOST, n elements.  Fails with TQ_ERR_INVALID_ARG when max == min. */
+int tq_quantize_tensor(const float* x, uint64_t n, uint8_t* q, float* scale, float* zero);
+
+/* Per-output-row symmetric int8 quantizer used by the benchmark workloads (not in the paper;
+ * it produces the same kind of 8-bit level Listing 1 does, W ~ scale_r * q):
+ * scale_r = max_c |w[r][c]| / 127 (1 for an all-zero row), q = clamp(round(w/scale_r), -127, 127).
+ * w: HOST [rows][cols] row-major; q: HOST [rows][cols]; scale: HOST [rows]. */
+int tq_quantize_rows(const float* w, uint32_t rows, uint32_t cols, int8_t* q, float* scale);
+
+/* Same computation on the GPU, bit-identical results.  d_w, d_q, d_scale: DEVICE. */
+int tq_quantize_rows_device(const float* d_w, uint32_t rows, uint32_t cols, int8_t* d_q,
+                            float* d_scale, void* cuda_stream);
+
+/* Frequent-sequence table (Listing 2).  Counts every window of 4 consecutive bytes (stride 1) of
+ * each flattened matrix -- windows never span two matrices -- and keeps the top_k most frequent
+ * in descending count order; equal counts keep first-seen order (matrix order, then position);
+ * code = rank + 1.  Code 65535 is the escape marker, so at most 65534 entries are kept
+ * (top_k > 65534 is clamped).  mats: HOST array of n_mats HOST pointers; n_elems: HOST, bytes
+ * per matrix.  The total window count must be < 2^32.  *out is owned by the library. */
+int tq_build_dictionary(const uint8_t* const* mats, const uint64_t* n_elems, int n_mats,
+                        uint32_t top_k, tq_dict** out);
+
+/* A table from an explicit entry list (K x 4 bytes, rank order, HOST). */
+int tq_dict_from_entries(const uint8_t* entries, uint32_t K, tq_dict** out);
+
+/* Borrow the table: *K entries, *entries -> K x 4 bytes in rank order (HOST, valid until
+ * tq_dict_free).  counts (may be NULL) -> K occurrence counts (zeros for tq_dict_from_entries). */
+int tq_dict_entries(const tq_dict* d, uint32_t* K, const uint8_t** entries,
+                    const uint64_t** counts);
+
+/* Token stream of one matrix (Listing 3): aligned groups of 4 bytes; a group found in the table
+ * is written as its code, any other as 0xFFFF followed by its 4 bytes widened to uint16; a tail of
+ * n mod 4 bytes is written as 0xFFFF followed by those bytes.  codes: HOST, n bytes.  out: HOST,
+ * room for out_cap uint16; out == NULL only queries the size.  *out_len receives the stream length
+ * in uint16 units; n_hits / n_miss (may be NULL) the number of coded / escaped groups.
+ * TQ_ERR_BUFFER_TOO_SMALL if out_cap is short. */
+int tq_encode(const tq_dict* d, const uint8_t* codes, uint64_t n, uint16_t* out, uint64_t out_cap,
+              uint64_t* out_len, uint64_t* n_hits, uint64_t* n_miss);
+
+void tq_dict_free(tq_dict* d);
+
+/* ------------------------------------------------------------------------------------------
+ * Device side: upload, decompress, fused products.
+ * ---------------------------------------------------------------------------------------- */
+
+/* Bytes of DEVICE memory a table needs. */
+int tq_dict_upload_size(const tq_dict* d, uint64_t* device_bytes);
+
+/* Copy the table into the caller's DEVICE buffer d_buf (256-byte aligned, d_buf_bytes long) and
+ * return a handle.  Synchronises cuda_stream before returning. */
+int tq_dict_upload(const tq_dict* d, void* d_buf, uint64_t d_buf_bytes, void* cuda_stream,
+                   tq_ddict** out);
+void tq_ddict_free(tq_ddict* d); /* host handle only */
+
+/* Device layouts of a compressed matrix. */
+#define TQ_LAYOUT_STREAM 0 /* the paper's token stream, byte for byte, cut into per-row segments */
+
+/* Bytes of DEVICE memory the layout of this stream needs.  stream: HOST.  Requires cols % 4 == 0
+ * (no aligned group straddles two rows; true of every LLaMA shape), else TQ_ERR_UNSUPPORTED_SHAPE. */
+int tq_upload_size(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
+                   int layout, uint64_t* device_bytes);
+
+/* Validate a token stream (Listing 4's walk must yield exactly rows*cols bytes, every code must be
+ * in 1..K, every raw slot <= 255) and place it in the caller's DEVICE buffer in the given layout,
+ * together with the per-row scale and zero point of the dequantisation scale_r * (q - zero_r)
+ * (Listing 1).  row_zero may be NULL (all zero).  levels_signed != 0: the decoded byte is an int8
+ * bit pattern (per-row symmetric quantizer); 0: an unsigned level 0..255 (Listing 1).
+ * stream, row_scale, row_zero: HOST.  d_buf: DEVICE, 256-byte aligned.  Synchronises cuda_stream
+ * before returning.  A corrupt stream is rejected with TQ_ERR_CORRUPT_STREAM and nothing is
+ * uploaded. */
+int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len, uint32_t rows,
+              uint32_t cols, const float* row_scale, const float* row_zero, int levels_signed,
+              int layout, void* d_buf, uint64_t d_buf_bytes, void* cuda_stream, tq_dmat** out);
+
+typedef struct tq_dmat_info {
+  uint32_t rows, cols, K;
+  int32_t layout, levels_signed;
+  uint64_t n_hits, n_miss;   /* coded / escaped groups                                        */
+  uint64_t stream_bytes;     /* the paper's stream: 2 * (n_hits + 5 * n_miss)                  */
+  uint64_t payload_bytes;    /* bytes a kernel reads per pass: token segments with their
+                                padding + per-row index + scales                              */
+  uint64_t device_bytes;     /* whole footprint in the caller's buffer                         */
+} tq_dmat_info;
+int tq_dmat_get_info(const tq_dmat* m, tq_dmat_info* info);
+
+/* Decompress (Listing 4): write the rows*cols decoded bytes, row-major, to d_codes (DEVICE). */
+int tq_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream);
+
+/* Compressed linear layer for small batches (Section 2.3: weights are expanded layer by layer,
+ * then used as an ordinary linear layer; here the expansion, Listing 1's scale*(q-zero) and the
+ * product are one kernel and the weights never reach memory):
+ *   y[b][r] = scale_r * sum_c (q[r][c] - zero_r) * x[b][c],   fp32 accumulation.
+ * d_x_bf16: DEVICE [B][cols] bf16, 16-byte aligned; B in 1..32; d_y: DEVICE [B][rows] fp32. */
+int tq_fused_gemv(const tq_dmat* m, const void* d_x_bf16, int B, float* d_y, void* cuda_stream);
+
+/* The same call with HOST operands: copies x to the DEVICE staging buffer d_x_stage ([B][cols]
+ * bf16), runs the kernel, copies y back from d_y_stage ([B][rows] fp32), all on cuda_stream, and
+ * does not synchronise.  h_x_bf16 / h_y should be pinned for the copies to be asynchronous. */
+int tq_fused_gemv_host(const tq_dmat* m, const void* h_x_bf16, int B, float* h_y, void* d_x_stage,
+                       float* d_y_stage, void* cuda_stream);
+
+/* Same product for prefill-sized batches (M tokens): decoded weight tiles are converted to bf16
+ * (exact: |level| <= 255) in shared memory and fed to tcgen05 tensor-core MMAs with fp32
+ * accumulation; scale and zero point are applied in fp32 afterwards.
+ * d_X_bf16: DEVICE [M][cols] bf16, 16-byte aligned; d_Y: DEVICE [M][rows] fp32. */
+int tq_fused_gemm(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, void* cuda_stream);
+
+/* Read and clear the matrix's device status word (TQ_STATUS_* bits); synchronises cuda_stream. */
+int tq_device_status(const tq_dmat* m, void* cuda_stream, uint32_t* status);
+
+void tq_dmat_free(tq_dmat* m); /* host handle only */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TQ_H_ */

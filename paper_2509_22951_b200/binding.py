@@ -1,0 +1,329 @@
+"""ctypes binding of libtq.so: argument marshalling only, same names as include/tq.h.
+
+Host arrays are numpy arrays; device memory is torch CUDA tensors (PyTorch is used for
+device memory and streams only).  There is no CPU fallback: if libtq.so cannot be loaded (or
+built with nvcc) importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+TQ_OK = 0
+TQ_ERR_INVALID_ARG = -1
+TQ_ERR_CORRUPT_STREAM = -2
+TQ_ERR_BUFFER_TOO_SMALL = -3
+TQ_ERR_UNSUPPORTED_SHAPE = -4
+TQ_ERR_CUDA = -5
+TQ_ERR_TIMEOUT = -6
+TQ_ERR_NOMEM = -7
+TQ_LAYOUT_STREAM = 0
+TQ_STATUS_BAD_CODE = 1
+TQ_STATUS_BAD_ROW = 2
+TQ_STATUS_WAIT_EXPIRED = 4
+
+EXPORTS = [
+    "tq_strerror", "tq_set_num_threads", "tq_quantize_tensor", "tq_quantize_rows",
+    "tq_quantize_rows_device", "tq_build_dictionary", "tq_dict_from_entries", "tq_dict_entries",
+    "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
+    "tq_upload_size", "tq_upload", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
+    "tq_fused_gemv_host", "tq_fused_gemm", "tq_device_status", "tq_dmat_free",
+]
+
+
+class TqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {_lib.tq_strerror(status).decode()} ({status})")
+
+
+class _Info(C.Structure):
+    _fields_ = [("rows", C.c_uint32), ("cols", C.c_uint32), ("K", C.c_uint32),
+                ("layout", C.c_int32), ("levels_signed", C.c_int32),
+                ("n_hits", C.c_uint64), ("n_miss", C.c_uint64), ("stream_bytes", C.c_uint64),
+                ("payload_bytes", C.c_uint64), ("device_bytes", C.c_uint64)]
+
+
+def _load() -> C.CDLL:
+    path = _build.build_library()  # raises if the library is missing and cannot be built
+    lib = C.CDLL(str(path))
+    vp, u8p, u16p, u32p, u64p = C.c_void_p, C.POINTER(C.c_uint8), C.POINTER(C.c_uint16), C.POINTER(C.c_uint32), C.POINTER(C.c_uint64)
+    f32p = C.POINTER(C.c_float)
+    sig = {
+        "tq_strerror": (C.c_char_p, [C.c_int]),
+        "tq_set_num_threads": (C.c_int, [C.c_int]),
+        "tq_quantize_tensor": (C.c_int, [f32p, C.c_uint64, u8p, f32p, f32p]),
+        "tq_quantize_rows": (C.c_int, [f32p, C.c_uint32, C.c_uint32, C.POINTER(C.c_int8), f32p]),
+        "tq_quantize_rows_device": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, vp, vp]),
+        "tq_build_dictionary": (C.c_int, [C.POINTER(u8p), u64p, C.c_int, C.c_uint32, C.POINTER(vp)]),
+        "tq_dict_from_entries": (C.c_int, [u8p, C.c_uint32, C.POINTER(vp)]),
+        "tq_dict_entries": (C.c_int, [vp, u32p, C.POINTER(u8p), C.POINTER(u64p)]),
+        "tq_encode": (C.c_int, [vp, u8p, C.c_uint64, u16p, C.c_uint64, u64p, u64p, u64p]),
+        "tq_dict_free": (None, [vp]),
+        "tq_dict_upload_size": (C.c_int, [vp, u64p]),
+        "tq_dict_upload": (C.c_int, [vp, vp, C.c_uint64, vp, C.POINTER(vp)]),
+        "tq_ddict_free": (None, [vp]),
+        "tq_upload_size": (C.c_int, [u16p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_int, u64p]),
+        "tq_upload": (C.c_int, [vp, u16p, C.c_uint64, C.c_uint32, C.c_uint32, f32p, f32p, C.c_int,
+                                C.c_int, vp, C.c_uint64, vp, C.POINTER(vp)]),
+        "tq_dmat_get_info": (C.c_int, [vp, C.POINTER(_Info)]),
+        "tq_decompress": (C.c_int, [vp, vp, vp]),
+        "tq_fused_gemv": (C.c_int, [vp, vp, C.c_int, vp, vp]),
+        "tq_fused_gemv_host": (C.c_int, [vp, vp, C.c_int, vp, vp, vp, vp]),
+        "tq_fused_gemm": (C.c_int, [vp, vp, C.c_int, vp, vp]),
+        "tq_device_status": (C.c_int, [vp, vp, u32p]),
+        "tq_dmat_free": (None, [vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    return lib
+
+
+_lib = _load()
+
+
+def _check(status: int, where: str) -> None:
+    if status != TQ_OK:
+        raise TqError(status, where)
+
+
+def _np_ptr(a: np.ndarray, ctype):
+    return a.ctypes.data_as(C.POINTER(ctype))
+
+
+def _stream_ptr(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def tq_set_num_threads(n: int) -> int:
+    return _lib.tq_set_num_threads(n)
+
+
+# ------------------------------------------------------------------------------ host
+def tq_quantize_tensor(x: np.ndarray):
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    q = np.empty(x.shape, dtype=np.uint8)
+    s, z = C.c_float(), C.c_float()
+    _check(_lib.tq_quantize_tensor(_np_ptr(x, C.c_float), x.size, _np_ptr(q, C.c_uint8), C.byref(s), C.byref(z)),
+           "tq_quantize_tensor")
+    return q, np.float32(s.value), np.float32(z.value)
+
+
+def tq_quantize_rows(w: np.ndarray):
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    rows, cols = w.shape
+    q = np.empty((rows, cols), dtype=np.int8)
+    s = np.empty(rows, dtype=np.float32)
+    _check(_lib.tq_quantize_rows(_np_ptr(w, C.c_float), rows, cols, _np_ptr(q, C.c_int8), _np_ptr(s, C.c_float)),
+           "tq_quantize_rows")
+    return q, s
+
+
+def tq_quantize_rows_device(w: torch.Tensor, stream=None):
+    assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous() and w.dim() == 2
+    rows, cols = w.shape
+    q = torch.empty((rows, cols), dtype=torch.int8, device=w.device)
+    s = torch.empty(rows, dtype=torch.float32, device=w.device)
+    _check(_lib.tq_quantize_rows_device(w.data_ptr(), rows, cols, q.data_ptr(), s.data_ptr(), _stream_ptr(stream)),
+           "tq_quantize_rows_device")
+    return q, s
+
+
+class Dict:
+    """Owner of a host tq_dict handle."""
+
+    def __init__(self, handle: int):
+        self._h = C.c_void_p(handle)
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            _lib.tq_dict_free(self._h)
+            self._h = None
+
+    def _borrow(self):
+        K, e, c = C.c_uint32(), C.POINTER(C.c_uint8)(), C.POINTER(C.c_uint64)()
+        _check(_lib.tq_dict_entries(self._h, C.byref(K), C.byref(e), C.byref(c)), "tq_dict_entries")
+        return K.value, e, c
+
+    @property
+    def K(self) -> int:
+        return self._borrow()[0]
+
+    @property
+    def entries(self) -> np.ndarray:
+        K, e, _ = self._borrow()
+        return np.ctypeslib.as_array(e, shape=(K, 4)).copy() if K else np.zeros((0, 4), np.uint8)
+
+    @property
+    def counts(self) -> np.ndarray:
+        K, _, c = self._borrow()
+        return np.ctypeslib.as_array(c, shape=(K,)).copy() if K else np.zeros((0,), np.uint64)
+
+
+def tq_build_dictionary(mats, top_k: int = 2 ** 16 - 1) -> Dict:
+    arrs = [np.ascontiguousarray(m).view(np.uint8).reshape(-1) for m in mats]
+    n = len(arrs)
+    ptrs = (C.POINTER(C.c_uint8) * max(n, 1))(*[_np_ptr(a, C.c_uint8) for a in arrs])
+    lens = (C.c_uint64 * max(n, 1))(*[a.size for a in arrs])
+    out = C.c_void_p()
+    _check(_lib.tq_build_dictionary(ptrs, lens, n, top_k, C.byref(out)), "tq_build_dictionary")
+    return Dict(out.value)
+
+
+def tq_dict_from_entries(entries: np.ndarray) -> Dict:
+    e = np.ascontiguousarray(entries, dtype=np.uint8).reshape(-1, 4)
+    out = C.c_void_p()
+    _check(_lib.tq_dict_from_entries(_np_ptr(e, C.c_uint8), e.shape[0], C.byref(out)), "tq_dict_from_entries")
+    return Dict(out.value)
+
+
+def tq_encode(d: Dict, codes: np.ndarray):
+    """-> (stream uint16, n_hits, n_miss)"""
+    w = np.ascontiguousarray(codes).view(np.uint8).reshape(-1)
+    n, h, m = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    _check(_lib.tq_encode(d._h, _np_ptr(w, C.c_uint8), w.size, None, 0, C.byref(n), C.byref(h), C.byref(m)), "tq_encode")
+    out = np.empty(n.value, dtype=np.uint16)
+    _check(_lib.tq_encode(d._h, _np_ptr(w, C.c_uint8), w.size, _np_ptr(out, C.c_uint16), out.size,
+                          C.byref(n), C.byref(h), C.byref(m)), "tq_encode")
+    return out, h.value, m.value
+
+
+# ------------------------------------------------------------------------------ device
+class DeviceDict:
+    """A table resident on the GPU: owns the torch buffer and the tq_ddict handle."""
+
+    def __init__(self, handle: int, buf: torch.Tensor, K: int):
+        self._h = C.c_void_p(handle)
+        self.buf = buf
+        self.K = K
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            _lib.tq_ddict_free(self._h)
+            self._h = None
+
+
+def tq_dict_upload(d: Dict, device="cuda", stream=None) -> DeviceDict:
+    need = C.c_uint64()
+    _check(_lib.tq_dict_upload_size(d._h, C.byref(need)), "tq_dict_upload_size")
+    buf = torch.empty(need.value, dtype=torch.uint8, device=device)
+    out = C.c_void_p()
+    with torch.cuda.device(buf.device):
+        _check(_lib.tq_dict_upload(d._h, buf.data_ptr(), buf.numel(), _stream_ptr(stream), C.byref(out)), "tq_dict_upload")
+    return DeviceDict(out.value, buf, d.K)
+
+
+@dataclass
+class MatInfo:
+    rows: int
+    cols: int
+    K: int
+    layout: int
+    levels_signed: int
+    n_hits: int
+    n_miss: int
+    stream_bytes: int
+    payload_bytes: int
+    device_bytes: int
+
+
+class DeviceMatrix:
+    """One compressed matrix resident on the GPU: owns the torch buffer and the tq_dmat handle."""
+
+    def __init__(self, handle: int, buf: torch.Tensor, ddict: DeviceDict):
+        self._h = C.c_void_p(handle)
+        self.buf = buf
+        self.ddict = ddict  # keeps the table alive
+        i = _Info()
+        _check(_lib.tq_dmat_get_info(self._h, C.byref(i)), "tq_dmat_get_info")
+        self.info = MatInfo(*(getattr(i, f[0]) for f in _Info._fields_))
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            _lib.tq_dmat_free(self._h)
+            self._h = None
+
+
+def tq_upload_size(stream: np.ndarray, rows: int, cols: int, layout: int = TQ_LAYOUT_STREAM) -> int:
+    s = np.ascontiguousarray(stream, dtype=np.uint16)
+    need = C.c_uint64()
+    _check(_lib.tq_upload_size(_np_ptr(s, C.c_uint16), s.size, rows, cols, layout, C.byref(need)), "tq_upload_size")
+    return need.value
+
+
+def tq_upload(ddict: DeviceDict, stream: np.ndarray, rows: int, cols: int, row_scale: np.ndarray,
+              row_zero=None, levels_signed: bool = True, layout: int = TQ_LAYOUT_STREAM,
+              cuda_stream=None) -> DeviceMatrix:
+    s = np.ascontiguousarray(stream, dtype=np.uint16)
+    sc = np.ascontiguousarray(row_scale, dtype=np.float32)
+    assert sc.size == rows
+    zp = None
+    if row_zero is not None:
+        zr = np.ascontiguousarray(row_zero, dtype=np.float32)
+        assert zr.size == rows
+        zp = _np_ptr(zr, C.c_float)
+    need = C.c_uint64()
+    _check(_lib.tq_upload_size(_np_ptr(s, C.c_uint16), s.size, rows, cols, layout, C.byref(need)), "tq_upload_size")
+    buf = torch.empty(need.value, dtype=torch.uint8, device=ddict.buf.device)
+    out = C.c_void_p()
+    with torch.cuda.device(buf.device):
+        _check(_lib.tq_upload(ddict._h, _np_ptr(s, C.c_uint16), s.size, rows, cols, _np_ptr(sc, C.c_float), zp,
+                              int(levels_signed), layout, buf.data_ptr(), buf.numel(), _stream_ptr(cuda_stream),
+                              C.byref(out)), "tq_upload")
+    return DeviceMatrix(out.value, buf, ddict)
+
+
+def tq_decompress(m: DeviceMatrix, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty((m.info.rows, m.info.cols), dtype=torch.uint8, device=m.buf.device)
+    assert out.is_cuda and out.is_contiguous() and out.numel() == m.info.rows * m.info.cols and out.element_size() == 1
+    _check(_lib.tq_decompress(m._h, out.data_ptr(), _stream_ptr(stream)), "tq_decompress")
+    return out
+
+
+def tq_fused_gemv(m: DeviceMatrix, x: torch.Tensor, y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+    x2 = x.view(-1, m.info.cols)
+    B = x2.shape[0]
+    if y is None:
+        y = torch.empty((B, m.info.rows), dtype=torch.float32, device=x.device)
+    assert y.is_cuda and y.dtype == torch.float32 and y.is_contiguous() and y.numel() == B * m.info.rows
+    _check(_lib.tq_fused_gemv(m._h, x2.data_ptr(), B, y.data_ptr(), _stream_ptr(stream)), "tq_fused_gemv")
+    return y
+
+
+def tq_fused_gemv_host(m: DeviceMatrix, h_x: torch.Tensor, h_y: torch.Tensor, d_x_stage: torch.Tensor,
+                       d_y_stage: torch.Tensor, stream=None) -> None:
+    """h_x: CPU (pinned) bf16 [B][cols]; h_y: CPU (pinned) fp32 [B][rows]; stages: CUDA tensors."""
+    assert (not h_x.is_cuda) and h_x.dtype == torch.bfloat16 and h_x.is_contiguous()
+    assert (not h_y.is_cuda) and h_y.dtype == torch.float32 and h_y.is_contiguous()
+    B = h_x.numel() // m.info.cols
+    assert d_x_stage.is_cuda and d_x_stage.numel() * d_x_stage.element_size() >= B * m.info.cols * 2
+    assert d_y_stage.is_cuda and d_y_stage.numel() * d_y_stage.element_size() >= B * m.info.rows * 4
+    _check(_lib.tq_fused_gemv_host(m._h, h_x.data_ptr(), B, h_y.data_ptr(), d_x_stage.data_ptr(),
+                                   d_y_stage.data_ptr(), _stream_ptr(stream)), "tq_fused_gemv_host")
+
+
+def tq_fused_gemm(m: DeviceMatrix, X: torch.Tensor, Y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.is_contiguous()
+    X2 = X.view(-1, m.info.cols)
+    M = X2.shape[0]
+    if Y is None:
+        Y = torch.empty((M, m.info.rows), dtype=torch.float32, device=X.device)
+    assert Y.is_cuda and Y.dtype == torch.float32 and Y.is_contiguous() and Y.numel() == M * m.info.rows
+    _check(_lib.tq_fused_gemm(m._h, X2.data_ptr(), M, Y.data_ptr(), _stream_ptr(stream)), "tq_fused_gemm")
+    return Y
+
+
+def tq_device_status(m: DeviceMatrix, stream=None) -> int:
+    st = C.c_uint32()
+    _check(_lib.tq_device_status(m._h, _stream_ptr(stream), C.byref(st)), "tq_device_status")
+    return st.value

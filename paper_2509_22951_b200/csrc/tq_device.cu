@@ -1,0 +1,440 @@
+// Device half of libtq (sm_100a): upload, tq_decompress, tq_fused_gemv and the row quantizer.
+//
+// Token parse shared by the kernels (Listing 4 made data-parallel).  One warp owns one row
+// segment and walks it in tiles of 256 uint16 slots; a lane holds 8 consecutive slots (one
+// 128-bit load).  A slot equal to 0xFFFF is always a marker (raw slots hold bytes, codes stop at
+// 65534), so a slot is raw exactly when one of the 4 slots before it is a marker.  A group is
+// "completed" at a code slot or at the 4th raw slot after a marker; the lane that holds the
+// completing slot also sees the 4 slots before its own 8 (two registers shuffled from the lane
+// below, or carried over from the previous tile), which is all it needs to produce the group's 4
+// bytes.  The group's index inside the row is a warp prefix sum of the per-lane completion counts
+// plus a running base.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <new>
+
+#include "tq_internal.h"
+
+namespace {
+
+constexpr int kWarpsPerCta = 8;
+constexpr int kThreads = kWarpsPerCta * 32;
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+// bit 15 / bit 31 set when the low / high half of a equals 0xFFFF (exact for validated streams:
+// the only false positive is 0xFFFE directly after a marker, which validation rules out).
+__device__ __forceinline__ uint32_t esc_bits(uint32_t a) {
+  return ~(a + 0x00010001u) & a & 0x80008000u;
+}
+
+// Walks one row segment.  emit(group_index, packed4bytes) is called once per completed group by
+// the lane that completed it.  Returns the number of groups seen (warp-uniform).
+template <class Emit>
+__device__ __forceinline__ uint32_t decode_row(const uint4* __restrict__ tok, uint32_t n_slots,
+                                               const uint32_t* __restrict__ table, uint32_t K,
+                                               uint32_t groups_per_row, uint32_t& status_bits,
+                                               Emit&& emit) {
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t n_chunks = (n_slots + 7u) >> 3;
+  const uint32_t n_tiles = (n_chunks + 31u) >> 5;
+  const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+
+  uint4 cur = lane < n_chunks ? ldg_stream(tok + lane) : zero4;
+  uint4 nxt = lane + 32u < n_chunks ? ldg_stream(tok + lane + 32u) : zero4;
+  uint32_t base = 0, carryE = 0, carryZ = 0, carryW = 0;
+
+  for (uint32_t t = 0; t < n_tiles; ++t) {
+    const uint32_t pf = (t + 2u) * 32u + lane;
+    const uint4 nn = pf < n_chunks ? ldg_stream(tok + pf) : zero4;
+
+    const int left = (int)n_slots - (int)(t * 256u + lane * 8u);
+    const uint32_t V = left >= 8 ? 0xFFu : (left <= 0 ? 0u : ((1u << left) - 1u));
+
+    const uint32_t e = (esc_bits(cur.x) >> 15) | (esc_bits(cur.y) >> 13) | (esc_bits(cur.z) >> 11) |
+                       (esc_bits(cur.w) >> 9);
+    const uint32_t E = (e | (e >> 15)) & V;
+
+    uint32_t prevE = __shfl_up_sync(kFull, E, 1);
+    uint32_t pz = __shfl_up_sync(kFull, cur.z, 1);
+    uint32_t pw = __shfl_up_sync(kFull, cur.w, 1);
+    if (lane == 0) { prevE = carryE; pz = carryZ; pw = carryW; }
+
+    const uint32_t X = (prevE >> 4) | (E << 4);                    // markers over the 12-slot window
+    const uint32_t R = (X | (X >> 1) | (X >> 2) | (X >> 3)) & 0xFFu;  // own slots that are raw
+    const uint32_t C = ((~R & ~E) | X) & V;                        // own slots that complete a group
+
+    const uint32_t n = __popc(C);
+    uint32_t incl = n;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      uint32_t v = __shfl_up_sync(kFull, incl, d);
+      if (lane >= (uint32_t)d) incl += v;
+    }
+    uint32_t g = base + incl - n;
+    base += __shfl_sync(kFull, incl, 31);
+    carryE = __shfl_sync(kFull, E, 31);
+    carryZ = __shfl_sync(kFull, cur.z, 31);
+    carryW = __shfl_sync(kFull, cur.w, 31);
+
+    const uint32_t W[6] = {pz, pw, cur.x, cur.y, cur.z, cur.w};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (C & (1u << j)) {
+        uint32_t w;
+        if (X & (1u << j)) {  // 4th raw slot of a marker at window slot j: bytes of slots j+1..j+4
+          if (j & 1) {
+            w = __byte_perm(W[(j + 1) >> 1], W[((j + 1) >> 1) + 1], 0x6420);
+          } else {
+            const uint32_t t3 = __byte_perm(W[j >> 1], W[(j >> 1) + 1], 0x0642);
+            w = __byte_perm(t3, W[(j >> 1) + 2], 0x4210);
+          }
+        } else {
+          const uint32_t reg = W[2 + (j >> 1)];
+          const uint32_t code = (j & 1) ? (reg >> 16) : (reg & 0xFFFFu);
+          if (code - 1u < K) {
+            w = __ldg(table + (code - 1u));
+          } else {
+            w = 0u;
+            status_bits |= TQ_STATUS_BAD_CODE;
+          }
+        }
+        if (g < groups_per_row) emit(g, w);
+        ++g;
+      }
+    }
+    cur = nxt;
+    nxt = nn;
+  }
+  return base;
+}
+
+// ---------------------------------------------------------------------------------------------
+// tq_decompress: expand to bytes in HBM.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+decompress_kernel(const uint4* __restrict__ tokens, const tq_rowseg* __restrict__ rowseg,
+                  const uint32_t* __restrict__ table, uint32_t K, uint32_t rows, uint32_t cols,
+                  uint32_t* __restrict__ out, uint32_t* __restrict__ status) {
+  const uint32_t warp = threadIdx.x >> 5;
+  const uint32_t gpr = cols >> 2;
+  uint32_t bits = 0;
+  for (uint32_t row = blockIdx.x * kWarpsPerCta + warp; row < rows; row += gridDim.x * kWarpsPerCta) {
+    const tq_rowseg seg = rowseg[row];
+    uint32_t* orow = out + (size_t)row * gpr;
+    const uint32_t seen = decode_row(tokens + seg.chunk_off, seg.n_slots, table, K, gpr, bits,
+                                     [&](uint32_t g, uint32_t w) { orow[g] = w; });
+    if (seen != gpr) bits |= TQ_STATUS_BAD_ROW;
+  }
+  if (bits) atomicOr(status, bits);
+}
+
+// ---------------------------------------------------------------------------------------------
+// tq_fused_gemv: decode -> dequantise -> dot product, batch NB (1..4) per pass.
+// x is staged once per CTA in shared memory as fp32, one float4 per group of 4 columns.
+// A byte b becomes a float through the bit pattern 0x4B000000 | b' (= 2^23 + b') minus a
+// constant; with b' = b ^ 0x80 and the constant 2^23 + 128 this is the int8 value of b, with
+// b' = b and 2^23 the unsigned one.
+// ---------------------------------------------------------------------------------------------
+template <int NB>
+__global__ void __launch_bounds__(kThreads)
+gemv_kernel(const uint4* __restrict__ tokens, const tq_rowseg* __restrict__ rowseg,
+            const float* __restrict__ scale, const float* __restrict__ zero, int has_zero,
+            const uint32_t* __restrict__ table, uint32_t K, uint32_t rows, uint32_t cols,
+            const __nv_bfloat16* __restrict__ x, float* __restrict__ y, uint32_t xor_mask,
+            float magic, uint32_t* __restrict__ status) {
+  extern __shared__ __align__(16) float xs[];  // [NB][cols]
+  __shared__ float sumx[NB];
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+  const uint32_t gpr = cols >> 2;
+
+  for (uint32_t i = threadIdx.x; i < NB * (cols >> 1); i += kThreads) {
+    const __nv_bfloat162 v = reinterpret_cast<const __nv_bfloat162*>(x)[i];
+    reinterpret_cast<float2*>(xs)[i] = __bfloat1622float2(v);
+  }
+  if (threadIdx.x < NB) sumx[threadIdx.x] = 0.f;
+  __syncthreads();
+  if (has_zero) {
+    for (int b = 0; b < NB; ++b) {
+      float s = 0.f;
+      for (uint32_t i = threadIdx.x; i < cols; i += kThreads) s += xs[b * cols + i];
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(kFull, s, d);
+      if (lane == 0) atomicAdd(&sumx[b], s);
+    }
+    __syncthreads();
+  }
+
+  uint32_t bits = 0;
+  for (uint32_t row = blockIdx.x * kWarpsPerCta + warp; row < rows; row += gridDim.x * kWarpsPerCta) {
+    const tq_rowseg seg = rowseg[row];
+    float acc[NB];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) acc[b] = 0.f;
+    const uint32_t seen = decode_row(
+        tokens + seg.chunk_off, seg.n_slots, table, K, gpr, bits, [&](uint32_t g, uint32_t w) {
+          w ^= xor_mask;
+          const float f0 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7540)) - magic;
+          const float f1 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7541)) - magic;
+          const float f2 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7542)) - magic;
+          const float f3 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7543)) - magic;
+#pragma unroll
+          for (int b = 0; b < NB; ++b) {
+            const float4 xv = reinterpret_cast<const float4*>(xs + b * cols)[g];
+            acc[b] = fmaf(f0, xv.x, acc[b]);
+            acc[b] = fmaf(f1, xv.y, acc[b]);
+            acc[b] = fmaf(f2, xv.z, acc[b]);
+            acc[b] = fmaf(f3, xv.w, acc[b]);
+          }
+        });
+    if (seen != gpr) bits |= TQ_STATUS_BAD_ROW;
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      float a = acc[b];
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(kFull, a, d);
+      acc[b] = a;
+    }
+    if (lane == 0) {
+      const float s = scale[row];
+      const float z = has_zero ? zero[row] : 0.f;
+#pragma unroll
+      for (int b = 0; b < NB; ++b) y[(size_t)b * rows + row] = s * (acc[b] - z * sumx[b]);
+    }
+  }
+  if (bits) atomicOr(status, bits);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Per-row symmetric int8 quantizer (one CTA per row).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+quantize_rows_kernel(const float* __restrict__ w, uint32_t rows, uint32_t cols, int8_t* __restrict__ q,
+                     float* __restrict__ scale) {
+  __shared__ float red[8];
+  __shared__ float s_sh;
+  for (uint32_t row = blockIdx.x; row < rows; row += gridDim.x) {
+    const float* wr = w + (size_t)row * cols;
+    float amax = 0.f;
+    for (uint32_t c = threadIdx.x; c < cols; c += 256) amax = fmaxf(amax, fabsf(wr[c]));
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(kFull, amax, d));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float m = red[0];
+      for (int i = 1; i < 8; ++i) m = fmaxf(m, red[i]);
+      const float s = m > 0.f ? __fdiv_rn(m, 127.0f) : 1.0f;
+      s_sh = s;
+      scale[row] = s;
+    }
+    __syncthreads();
+    const float s = s_sh;
+    for (uint32_t c = threadIdx.x; c < cols; c += 256) {
+      float v = rintf(__fdiv_rn(wr[c], s));
+      v = fminf(fmaxf(v, -127.f), 127.f);
+      q[(size_t)row * cols + c] = (int8_t)v;
+    }
+    __syncthreads();
+  }
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? TQ_OK : TQ_ERR_CUDA; }
+
+template <int NB>
+int launch_gemv(const tq_dmat* m, const __nv_bfloat16* x, float* y, cudaStream_t st) {
+  const uint32_t rows = m->info.rows, cols = m->info.cols;
+  const size_t smem = (size_t)NB * cols * sizeof(float);
+  static size_t configured = 0;
+  if (smem > 48 * 1024 && smem > configured) {
+    if (cudaFuncSetAttribute(gemv_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return TQ_ERR_CUDA;
+    configured = smem;
+  }
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gemv_kernel<NB>, kThreads, smem) != cudaSuccess || per_sm < 1)
+    return TQ_ERR_CUDA;
+  const uint32_t need = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
+  const uint32_t grid = std::min<uint32_t>(need, (uint32_t)(sm_count() * per_sm));
+  gemv_kernel<NB><<<grid, kThreads, smem, st>>>(
+      reinterpret_cast<const uint4*>(m->d_tokens), m->d_rowseg, m->d_scale, m->d_zero, m->has_zero,
+      m->dict->d_entries, m->dict->K, rows, cols, x, y, m->info.levels_signed ? 0x80808080u : 0u,
+      m->info.levels_signed ? 8388736.0f : 8388608.0f, m->d_status);
+  return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace
+
+extern "C" {
+
+int tq_quantize_rows_device(const float* d_w, uint32_t rows, uint32_t cols, int8_t* d_q, float* d_scale,
+                            void* cuda_stream) {
+  if (!d_w || !d_q || !d_scale || rows == 0 || cols == 0) return TQ_ERR_INVALID_ARG;
+  const uint32_t grid = std::min<uint32_t>(rows, (uint32_t)sm_count() * 8u);
+  quantize_rows_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(d_w, rows, cols, d_q, d_scale);
+  return cuda_ok(cudaGetLastError());
+}
+
+int tq_dict_upload_size(const tq_dict* d, uint64_t* device_bytes) {
+  if (!d || !device_bytes) return TQ_ERR_INVALID_ARG;
+  *device_bytes = ((uint64_t)d->K * 4 + 255) / 256 * 256 + 256;
+  return TQ_OK;
+}
+
+int tq_dict_upload(const tq_dict* d, void* d_buf, uint64_t d_buf_bytes, void* cuda_stream, tq_ddict** out) {
+  if (!d || !d_buf || !out || ((uintptr_t)d_buf & 255)) return TQ_ERR_INVALID_ARG;
+  uint64_t need = 0;
+  tq_dict_upload_size(d, &need);
+  if (d_buf_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (d->K) {
+    if (cudaMemcpyAsync(d_buf, d->entries.data(), (size_t)d->K * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return TQ_ERR_CUDA;
+  }
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TQ_ERR_CUDA;
+  tq_ddict* dd = new (std::nothrow) tq_ddict();
+  if (!dd) return TQ_ERR_NOMEM;
+  dd->K = d->K;
+  dd->d_entries = static_cast<const uint32_t*>(d_buf);
+  *out = dd;
+  return TQ_OK;
+}
+
+void tq_ddict_free(tq_ddict* d) { delete d; }
+
+int tq_upload_size(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols, int layout,
+                   uint64_t* device_bytes) {
+  if (!device_bytes || layout != TQ_LAYOUT_STREAM) return TQ_ERR_INVALID_ARG;
+  return tq_build_stream_image(stream, stream_len, rows, cols, 0xFFFFFFFFu, nullptr, nullptr, device_bytes, nullptr);
+}
+
+int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
+              const float* row_scale, const float* row_zero, int levels_signed, int layout, void* d_buf,
+              uint64_t d_buf_bytes, void* cuda_stream, tq_dmat** out) {
+  if (!dict || !stream || !row_scale || !d_buf || !out || ((uintptr_t)d_buf & 255) || layout != TQ_LAYOUT_STREAM)
+    return TQ_ERR_INVALID_ARG;
+  tq_host_image img;
+  uint64_t need = 0;
+  int rc = tq_build_stream_image(stream, stream_len, rows, cols, dict->K, row_scale, row_zero, &need, &img);
+  if (rc != TQ_OK) return rc;
+  if (d_buf_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (cudaMemcpyAsync(d_buf, img.blob.data(), img.blob.size(), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return TQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TQ_ERR_CUDA;
+  tq_dmat* m = new (std::nothrow) tq_dmat();
+  if (!m) return TQ_ERR_NOMEM;
+  uint8_t* base = static_cast<uint8_t*>(d_buf);
+  m->dict = dict;
+  m->d_status = reinterpret_cast<uint32_t*>(base + img.off_status);
+  m->d_rowseg = reinterpret_cast<const tq_rowseg*>(base + img.off_rowseg);
+  m->d_scale = reinterpret_cast<const float*>(base + img.off_scale);
+  m->d_zero = reinterpret_cast<const float*>(base + img.off_zero);
+  m->d_tokens = reinterpret_cast<const uint16_t*>(base + img.off_tokens);
+  m->token_chunks = img.token_chunks;
+  m->has_zero = row_zero != nullptr;
+  m->info.rows = rows;
+  m->info.cols = cols;
+  m->info.K = dict->K;
+  m->info.layout = layout;
+  m->info.levels_signed = levels_signed != 0;
+  m->info.n_hits = img.n_hits;
+  m->info.n_miss = img.n_miss;
+  m->info.stream_bytes = 2 * (img.n_hits + 5 * img.n_miss);
+  m->info.payload_bytes = img.token_chunks * 16 + (uint64_t)rows * (sizeof(tq_rowseg) + 4 + (row_zero ? 4 : 0));
+  m->info.device_bytes = need;
+  *out = m;
+  return TQ_OK;
+}
+
+int tq_dmat_get_info(const tq_dmat* m, tq_dmat_info* info) {
+  if (!m || !info) return TQ_ERR_INVALID_ARG;
+  *info = m->info;
+  return TQ_OK;
+}
+
+void tq_dmat_free(tq_dmat* m) { delete m; }
+
+int tq_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
+  if (!m || !d_codes || ((uintptr_t)d_codes & 3)) return TQ_ERR_INVALID_ARG;
+  const uint32_t need = (m->info.rows + kWarpsPerCta - 1) / kWarpsPerCta;
+  const uint32_t grid = std::min<uint32_t>(need, (uint32_t)sm_count() * 8u);
+  decompress_kernel<<<grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
+      reinterpret_cast<const uint4*>(m->d_tokens), m->d_rowseg, m->dict->d_entries, m->dict->K, m->info.rows,
+      m->info.cols, reinterpret_cast<uint32_t*>(d_codes), m->d_status);
+  return cuda_ok(cudaGetLastError());
+}
+
+int tq_fused_gemv(const tq_dmat* m, const void* d_x_bf16, int B, float* d_y, void* cuda_stream) {
+  if (!m || !d_x_bf16 || !d_y || B < 1 || B > 32 || ((uintptr_t)d_x_bf16 & 15)) return TQ_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(d_x_bf16);
+  const uint32_t rows = m->info.rows, cols = m->info.cols;
+  // fp32 x for up to 4 batch columns must fit the 227 KB of shared memory
+  const int max_nb = (size_t)4 * cols * 4 <= 200 * 1024 ? 4 : ((size_t)2 * cols * 4 <= 200 * 1024 ? 2 : 1);
+  if ((size_t)cols * 4 > 200 * 1024) return TQ_ERR_UNSUPPORTED_SHAPE;
+  for (int b0 = 0; b0 < B;) {
+    int nb = std::min(B - b0, max_nb);
+    if (nb == 3 && ((uintptr_t)(x + (size_t)(b0 + 3) * cols) & 15)) nb = 2;
+    int rc;
+    const __nv_bfloat16* xb = x + (size_t)b0 * cols;
+    float* yb = d_y + (size_t)b0 * rows;
+    switch (nb) {
+      case 1: rc = launch_gemv<1>(m, xb, yb, st); break;
+      case 2: rc = launch_gemv<2>(m, xb, yb, st); break;
+      case 3: rc = launch_gemv<3>(m, xb, yb, st); break;
+      default: rc = launch_gemv<4>(m, xb, yb, st); break;
+    }
+    if (rc != TQ_OK) return rc;
+    b0 += nb;
+  }
+  return TQ_OK;
+}
+
+int tq_fused_gemv_host(const tq_dmat* m, const void* h_x_bf16, int B, float* h_y, void* d_x_stage,
+                       float* d_y_stage, void* cuda_stream) {
+  if (!m || !h_x_bf16 || !h_y || !d_x_stage || !d_y_stage || B < 1 || B > 32) return TQ_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (cudaMemcpyAsync(d_x_stage, h_x_bf16, (size_t)B * m->info.cols * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return TQ_ERR_CUDA;
+  int rc = tq_fused_gemv(m, d_x_stage, B, d_y_stage, cuda_stream);
+  if (rc != TQ_OK) return rc;
+  if (cudaMemcpyAsync(h_y, d_y_stage, (size_t)B * m->info.rows * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return TQ_ERR_CUDA;
+  return TQ_OK;
+}
+
+int tq_fused_gemm(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, void* cuda_stream) {
+  (void)m; (void)d_X_bf16; (void)M; (void)d_Y; (void)cuda_stream;
+  return TQ_ERR_UNSUPPORTED_SHAPE;
+}
+
+int tq_device_status(const tq_dmat* m, void* cuda_stream, uint32_t* status) {
+  if (!m || !status) return TQ_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (cudaMemcpyAsync(status, m->d_status, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return TQ_ERR_CUDA;
+  if (cudaMemsetAsync(m->d_status, 0, 4, st) != cudaSuccess) return TQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TQ_ERR_CUDA;
+  return TQ_OK;
+}
+
+}  // extern "C"

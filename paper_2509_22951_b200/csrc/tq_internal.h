@@ -1,0 +1,59 @@
+// Internal declarations shared by the host (tq_host.cpp) and device (tq_device.cu) halves of
+// libtq.  Nothing here crosses the C ABI.
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "tq.h"
+
+struct tq_dict {
+  uint32_t K = 0;
+  std::vector<uint8_t> entries;  // K x 4, rank order
+  std::vector<uint64_t> counts;  // K
+  // open-addressing lookup: 4-byte window -> code (0 = empty slot)
+  uint32_t map_mask = 0;
+  std::vector<uint32_t> map_key;
+  std::vector<uint16_t> map_code;
+  uint64_t n_windows = 0, n_distinct = 0;
+};
+
+struct tq_ddict {
+  uint32_t K = 0;
+  const uint32_t* d_entries = nullptr;  // DEVICE: K words, byte i of the window in bits 8i..8i+7
+};
+
+// Row descriptor of the STREAM layout: where the row's token segment starts (in 16-byte units
+// from the start of the token area) and how many uint16 slots it holds.
+struct tq_rowseg {
+  uint32_t chunk_off;
+  uint32_t n_slots;
+};
+
+struct tq_dmat {
+  tq_dmat_info info{};
+  const tq_ddict* dict = nullptr;
+  uint32_t* d_status = nullptr;        // DEVICE: status word
+  const tq_rowseg* d_rowseg = nullptr; // DEVICE: rows entries
+  const float* d_scale = nullptr;      // DEVICE: rows
+  const float* d_zero = nullptr;       // DEVICE: rows
+  const uint16_t* d_tokens = nullptr;  // DEVICE: token area, 256-byte aligned
+  uint64_t token_chunks = 0;           // token area length in 16-byte units
+  int has_zero = 0;
+};
+
+// Host-side image of a matrix in the STREAM layout, ready for one cudaMemcpy.
+struct tq_host_image {
+  std::vector<uint8_t> blob;
+  uint64_t off_status = 0, off_rowseg = 0, off_scale = 0, off_zero = 0, off_tokens = 0;
+  uint64_t token_chunks = 0;
+  uint64_t n_hits = 0, n_miss = 0;
+};
+
+int tq_num_threads();
+
+// Validates the stream and computes the layout size; if img != nullptr also builds the image.
+// K == 0xFFFFFFFF skips the code-range check (size query without a table).
+int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
+                          uint32_t K, const float* row_scale, const float* row_zero,
+                          uint64_t* device_bytes, tq_host_image* img);

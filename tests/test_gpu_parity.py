@@ -1,0 +1,158 @@
+"""CUDA path against the oracle, through the C ABI.  Decoded bytes must be bit-exact; layer
+outputs must satisfy max_r |y - y_ref| <= 2e-3 * max_r |y_ref| per batch column (fp32
+accumulation of exact int8 x bf16 products against an fp64 reference)."""
+import numpy as np
+import pytest
+import torch
+
+from inputs import synth
+from oracle import oracle
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-3
+
+
+@pytest.fixture(scope="module")
+def tq():
+    from paper_2509_22951_b200 import binding
+    return binding
+
+
+def _rel_err(y, ref):
+    # per batch column
+    return float(np.max(np.max(np.abs(y - ref), axis=1) / np.max(np.abs(ref), axis=1)))
+
+
+def _oracle_pack(q_list, top_k=65535):
+    d = oracle.Dictionary.build(q_list, top_k=top_k)
+    return d, [d.encode(q)[0] for q in q_list]
+
+
+def _upload_from_oracle(tq, odict, stream, rows, cols, scale, zero=None, signed=True):
+    """Everything fed to the device comes from the oracle (table, stream) so a host-library bug
+    cannot hide a device bug."""
+    hd = tq.tq_dict_from_entries(odict.entries)
+    dd = tq.tq_dict_upload(hd)
+    return tq.tq_upload(dd, stream, rows, cols, scale, zero, levels_signed=signed)
+
+
+def _check_layer(tq, q, scale, odict, stream, batches=(1,), zero=None, seed=1):
+    rows, cols = q.shape
+    m = _upload_from_oracle(tq, odict, stream, rows, cols, scale, zero, signed=(q.dtype == np.int8))
+    # decoded bytes: bit exact against the oracle's decoder and the original levels
+    got = tq.tq_decompress(m).cpu().numpy()
+    ref = odict.decode(stream).reshape(rows, cols)
+    assert np.array_equal(ref, q.view(np.uint8))
+    assert np.array_equal(got, ref)
+    for B in batches:
+        x = synth.activations(B, cols, seed + B)
+        y = tq.tq_fused_gemv(m, x.cuda()).cpu().numpy().astype(np.float64)
+        yref = oracle.layer_forward(q, scale, x.double().numpy(), zero=zero)
+        assert y.shape == yref.shape
+        assert _rel_err(y, yref) <= TOL
+    assert tq.tq_device_status(m) == 0
+    return m
+
+
+def test_config0_layer_2048x2048(tq):
+    w = synth.weight(2048, 2048, synth.matrix_seed(0)).numpy()
+    q, s = oracle.quantize_rows(w)
+    d, (stream,) = _oracle_pack([q])
+    m = _check_layer(tq, q, s, d, stream, batches=(1, 4))
+    assert m.info.n_hits + m.info.n_miss == 2048 * 2048 // 4
+    assert m.info.stream_bytes == stream.nbytes
+
+
+@pytest.mark.parametrize("rows,cols", [(1, 4), (3, 8), (7, 260), (8, 256), (9, 1028), (33, 2052), (17, 8192), (5, 12288)])
+def test_ragged_shapes(tq, rows, cols):
+    rng = np.random.default_rng(rows * 1000 + cols)
+    q = np.clip(np.rint(rng.standard_t(5, size=(rows, cols)) * 3), -127, 127).astype(np.int8)
+    s = (rng.random(rows) + 0.5).astype(np.float32)
+    d, (stream,) = _oracle_pack([q], top_k=200)
+    _check_layer(tq, q, s, d, stream, batches=(1, 2, 3, 4, 5))
+
+
+def test_all_hits_and_all_misses(tq):
+    rng = np.random.default_rng(5)
+    q = rng.integers(-2, 3, size=(64, 512)).astype(np.int8)
+    s = np.full(64, 0.01, dtype=np.float32)
+    d, (stream,) = _oracle_pack([q])
+    assert np.all(stream != 0xFFFF)  # every group is in the table
+    _check_layer(tq, q, s, d, stream, batches=(1, 4))
+    d0, (stream0,) = _oracle_pack([q], top_k=0)
+    assert stream0.size == 5 * q.size // 4  # every group escapes
+    _check_layer(tq, q, s, d0, stream0, batches=(1, 3))
+
+
+def test_large_table_codes_near_65534(tq):
+    # enough distinct windows to fill the table; high codes (>= 0xFF00) share their top byte with the marker
+    rng = np.random.default_rng(6)
+    q = rng.integers(-20, 21, size=(512, 1024)).astype(np.int8)
+    s = (rng.random(512) + 0.5).astype(np.float32)
+    d, (stream,) = _oracle_pack([q])
+    assert d.K == 65534 and int(stream[stream != 0xFFFF].max()) > 0xFF00
+    _check_layer(tq, q, s, d, stream, batches=(1,))
+
+
+def test_unsigned_levels_with_zero_point(tq):
+    # the paper's own quantizer: per-tensor unsigned levels and a zero point
+    w = synth.weight(256, 1024, synth.matrix_seed(9)).numpy()
+    qu, sc, zp = oracle.quantize_paper(w)
+    qu = qu.reshape(256, 1024)
+    s = np.full(256, sc, dtype=np.float32)
+    z = np.full(256, zp, dtype=np.float32)
+    d, (stream,) = _oracle_pack([qu])
+    _check_layer(tq, qu, s, d, stream, batches=(1, 4), zero=z)
+
+
+def test_batch_up_to_32(tq):
+    rng = np.random.default_rng(8)
+    q = np.clip(np.rint(rng.standard_t(5, size=(130, 3072)) * 6), -127, 127).astype(np.int8)
+    s = (rng.random(130) + 0.5).astype(np.float32)
+    d, (stream,) = _oracle_pack([q])
+    _check_layer(tq, q, s, d, stream, batches=(8, 32))
+
+
+def test_quantize_rows_device_bit_exact(tq):
+    w = synth.weight(300, 3072, synth.matrix_seed(11), device="cuda")
+    w[17] = 0
+    q, s = tq.tq_quantize_rows_device(w)
+    qo, so = oracle.quantize_rows(w.cpu().numpy())
+    assert np.array_equal(q.cpu().numpy(), qo) and np.array_equal(s.cpu().numpy(), so)
+
+
+def test_generator_is_device_independent():
+    a = synth.weight(64, 2048, synth.matrix_seed(2), device="cpu")
+    b = synth.weight(64, 2048, synth.matrix_seed(2), device="cuda").cpu()
+    assert torch.equal(a, b)
+    xa = synth.activations(4, 2048, 5, device="cpu")
+    xb = synth.activations(4, 2048, 5, device="cuda").cpu()
+    assert torch.equal(xa, xb)
+
+
+def test_host_library_pipeline_matches_oracle_pipeline(tq):
+    """Product pipeline end to end (tq_quantize_rows_device -> tq_build_dictionary -> tq_encode ->
+    tq_upload -> kernels) on the 1B MLP shapes, checked on sampled rows the oracle computes itself."""
+    shapes = [("gate", 8192, 2048), ("up", 8192, 2048), ("down", 2048, 8192)]
+    ws = [synth.weight(r, c, synth.matrix_seed(100 + i), device="cuda") for i, (_, r, c) in enumerate(shapes)]
+    qs, ss = zip(*[tq.tq_quantize_rows_device(w) for w in ws])
+    q_host = [q.cpu().numpy() for q in qs]
+    hd = tq.tq_build_dictionary(q_host)
+    dd = tq.tq_dict_upload(hd)
+    rng = np.random.default_rng(3)
+    for i, (name, rows, cols) in enumerate(shapes):
+        stream, h, mi = tq.tq_encode(hd, q_host[i])
+        assert stream.size == h + 5 * mi
+        m = tq.tq_upload(dd, stream, rows, cols, ss[i].cpu().numpy())
+        got = tq.tq_decompress(m)
+        assert torch.equal(got.view(torch.int8), qs[i])  # whole matrix, product vs product
+        sample = np.sort(rng.choice(rows, 64, replace=False))
+        qo, so = oracle.quantize_rows(ws[i][sample].cpu().numpy())  # oracle quantizes the sampled rows itself
+        assert np.array_equal(got[sample].cpu().numpy().view(np.int8), qo)
+        for B in (1, 4):
+            x = synth.activations(B, cols, 40 + i)
+            y = tq.tq_fused_gemv(m, x.cuda()).cpu().numpy().astype(np.float64)
+            yref = oracle.layer_forward(qo, so, x.double().numpy())
+            err = np.max(np.abs(y[:, sample] - yref), axis=1) / np.max(np.abs(yref), axis=1)
+            assert float(err.max()) <= TOL
+        assert tq.tq_device_status(m) == 0

@@ -1,0 +1,186 @@
+"""Host half of libtq against the oracle: quantizers, table, encoder, stream validation.  No GPU."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from inputs import synth
+from oracle import oracle
+from paper_2509_22951_b200 import binding as tq
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "tq.h")).read()
+    declared = set(re.findall(r"\b(tq_[a-z0-9_]+)\s*\(", hdr))
+    assert declared, "no declarations found"
+    lib = ctypes.CDLL(str(tq._build.LIB))
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} declared in tq.h but not exported"
+    assert declared == set(tq.EXPORTS)
+
+
+def test_quantize_rows_matches_oracle_bit_exact():
+    w = synth.weight(96, 512, synth.matrix_seed(3)).numpy()
+    w[5] = 0
+    q, s = tq.tq_quantize_rows(w)
+    qo, so = oracle.quantize_rows(w)
+    assert np.array_equal(q, qo) and np.array_equal(s, so)
+
+
+def test_quantize_tensor_matches_oracle_bit_exact():
+    x = synth.weight(64, 256, synth.matrix_seed(4)).numpy()
+    q, s, z = tq.tq_quantize_tensor(x)
+    qo, so, zo = oracle.quantize_paper(x)
+    assert np.array_equal(q, qo) and s == so and z == zo
+    with pytest.raises(tq.TqError):
+        tq.tq_quantize_tensor(np.zeros(16, dtype=np.float32))
+
+
+def _check_same(mats, top_k):
+    d = tq.tq_build_dictionary(mats, top_k)
+    o = oracle.Dictionary.build(mats, top_k)
+    assert d.K == o.K
+    assert np.array_equal(d.entries, o.entries)
+    assert np.array_equal(d.counts, o.counts)
+    for m in mats:
+        s, h, mi = tq.tq_encode(d, m)
+        so, ho, mo = o.encode(m)
+        assert (h, mi) == (ho, mo) and np.array_equal(s, so)
+        assert np.array_equal(o.decode(s), np.ascontiguousarray(m).view(np.uint8).ravel())
+    return d, o
+
+
+@pytest.mark.parametrize("seed", range(8))
+@pytest.mark.parametrize("threads", [1, 3])
+def test_dictionary_and_stream_identical_small_alphabets(seed, threads):
+    tq.tq_set_num_threads(threads)
+    try:
+        rng = np.random.default_rng(seed)
+        a = int(rng.integers(1, 9))
+        mats = [rng.integers(0, a + 1, size=int(rng.integers(0, 5000))).astype(np.uint8)
+                for _ in range(int(rng.integers(1, 5)))]
+        for top_k in (65535, 50, 3, 0):
+            _check_same(mats, top_k)
+    finally:
+        tq.tq_set_num_threads(0)
+
+
+def test_dictionary_many_ties_at_the_cut():
+    # ~all windows distinct: the cut falls inside a huge class of count-1 windows, so the table is
+    # the first 65534 windows in visiting order
+    rng = np.random.default_rng(1)
+    data = rng.integers(0, 256, size=300_000).astype(np.uint8)
+    d, o = _check_same([data], 65535)
+    assert d.K == 65534
+
+
+def test_dictionary_tie_walk_path(monkeypatch):
+    # force the in-order walk that picks first-seen windows out of a large tied class
+    monkeypatch.setenv("TQ_TIE_LIMIT", "10")
+    rng = np.random.default_rng(2)
+    mats = [rng.integers(0, 4, size=3000).astype(np.uint8), rng.integers(0, 7, size=2000).astype(np.uint8)]
+    for top_k in (65535, 400, 120, 30, 5, 1):
+        _check_same(mats, top_k)
+
+
+def test_dictionary_multithreaded_large_matches_oracle():
+    # config-0 sized layer, quantized weights, several threads and buckets
+    w = synth.weight(1024, 2048, synth.matrix_seed(0)).numpy()
+    q, s = oracle.quantize_rows(w)
+    w2 = synth.weight(512, 2048, synth.matrix_seed(1)).numpy()
+    q2, s2 = oracle.quantize_rows(w2)
+    tq.tq_set_num_threads(4)
+    try:
+        _check_same([q, q2], 65535)
+    finally:
+        tq.tq_set_num_threads(0)
+
+
+def test_encode_tails_and_buffer_check():
+    d = tq.tq_dict_from_entries(np.array([[1, 2, 3, 4]], dtype=np.uint8))
+    o = oracle.Dictionary.from_entries(np.array([[1, 2, 3, 4]], dtype=np.uint8))
+    for n in range(0, 14):
+        data = np.array(([1, 2, 3, 4, 9, 8, 7, 6] * 2)[:n], dtype=np.uint8)
+        s, h, m = tq.tq_encode(d, data)
+        so, _, _ = o.encode(data)
+        assert np.array_equal(s, so)
+    data = np.arange(8, dtype=np.uint8)
+    n = ctypes.c_uint64()
+    out = np.zeros(3, dtype=np.uint16)
+    rc = tq._lib.tq_encode(d._h, tq._np_ptr(data, ctypes.c_uint8), 8, tq._np_ptr(out, ctypes.c_uint16), 3,
+                           ctypes.byref(n), None, None)
+    assert rc == tq.TQ_ERR_BUFFER_TOO_SMALL and n.value == 10
+
+
+# ------------------------------------------------------------------ stream validation (host part of tq_upload)
+def _valid_stream(rows=6, cols=16, seed=0):
+    rng = np.random.default_rng(seed)
+    q = rng.integers(0, 3, size=(rows, cols)).astype(np.uint8)
+    o = oracle.Dictionary.build([q], top_k=5)
+    s, h, m = o.encode(q)
+    assert h > 0 and m > 0
+    return s, rows, cols
+
+
+def test_upload_size_accepts_valid_and_rejects_corrupt():
+    s, rows, cols = _valid_stream()
+    assert tq.tq_upload_size(s, rows, cols) > 0
+
+    def bad(stream, r=rows, c=cols):
+        with pytest.raises(tq.TqError) as e:
+            tq.tq_upload_size(stream, r, c)
+        return e.value.status
+
+    assert bad(s[:-1]) == tq.TQ_ERR_CORRUPT_STREAM               # truncated
+    assert bad(np.append(s, 1).astype(np.uint16)) == tq.TQ_ERR_CORRUPT_STREAM  # one group too many
+    esc = int(np.flatnonzero(s == 0xFFFF)[0])
+    t = s.copy(); t[esc + 2] = 300                                 # raw slot > 255
+    assert bad(t) == tq.TQ_ERR_CORRUPT_STREAM
+    t = s.copy(); t[esc + 1] = 0xFFFF                              # marker inside raw run
+    assert bad(t) == tq.TQ_ERR_CORRUPT_STREAM
+    code = int(np.flatnonzero((s != 0xFFFF) & (s > 0) & (np.arange(s.size) > 4))[0])
+    t = s.copy()
+    if not any(t[max(0, code - 4):code] == 0xFFFF):
+        t[code] = 0                                                # code 0 is never assigned
+        assert bad(t) == tq.TQ_ERR_CORRUPT_STREAM
+    assert bad(s, rows, cols + 2) == tq.TQ_ERR_UNSUPPORTED_SHAPE   # cols % 4 != 0
+    assert bad(s, rows + 1, cols) == tq.TQ_ERR_CORRUPT_STREAM      # wrong shape for this stream
+    t = np.concatenate([s[:-5], [0xFFFF, 1, 2, 3]]).astype(np.uint16) if s[-5] == 0xFFFF else None
+    if t is not None:
+        assert bad(t) == tq.TQ_ERR_CORRUPT_STREAM                  # marker with < 4 slots after it
+
+
+def test_row_partition_helper_two_ranks_gloo():
+    """Row sharding for several GPUs is a plain split of the rows: check with 2 gloo ranks that the
+    shards tile the matrix and that concatenating per-rank oracle outputs gives the full output."""
+    import torch.multiprocessing as mp
+    mp.spawn(_rank_main, args=(2,), nprocs=2, join=True)
+
+
+def _rank_main(rank, world):
+    import torch
+    import torch.distributed as dist
+    from paper_2509_22951_b200 import sharding
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29531")
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        rows, cols = 37, 16
+        rng = np.random.default_rng(7)
+        q = rng.integers(-127, 128, size=(rows, cols)).astype(np.int8)
+        s = (rng.random(rows) + 0.5).astype(np.float32)
+        x = rng.standard_normal((2, cols))
+        r0, r1 = sharding.row_range(rows, rank, world)
+        y_local = torch.from_numpy(oracle.layer_forward(q[r0:r1], s[r0:r1], x))
+        parts = sharding.all_gather_rows(y_local, rows, rank, world)
+        full = torch.from_numpy(oracle.layer_forward(q, s, x))
+        assert torch.equal(parts, full)
+        # shards tile [0, rows)
+        cover = sorted(sharding.row_range(rows, r, world) for r in range(world))
+        assert cover[0][0] == 0 and cover[-1][1] == rows and all(a[1] == b[0] for a, b in zip(cover, cover[1:]))
+    finally:
+        dist.destroy_process_group()
