@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the fused dictionary-decode + GEMV path (one JSON line on stdout).
+
+A step is one pass over every linear layer of one LLaMA-3.2-3B decode step at batch 1 (197 fused
+decode+GEMV launches, replayed as one CUDA graph).  Weights are seeded synthetic Student-t values,
+quantized per row to int8 on the GPU, dictionary-coded with one table for the whole model by the
+host library, and resident in HBM before the timed region starts.  `value` is the effective
+bandwidth on algorithmic bytes (token stream + per-row index and scales + x + y) per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--model 3b|1b] [--batch B] [--layers L]
+  python bench.py --impl reference ...     # the CPU oracle on a bounded sample of the workload
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from inputs import synth  # noqa: E402
+
+METRIC = "fused_decode_gemv_effective_bandwidth"
+UNIT = "GB/s"
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            j = json.load(f)
+        return float(j["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines: list[str] = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_model(tq, shapes, batch, device, threads=0, table_entries=None):
+    """Generate, quantize (GPU), build the table and encode (host), upload.  Returns
+    (matrices, xs, ys, table, stats)."""
+    t0 = time.time()
+    if threads:
+        tq.tq_set_num_threads(threads)
+    q_host, scales = [], []
+    for i, (name, rows, cols) in enumerate(shapes):
+        w = synth.weight(rows, cols, synth.matrix_seed(i), device=device)
+        q, s = tq.tq_quantize_rows_device(w)
+        q_host.append(q.cpu().numpy())
+        scales.append(s.cpu().numpy())
+        del w, q, s
+    t1 = time.time()
+    hd = tq.tq_build_dictionary(q_host) if table_entries is None else tq.tq_dict_from_entries(table_entries)
+    t2 = time.time()
+    dd = tq.tq_dict_upload(hd, device=device)
+    mats = []
+    for i, (name, rows, cols) in enumerate(shapes):
+        stream, h, m = tq.tq_encode(hd, q_host[i])
+        mats.append(tq.tq_upload(dd, stream, rows, cols, scales[i]))
+        del stream
+    t3 = time.time()
+    xs = [synth.activations(batch, cols, 7000 + i, device=device) for i, (_, rows, cols) in enumerate(shapes)]
+    ys = [torch.empty((batch, rows), dtype=torch.float32, device=device) for (_, rows, cols) in shapes]
+    stats = {"gen_quant_s": t1 - t0, "table_s": t2 - t1, "encode_upload_s": t3 - t2, "K": hd.K}
+    return mats, xs, ys, hd, q_host, scales, stats
+
+
+def algorithmic_bytes(info, batch):
+    return (info.stream_bytes + info.rows * (8 + 4) + 2 * batch * info.cols + 4 * batch * info.rows)
+
+
+def oracle_sample_run(hd_entries, q_host, scales, shapes, batch, sample_idx, reps=1):
+    """The CPU oracle on a bounded sample: Listing 4 decode + fp64 layer product per matrix.
+    Streams are produced beforehand by the oracle's own encoder (untimed).  Returns
+    (algorithmic bytes of the sample, [seconds per repetition])."""
+    from oracle import oracle
+    od = oracle.Dictionary.from_entries(hd_entries)
+    times = [0.0] * reps
+    total = 0
+    for i in sample_idx:
+        name, rows, cols = shapes[i]
+        stream, h, m = od.encode(q_host[i])
+        x = synth.activations(batch, cols, 7000 + i).double().numpy()
+        total += 2 * (h + 5 * m) + rows * 12 + 2 * batch * cols + 4 * batch * rows
+        for r in range(reps):
+            t0 = time.perf_counter()
+            codes = od.decode(stream, rows * cols).reshape(rows, cols).view(np.int8)
+            oracle.layer_forward(codes, scales[i], x)
+            times[r] += time.perf_counter() - t0
+        del stream
+    return total, times
+
+
+def pick_sample(shapes, max_weights):
+    idx, tot = [], 0
+    for i, (_, r, c) in enumerate(shapes):
+        if tot + r * c > max_weights and idx:
+            break
+        idx.append(i)
+        tot += r * c
+    return idx
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="tq", choices=["tq", "reference"])
+    ap.add_argument("--model", default="3b", choices=["1b", "3b"])
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--layers", type=int, default=None, help="decoder layers to build (default: all)")
+    ap.add_argument("--no-lm-head", action="store_true")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    shapes = synth.llama32_linear_shapes(args.model, args.layers, lm_head=not args.no_lm_head)
+    workload = f"llama3.2-{args.model} linear stack ({len(shapes)} matrices), batch {args.batch}"
+    n_weights = sum(r * c for _, r, c in shapes)
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        run_reference(args, shapes, workload)
+        return
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2509_22951_b200 import binding as tq
+
+    ncores = os.cpu_count() or 1
+    threads = max(1, ncores // world)
+    table_entries = None
+    if world > 1:
+        # the table is a property of the model: rank 0 builds it, the others receive the entries
+        import torch.distributed as dist
+        if rank == 0:
+            q0 = []
+            for i, (name, rows, cols) in enumerate(shapes):
+                w = synth.weight(rows, cols, synth.matrix_seed(i), device=device)
+                q0.append(tq.tq_quantize_rows_device(w)[0].cpu().numpy())
+            ent = torch.from_numpy(tq.tq_build_dictionary(q0).entries).to(device)
+            del q0
+            meta = torch.tensor([ent.shape[0]], device=device)
+        else:
+            meta = torch.zeros(1, dtype=torch.int64, device=device)
+        dist.broadcast(meta, 0)
+        if rank != 0:
+            ent = torch.empty((int(meta.item()), 4), dtype=torch.uint8, device=device)
+        dist.broadcast(ent, 0)
+        table_entries = ent.cpu().numpy()
+
+    mats, xs, ys, hd, q_host, scales, stats = build_model(tq, shapes, args.batch, device, threads, table_entries)
+    infos = [m.info for m in mats]
+    hits = sum(i.n_hits for i in infos)
+    miss = sum(i.n_miss for i in infos)
+    alg_bytes = sum(algorithmic_bytes(i, args.batch) for i in infos)
+    stream_bytes = sum(i.stream_bytes for i in infos)
+    payload_bytes = sum(i.payload_bytes for i in infos)
+    log(f"[rank {rank}] built {len(mats)} matrices, {n_weights/1e9:.3f} G weights, hit rate {hits/(hits+miss):.4f}, "
+        f"stream {stream_bytes/1e9:.3f} GB, setup {stats}")
+
+    stream = torch.cuda.Stream(device)
+    launches_per_step = len(mats) * ((args.batch + 3) // 4)
+
+    def step_plain():
+        for m, x, y in zip(mats, xs, ys):
+            tq.tq_fused_gemv(m, x, y)
+
+    with torch.cuda.stream(stream):
+        step_plain()  # sets kernel attributes before any capture
+        stream.synchronize()
+        graph = None
+        if not args.no_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                step_plain()
+        run_step = graph.replay if graph is not None else step_plain
+
+        for _ in range(max(args.warmup, 3)):
+            run_step()
+        stream.synchronize()
+
+        def barrier():
+            if world > 1:
+                import torch.distributed as dist
+                dist.barrier()
+
+        sampler = ClockSampler(local_rank)
+        barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for _ in range(args.steps):
+            run_step()
+        ev1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        barrier()
+        clocks = sampler.stop()
+        ms_total = ev0.elapsed_time(ev1)
+
+        status = 0
+        for m in mats:
+            status |= tq.tq_device_status(m)
+        assert status == 0, f"device status {status}"
+
+        # ---- end to end through the host-buffer call: H2D of x and D2H of y every step ----
+        e2e = None
+        if not args.no_e2e:
+            hx = [x.cpu().pin_memory() for x in xs]
+            hy = [torch.empty(y.shape, dtype=torch.float32).pin_memory() for y in ys]
+            e_steps = max(3, min(args.steps, 10))
+
+            def step_e2e():
+                for m, a, b, dx, dy in zip(mats, hx, hy, xs, ys):
+                    tq.tq_fused_gemv_host(m, a, b, dx, dy)
+
+            for _ in range(3):
+                step_e2e()
+            stream.synchronize()
+            barrier()
+            t0 = time.perf_counter()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(e_steps):
+                step_e2e()
+                stream.synchronize()  # the step's result is on the host
+            e1.record(stream)
+            stream.synchronize()
+            wall = time.perf_counter() - t0
+            e2e_ms = max(e0.elapsed_time(e1), wall * 1e3) / e_steps
+            e2e = {"ms_per_step": e2e_ms, "steps": e_steps,
+                   "h2d": sum(2 * args.batch * i.cols for i in infos),
+                   "d2h": sum(4 * args.batch * i.rows for i in infos)}
+
+    ms_step = ms_total / args.steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_step, e2e["ms_per_step"] if e2e else 0.0], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t[0].item())
+        if e2e:
+            e2e["ms_per_step"] = float(t[1].item())
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peaks()
+    value = world * alg_bytes / (ms_step * 1e-3) / 1e9
+    per_gpu = alg_bytes / (ms_step * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8 weights x bf16 activations, fp32 accumulate",
+        "data": "synthetic",
+        "config": {"workload": workload, "n_weights": n_weights, "hit_rate": hits / (hits + miss), "K": stats["K"],
+                   "layout": "paper token stream, per-row segments", "cuda_graph": graph is not None,
+                   "l2": "inputs larger than L2: each step streams %.2f GB" % (payload_bytes / 1e9),
+                   "multi_gpu": "independent replicas, no data-path collective" if world > 1 else "single GPU"},
+        "us_per_token": ms_step * 1e3 / args.batch,
+        "bytes_per_step": {"algorithmic": alg_bytes, "paper_stream": stream_bytes, "device_payload": payload_bytes,
+                           "int8_equivalent": n_weights},
+        "pct_of_8TBs_nominal": 100.0 * per_gpu / 8000.0,
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
+                     "traffic": None, "kernel": "gemv_kernel", "peak_source": peak_src,
+                     "note": "achieved = algorithmic bytes of the %d launches of a step / step time (launch gaps included)" % launches_per_step},
+        "setup_s": stats,
+    }
+    if e2e:
+        out["e2e"] = {"value": world * alg_bytes / (e2e["ms_per_step"] * 1e-3) / 1e9, "unit": UNIT,
+                      "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                      "ms_per_step": e2e["ms_per_step"], "steps": e2e["steps"]}
+
+    if not args.no_cpu_baseline:
+        sample = pick_sample(shapes, 3_300_000_000)  # ~13 s of single-thread oracle work for the 3B stack
+        total, times = oracle_sample_run(hd.entries, q_host, scales, shapes, args.batch, sample, reps=1)
+        best = min(times)
+        out["cpu_baseline"] = {"value": total / best / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                               "sample": f"first {len(sample)} matrices of the workload "
+                                         f"({sum(shapes[i][1]*shapes[i][2] for i in sample)/1e6:.1f} M weights), "
+                                         f"Listing-4 decode + fp64 product, one pass, {best:.2f} s",
+                               "host_cores_available": ncores}
+    print(json.dumps(out), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_reference(args, shapes, workload):
+    """The oracle as it stands on the host cores: each step = one bounded sample of the workload."""
+    from oracle import oracle
+    t0 = time.time()
+    sample = pick_sample(shapes, 60_000_000)
+    q_host, scales = {}, {}
+    for i in sample:
+        name, rows, cols = shapes[i]
+        w = synth.weight(rows, cols, synth.matrix_seed(i)).numpy()
+        q_host[i], scales[i] = oracle.quantize_rows(w)
+    od = oracle.Dictionary.build([q_host[i] for i in sample])  # the oracle's own table over the sample
+    log(f"reference setup {time.time()-t0:.1f} s, sample {sample}")
+    total, times = oracle_sample_run(od.entries, q_host, scales, shapes, args.batch, sample,
+                                     reps=max(args.warmup, 1) + args.steps)
+    times = times[max(args.warmup, 1):]
+    ms = 1e3 * sum(times) / len(times)
+    v = total / (ms * 1e-3) / 1e9
+    nw = sum(shapes[i][1] * shapes[i][2] for i in sample)
+    desc = f"first {len(sample)} matrices of the workload ({nw/1e6:.1f} M weights) per step, table built over the sample"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": max(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8 weights x bf16 activations, fp64 accumulate", "data": "synthetic",
+        "config": {"workload": workload, "sample": desc},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -47,6 +47,10 @@ typedef struct tq_dmat tq_dmat;   /* handle of one compressed matrix resident in
 /* Human-readable text for a status code (static storage). */
 const char* tq_strerror(int status);
 
+/* Text of the calling thread's most recent CUDA failure behind a TQ_ERR_CUDA (static storage,
+ * empty if none). */
+const char* tq_last_cuda_error(void);
+
 /* Worker threads used by the host calls below (0 = hardware concurrency).  Returns the value in
  * effect. */
 int tq_set_num_threads(int n);

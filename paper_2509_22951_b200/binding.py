@@ -28,7 +28,7 @@ TQ_STATUS_BAD_ROW = 2
 TQ_STATUS_WAIT_EXPIRED = 4
 
 EXPORTS = [
-    "tq_strerror", "tq_set_num_threads", "tq_quantize_tensor", "tq_quantize_rows",
+    "tq_strerror", "tq_last_cuda_error", "tq_set_num_threads", "tq_quantize_tensor", "tq_quantize_rows",
     "tq_quantize_rows_device", "tq_build_dictionary", "tq_dict_from_entries", "tq_dict_entries",
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
@@ -39,7 +39,8 @@ EXPORTS = [
 class TqError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: {_lib.tq_strerror(status).decode()} ({status})")
+        detail = _lib.tq_last_cuda_error().decode() if status == TQ_ERR_CUDA else ""
+        super().__init__(f"{where}: {_lib.tq_strerror(status).decode()} ({status}) {detail}")
 
 
 class _Info(C.Structure):
@@ -56,6 +57,7 @@ def _load() -> C.CDLL:
     f32p = C.POINTER(C.c_float)
     sig = {
         "tq_strerror": (C.c_char_p, [C.c_int]),
+        "tq_last_cuda_error": (C.c_char_p, []),
         "tq_set_num_threads": (C.c_int, [C.c_int]),
         "tq_quantize_tensor": (C.c_int, [f32p, C.c_uint64, u8p, f32p, f32p]),
         "tq_quantize_rows": (C.c_int, [f32p, C.c_uint32, C.c_uint32, C.POINTER(C.c_int8), f32p]),

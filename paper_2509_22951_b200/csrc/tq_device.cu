@@ -258,7 +258,14 @@ int sm_count() {
   return n;
 }
 
-inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? TQ_OK : TQ_ERR_CUDA; }
+thread_local char g_cuda_msg[256] = "";
+
+// Records the text of a CUDA failure for tq_last_cuda_error and maps it to TQ_ERR_CUDA.
+inline int cuda_ok(cudaError_t e, const char* what = "") {
+  if (e == cudaSuccess) return TQ_OK;
+  snprintf(g_cuda_msg, sizeof(g_cuda_msg), "%s: %s (%s)", what, cudaGetErrorString(e), cudaGetErrorName(e));
+  return TQ_ERR_CUDA;
+}
 
 template <int NB>
 int launch_gemv(const tq_dmat* m, const __nv_bfloat16* x, float* y, cudaStream_t st) {
@@ -266,25 +273,33 @@ int launch_gemv(const tq_dmat* m, const __nv_bfloat16* x, float* y, cudaStream_t
   const size_t smem = (size_t)NB * cols * sizeof(float);
   static size_t configured = 0;
   if (smem > 48 * 1024 && smem > configured) {
-    if (cudaFuncSetAttribute(gemv_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return TQ_ERR_CUDA;
+    if (int rc = cuda_ok(cudaFuncSetAttribute(gemv_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+                         "gemv: raising the dynamic shared memory limit"))
+      return rc;
     configured = smem;
   }
   int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gemv_kernel<NB>, kThreads, smem) != cudaSuccess || per_sm < 1)
+  if (int rc = cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gemv_kernel<NB>, kThreads, smem),
+                       "gemv: occupancy query"))
+    return rc;
+  if (per_sm < 1) {
+    snprintf(g_cuda_msg, sizeof(g_cuda_msg), "gemv: %zu bytes of shared memory do not fit one CTA", smem);
     return TQ_ERR_CUDA;
+  }
   const uint32_t need = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
   const uint32_t grid = std::min<uint32_t>(need, (uint32_t)(sm_count() * per_sm));
   gemv_kernel<NB><<<grid, kThreads, smem, st>>>(
       reinterpret_cast<const uint4*>(m->d_tokens), m->d_rowseg, m->d_scale, m->d_zero, m->has_zero,
       m->dict->d_entries, m->dict->K, rows, cols, x, y, m->info.levels_signed ? 0x80808080u : 0u,
       m->info.levels_signed ? 8388736.0f : 8388608.0f, m->d_status);
-  return cuda_ok(cudaGetLastError());
+  return cuda_ok(cudaGetLastError(), "gemv launch");
 }
 
 }  // namespace
 
 extern "C" {
+
+const char* tq_last_cuda_error(void) { return g_cuda_msg; }
 
 int tq_quantize_rows_device(const float* d_w, uint32_t rows, uint32_t cols, int8_t* d_q, float* d_scale,
                             void* cuda_stream) {
@@ -393,8 +408,7 @@ int tq_fused_gemv(const tq_dmat* m, const void* d_x_bf16, int B, float* d_y, voi
   const int max_nb = (size_t)4 * cols * 4 <= 200 * 1024 ? 4 : ((size_t)2 * cols * 4 <= 200 * 1024 ? 2 : 1);
   if ((size_t)cols * 4 > 200 * 1024) return TQ_ERR_UNSUPPORTED_SHAPE;
   for (int b0 = 0; b0 < B;) {
-    int nb = std::min(B - b0, max_nb);
-    if (nb == 3 && ((uintptr_t)(x + (size_t)(b0 + 3) * cols) & 15)) nb = 2;
+    const int nb = std::min(B - b0, max_nb);
     int rc;
     const __nv_bfloat16* xb = x + (size_t)b0 * cols;
     float* yb = d_y + (size_t)b0 * rows;
