@@ -70,9 +70,14 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
 
-    def stop(self):
+    def wait_first(self, timeout=5.0):
+        t0 = time.time()
+        while not self.lines and time.time() - t0 < timeout and self.proc is not None:
+            time.sleep(0.02)
+
+    def stop(self, t_start=0.0, t_end=float("inf")):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -81,7 +86,9 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
-        for ln in self.lines:
+        for ts, ln in self.lines:
+            if ts < t_start or ts > t_end:
+                continue
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 8:
                 continue
@@ -164,7 +171,7 @@ def pick_sample(shapes, max_weights):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="tq", choices=["tq", "reference"])
     ap.add_argument("--model", default="3b", choices=["1b", "3b"])
@@ -256,9 +263,11 @@ def main():
                 dist.barrier()
 
         sampler = ClockSampler(local_rank)
+        sampler.start()
+        sampler.wait_first()
         barrier()
         torch.cuda.synchronize()
-        sampler.start()
+        t_start = time.time()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record(stream)
         for _ in range(args.steps):
@@ -266,8 +275,17 @@ def main():
         ev1.record(stream)
         stream.synchronize()
         torch.cuda.synchronize()
+        t_end = time.time()
         barrier()
-        clocks = sampler.stop()
+        extended = False
+        if t_end - t_start < 0.6:  # too short for nvidia-smi's 100 ms period: keep the same load running, untimed
+            extended = True
+            while time.time() - t_start < 0.8:
+                run_step()
+                stream.synchronize()
+            t_end = time.time()
+        clocks = sampler.stop(t_start, t_end)
+        clocks["sampled_over"] = "timed region" if not extended else "timed region plus identical untimed steps"
         ms_total = ev0.elapsed_time(ev1)
 
         status = 0

@@ -146,7 +146,7 @@ class Dict:
         self._h = C.c_void_p(handle)
 
     def __del__(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:
             _lib.tq_dict_free(self._h)
             self._h = None
 
@@ -208,7 +208,7 @@ class DeviceDict:
         self.K = K
 
     def __del__(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:
             _lib.tq_ddict_free(self._h)
             self._h = None
 
@@ -249,7 +249,7 @@ class DeviceMatrix:
         self.info = MatInfo(*(getattr(i, f[0]) for f in _Info._fields_))
 
     def __del__(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:
             _lib.tq_dmat_free(self._h)
             self._h = None
 

@@ -37,21 +37,29 @@ __device__ __forceinline__ uint32_t esc_bits(uint32_t a) {
   return ~(a + 0x00010001u) & a & 0x80008000u;
 }
 
-// Walks one row segment.  emit(group_index, packed4bytes) is called once per completed group by
-// the lane that completed it.  Returns the number of groups seen (warp-uniform).
-template <class Emit>
+constexpr uint32_t kRing = 512;  // per-warp ring of decoded groups (uint32 each); > 256 + 31
+
+// Walks one row segment.  Each tile is handled in two phases.  Phase 1: every lane turns the
+// groups completed inside its 8 slots into packed 4-byte words (table loads are issued together,
+// before any use) and stores them, in row order, into the warp's ring in shared memory.  Phase 2:
+// the ring is drained 32 groups at a time, lane i taking group done+i, so the consumer sees
+// consecutive groups on consecutive lanes (conflict-free x reads, coalesced stores).  Fewer than
+// 32 left-over groups wait for the next tile; the row end flushes them.
+// consume(group_index, packed4bytes) is called once per group.  Returns the groups seen.
+template <class Consume>
 __device__ __forceinline__ uint32_t decode_row(const uint4* __restrict__ tok, uint32_t n_slots,
                                                const uint32_t* __restrict__ table, uint32_t K,
-                                               uint32_t groups_per_row, uint32_t& status_bits,
-                                               Emit&& emit) {
+                                               uint32_t groups_per_row, uint32_t* __restrict__ ring,
+                                               uint32_t& status_bits, Consume&& consume) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t n_chunks = (n_slots + 7u) >> 3;
   const uint32_t n_tiles = (n_chunks + 31u) >> 5;
+  const uint32_t kmax = K ? K - 1u : 0u;
   const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
 
   uint4 cur = lane < n_chunks ? ldg_stream(tok + lane) : zero4;
   uint4 nxt = lane + 32u < n_chunks ? ldg_stream(tok + lane + 32u) : zero4;
-  uint32_t base = 0, carryE = 0, carryZ = 0, carryW = 0;
+  uint32_t base = 0, done = 0, carryE = 0, carryZ = 0, carryW = 0, bad = 0;
 
   for (uint32_t t = 0; t < n_tiles; ++t) {
     const uint32_t pf = (t + 2u) * 32u + lane;
@@ -69,9 +77,10 @@ __device__ __forceinline__ uint32_t decode_row(const uint4* __restrict__ tok, ui
     uint32_t pw = __shfl_up_sync(kFull, cur.w, 1);
     if (lane == 0) { prevE = carryE; pz = carryZ; pw = carryW; }
 
-    const uint32_t X = (prevE >> 4) | (E << 4);                    // markers over the 12-slot window
+    const uint32_t X = (prevE >> 4) | (E << 4);                       // markers over the 12-slot window
     const uint32_t R = (X | (X >> 1) | (X >> 2) | (X >> 3)) & 0xFFu;  // own slots that are raw
-    const uint32_t C = ((~R & ~E) | X) & V;                        // own slots that complete a group
+    const uint32_t CODE = ~R & ~E & V;                                // own slots holding a code
+    const uint32_t C = (CODE | X) & V;                                // own slots completing a group
 
     const uint32_t n = __popc(C);
     uint32_t incl = n;
@@ -86,52 +95,76 @@ __device__ __forceinline__ uint32_t decode_row(const uint4* __restrict__ tok, ui
     carryZ = __shfl_sync(kFull, cur.z, 31);
     carryW = __shfl_sync(kFull, cur.w, 31);
 
+    // ---- phase 1: words of the completed groups ----
     const uint32_t W[6] = {pz, pw, cur.x, cur.y, cur.z, cur.w};
+    uint32_t w[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const uint32_t reg = W[2 + (j >> 1)];
+      const uint32_t idx = ((j & 1) ? (reg >> 16) : (reg & 0xFFFFu)) - 1u;
+      const uint32_t cl = min(idx, kmax);
+      uint32_t v = 0u;
+      if (CODE & (1u << j)) {
+        v = __ldg(table + cl);
+        bad |= idx ^ cl;
+      }
+      w[j] = v;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (X & (1u << j)) {  // 4th raw slot after a marker at window slot j: low bytes of slots j+1..j+4
+        if (j & 1) {
+          w[j] = __byte_perm(W[(j + 1) >> 1], W[((j + 1) >> 1) + 1], 0x6420);
+        } else {
+          const uint32_t t3 = __byte_perm(W[j >> 1], W[(j >> 1) + 1], 0x0642);
+          w[j] = __byte_perm(t3, W[(j >> 1) + 2], 0x4210);
+        }
+      }
+    }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       if (C & (1u << j)) {
-        uint32_t w;
-        if (X & (1u << j)) {  // 4th raw slot of a marker at window slot j: bytes of slots j+1..j+4
-          if (j & 1) {
-            w = __byte_perm(W[(j + 1) >> 1], W[((j + 1) >> 1) + 1], 0x6420);
-          } else {
-            const uint32_t t3 = __byte_perm(W[j >> 1], W[(j >> 1) + 1], 0x0642);
-            w = __byte_perm(t3, W[(j >> 1) + 2], 0x4210);
-          }
-        } else {
-          const uint32_t reg = W[2 + (j >> 1)];
-          const uint32_t code = (j & 1) ? (reg >> 16) : (reg & 0xFFFFu);
-          if (code - 1u < K) {
-            w = __ldg(table + (code - 1u));
-          } else {
-            w = 0u;
-            status_bits |= TQ_STATUS_BAD_CODE;
-          }
-        }
-        if (g < groups_per_row) emit(g, w);
+        ring[g & (kRing - 1u)] = w[j];
         ++g;
       }
+    }
+    __syncwarp();
+
+    // ---- phase 2: drain full batches of 32 groups ----
+    const uint32_t lim = min(base, groups_per_row);
+    while (done + 32u <= lim) {
+      const uint32_t grp = done + lane;
+      consume(grp, ring[grp & (kRing - 1u)]);
+      done += 32u;
     }
     cur = nxt;
     nxt = nn;
   }
+  {
+    const uint32_t lim = min(base, groups_per_row);
+    const uint32_t grp = done + lane;
+    if (grp < lim) consume(grp, ring[grp & (kRing - 1u)]);
+  }
+  __syncwarp();  // the ring is reused by this warp's next row
+  if (bad) status_bits |= TQ_STATUS_BAD_CODE;
   return base;
 }
 
 // ---------------------------------------------------------------------------------------------
 // tq_decompress: expand to bytes in HBM.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 decompress_kernel(const uint4* __restrict__ tokens, const tq_rowseg* __restrict__ rowseg,
                   const uint32_t* __restrict__ table, uint32_t K, uint32_t rows, uint32_t cols,
                   uint32_t* __restrict__ out, uint32_t* __restrict__ status) {
+  __shared__ uint32_t rings[kWarpsPerCta][kRing];
   const uint32_t warp = threadIdx.x >> 5;
   const uint32_t gpr = cols >> 2;
   uint32_t bits = 0;
   for (uint32_t row = blockIdx.x * kWarpsPerCta + warp; row < rows; row += gridDim.x * kWarpsPerCta) {
     const tq_rowseg seg = rowseg[row];
     uint32_t* orow = out + (size_t)row * gpr;
-    const uint32_t seen = decode_row(tokens + seg.chunk_off, seg.n_slots, table, K, gpr, bits,
+    const uint32_t seen = decode_row(tokens + seg.chunk_off, seg.n_slots, table, K, gpr, rings[warp], bits,
                                      [&](uint32_t g, uint32_t w) { orow[g] = w; });
     if (seen != gpr) bits |= TQ_STATUS_BAD_ROW;
   }
@@ -146,13 +179,14 @@ decompress_kernel(const uint4* __restrict__ tokens, const tq_rowseg* __restrict_
 // b' = b and 2^23 the unsigned one.
 // ---------------------------------------------------------------------------------------------
 template <int NB>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 gemv_kernel(const uint4* __restrict__ tokens, const tq_rowseg* __restrict__ rowseg,
             const float* __restrict__ scale, const float* __restrict__ zero, int has_zero,
             const uint32_t* __restrict__ table, uint32_t K, uint32_t rows, uint32_t cols,
             const __nv_bfloat16* __restrict__ x, float* __restrict__ y, uint32_t xor_mask,
             float magic, uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) float xs[];  // [NB][cols]
+  __shared__ uint32_t rings[kWarpsPerCta][kRing];
   __shared__ float sumx[NB];
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
   const uint32_t gpr = cols >> 2;
@@ -181,7 +215,7 @@ gemv_kernel(const uint4* __restrict__ tokens, const tq_rowseg* __restrict__ rows
 #pragma unroll
     for (int b = 0; b < NB; ++b) acc[b] = 0.f;
     const uint32_t seen = decode_row(
-        tokens + seg.chunk_off, seg.n_slots, table, K, gpr, bits, [&](uint32_t g, uint32_t w) {
+        tokens + seg.chunk_off, seg.n_slots, table, K, gpr, rings[warp], bits, [&](uint32_t g, uint32_t w) {
           w ^= xor_mask;
           const float f0 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7540)) - magic;
           const float f1 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7541)) - magic;
@@ -272,7 +306,7 @@ int launch_gemv(const tq_dmat* m, const __nv_bfloat16* x, float* y, cudaStream_t
   const uint32_t rows = m->info.rows, cols = m->info.cols;
   const size_t smem = (size_t)NB * cols * sizeof(float);
   static size_t configured = 0;
-  if (smem > 48 * 1024 && smem > configured) {
+  if (smem + 20 * 1024 > 48 * 1024 && smem > configured) {  // static shared memory counts too
     if (int rc = cuda_ok(cudaFuncSetAttribute(gemv_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
                          "gemv: raising the dynamic shared memory limit"))
       return rc;
