@@ -178,6 +178,7 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--layers", type=int, default=None, help="decoder layers to build (default: all)")
     ap.add_argument("--no-lm-head", action="store_true")
+    ap.add_argument("--shapes", default=None, help="custom workload, e.g. 32768x3072,3072x8192 (profiling cases)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -188,6 +189,9 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     shapes = synth.llama32_linear_shapes(args.model, args.layers, lm_head=not args.no_lm_head)
     workload = f"llama3.2-{args.model} linear stack ({len(shapes)} matrices), batch {args.batch}"
+    if args.shapes:
+        shapes = [(f"m{i}", int(t.split("x")[0]), int(t.split("x")[1])) for i, t in enumerate(args.shapes.split(","))]
+        workload = f"custom shapes {args.shapes}, batch {args.batch}"
     n_weights = sum(r * c for _, r, c in shapes)
 
     if args.impl == "reference":
