@@ -103,7 +103,7 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def build_model(tq, shapes, batch, device, threads=0, table_entries=None):
+def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout=1):
     """Generate, quantize (GPU), build the table and encode (host), upload.  Returns
     (matrices, xs, ys, table, stats)."""
     t0 = time.time()
@@ -123,7 +123,7 @@ def build_model(tq, shapes, batch, device, threads=0, table_entries=None):
     mats = []
     for i, (name, rows, cols) in enumerate(shapes):
         stream, h, m = tq.tq_encode(hd, q_host[i])
-        mats.append(tq.tq_upload(dd, stream, rows, cols, scales[i]))
+        mats.append(tq.tq_upload(dd, stream, rows, cols, scales[i], layout=layout))
         del stream
     t3 = time.time()
     xs = [synth.activations(batch, cols, 7000 + i, device=device) for i, (_, rows, cols) in enumerate(shapes)]
@@ -133,7 +133,13 @@ def build_model(tq, shapes, batch, device, threads=0, table_entries=None):
 
 
 def algorithmic_bytes(info, batch):
-    return (info.stream_bytes + info.rows * (8 + 4) + 2 * batch * info.cols + 4 * batch * info.rows)
+    """Bytes the method has to move for one call: the tokens of the layout in use, an 8-byte row
+    index, the row scale, x and y.  Padding is not counted."""
+    if info.layout == 0:   # paper stream: 2 bytes per code, 10 per escaped group
+        tokens = info.stream_bytes
+    else:                  # planes: one 2-byte token per group + one 4-byte word per escaped group
+        tokens = 2 * (info.n_hits + info.n_miss) + 4 * info.n_miss
+    return tokens + info.rows * (8 + 4) + 2 * batch * info.cols + 4 * batch * info.rows
 
 
 def oracle_sample_run(hd_entries, q_host, scales, shapes, batch, sample_idx, reps=1):
@@ -179,6 +185,7 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="decoder layers to build (default: all)")
     ap.add_argument("--no-lm-head", action="store_true")
     ap.add_argument("--shapes", default=None, help="custom workload, e.g. 32768x3072,3072x8192 (profiling cases)")
+    ap.add_argument("--layout", default="planes", choices=["stream", "planes"])
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -230,7 +237,7 @@ def main():
         dist.broadcast(ent, 0)
         table_entries = ent.cpu().numpy()
 
-    mats, xs, ys, hd, q_host, scales, stats = build_model(tq, shapes, args.batch, device, threads, table_entries)
+    mats, xs, ys, hd, q_host, scales, stats = build_model(tq, shapes, args.batch, device, threads, table_entries, layout=0 if args.layout == "stream" else 1)
     infos = [m.info for m in mats]
     hits = sum(i.n_hits for i in infos)
     miss = sum(i.n_miss for i in infos)
@@ -351,7 +358,7 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "int8 weights x bf16 activations, fp32 accumulate",
         "data": "synthetic",
         "config": {"workload": workload, "n_weights": n_weights, "hit_rate": hits / (hits + miss), "K": stats["K"],
-                   "layout": "paper token stream, per-row segments", "cuda_graph": graph is not None,
+                   "layout": "paper token stream, per-row segments" if args.layout == "stream" else "two planes: fixed-stride tokens + packed raw words", "cuda_graph": graph is not None,
                    "l2": "inputs larger than L2: each step streams %.2f GB" % (payload_bytes / 1e9),
                    "multi_gpu": "independent replicas, no data-path collective" if world > 1 else "single GPU"},
         "us_per_token": ms_step * 1e3 / args.batch,

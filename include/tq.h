@@ -117,6 +117,10 @@ void tq_ddict_free(tq_ddict* d); /* host handle only */
 
 /* Device layouts of a compressed matrix. */
 #define TQ_LAYOUT_STREAM 0 /* the paper's token stream, byte for byte, cut into per-row segments */
+#define TQ_LAYOUT_PLANES 1 /* the same tokens re-tiled without loss: one 16-bit token per group in a
+                              fixed-stride plane (code, or 0xFFFF), and the 4 bytes that followed each
+                              0xFFFF packed into one word of a second, compact plane.  2 + 4*miss_rate
+                              bytes per group instead of 2 + 8*miss_rate, and no sequential parse. */
 
 /* Bytes of DEVICE memory the layout of this stream needs.  stream: HOST.  Requires cols % 4 == 0
  * (no aligned group straddles two rows; true of every LLaMA shape), else TQ_ERR_UNSUPPORTED_SHAPE. */

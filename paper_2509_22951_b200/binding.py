@@ -23,6 +23,7 @@ TQ_ERR_CUDA = -5
 TQ_ERR_TIMEOUT = -6
 TQ_ERR_NOMEM = -7
 TQ_LAYOUT_STREAM = 0
+TQ_LAYOUT_PLANES = 1
 TQ_STATUS_BAD_CODE = 1
 TQ_STATUS_BAD_ROW = 2
 TQ_STATUS_WAIT_EXPIRED = 4

@@ -54,7 +54,6 @@ __device__ __forceinline__ uint32_t decode_row(const uint4* __restrict__ tok, ui
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t n_chunks = (n_slots + 7u) >> 3;
   const uint32_t n_tiles = (n_chunks + 31u) >> 5;
-  const uint32_t kmax = K ? K - 1u : 0u;
   const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
 
   uint4 cur = lane < n_chunks ? ldg_stream(tok + lane) : zero4;
@@ -101,12 +100,12 @@ __device__ __forceinline__ uint32_t decode_row(const uint4* __restrict__ tok, ui
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const uint32_t reg = W[2 + (j >> 1)];
-      const uint32_t idx = ((j & 1) ? (reg >> 16) : (reg & 0xFFFFu)) - 1u;
-      const uint32_t cl = min(idx, kmax);
+      const uint32_t idx = (j & 1) ? (reg >> 16) : (reg & 0xFFFFu);
+      const uint32_t cl = min(idx, K);
       uint32_t v = 0u;
       if (CODE & (1u << j)) {
-        v = __ldg(table + cl);
-        bad |= idx ^ cl;
+        v = __ldg(table + cl);  // word 0 of the table is zero
+        bad |= (idx ^ cl) | (idx == 0u);
       }
       w[j] = v;
     }
@@ -249,6 +248,177 @@ gemv_kernel(const uint4* __restrict__ tokens, const tq_rowseg* __restrict__ rows
 }
 
 // ---------------------------------------------------------------------------------------------
+// PLANES layout.  One warp owns one row and walks it in passes of 256 groups; lane L holds the 8
+// consecutive tokens of groups 8L..8L+7 of the pass (one 128-bit load).  A token is a code, the
+// marker 0xFFFF (its 4 bytes are the next word of the row's raw plane; the word's rank is the
+// number of markers before it, a warp prefix sum plus a popcount) or 0 (padding, decodes to zero
+// bytes through word 0 of the table).  All loads of a pass are issued before any use.
+// done(j, w) receives the packed bytes of the lane's j-th group, j = 0..7 (static).
+// ---------------------------------------------------------------------------------------------
+template <class Pass>
+__device__ __forceinline__ void planes_row(const uint4* __restrict__ codes, uint32_t gpr_pad,
+                                           const uint32_t* __restrict__ raw, const uint32_t* __restrict__ table,
+                                           uint32_t K, uint32_t& bad, Pass&& pass_done) {
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t n_vec = gpr_pad >> 3;           // 128-bit loads in the row
+  const uint32_t n_pass = (n_vec + 31u) >> 5;
+  const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+  uint4 cur = lane < n_vec ? ldg_stream(codes + lane) : zero4;
+  uint4 nxt = lane + 32u < n_vec ? ldg_stream(codes + lane + 32u) : zero4;
+  uint32_t rawcur = 0;
+  for (uint32_t p = 0; p < n_pass; ++p) {
+    const uint32_t pf = (p + 2u) * 32u + lane;
+    const uint4 nn = pf < n_vec ? ldg_stream(codes + pf) : zero4;
+    const uint32_t e = (esc_bits(cur.x) >> 15) | (esc_bits(cur.y) >> 13) | (esc_bits(cur.z) >> 11) |
+                       (esc_bits(cur.w) >> 9);
+    const uint32_t E = (e | (e >> 15)) & 0xFFu;
+    const uint32_t n = __popc(E);
+    uint32_t incl = n;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      uint32_t v = __shfl_up_sync(kFull, incl, d);
+      if (lane >= (uint32_t)d) incl += v;
+    }
+    const uint32_t* rp = raw + rawcur + (incl - n);
+    rawcur += __shfl_sync(kFull, incl, 31);
+    const uint32_t T[4] = {cur.x, cur.y, cur.z, cur.w};
+    uint32_t w[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const uint32_t tok = (j & 1) ? (T[j >> 1] >> 16) : (T[j >> 1] & 0xFFFFu);
+      if (E & (1u << j)) {
+        w[j] = __ldg(rp + __popc(E & ((1u << j) - 1u)));
+      } else {
+        const uint32_t cl = min(tok, K);
+        bad |= tok ^ cl;
+        w[j] = __ldg(table + cl);
+      }
+    }
+    pass_done(p, w);
+    cur = nxt;
+    nxt = nn;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+decompress_planes_kernel(const uint16_t* __restrict__ codes, uint32_t gpr_pad, const uint32_t* __restrict__ rawbase,
+                         const uint32_t* __restrict__ raw, const uint32_t* __restrict__ table, uint32_t K,
+                         uint32_t rows, uint32_t cols, uint32_t* __restrict__ out, uint32_t* __restrict__ status) {
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+  const uint32_t gpr = cols >> 2;
+  const bool vec_ok = (cols & 15u) == 0u;
+  uint32_t bad = 0;
+  for (uint32_t row = blockIdx.x * kWarpsPerCta + warp; row < rows; row += gridDim.x * kWarpsPerCta) {
+    uint32_t* orow = out + (size_t)row * gpr;
+    planes_row(reinterpret_cast<const uint4*>(codes + (size_t)row * gpr_pad), gpr_pad, raw + rawbase[row], table, K,
+               bad, [&](uint32_t p, const uint32_t (&w)[8]) {
+                 const uint32_t g0 = p * 256u + lane * 8u;
+                 if (vec_ok && g0 + 8u <= gpr) {
+                   uint4* o = reinterpret_cast<uint4*>(orow + g0);
+                   o[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                   o[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                 } else {
+#pragma unroll
+                   for (int j = 0; j < 8; ++j)
+                     if (g0 + j < gpr) orow[g0 + j] = w[j];
+                 }
+               });
+  }
+  if (bad) atomicOr(status, TQ_STATUS_BAD_CODE);
+}
+
+// x is staged per CTA as fp32 float4 per group, permuted so that the group 8L+j of pass p sits at
+// slot p*256 + j*32 + L: the 32 lanes of a warp read 32 consecutive float4 at every step j.
+template <int NB>
+__global__ void __launch_bounds__(kThreads, 4)
+gemv_planes_kernel(const uint16_t* __restrict__ codes, uint32_t gpr_pad, const uint32_t* __restrict__ rawbase,
+                   const uint32_t* __restrict__ raw, const float* __restrict__ scale, const float* __restrict__ zero,
+                   int has_zero, const uint32_t* __restrict__ table, uint32_t K, uint32_t rows, uint32_t cols,
+                   const __nv_bfloat16* __restrict__ x, float* __restrict__ y, uint32_t xor_mask, float magic,
+                   uint32_t* __restrict__ status) {
+  extern __shared__ __align__(16) float xs[];  // [NB][n_pass*256] float4
+  __shared__ float sumx[NB];
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+  const uint32_t gpr = cols >> 2;
+  const uint32_t slots = ((gpr_pad + 255u) >> 8) << 8;  // float4 slots per batch column
+  float4* xs4 = reinterpret_cast<float4*>(xs);
+
+  float part[NB];
+#pragma unroll
+  for (int b = 0; b < NB; ++b) part[b] = 0.f;
+  for (uint32_t i = threadIdx.x; i < slots; i += kThreads) {
+    const uint32_t r = i & 255u;
+    const uint32_t g = (i & ~255u) + ((r & 31u) << 3) + (r >> 5);
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (g < gpr) {
+        const uint2 raw2 = reinterpret_cast<const uint2*>(x + (size_t)b * cols)[g];
+        v.x = __uint_as_float(raw2.x << 16);
+        v.y = __uint_as_float(raw2.x & 0xFFFF0000u);
+        v.z = __uint_as_float(raw2.y << 16);
+        v.w = __uint_as_float(raw2.y & 0xFFFF0000u);
+      }
+      xs4[(size_t)b * slots + i] = v;
+      part[b] += (v.x + v.y) + (v.z + v.w);
+    }
+  }
+  if (threadIdx.x < NB) sumx[threadIdx.x] = 0.f;
+  __syncthreads();
+  if (has_zero) {
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      float s = part[b];
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(kFull, s, d);
+      if (lane == 0) atomicAdd(&sumx[b], s);
+    }
+  }
+  __syncthreads();
+
+  uint32_t bad = 0;
+  for (uint32_t row = blockIdx.x * kWarpsPerCta + warp; row < rows; row += gridDim.x * kWarpsPerCta) {
+    float acc[NB];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) acc[b] = 0.f;
+    planes_row(reinterpret_cast<const uint4*>(codes + (size_t)row * gpr_pad), gpr_pad, raw + rawbase[row], table, K,
+               bad, [&](uint32_t p, const uint32_t (&w)[8]) {
+                 const float4* xp = xs4 + p * 256u + lane;
+#pragma unroll
+                 for (int j = 0; j < 8; ++j) {
+                   const uint32_t v = w[j] ^ xor_mask;
+                   const float f0 = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7540)) - magic;
+                   const float f1 = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7541)) - magic;
+                   const float f2 = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7542)) - magic;
+                   const float f3 = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7543)) - magic;
+#pragma unroll
+                   for (int b = 0; b < NB; ++b) {
+                     const float4 xv = xp[(size_t)b * slots + j * 32];
+                     acc[b] = fmaf(f0, xv.x, acc[b]);
+                     acc[b] = fmaf(f1, xv.y, acc[b]);
+                     acc[b] = fmaf(f2, xv.z, acc[b]);
+                     acc[b] = fmaf(f3, xv.w, acc[b]);
+                   }
+                 }
+               });
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      float a = acc[b];
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(kFull, a, d);
+      acc[b] = a;
+    }
+    if (lane == 0) {
+      const float s = scale[row];
+      const float z = has_zero ? zero[row] : 0.f;
+#pragma unroll
+      for (int b = 0; b < NB; ++b) y[(size_t)b * rows + row] = s * (acc[b] - z * sumx[b]);
+    }
+  }
+  if (bad) atomicOr(status, TQ_STATUS_BAD_CODE);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Per-row symmetric int8 quantizer (one CTA per row).
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
@@ -324,9 +494,38 @@ int launch_gemv(const tq_dmat* m, const __nv_bfloat16* x, float* y, cudaStream_t
   const uint32_t grid = std::min<uint32_t>(need, (uint32_t)(sm_count() * per_sm));
   gemv_kernel<NB><<<grid, kThreads, smem, st>>>(
       reinterpret_cast<const uint4*>(m->d_tokens), m->d_rowseg, m->d_scale, m->d_zero, m->has_zero,
-      m->dict->d_entries, m->dict->K, rows, cols, x, y, m->info.levels_signed ? 0x80808080u : 0u,
+      m->dict->d_table, m->dict->K, rows, cols, x, y, m->info.levels_signed ? 0x80808080u : 0u,
       m->info.levels_signed ? 8388736.0f : 8388608.0f, m->d_status);
   return cuda_ok(cudaGetLastError(), "gemv launch");
+}
+
+template <int NB>
+int launch_gemv_planes(const tq_dmat* m, const __nv_bfloat16* x, float* y, cudaStream_t st) {
+  const uint32_t rows = m->info.rows, cols = m->info.cols;
+  const size_t slots = ((size_t)(m->gpr_pad + 255u) >> 8) << 8;
+  const size_t smem = (size_t)NB * slots * sizeof(float4);
+  static size_t configured = 0;
+  if (smem + 4 * 1024 > 48 * 1024 && smem > configured) {
+    if (int rc = cuda_ok(cudaFuncSetAttribute(gemv_planes_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+                         "gemv(planes): raising the dynamic shared memory limit"))
+      return rc;
+    configured = smem;
+  }
+  int per_sm = 0;
+  if (int rc = cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gemv_planes_kernel<NB>, kThreads, smem),
+                       "gemv(planes): occupancy query"))
+    return rc;
+  if (per_sm < 1) {
+    snprintf(g_cuda_msg, sizeof(g_cuda_msg), "gemv(planes): %zu bytes of shared memory do not fit one CTA", smem);
+    return TQ_ERR_CUDA;
+  }
+  const uint32_t need = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
+  const uint32_t grid = std::min<uint32_t>(need, (uint32_t)(sm_count() * per_sm));
+  gemv_planes_kernel<NB><<<grid, kThreads, smem, st>>>(
+      m->d_codes, m->gpr_pad, m->d_rawbase, m->d_raw, m->d_scale, m->d_zero, m->has_zero, m->dict->d_table,
+      m->dict->K, rows, cols, x, y, m->info.levels_signed ? 0x80808080u : 0u,
+      m->info.levels_signed ? 8388736.0f : 8388608.0f, m->d_status);
+  return cuda_ok(cudaGetLastError(), "gemv(planes) launch");
 }
 
 }  // namespace
@@ -345,7 +544,7 @@ int tq_quantize_rows_device(const float* d_w, uint32_t rows, uint32_t cols, int8
 
 int tq_dict_upload_size(const tq_dict* d, uint64_t* device_bytes) {
   if (!d || !device_bytes) return TQ_ERR_INVALID_ARG;
-  *device_bytes = ((uint64_t)d->K * 4 + 255) / 256 * 256 + 256;
+  *device_bytes = (((uint64_t)d->K + 1) * 4 + 255) / 256 * 256 + 256;
   return TQ_OK;
 }
 
@@ -355,15 +554,17 @@ int tq_dict_upload(const tq_dict* d, void* d_buf, uint64_t d_buf_bytes, void* cu
   tq_dict_upload_size(d, &need);
   if (d_buf_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (int rc = cuda_ok(cudaMemsetAsync(d_buf, 0, 256, st), "table upload")) return rc;
   if (d->K) {
-    if (cudaMemcpyAsync(d_buf, d->entries.data(), (size_t)d->K * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
-      return TQ_ERR_CUDA;
+    if (int rc = cuda_ok(cudaMemcpyAsync(static_cast<uint8_t*>(d_buf) + 4, d->entries.data(), (size_t)d->K * 4,
+                                         cudaMemcpyHostToDevice, st), "table upload"))
+      return rc;
   }
-  if (cudaStreamSynchronize(st) != cudaSuccess) return TQ_ERR_CUDA;
+  if (int rc = cuda_ok(cudaStreamSynchronize(st), "table upload")) return rc;
   tq_ddict* dd = new (std::nothrow) tq_ddict();
   if (!dd) return TQ_ERR_NOMEM;
   dd->K = d->K;
-  dd->d_entries = static_cast<const uint32_t*>(d_buf);
+  dd->d_table = static_cast<const uint32_t*>(d_buf);
   *out = dd;
   return TQ_OK;
 }
@@ -372,44 +573,73 @@ void tq_ddict_free(tq_ddict* d) { delete d; }
 
 int tq_upload_size(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols, int layout,
                    uint64_t* device_bytes) {
-  if (!device_bytes || layout != TQ_LAYOUT_STREAM) return TQ_ERR_INVALID_ARG;
-  return tq_build_stream_image(stream, stream_len, rows, cols, 0xFFFFFFFFu, nullptr, nullptr, device_bytes, nullptr);
+  if (!device_bytes) return TQ_ERR_INVALID_ARG;
+  if (layout == TQ_LAYOUT_STREAM)
+    return tq_build_stream_image(stream, stream_len, rows, cols, 0xFFFFFFFFu, nullptr, nullptr, device_bytes, nullptr);
+  if (layout == TQ_LAYOUT_PLANES)
+    return tq_build_planes_image(stream, stream_len, rows, cols, 0xFFFFFFFFu, nullptr, nullptr, device_bytes, nullptr);
+  return TQ_ERR_INVALID_ARG;
 }
 
 int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
               const float* row_scale, const float* row_zero, int levels_signed, int layout, void* d_buf,
               uint64_t d_buf_bytes, void* cuda_stream, tq_dmat** out) {
-  if (!dict || !stream || !row_scale || !d_buf || !out || ((uintptr_t)d_buf & 255) || layout != TQ_LAYOUT_STREAM)
+  if (!dict || !stream || !row_scale || !d_buf || !out || ((uintptr_t)d_buf & 255) ||
+      (layout != TQ_LAYOUT_STREAM && layout != TQ_LAYOUT_PLANES))
     return TQ_ERR_INVALID_ARG;
-  tq_host_image img;
-  uint64_t need = 0;
-  int rc = tq_build_stream_image(stream, stream_len, rows, cols, dict->K, row_scale, row_zero, &need, &img);
-  if (rc != TQ_OK) return rc;
-  if (d_buf_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
+  if (cols / 4 > 65504u) return TQ_ERR_UNSUPPORTED_SHAPE;  // per-row marker counts are 16-bit
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  if (cudaMemcpyAsync(d_buf, img.blob.data(), img.blob.size(), cudaMemcpyHostToDevice, st) != cudaSuccess)
-    return TQ_ERR_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return TQ_ERR_CUDA;
   tq_dmat* m = new (std::nothrow) tq_dmat();
   if (!m) return TQ_ERR_NOMEM;
   uint8_t* base = static_cast<uint8_t*>(d_buf);
+  uint64_t need = 0, n_hits = 0, n_miss = 0;
+  int rc;
+  if (layout == TQ_LAYOUT_STREAM) {
+    tq_host_image img;
+    rc = tq_build_stream_image(stream, stream_len, rows, cols, dict->K, row_scale, row_zero, &need, &img);
+    if (rc == TQ_OK && d_buf_bytes < need) rc = TQ_ERR_BUFFER_TOO_SMALL;
+    if (rc == TQ_OK) rc = cuda_ok(cudaMemcpyAsync(d_buf, img.blob.data(), img.blob.size(), cudaMemcpyHostToDevice, st), "upload");
+    if (rc == TQ_OK) rc = cuda_ok(cudaStreamSynchronize(st), "upload");
+    if (rc != TQ_OK) { delete m; return rc; }
+    m->d_status = reinterpret_cast<uint32_t*>(base + img.off_status);
+    m->d_rowseg = reinterpret_cast<const tq_rowseg*>(base + img.off_rowseg);
+    m->d_scale = reinterpret_cast<const float*>(base + img.off_scale);
+    m->d_zero = reinterpret_cast<const float*>(base + img.off_zero);
+    m->d_tokens = reinterpret_cast<const uint16_t*>(base + img.off_tokens);
+    m->token_chunks = img.token_chunks;
+    n_hits = img.n_hits;
+    n_miss = img.n_miss;
+    m->info.payload_bytes = img.token_chunks * 16 + (uint64_t)rows * (sizeof(tq_rowseg) + 4 + (row_zero ? 4 : 0));
+  } else {
+    tq_planes_image img;
+    rc = tq_build_planes_image(stream, stream_len, rows, cols, dict->K, row_scale, row_zero, &need, &img);
+    if (rc == TQ_OK && d_buf_bytes < need) rc = TQ_ERR_BUFFER_TOO_SMALL;
+    if (rc == TQ_OK) rc = cuda_ok(cudaMemcpyAsync(d_buf, img.blob.data(), img.blob.size(), cudaMemcpyHostToDevice, st), "upload");
+    if (rc == TQ_OK) rc = cuda_ok(cudaStreamSynchronize(st), "upload");
+    if (rc != TQ_OK) { delete m; return rc; }
+    m->d_status = reinterpret_cast<uint32_t*>(base + img.off_status);
+    m->d_rawbase = reinterpret_cast<const uint32_t*>(base + img.off_rawbase);
+    m->d_rawidx = reinterpret_cast<const uint16_t*>(base + img.off_rawidx);
+    m->d_scale = reinterpret_cast<const float*>(base + img.off_scale);
+    m->d_zero = reinterpret_cast<const float*>(base + img.off_zero);
+    m->d_codes = reinterpret_cast<const uint16_t*>(base + img.off_codes);
+    m->d_raw = reinterpret_cast<const uint32_t*>(base + img.off_raw);
+    m->gpr_pad = img.gpr_pad;
+    m->nidx_pad = img.nidx_pad;
+    n_hits = img.n_hits;
+    n_miss = img.n_miss;
+    m->info.payload_bytes = (uint64_t)rows * img.gpr_pad * 2 + n_miss * 4 + (uint64_t)rows * (4 + 4 + (row_zero ? 4 : 0));
+  }
   m->dict = dict;
-  m->d_status = reinterpret_cast<uint32_t*>(base + img.off_status);
-  m->d_rowseg = reinterpret_cast<const tq_rowseg*>(base + img.off_rowseg);
-  m->d_scale = reinterpret_cast<const float*>(base + img.off_scale);
-  m->d_zero = reinterpret_cast<const float*>(base + img.off_zero);
-  m->d_tokens = reinterpret_cast<const uint16_t*>(base + img.off_tokens);
-  m->token_chunks = img.token_chunks;
   m->has_zero = row_zero != nullptr;
   m->info.rows = rows;
   m->info.cols = cols;
   m->info.K = dict->K;
   m->info.layout = layout;
   m->info.levels_signed = levels_signed != 0;
-  m->info.n_hits = img.n_hits;
-  m->info.n_miss = img.n_miss;
-  m->info.stream_bytes = 2 * (img.n_hits + 5 * img.n_miss);
-  m->info.payload_bytes = img.token_chunks * 16 + (uint64_t)rows * (sizeof(tq_rowseg) + 4 + (row_zero ? 4 : 0));
+  m->info.n_hits = n_hits;
+  m->info.n_miss = n_miss;
+  m->info.stream_bytes = 2 * (n_hits + 5 * n_miss);
   m->info.device_bytes = need;
   *out = m;
   return TQ_OK;
@@ -424,11 +654,17 @@ int tq_dmat_get_info(const tq_dmat* m, tq_dmat_info* info) {
 void tq_dmat_free(tq_dmat* m) { delete m; }
 
 int tq_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
-  if (!m || !d_codes || ((uintptr_t)d_codes & 3)) return TQ_ERR_INVALID_ARG;
+  if (!m || !d_codes || ((uintptr_t)d_codes & 15)) return TQ_ERR_INVALID_ARG;
   const uint32_t need = (m->info.rows + kWarpsPerCta - 1) / kWarpsPerCta;
   const uint32_t grid = std::min<uint32_t>(need, (uint32_t)sm_count() * 8u);
+  if (m->info.layout == TQ_LAYOUT_PLANES) {
+    decompress_planes_kernel<<<grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
+        m->d_codes, m->gpr_pad, m->d_rawbase, m->d_raw, m->dict->d_table, m->dict->K, m->info.rows, m->info.cols,
+        reinterpret_cast<uint32_t*>(d_codes), m->d_status);
+    return cuda_ok(cudaGetLastError(), "decompress(planes) launch");
+  }
   decompress_kernel<<<grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
-      reinterpret_cast<const uint4*>(m->d_tokens), m->d_rowseg, m->dict->d_entries, m->dict->K, m->info.rows,
+      reinterpret_cast<const uint4*>(m->d_tokens), m->d_rowseg, m->dict->d_table, m->dict->K, m->info.rows,
       m->info.cols, reinterpret_cast<uint32_t*>(d_codes), m->d_status);
   return cuda_ok(cudaGetLastError());
 }
@@ -439,18 +675,20 @@ int tq_fused_gemv(const tq_dmat* m, const void* d_x_bf16, int B, float* d_y, voi
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(d_x_bf16);
   const uint32_t rows = m->info.rows, cols = m->info.cols;
   // fp32 x for up to 4 batch columns must fit the 227 KB of shared memory
-  const int max_nb = (size_t)4 * cols * 4 <= 200 * 1024 ? 4 : ((size_t)2 * cols * 4 <= 200 * 1024 ? 2 : 1);
-  if ((size_t)cols * 4 > 200 * 1024) return TQ_ERR_UNSUPPORTED_SHAPE;
+  const bool planes = m->info.layout == TQ_LAYOUT_PLANES;
+  const size_t xcols = planes ? ((((size_t)m->gpr_pad + 255) >> 8) << 10) : cols;  // staged columns per batch column
+  const int max_nb = 4 * xcols * 4 <= 200 * 1024 ? 4 : (2 * xcols * 4 <= 200 * 1024 ? 2 : 1);
+  if (xcols * 4 > 200 * 1024) return TQ_ERR_UNSUPPORTED_SHAPE;
   for (int b0 = 0; b0 < B;) {
     const int nb = std::min(B - b0, max_nb);
     int rc;
     const __nv_bfloat16* xb = x + (size_t)b0 * cols;
     float* yb = d_y + (size_t)b0 * rows;
     switch (nb) {
-      case 1: rc = launch_gemv<1>(m, xb, yb, st); break;
-      case 2: rc = launch_gemv<2>(m, xb, yb, st); break;
-      case 3: rc = launch_gemv<3>(m, xb, yb, st); break;
-      default: rc = launch_gemv<4>(m, xb, yb, st); break;
+      case 1: rc = planes ? launch_gemv_planes<1>(m, xb, yb, st) : launch_gemv<1>(m, xb, yb, st); break;
+      case 2: rc = planes ? launch_gemv_planes<2>(m, xb, yb, st) : launch_gemv<2>(m, xb, yb, st); break;
+      case 3: rc = planes ? launch_gemv_planes<3>(m, xb, yb, st) : launch_gemv<3>(m, xb, yb, st); break;
+      default: rc = planes ? launch_gemv_planes<4>(m, xb, yb, st) : launch_gemv<4>(m, xb, yb, st); break;
     }
     if (rc != TQ_OK) return rc;
     b0 += nb;

@@ -487,9 +487,9 @@ namespace {
 inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 }  // namespace
 
-int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
-                          uint32_t K, const float* row_scale, const float* row_zero,
-                          uint64_t* device_bytes, tq_host_image* img) {
+// Validates the stream and finds where every row's tokens start.
+static int scan_stream(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols, uint32_t K,
+                       std::vector<uint64_t>& row_start, uint64_t& H, uint64_t& M) {
   if (!stream || rows == 0 || cols == 0) return TQ_ERR_INVALID_ARG;
   if (cols % 4 != 0) return TQ_ERR_UNSUPPORTED_SHAPE;
   const uint64_t bpr = cols / 4, nb = (uint64_t)rows * bpr;
@@ -525,7 +525,8 @@ int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t 
     miss[t] = m;
   });
   if (bad.load()) return TQ_ERR_CORRUPT_STREAM;
-  uint64_t H = 0, M = 0;
+  H = 0;
+  M = 0;
   std::vector<uint64_t> first_block(T + 1, 0);
   for (int t = 0; t < T; ++t) {
     H += hits[t];
@@ -534,8 +535,7 @@ int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t 
   }
   if (H + M != nb || H + 5 * M != stream_len) return TQ_ERR_CORRUPT_STREAM;
 
-  // row starts
-  std::vector<uint64_t> row_start((size_t)rows + 1, 0);
+  row_start.assign((size_t)rows + 1, 0);
   row_start[rows] = stream_len;
   parallel_run(T, [&](int t) {
     uint64_t p = cut(t), e = cut(t + 1), blk = first_block[t];
@@ -551,6 +551,16 @@ int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t 
       if (stream[p] == TQ_ESCAPE) raw = 4;
     }
   });
+  return TQ_OK;
+}
+
+int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
+                          uint32_t K, const float* row_scale, const float* row_zero,
+                          uint64_t* device_bytes, tq_host_image* img) {
+  std::vector<uint64_t> row_start;
+  uint64_t H = 0, M = 0;
+  int rc = scan_stream(stream, stream_len, rows, cols, K, row_start, H, M);
+  if (rc != TQ_OK) return rc;
 
   std::vector<uint64_t> chunk_off((size_t)rows + 1, 0);
   for (uint32_t r = 0; r < rows; ++r) chunk_off[r + 1] = chunk_off[r] + (row_start[r + 1] - row_start[r] + 7) / 8;
@@ -593,6 +603,92 @@ int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t 
       seg[r].chunk_off = (uint32_t)chunk_off[r];
       seg[r].n_slots = (uint32_t)n;
       std::memcpy(tok + chunk_off[r] * 8, stream + row_start[r], n * 2);
+    }
+  });
+  return TQ_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// PLANES layout: a lossless re-tiling of the same tokens.  Every group keeps its 16-bit token in a
+// fixed-stride code plane (row-major, row stride padded to a multiple of 32 groups with token 0,
+// which decodes to four zero bytes); the 4 raw bytes that follow a marker move, packed into one
+// 32-bit word, to a compact raw plane in row-major group order.  raw_base[r] is the index of row
+// r's first raw word; raw_idx[r][c] counts the row's markers before group 32*c.
+// ---------------------------------------------------------------------------------------------
+int tq_build_planes_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
+                          uint32_t K, const float* row_scale, const float* row_zero,
+                          uint64_t* device_bytes, tq_planes_image* img) {
+  std::vector<uint64_t> row_start;
+  uint64_t H = 0, M = 0;
+  int rc = scan_stream(stream, stream_len, rows, cols, K, row_start, H, M);
+  if (rc != TQ_OK) return rc;
+  if (M >= (1ull << 32)) return TQ_ERR_UNSUPPORTED_SHAPE;
+
+  const uint32_t gpr = cols / 4;
+  const uint32_t gpr_pad = (gpr + 31u) / 32u * 32u;
+  const uint32_t nidx = gpr_pad / 32u + 1u;
+  const uint32_t nidx_pad = (nidx + 1u) & ~1u;
+
+  const uint64_t off_status = 0;
+  const uint64_t off_rawbase = 256;
+  const uint64_t off_rawidx = align_up(off_rawbase + ((uint64_t)rows + 1) * 4, 256);
+  const uint64_t off_scale = align_up(off_rawidx + (uint64_t)rows * nidx_pad * 2, 256);
+  const uint64_t off_zero = align_up(off_scale + (uint64_t)rows * 4, 256);
+  const uint64_t off_codes = align_up(off_zero + (uint64_t)rows * 4, 256);
+  const uint64_t off_raw = align_up(off_codes + (uint64_t)rows * gpr_pad * 2 + 256, 256);
+  const uint64_t total = align_up(off_raw + M * 4 + 256, 256);
+  if (device_bytes) *device_bytes = total;
+  if (!img) return TQ_OK;
+  if (!row_scale) return TQ_ERR_INVALID_ARG;
+  try {
+    img->blob.assign(total, 0);
+  } catch (const std::bad_alloc&) {
+    return TQ_ERR_NOMEM;
+  }
+  img->off_status = off_status;
+  img->off_rawbase = off_rawbase;
+  img->off_rawidx = off_rawidx;
+  img->off_scale = off_scale;
+  img->off_zero = off_zero;
+  img->off_codes = off_codes;
+  img->off_raw = off_raw;
+  img->gpr_pad = gpr_pad;
+  img->nidx_pad = nidx_pad;
+  img->n_hits = H;
+  img->n_miss = M;
+  uint8_t* base = img->blob.data();
+  std::memcpy(base + off_scale, row_scale, (size_t)rows * 4);
+  if (row_zero) std::memcpy(base + off_zero, row_zero, (size_t)rows * 4);
+  uint32_t* rawbase = reinterpret_cast<uint32_t*>(base + off_rawbase);
+  uint16_t* rawidx = reinterpret_cast<uint16_t*>(base + off_rawidx);
+  uint16_t* codes = reinterpret_cast<uint16_t*>(base + off_codes);
+  uint32_t* raw = reinterpret_cast<uint32_t*>(base + off_raw);
+
+  // markers per row: a row with h coded groups and m escaped ones occupies h + 5m slots
+  for (uint32_t r = 0; r < rows; ++r) {
+    const uint64_t n = row_start[r + 1] - row_start[r];
+    rawbase[r + 1] = rawbase[r] + (uint32_t)((n - gpr) / 4);
+  }
+  const int T = (int)std::min<uint64_t>(tq_num_threads(), stream_len / (1u << 18) + 1);
+  parallel_run(T, [&](int t) {
+    uint32_t r0 = (uint32_t)((uint64_t)rows * t / T), r1 = (uint32_t)((uint64_t)rows * (t + 1) / T);
+    for (uint32_t r = r0; r < r1; ++r) {
+      const uint16_t* s = stream + row_start[r];
+      uint16_t* c = codes + (uint64_t)r * gpr_pad;
+      uint16_t* ix = rawidx + (uint64_t)r * nidx_pad;
+      uint32_t* rw = raw + rawbase[r];
+      uint32_t nraw = 0;
+      for (uint32_t g = 0; g < gpr; ++g) {
+        if ((g & 31u) == 0) ix[g >> 5] = (uint16_t)nraw;
+        const uint16_t v = *s++;
+        c[g] = v;
+        if (v == TQ_ESCAPE) {
+          rw[nraw++] = (uint32_t)(s[0] & 0xFF) | ((uint32_t)(s[1] & 0xFF) << 8) | ((uint32_t)(s[2] & 0xFF) << 16) |
+                       ((uint32_t)(s[3] & 0xFF) << 24);
+          s += 4;
+        }
+      }
+      for (uint32_t k = (gpr + 31u) >> 5; k < nidx; ++k) ix[k] = (uint16_t)nraw;
     }
   });
   return TQ_OK;

@@ -20,7 +20,9 @@ struct tq_dict {
 
 struct tq_ddict {
   uint32_t K = 0;
-  const uint32_t* d_entries = nullptr;  // DEVICE: K words, byte i of the window in bits 8i..8i+7
+  // DEVICE: K + 1 words indexed by code; word 0 is zero (token 0 = padding), word c holds entry
+  // c - 1 with byte i of the window in bits 8i..8i+7
+  const uint32_t* d_table = nullptr;
 };
 
 // Row descriptor of the STREAM layout: where the row's token segment starts (in 16-byte units
@@ -37,9 +39,15 @@ struct tq_dmat {
   const tq_rowseg* d_rowseg = nullptr; // DEVICE: rows entries
   const float* d_scale = nullptr;      // DEVICE: rows
   const float* d_zero = nullptr;       // DEVICE: rows
-  const uint16_t* d_tokens = nullptr;  // DEVICE: token area, 256-byte aligned
+  const uint16_t* d_tokens = nullptr;  // DEVICE: token area, 256-byte aligned (STREAM layout)
   uint64_t token_chunks = 0;           // token area length in 16-byte units
   int has_zero = 0;
+  // PLANES layout
+  const uint32_t* d_rawbase = nullptr; // DEVICE: rows + 1, index of each row's first raw word
+  const uint16_t* d_rawidx = nullptr;  // DEVICE: rows x nidx_pad, markers before group 32*c of the row
+  const uint16_t* d_codes = nullptr;   // DEVICE: rows x gpr_pad tokens
+  const uint32_t* d_raw = nullptr;     // DEVICE: raw words
+  uint32_t gpr_pad = 0, nidx_pad = 0;
 };
 
 // Host-side image of a matrix in the STREAM layout, ready for one cudaMemcpy.
@@ -50,6 +58,13 @@ struct tq_host_image {
   uint64_t n_hits = 0, n_miss = 0;
 };
 
+struct tq_planes_image {
+  std::vector<uint8_t> blob;
+  uint64_t off_status = 0, off_rawbase = 0, off_rawidx = 0, off_scale = 0, off_zero = 0, off_codes = 0, off_raw = 0;
+  uint32_t gpr_pad = 0, nidx_pad = 0;
+  uint64_t n_hits = 0, n_miss = 0;
+};
+
 int tq_num_threads();
 
 // Validates the stream and computes the layout size; if img != nullptr also builds the image.
@@ -57,3 +72,6 @@ int tq_num_threads();
 int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
                           uint32_t K, const float* row_scale, const float* row_zero,
                           uint64_t* device_bytes, tq_host_image* img);
+int tq_build_planes_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
+                          uint32_t K, const float* row_scale, const float* row_zero,
+                          uint64_t* device_bytes, tq_planes_image* img);

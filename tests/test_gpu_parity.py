@@ -18,6 +18,14 @@ def tq():
     return binding
 
 
+LAYOUTS = [0, 1]  # TQ_LAYOUT_STREAM, TQ_LAYOUT_PLANES
+
+
+@pytest.fixture(params=LAYOUTS, ids=["stream", "planes"])
+def layout(request):
+    return request.param
+
+
 def _rel_err(y, ref):
     # per batch column
     return float(np.max(np.max(np.abs(y - ref), axis=1) / np.max(np.abs(ref), axis=1)))
@@ -28,17 +36,17 @@ def _oracle_pack(q_list, top_k=65535):
     return d, [d.encode(q)[0] for q in q_list]
 
 
-def _upload_from_oracle(tq, odict, stream, rows, cols, scale, zero=None, signed=True):
+def _upload_from_oracle(tq, odict, stream, rows, cols, scale, zero=None, signed=True, layout=0):
     """Everything fed to the device comes from the oracle (table, stream) so a host-library bug
     cannot hide a device bug."""
     hd = tq.tq_dict_from_entries(odict.entries)
     dd = tq.tq_dict_upload(hd)
-    return tq.tq_upload(dd, stream, rows, cols, scale, zero, levels_signed=signed)
+    return tq.tq_upload(dd, stream, rows, cols, scale, zero, levels_signed=signed, layout=layout)
 
 
-def _check_layer(tq, q, scale, odict, stream, batches=(1,), zero=None, seed=1):
+def _check_layer(tq, q, scale, odict, stream, batches=(1,), zero=None, seed=1, layout=0):
     rows, cols = q.shape
-    m = _upload_from_oracle(tq, odict, stream, rows, cols, scale, zero, signed=(q.dtype == np.int8))
+    m = _upload_from_oracle(tq, odict, stream, rows, cols, scale, zero, signed=(q.dtype == np.int8), layout=layout)
     # decoded bytes: bit exact against the oracle's decoder and the original levels
     got = tq.tq_decompress(m).cpu().numpy()
     ref = odict.decode(stream).reshape(rows, cols)
@@ -54,47 +62,47 @@ def _check_layer(tq, q, scale, odict, stream, batches=(1,), zero=None, seed=1):
     return m
 
 
-def test_config0_layer_2048x2048(tq):
+def test_config0_layer_2048x2048(tq, layout):
     w = synth.weight(2048, 2048, synth.matrix_seed(0)).numpy()
     q, s = oracle.quantize_rows(w)
     d, (stream,) = _oracle_pack([q])
-    m = _check_layer(tq, q, s, d, stream, batches=(1, 4))
+    m = _check_layer(tq, q, s, d, stream, batches=(1, 4), layout=layout)
     assert m.info.n_hits + m.info.n_miss == 2048 * 2048 // 4
     assert m.info.stream_bytes == stream.nbytes
 
 
-@pytest.mark.parametrize("rows,cols", [(1, 4), (3, 8), (7, 260), (8, 256), (9, 1028), (33, 2052), (17, 8192), (5, 12288)])
-def test_ragged_shapes(tq, rows, cols):
+@pytest.mark.parametrize("rows,cols", [(1, 4), (3, 8), (7, 260), (8, 256), (9, 1028), (33, 2052), (17, 8192), (5, 12288), (40, 4 * 300)])
+def test_ragged_shapes(tq, rows, cols, layout):
     rng = np.random.default_rng(rows * 1000 + cols)
     q = np.clip(np.rint(rng.standard_t(5, size=(rows, cols)) * 3), -127, 127).astype(np.int8)
     s = (rng.random(rows) + 0.5).astype(np.float32)
     d, (stream,) = _oracle_pack([q], top_k=200)
-    _check_layer(tq, q, s, d, stream, batches=(1, 2, 3, 4, 5))
+    _check_layer(tq, q, s, d, stream, batches=(1, 2, 3, 4, 5), layout=layout)
 
 
-def test_all_hits_and_all_misses(tq):
+def test_all_hits_and_all_misses(tq, layout):
     rng = np.random.default_rng(5)
     q = rng.integers(-2, 3, size=(64, 512)).astype(np.int8)
     s = np.full(64, 0.01, dtype=np.float32)
     d, (stream,) = _oracle_pack([q])
     assert np.all(stream != 0xFFFF)  # every group is in the table
-    _check_layer(tq, q, s, d, stream, batches=(1, 4))
+    _check_layer(tq, q, s, d, stream, batches=(1, 4), layout=layout)
     d0, (stream0,) = _oracle_pack([q], top_k=0)
     assert stream0.size == 5 * q.size // 4  # every group escapes
-    _check_layer(tq, q, s, d0, stream0, batches=(1, 3))
+    _check_layer(tq, q, s, d0, stream0, batches=(1, 3), layout=layout)
 
 
-def test_large_table_codes_near_65534(tq):
+def test_large_table_codes_near_65534(tq, layout):
     # enough distinct windows to fill the table; high codes (>= 0xFF00) share their top byte with the marker
     rng = np.random.default_rng(6)
     q = rng.integers(-20, 21, size=(512, 1024)).astype(np.int8)
     s = (rng.random(512) + 0.5).astype(np.float32)
     d, (stream,) = _oracle_pack([q])
     assert d.K == 65534 and int(stream[stream != 0xFFFF].max()) > 0xFF00
-    _check_layer(tq, q, s, d, stream, batches=(1,))
+    _check_layer(tq, q, s, d, stream, batches=(1,), layout=layout)
 
 
-def test_unsigned_levels_with_zero_point(tq):
+def test_unsigned_levels_with_zero_point(tq, layout):
     # the paper's own quantizer: per-tensor unsigned levels and a zero point
     w = synth.weight(256, 1024, synth.matrix_seed(9)).numpy()
     qu, sc, zp = oracle.quantize_paper(w)
@@ -102,15 +110,15 @@ def test_unsigned_levels_with_zero_point(tq):
     s = np.full(256, sc, dtype=np.float32)
     z = np.full(256, zp, dtype=np.float32)
     d, (stream,) = _oracle_pack([qu])
-    _check_layer(tq, qu, s, d, stream, batches=(1, 4), zero=z)
+    _check_layer(tq, qu, s, d, stream, batches=(1, 4), zero=z, layout=layout)
 
 
-def test_batch_up_to_32(tq):
+def test_batch_up_to_32(tq, layout):
     rng = np.random.default_rng(8)
     q = np.clip(np.rint(rng.standard_t(5, size=(130, 3072)) * 6), -127, 127).astype(np.int8)
     s = (rng.random(130) + 0.5).astype(np.float32)
     d, (stream,) = _oracle_pack([q])
-    _check_layer(tq, q, s, d, stream, batches=(8, 32))
+    _check_layer(tq, q, s, d, stream, batches=(8, 32), layout=layout)
 
 
 def test_quantize_rows_device_bit_exact(tq):
@@ -130,7 +138,7 @@ def test_generator_is_device_independent():
     assert torch.equal(xa, xb)
 
 
-def test_host_library_pipeline_matches_oracle_pipeline(tq):
+def test_host_library_pipeline_matches_oracle_pipeline(tq, layout):
     """Product pipeline end to end (tq_quantize_rows_device -> tq_build_dictionary -> tq_encode ->
     tq_upload -> kernels) on the 1B MLP shapes, checked on sampled rows the oracle computes itself."""
     shapes = [("gate", 8192, 2048), ("up", 8192, 2048), ("down", 2048, 8192)]
@@ -143,7 +151,7 @@ def test_host_library_pipeline_matches_oracle_pipeline(tq):
     for i, (name, rows, cols) in enumerate(shapes):
         stream, h, mi = tq.tq_encode(hd, q_host[i])
         assert stream.size == h + 5 * mi
-        m = tq.tq_upload(dd, stream, rows, cols, ss[i].cpu().numpy())
+        m = tq.tq_upload(dd, stream, rows, cols, ss[i].cpu().numpy(), layout=layout)
         got = tq.tq_decompress(m)
         assert torch.equal(got.view(torch.int8), qs[i])  # whole matrix, product vs product
         sample = np.sort(rng.choice(rows, 64, replace=False))

@@ -126,13 +126,14 @@ def _valid_stream(rows=6, cols=16, seed=0):
     return s, rows, cols
 
 
-def test_upload_size_accepts_valid_and_rejects_corrupt():
+@pytest.mark.parametrize("layout", [0, 1], ids=["stream", "planes"])
+def test_upload_size_accepts_valid_and_rejects_corrupt(layout):
     s, rows, cols = _valid_stream()
-    assert tq.tq_upload_size(s, rows, cols) > 0
+    assert tq.tq_upload_size(s, rows, cols, layout) > 0
 
     def bad(stream, r=rows, c=cols):
         with pytest.raises(tq.TqError) as e:
-            tq.tq_upload_size(stream, r, c)
+            tq.tq_upload_size(stream, r, c, layout)
         return e.value.status
 
     assert bad(s[:-1]) == tq.TQ_ERR_CORRUPT_STREAM               # truncated
