@@ -39,6 +39,13 @@ __device__ __forceinline__ uint32_t esc_bits(uint32_t a) {
 
 constexpr uint32_t kRing = 512;  // per-warp ring of decoded groups (uint32 each); > 256 + 31
 
+// Exact variant for token planes, where any token may follow a marker: bit 15 / 31 set iff the
+// low / high half equals 0xFFFF.
+__device__ __forceinline__ uint32_t esc_bits_exact(uint32_t a) {
+  const uint32_t t = (~a & 0x7FFF7FFFu) + 0x7FFF7FFFu;
+  return ~t & a & 0x80008000u;
+}
+
 // Walks one row segment.  Each tile is handled in two phases.  Phase 1: every lane turns the
 // groups completed inside its 8 slots into packed 4-byte words (table loads are issued together,
 // before any use) and stores them, in row order, into the warp's ring in shared memory.  Phase 2:
@@ -269,8 +276,8 @@ __device__ __forceinline__ void planes_row(const uint4* __restrict__ codes, uint
   for (uint32_t p = 0; p < n_pass; ++p) {
     const uint32_t pf = (p + 2u) * 32u + lane;
     const uint4 nn = pf < n_vec ? ldg_stream(codes + pf) : zero4;
-    const uint32_t e = (esc_bits(cur.x) >> 15) | (esc_bits(cur.y) >> 13) | (esc_bits(cur.z) >> 11) |
-                       (esc_bits(cur.w) >> 9);
+    const uint32_t e = (esc_bits_exact(cur.x) >> 15) | (esc_bits_exact(cur.y) >> 13) | (esc_bits_exact(cur.z) >> 11) |
+                       (esc_bits_exact(cur.w) >> 9);
     const uint32_t E = (e | (e >> 15)) & 0xFFu;
     const uint32_t n = __popc(E);
     uint32_t incl = n;
