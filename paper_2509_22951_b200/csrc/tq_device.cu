@@ -537,6 +537,8 @@ int launch_gemv_planes(const tq_dmat* m, const __nv_bfloat16* x, float* y, cudaS
 
 }  // namespace
 
+int tq_cuda_status(int cuda_error, const char* what) { return cuda_ok((cudaError_t)cuda_error, what); }
+
 extern "C" {
 
 const char* tq_last_cuda_error(void) { return g_cuda_msg; }
@@ -714,11 +716,6 @@ int tq_fused_gemv_host(const tq_dmat* m, const void* h_x_bf16, int B, float* h_y
   if (cudaMemcpyAsync(h_y, d_y_stage, (size_t)B * m->info.rows * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return TQ_ERR_CUDA;
   return TQ_OK;
-}
-
-int tq_fused_gemm(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, void* cuda_stream) {
-  (void)m; (void)d_X_bf16; (void)M; (void)d_Y; (void)cuda_stream;
-  return TQ_ERR_UNSUPPORTED_SHAPE;
 }
 
 int tq_device_status(const tq_dmat* m, void* cuda_stream, uint32_t* status) {

@@ -67,6 +67,9 @@ struct tq_planes_image {
 
 int tq_num_threads();
 
+// Maps a cudaError_t (passed as int) to TQ_OK / TQ_ERR_CUDA and records its text for tq_last_cuda_error.
+int tq_cuda_status(int cuda_error, const char* what);
+
 // Validates the stream and computes the layout size; if img != nullptr also builds the image.
 // K == 0xFFFFFFFF skips the code-range check (size query without a table).
 int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
