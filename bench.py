@@ -164,6 +164,58 @@ def oracle_sample_run(hd_entries, q_host, scales, shapes, batch, sample_idx, rep
     return total, times
 
 
+def time_extras(tq, mats, infos, shapes, args, device, stream):
+    """Standalone tq_decompress of the whole weight set and the prefill product (tq_fused_gemm) at
+    M tokens, timed with CUDA events on the launching stream (3 warm-ups, inputs far larger than L2)."""
+    out = {}
+    n_weights = sum(i.rows * i.cols for i in infos)
+    max_elems = max(i.rows * i.cols for i in infos)
+    buf = torch.empty(max_elems, dtype=torch.uint8, device=device)
+
+    def run_dec():
+        for m in mats:
+            tq.tq_decompress(m, buf[: m.info.rows * m.info.cols])
+
+    def timed(fn, reps):
+        for _ in range(3):
+            fn()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        stream.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    ms = timed(run_dec, 10)
+    rd = sum(algorithmic_bytes(i, 0) for i in infos)
+    out["decompress"] = {"ms": ms, "GB_per_s": (rd + n_weights) / (ms * 1e-3) / 1e9,
+                         "bytes": {"read": rd, "written": n_weights},
+                         "frac_of_measured_hbm": (rd + n_weights) / (ms * 1e-3) / 1e9 / measured_peaks()[0]}
+    if args.layout == "planes":
+        M = args.prefill_tokens
+        max_rows = max(i.rows for i in infos)
+        Y = torch.empty(M * max_rows, dtype=torch.float32, device=device)
+        Xs = {c: synth.activations(M, c, 99, device=device) for c in sorted({i.cols for i in infos})}
+
+        def run_gemm():
+            for m in mats:
+                tq.tq_fused_gemm(m, Xs[m.info.cols], Y[: M * m.info.rows].view(M, m.info.rows))
+
+        ms = timed(run_gemm, 3)
+        flops = 2.0 * M * n_weights
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+        pk = float(peaks.get("bf16_tflops_sustained", 1400.0))
+        out["prefill"] = {"tokens": M, "ms": ms, "TFLOP_per_s": flops / (ms * 1e-3) / 1e12,
+                          "frac_of_measured_bf16_sustained": flops / (ms * 1e-3) / 1e12 / pk, "peak_TFLOP_per_s": pk}
+        status = 0
+        for m in mats:
+            status |= tq.tq_device_status(m)
+        assert status == 0, f"device status {status}"
+    return out
+
+
 def pick_sample(shapes, max_weights):
     idx, tot = [], 0
     for i, (_, r, c) in enumerate(shapes):
@@ -189,6 +241,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the tq_decompress / tq_fused_gemm timings")
+    ap.add_argument("--prefill-tokens", type=int, default=2048)
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -333,6 +387,11 @@ def main():
                    "h2d": sum(2 * args.batch * i.cols for i in infos),
                    "d2h": sum(4 * args.batch * i.rows for i in infos)}
 
+        # ---- the other device calls on the same resident model (single GPU only) ----
+        extras = {}
+        if not args.no_extras and world == 1:
+            extras = time_extras(tq, mats, infos, shapes, args, device, stream)
+
     ms_step = ms_total / args.steps
     if world > 1:
         import torch.distributed as dist
@@ -372,6 +431,7 @@ def main():
                      "note": "achieved = algorithmic bytes of the %d launches of a step / step time (launch gaps included)" % launches_per_step},
         "setup_s": stats,
     }
+    out.update(extras)
     if e2e:
         out["e2e"] = {"value": world * alg_bytes / (e2e["ms_per_step"] * 1e-3) / 1e9, "unit": UNIT,
                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
