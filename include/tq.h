@@ -166,6 +166,23 @@ int tq_fused_gemv(const tq_dmat* m, const void* d_x_bf16, int B, float* d_y, voi
 int tq_fused_gemv_host(const tq_dmat* m, const void* h_x_bf16, int B, float* h_y, void* d_x_stage,
                        float* d_y_stage, void* cuda_stream);
 
+/* tq_fused_gemv_host for callers that cannot allocate device memory (the paper has no counterpart:
+ * this is a convenience of the library).  Such callers exist: code running inside a stream
+ * capture or a latency-critical serving loop where cudaMalloc would synchronise the device, a
+ * plug-in handed a fixed memory budget by its host application, a process that only receives
+ * device pointers from elsewhere.  The staging copies of x and y live in a fixed 1.5 MiB array
+ * that is part of the library image (every GPU that loads the library keeps it until the process
+ * exits), so the call is limited to B * cols <= 262144 and B * rows <= 262144 and returns
+ * TQ_ERR_UNSUPPORTED_SHAPE (text in tq_last_cuda_error) beyond that.  No cudaMalloc, cudaFree or
+ * other allocating routine is called.  The first call on each device looks up the array's device
+ * address with that device current; make that first call outside any stream capture.  All calls
+ * on a device share the one array: nothing in it has to start at zero (x is overwritten by the
+ * copy, y by the kernel, before either is read), but two calls whose GPU work overlaps (different
+ * streams, or different threads) race on it -- serialise them.  h_x_bf16, h_y: HOST, as for
+ * tq_fused_gemv_host; asynchronous on cuda_stream. */
+int tq_fused_gemv_host_static(const tq_dmat* m, const void* h_x_bf16, int B, float* h_y,
+                              void* cuda_stream);
+
 /* Same product for prefill-sized batches (M tokens): decoded weight tiles are converted to bf16
  * (exact: |level| <= 255) in shared memory and fed to tcgen05 tensor-core MMAs with fp32
  * accumulation; scale and zero point are applied in fp32 afterwards.

@@ -33,14 +33,15 @@ EXPORTS = [
     "tq_quantize_rows_device", "tq_build_dictionary", "tq_dict_from_entries", "tq_dict_entries",
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
-    "tq_fused_gemv_host", "tq_fused_gemm", "tq_device_status", "tq_dmat_free",
+    "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_device_status", "tq_dmat_free",
 ]
 
 
 class TqError(RuntimeError):
-    def __init__(self, status: int, where: str):
+    def __init__(self, status: int, where: str, detail: str | None = None):
         self.status = status
-        detail = _lib.tq_last_cuda_error().decode() if status == TQ_ERR_CUDA else ""
+        if detail is None:
+            detail = _lib.tq_last_cuda_error().decode() if status == TQ_ERR_CUDA else ""
         super().__init__(f"{where}: {_lib.tq_strerror(status).decode()} ({status}) {detail}")
 
 
@@ -78,6 +79,7 @@ def _load() -> C.CDLL:
         "tq_decompress": (C.c_int, [vp, vp, vp]),
         "tq_fused_gemv": (C.c_int, [vp, vp, C.c_int, vp, vp]),
         "tq_fused_gemv_host": (C.c_int, [vp, vp, C.c_int, vp, vp, vp, vp]),
+        "tq_fused_gemv_host_static": (C.c_int, [vp, vp, C.c_int, vp, vp]),
         "tq_fused_gemm": (C.c_int, [vp, vp, C.c_int, vp, vp]),
         "tq_device_status": (C.c_int, [vp, vp, u32p]),
         "tq_dmat_free": (None, [vp]),
@@ -313,6 +315,20 @@ def tq_fused_gemv_host(m: DeviceMatrix, h_x: torch.Tensor, h_y: torch.Tensor, d_
     assert d_y_stage.is_cuda and d_y_stage.numel() * d_y_stage.element_size() >= B * m.info.rows * 4
     _check(_lib.tq_fused_gemv_host(m._h, h_x.data_ptr(), B, h_y.data_ptr(), d_x_stage.data_ptr(),
                                    d_y_stage.data_ptr(), _stream_ptr(stream)), "tq_fused_gemv_host")
+
+
+def tq_fused_gemv_host_static(m: DeviceMatrix, h_x: torch.Tensor, h_y: torch.Tensor, stream=None) -> None:
+    """tq_fused_gemv_host without caller staging: the library's built-in 1.5 MiB staging array is
+    used, nothing is allocated (B * cols and B * rows are limited to 262144 each)."""
+    assert (not h_x.is_cuda) and h_x.dtype == torch.bfloat16 and h_x.is_contiguous()
+    assert (not h_y.is_cuda) and h_y.dtype == torch.float32 and h_y.is_contiguous()
+    B = h_x.numel() // m.info.cols
+    assert h_y.numel() == B * m.info.rows
+    with torch.cuda.device(m.buf.device):
+        rc = _lib.tq_fused_gemv_host_static(m._h, h_x.data_ptr(), B, h_y.data_ptr(), _stream_ptr(stream))
+    if rc == TQ_ERR_UNSUPPORTED_SHAPE:  # the library left the limits in its error text
+        raise TqError(rc, "tq_fused_gemv_host_static", _lib.tq_last_cuda_error().decode())
+    _check(rc, "tq_fused_gemv_host_static")
 
 
 def tq_fused_gemm(m: DeviceMatrix, X: torch.Tensor, Y: torch.Tensor | None = None, stream=None) -> torch.Tensor:

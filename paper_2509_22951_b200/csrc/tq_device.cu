@@ -13,6 +13,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <mutex>
 #include <new>
 
 #include "tq_internal.h"
@@ -716,6 +717,48 @@ int tq_fused_gemv_host(const tq_dmat* m, const void* h_x_bf16, int B, float* h_y
   if (cudaMemcpyAsync(h_y, d_y_stage, (size_t)B * m->info.rows * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return TQ_ERR_CUDA;
   return TQ_OK;
+}
+
+// Staging memory of tq_fused_gemv_host_static: lives in the library image, so every GPU that
+// loads the library holds these 1.5 MiB until the process exits.  Host code cannot use the
+// symbol as a pointer; static_stage() asks the runtime for its address on the current device.
+constexpr uint64_t kStaticXElems = 262144;  // bf16 elements of x the staging area can hold
+constexpr uint64_t kStaticYElems = 262144;  // fp32 elements of y the staging area can hold
+static __device__ __align__(256) unsigned char g_static_stage[kStaticXElems * 2 + kStaticYElems * 4];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mu;
+static unsigned char* g_static_ptr[kMaxDevices] = {};
+
+// Device address of g_static_stage on the current device (looked up once per device).
+static int static_stage(unsigned char** out) {
+  int dev = -1;
+  if (int rc = cuda_ok(cudaGetDevice(&dev), "static staging: current device")) return rc;
+  if (dev < 0 || dev >= kMaxDevices) return TQ_ERR_UNSUPPORTED_SHAPE;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    if (int rc = cuda_ok(cudaGetSymbolAddress(&p, g_static_stage), "static staging: symbol address")) return rc;
+    g_static_ptr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_static_ptr[dev];
+  return TQ_OK;
+}
+
+int tq_fused_gemv_host_static(const tq_dmat* m, const void* h_x_bf16, int B, float* h_y, void* cuda_stream) {
+  if (!m || !h_x_bf16 || !h_y || B < 1 || B > 32) return TQ_ERR_INVALID_ARG;
+  if ((uint64_t)B * m->info.cols > kStaticXElems || (uint64_t)B * m->info.rows > kStaticYElems) {
+    snprintf(g_cuda_msg, sizeof(g_cuda_msg),
+             "tq_fused_gemv_host_static: B*cols = %llu (limit %llu) or B*rows = %llu (limit %llu) exceeds the "
+             "built-in staging area; use tq_fused_gemv_host with caller-provided staging",
+             (unsigned long long)B * m->info.cols, (unsigned long long)kStaticXElems,
+             (unsigned long long)B * m->info.rows, (unsigned long long)kStaticYElems);
+    return TQ_ERR_UNSUPPORTED_SHAPE;
+  }
+  unsigned char* stage = nullptr;
+  if (int rc = static_stage(&stage)) return rc;
+  return tq_fused_gemv_host(m, h_x_bf16, B, h_y, stage, reinterpret_cast<float*>(stage + kStaticXElems * 2),
+                            cuda_stream);
 }
 
 int tq_device_status(const tq_dmat* m, void* cuda_stream, uint32_t* status) {
