@@ -139,7 +139,11 @@ def algorithmic_bytes(info, batch):
         tokens = info.stream_bytes
     else:                  # planes: one 2-byte token per group + one 4-byte word per escaped group
         tokens = 2 * (info.n_hits + info.n_miss) + 4 * info.n_miss
-    return tokens + info.rows * (8 + 4) + 2 * batch * info.cols + 4 * batch * info.rows
+    if info.layout == 2:   # tiles: a 4-byte raw-stream index per tile of 16 rows x 128 columns
+        index = 4 * (-(-info.rows // 16) * -(-info.cols // 128) + 1)
+    else:
+        index = 8 * info.rows
+    return tokens + index + 4 * info.rows + 2 * batch * info.cols + 4 * batch * info.rows
 
 
 def oracle_sample_run(hd_entries, q_host, scales, shapes, batch, sample_idx, reps=1):
@@ -237,7 +241,7 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="decoder layers to build (default: all)")
     ap.add_argument("--no-lm-head", action="store_true")
     ap.add_argument("--shapes", default=None, help="custom workload, e.g. 32768x3072,3072x8192 (profiling cases)")
-    ap.add_argument("--layout", default="planes", choices=["stream", "planes"])
+    ap.add_argument("--layout", default="planes", choices=["stream", "planes", "tiles"])
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -291,7 +295,7 @@ def main():
         dist.broadcast(ent, 0)
         table_entries = ent.cpu().numpy()
 
-    mats, xs, ys, hd, q_host, scales, stats = build_model(tq, shapes, args.batch, device, threads, table_entries, layout=0 if args.layout == "stream" else 1)
+    mats, xs, ys, hd, q_host, scales, stats = build_model(tq, shapes, args.batch, device, threads, table_entries, layout={"stream": 0, "planes": 1, "tiles": 2}[args.layout])
     infos = [m.info for m in mats]
     hits = sum(i.n_hits for i in infos)
     miss = sum(i.n_miss for i in infos)
@@ -417,7 +421,8 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "int8 weights x bf16 activations, fp32 accumulate",
         "data": "synthetic",
         "config": {"workload": workload, "n_weights": n_weights, "hit_rate": hits / (hits + miss), "K": stats["K"],
-                   "layout": "paper token stream, per-row segments" if args.layout == "stream" else "two planes: fixed-stride tokens + packed raw words", "cuda_graph": graph is not None,
+                   "layout": {"stream": "paper token stream, per-row segments", "planes": "two planes: fixed-stride tokens + packed raw words",
+                              "tiles": "1 KB token tiles of 16 rows x 32 groups in integer-MMA operand order + one raw-word stream"}[args.layout], "cuda_graph": graph is not None,
                    "l2": "inputs larger than L2: each step streams %.2f GB" % (payload_bytes / 1e9),
                    "multi_gpu": "independent replicas, no data-path collective" if world > 1 else "single GPU"},
         "us_per_token": ms_step * 1e3 / args.batch,

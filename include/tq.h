@@ -106,7 +106,8 @@ void tq_dict_free(tq_dict* d);
  * Device side: upload, decompress, fused products.
  * ---------------------------------------------------------------------------------------- */
 
-/* Bytes of DEVICE memory a table needs. */
+/* Bytes of DEVICE memory a table needs (always the full 16-bit index range, 256 KB: words past
+ * the last entry are zero, so a kernel may index the table with any token). */
 int tq_dict_upload_size(const tq_dict* d, uint64_t* device_bytes);
 
 /* Copy the table into the caller's DEVICE buffer d_buf (256-byte aligned, d_buf_bytes long) and
@@ -121,6 +122,13 @@ void tq_ddict_free(tq_ddict* d); /* host handle only */
                               fixed-stride plane (code, or 0xFFFF), and the 4 bytes that followed each
                               0xFFFF packed into one word of a second, compact plane.  2 + 4*miss_rate
                               bytes per group instead of 2 + 8*miss_rate, and no sequential parse. */
+
+#define TQ_LAYOUT_TILES 2  /* the PLANES content ordered for the integer tensor-core GEMV: tokens in 1 KB
+                              tiles of 16 rows x 32 groups laid out in the register order of an 8-bit
+                              mma (so a looked-up word is an operand as it stands), raw words in one
+                              stream in the order a warp meets the markers.  Same bytes per group as
+                              PLANES.  tq_decompress and tq_fused_gemv accept it; tq_fused_gemm does not.
+                              Requires cols <= 65536. */
 
 /* Bytes of DEVICE memory the layout of this stream needs.  stream: HOST.  Requires cols % 4 == 0
  * (no aligned group straddles two rows; true of every LLaMA shape), else TQ_ERR_UNSUPPORTED_SHAPE. */
@@ -138,6 +146,17 @@ int tq_upload_size(const uint16_t* stream, uint64_t stream_len, uint32_t rows, u
 int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len, uint32_t rows,
               uint32_t cols, const float* row_scale, const float* row_zero, int levels_signed,
               int layout, void* d_buf, uint64_t d_buf_bytes, void* cuda_stream, tq_dmat** out);
+
+/* The TQ_LAYOUT_TILES image exactly as tq_upload would place it in device memory, built in HOST
+ * memory instead (for inspection, or to prepare images ahead of time).  out == NULL only queries
+ * *out_bytes.  K is the table size the codes are checked against.  offsets[5] receives the byte
+ * offsets of: row scales, row zero points, the tile_raw index (tiles + 1 uint32), the token tiles
+ * (1 KB each), the raw words; dims[2] receives tiles per row block and row blocks.  Tile layout:
+ * see TQ_LAYOUT_TILES; inside a tile, lane l = 4*g + t holds at byte h*512 + l*16 the 8 tokens of
+ * row 16*row_block + g + 8*h, groups 32*step + 8*t .. + 7. */
+int tq_tiles_image_host(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
+                        uint32_t K, const float* row_scale, const float* row_zero, uint8_t* out,
+                        uint64_t out_cap, uint64_t* out_bytes, uint64_t* offsets, uint32_t* dims);
 
 typedef struct tq_dmat_info {
   uint32_t rows, cols, K;

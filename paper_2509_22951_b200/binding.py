@@ -24,6 +24,7 @@ TQ_ERR_TIMEOUT = -6
 TQ_ERR_NOMEM = -7
 TQ_LAYOUT_STREAM = 0
 TQ_LAYOUT_PLANES = 1
+TQ_LAYOUT_TILES = 2
 TQ_STATUS_BAD_CODE = 1
 TQ_STATUS_BAD_ROW = 2
 TQ_STATUS_WAIT_EXPIRED = 4
@@ -32,7 +33,7 @@ EXPORTS = [
     "tq_strerror", "tq_last_cuda_error", "tq_set_num_threads", "tq_quantize_tensor", "tq_quantize_rows",
     "tq_quantize_rows_device", "tq_build_dictionary", "tq_dict_from_entries", "tq_dict_entries",
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
-    "tq_upload_size", "tq_upload", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
+    "tq_upload_size", "tq_upload", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
     "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_device_status", "tq_dmat_free",
 ]
 
@@ -75,6 +76,8 @@ def _load() -> C.CDLL:
         "tq_upload_size": (C.c_int, [u16p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_int, u64p]),
         "tq_upload": (C.c_int, [vp, u16p, C.c_uint64, C.c_uint32, C.c_uint32, f32p, f32p, C.c_int,
                                 C.c_int, vp, C.c_uint64, vp, C.POINTER(vp)]),
+        "tq_tiles_image_host": (C.c_int, [u16p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, f32p, f32p, u8p,
+                                          C.c_uint64, u64p, u64p, u32p]),
         "tq_dmat_get_info": (C.c_int, [vp, C.POINTER(_Info)]),
         "tq_decompress": (C.c_int, [vp, vp, vp]),
         "tq_fused_gemv": (C.c_int, [vp, vp, C.c_int, vp, vp]),
@@ -284,6 +287,26 @@ def tq_upload(ddict: DeviceDict, stream: np.ndarray, rows: int, cols: int, row_s
                               int(levels_signed), layout, buf.data_ptr(), buf.numel(), _stream_ptr(cuda_stream),
                               C.byref(out)), "tq_upload")
     return DeviceMatrix(out.value, buf, ddict)
+
+
+def tq_tiles_image_host(stream: np.ndarray, rows: int, cols: int, K: int, row_scale: np.ndarray, row_zero=None):
+    """-> (image uint8, dict of byte offsets, tiles per row block, row blocks)"""
+    s = np.ascontiguousarray(stream, dtype=np.uint16)
+    sc = np.ascontiguousarray(row_scale, dtype=np.float32)
+    zp = None
+    if row_zero is not None:
+        zr = np.ascontiguousarray(row_zero, dtype=np.float32)
+        zp = _np_ptr(zr, C.c_float)
+    need = C.c_uint64()
+    _check(_lib.tq_tiles_image_host(_np_ptr(s, C.c_uint16), s.size, rows, cols, K, None, None, None, 0,
+                                    C.byref(need), None, None), "tq_tiles_image_host")
+    out = np.zeros(need.value, dtype=np.uint8)
+    offs = (C.c_uint64 * 5)()
+    dims = (C.c_uint32 * 2)()
+    _check(_lib.tq_tiles_image_host(_np_ptr(s, C.c_uint16), s.size, rows, cols, K, _np_ptr(sc, C.c_float), zp,
+                                    _np_ptr(out, C.c_uint8), out.size, C.byref(need), offs, dims), "tq_tiles_image_host")
+    names = ("scale", "zero", "tile_raw", "tokens", "raw")
+    return out, dict(zip(names, (int(o) for o in offs))), int(dims[0]), int(dims[1])
 
 
 def tq_decompress(m: DeviceMatrix, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:

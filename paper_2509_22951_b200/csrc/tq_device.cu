@@ -554,7 +554,9 @@ int tq_quantize_rows_device(const float* d_w, uint32_t rows, uint32_t cols, int8
 
 int tq_dict_upload_size(const tq_dict* d, uint64_t* device_bytes) {
   if (!d || !device_bytes) return TQ_ERR_INVALID_ARG;
-  *device_bytes = (((uint64_t)d->K + 1) * 4 + 255) / 256 * 256 + 256;
+  // always the full 16-bit index range, zero past the last entry: any token is a safe index
+  (void)d;
+  *device_bytes = 65536ull * 4 + 256;
   return TQ_OK;
 }
 
@@ -564,7 +566,7 @@ int tq_dict_upload(const tq_dict* d, void* d_buf, uint64_t d_buf_bytes, void* cu
   tq_dict_upload_size(d, &need);
   if (d_buf_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  if (int rc = cuda_ok(cudaMemsetAsync(d_buf, 0, 256, st), "table upload")) return rc;
+  if (int rc = cuda_ok(cudaMemsetAsync(d_buf, 0, need, st), "table upload")) return rc;
   if (d->K) {
     if (int rc = cuda_ok(cudaMemcpyAsync(static_cast<uint8_t*>(d_buf) + 4, d->entries.data(), (size_t)d->K * 4,
                                          cudaMemcpyHostToDevice, st), "table upload"))
@@ -588,6 +590,8 @@ int tq_upload_size(const uint16_t* stream, uint64_t stream_len, uint32_t rows, u
     return tq_build_stream_image(stream, stream_len, rows, cols, 0xFFFFFFFFu, nullptr, nullptr, device_bytes, nullptr);
   if (layout == TQ_LAYOUT_PLANES)
     return tq_build_planes_image(stream, stream_len, rows, cols, 0xFFFFFFFFu, nullptr, nullptr, device_bytes, nullptr);
+  if (layout == TQ_LAYOUT_TILES)
+    return tq_build_tiles_image(stream, stream_len, rows, cols, 0xFFFFFFFFu, nullptr, nullptr, device_bytes, nullptr);
   return TQ_ERR_INVALID_ARG;
 }
 
@@ -595,7 +599,7 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
               const float* row_scale, const float* row_zero, int levels_signed, int layout, void* d_buf,
               uint64_t d_buf_bytes, void* cuda_stream, tq_dmat** out) {
   if (!dict || !stream || !row_scale || !d_buf || !out || ((uintptr_t)d_buf & 255) ||
-      (layout != TQ_LAYOUT_STREAM && layout != TQ_LAYOUT_PLANES))
+      (layout != TQ_LAYOUT_STREAM && layout != TQ_LAYOUT_PLANES && layout != TQ_LAYOUT_TILES))
     return TQ_ERR_INVALID_ARG;
   if (cols / 4 > 65504u) return TQ_ERR_UNSUPPORTED_SHAPE;  // per-row marker counts are 16-bit
   cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -620,6 +624,32 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
     n_hits = img.n_hits;
     n_miss = img.n_miss;
     m->info.payload_bytes = img.token_chunks * 16 + (uint64_t)rows * (sizeof(tq_rowseg) + 4 + (row_zero ? 4 : 0));
+  } else if (layout == TQ_LAYOUT_TILES) {
+    tq_tiles_image img;
+    rc = tq_build_tiles_image(stream, stream_len, rows, cols, dict->K, row_scale, row_zero, &need, &img);
+    if (rc == TQ_OK && d_buf_bytes < need) rc = TQ_ERR_BUFFER_TOO_SMALL;
+    if (rc == TQ_OK) rc = cuda_ok(cudaMemcpyAsync(d_buf, img.blob.data(), img.blob.size(), cudaMemcpyHostToDevice, st), "upload");
+    if (rc == TQ_OK) rc = cuda_ok(cudaStreamSynchronize(st), "upload");
+    if (rc != TQ_OK) { delete m; return rc; }
+    m->d_status = reinterpret_cast<uint32_t*>(base + img.off_status);
+    m->d_scale = reinterpret_cast<const float*>(base + img.off_scale);
+    m->d_zero = reinterpret_cast<const float*>(base + img.off_zero);
+    tq_tiles_desc& t = m->tiles;
+    t.tokens = reinterpret_cast<const uint4*>(base + img.off_tokens);
+    t.raw = reinterpret_cast<const uint32_t*>(base + img.off_raw);
+    t.tile_raw = reinterpret_cast<const uint32_t*>(base + img.off_tile_raw);
+    t.scale = m->d_scale;
+    t.zero = m->d_zero;
+    t.status = m->d_status;
+    t.rows = rows;
+    t.cols = cols;
+    t.steps = img.steps;
+    t.row_blocks = img.row_blocks;
+    t.has_zero = row_zero != nullptr;
+    n_hits = img.n_hits;
+    n_miss = img.n_miss;
+    const uint64_t n_tiles = (uint64_t)img.steps * img.row_blocks;
+    m->info.payload_bytes = n_tiles * 1024 + n_miss * 4 + (n_tiles + 1) * 4 + (uint64_t)rows * (4 + (row_zero ? 4 : 0));
   } else {
     tq_planes_image img;
     rc = tq_build_planes_image(stream, stream_len, rows, cols, dict->K, row_scale, row_zero, &need, &img);
@@ -667,6 +697,7 @@ int tq_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
   if (!m || !d_codes || ((uintptr_t)d_codes & 15)) return TQ_ERR_INVALID_ARG;
   const uint32_t need = (m->info.rows + kWarpsPerCta - 1) / kWarpsPerCta;
   const uint32_t grid = std::min<uint32_t>(need, (uint32_t)sm_count() * 8u);
+  if (m->info.layout == TQ_LAYOUT_TILES) return tq_tiles_decompress(m, d_codes, cuda_stream);
   if (m->info.layout == TQ_LAYOUT_PLANES) {
     decompress_planes_kernel<<<grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
         m->d_codes, m->gpr_pad, m->d_rawbase, m->d_raw, m->dict->d_table, m->dict->K, m->info.rows, m->info.cols,
@@ -684,6 +715,13 @@ int tq_fused_gemv(const tq_dmat* m, const void* d_x_bf16, int B, float* d_y, voi
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(d_x_bf16);
   const uint32_t rows = m->info.rows, cols = m->info.cols;
+  if (m->info.layout == TQ_LAYOUT_TILES) {  // two batch columns per pass of the integer-MMA kernel
+    for (int b0 = 0; b0 < B; b0 += 2) {
+      if (int rc = tq_tiles_gemv(m, x + (size_t)b0 * cols, std::min(2, B - b0), d_y + (size_t)b0 * rows, cuda_stream))
+        return rc;
+    }
+    return TQ_OK;
+  }
   // fp32 x for up to 4 batch columns must fit the 227 KB of shared memory
   const bool planes = m->info.layout == TQ_LAYOUT_PLANES;
   const size_t xcols = planes ? ((((size_t)m->gpr_pad + 255) >> 8) << 10) : cols;  // staged columns per batch column

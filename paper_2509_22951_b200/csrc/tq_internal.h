@@ -5,6 +5,8 @@
 #include <cstdint>
 #include <vector>
 
+#include <vector_types.h>
+
 #include "tq.h"
 
 struct tq_dict {
@@ -32,6 +34,23 @@ struct tq_rowseg {
   uint32_t n_slots;
 };
 
+// What a kernel needs to know about one matrix in the TILES layout (all pointers DEVICE).
+struct tq_tiles_desc {
+  const uint4* tokens;       // n_tiles x 1 KB token tiles
+  const uint32_t* raw;       // raw words in tile order (512-byte aligned, readable 16 KB past the end)
+  const uint32_t* tile_raw;  // n_tiles + 1: index of each tile's first raw word
+  const float* scale;        // rows
+  const float* zero;         // rows (valid when has_zero)
+  uint32_t* status;
+  const void* x;             // bf16 [B][cols]
+  float* y;                  // fp32 [B][rows]
+  uint32_t rows, cols;
+  uint32_t steps;            // tiles per row block = ceil(cols / 128)
+  uint32_t row_blocks;       // ceil(rows / 16)
+  uint32_t has_zero;
+  uint32_t pad_;
+};
+
 struct tq_dmat {
   tq_dmat_info info{};
   const tq_ddict* dict = nullptr;
@@ -48,6 +67,8 @@ struct tq_dmat {
   const uint16_t* d_codes = nullptr;   // DEVICE: rows x gpr_pad tokens
   const uint32_t* d_raw = nullptr;     // DEVICE: raw words
   uint32_t gpr_pad = 0, nidx_pad = 0;
+  // TILES layout
+  tq_tiles_desc tiles{};
 };
 
 // Host-side image of a matrix in the STREAM layout, ready for one cudaMemcpy.
@@ -65,6 +86,13 @@ struct tq_planes_image {
   uint64_t n_hits = 0, n_miss = 0;
 };
 
+struct tq_tiles_image {
+  std::vector<uint8_t> blob;
+  uint64_t off_status = 0, off_scale = 0, off_zero = 0, off_tile_raw = 0, off_tokens = 0, off_raw = 0;
+  uint32_t steps = 0, row_blocks = 0;
+  uint64_t n_hits = 0, n_miss = 0;
+};
+
 int tq_num_threads();
 
 // Maps a cudaError_t (passed as int) to TQ_OK / TQ_ERR_CUDA and records its text for tq_last_cuda_error.
@@ -75,6 +103,13 @@ int tq_cuda_status(int cuda_error, const char* what);
 int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
                           uint32_t K, const float* row_scale, const float* row_zero,
                           uint64_t* device_bytes, tq_host_image* img);
+int tq_build_tiles_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
+                         uint32_t K, const float* row_scale, const float* row_zero,
+                         uint64_t* device_bytes, tq_tiles_image* img);
 int tq_build_planes_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
                           uint32_t K, const float* row_scale, const float* row_zero,
                           uint64_t* device_bytes, tq_planes_image* img);
+
+// TILES layout entry points (tq_tiles.cu).  x: bf16 [nb][cols], nb in 1..2; y: fp32 [nb][rows].
+int tq_tiles_gemv(const tq_dmat* m, const void* x, int nb, float* y, void* cuda_stream);
+int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream);

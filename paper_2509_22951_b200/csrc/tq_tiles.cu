@@ -1,0 +1,616 @@
+// Kernels of the TILES layout (sm_100a): fused decode + GEMV on the 8-bit integer tensor-core
+// path, and decompress.
+//
+// Why integer MMAs for a matrix-vector product.  A decoded group is a 32-bit word holding four
+// 8-bit levels of one row -- exactly one A-operand register of mma.m16n8k32 (16 rows x 32 columns
+// of 8-bit values, 32-bit accumulators).  A warp that owns 16 rows therefore feeds every word it
+// looks up to the tensor core as is: no unpacking, no int->float conversion, no FMA chain.  The
+// activations take the B operand.  A bf16 activation vector is turned, once per CTA, into a
+// block-fixed-point integer X[c] = round(x[c] * 2^(22-e)) (2^e > max |x|, so |X| <= 2^22) and
+// split into three balanced base-256 digits X = d0 + 256 d1 + 65536 d2, each a signed byte; the
+// three digit vectors are three of the eight B columns.  All sums are exact integers, so
+//   y[r] = scale_r * ( 2^(e-22) * (D0 + 256 D1 + 65536 D2) - zero_r * 2^(e-22) * sum_c X[c] )
+// differs from the exact product only by the rounding of x to 22 bits below its largest element
+// (bf16 carries 8), far inside the fp32-accumulation tolerance, and is independent of how the
+// columns are split among warps.  Two batch columns fit one MMA (6 of 8 B columns).
+//
+// Data movement.  One persistent CTA per SM keeps the first KS words of the table in shared
+// memory (lookups there are bank-conflict limited, not tag limited like divergent global loads);
+// codes >= KS are read from the full table in global memory.  Each warp walks a contiguous run of
+// tiles: token tiles come through registers three tiles ahead; raw words come through a per-warp
+// ring in shared memory that a single lane keeps filled with 512-byte bulk copies
+// (cp.async.bulk + mbarrier), so neither stream sits on the dependent path.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+
+#include "tq_internal.h"
+
+namespace {
+
+constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kChunkWords = 128;                    // one bulk copy: 512 bytes of raw words
+constexpr int kSlots = 8;                           // chunks per ring
+constexpr int kRingWords = kChunkWords * kSlots;    // 4 KB per warp
+constexpr int kPrefetch = 3;                        // token tiles in flight per warp
+constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr uint32_t kNoBlock = 0xFFFFFFFFu;
+
+__host__ __device__ inline uint32_t align_up_u32(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
+
+// Shared-memory plan, identical on host and device.
+struct TilesSmem {
+  uint32_t ring, x, bar, part, stage, misc, total;
+};
+__host__ __device__ inline TilesSmem tiles_smem(uint32_t KS, uint32_t x_words, int warps) {
+  TilesSmem L;
+  L.ring = align_up_u32(KS * 4u, 4096u);  // rings start on a multiple of their size from the table base
+  L.x = L.ring + (uint32_t)warps * kRingWords * 4u;
+  L.bar = align_up_u32(L.x + x_words * 4u, 16u);
+  L.part = L.bar + (uint32_t)warps * kSlots * 8u;
+  L.stage = L.part + 2u * warps * 512u;
+  L.misc = L.stage + (uint32_t)warps * 512u;
+  L.total = L.misc + 512u;
+  return L;
+}
+
+struct TilesSeg {
+  uint32_t mat, rb_begin, rb_end;
+};
+
+struct TilesParams {
+  const tq_tiles_desc* mats;  // stack mode: DEVICE array; nullptr in single-matrix mode
+  const TilesSeg* segs;       // stack mode: segments, grouped by CTA
+  const uint32_t* cta_seg;    // stack mode: gridDim.x + 1 offsets into segs
+  tq_tiles_desc one;          // single-matrix mode
+  const uint32_t* table;      // 65536 words, zero past the last entry
+  uint32_t KS;                // table words kept in shared memory (multiple of 1024)
+  uint32_t xstride;           // words per digit column in shared memory
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+// One decoded word: from the table in shared memory (code < KS), from the warp's raw ring (marker;
+// `cursor` is the lane's next raw word and moves on), or from the table in global memory.
+__device__ __forceinline__ uint32_t lookup(uint32_t tk, uint32_t& cursor, uint32_t tbl_addr, uint32_t ring_idx,
+                                           uint32_t KS, const uint32_t* __restrict__ gtable) {
+  const bool mk = tk == 0xFFFFu;
+  const uint32_t idx = mk ? (ring_idx | (cursor & (kRingWords - 1u))) : tk;
+  cursor += mk ? 1u : 0u;
+  const uint32_t far = (tk >= KS && !mk) ? 1u : 0u;
+  uint32_t w;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.u32 p, %1, 0;\n\t"
+      "@p ld.global.nc.u32 %0, [%2];\n\t"
+      "@!p ld.shared.u32 %0, [%3];\n\t}"
+      : "=r"(w)
+      : "r"(far), "l"(gtable + tk), "r"(tbl_addr + idx * 4u));
+  return w;
+}
+
+template <bool SIGNED>
+__device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                       uint32_t b1) {
+  if (SIGNED) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  } else {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  }
+}
+
+// Per-CTA values of the activation vectors of the current segment.
+struct XInfo {
+  double out_scale[2];  // 2^(e-22), NaN for a vector with a non-finite element
+  double sum_x[2];      // out_scale * sum_c X[c]
+};
+
+template <int W, int NB, bool SIGNED>
+struct TilesCta {
+  static constexpr int kThreads = W * 32;
+  static constexpr int NCOL = 3 * NB;
+
+  uint8_t* smem;
+  TilesSmem L;
+  uint32_t tbl_addr;
+  uint32_t KS, xstride;
+  const uint32_t* gtable;
+  uint32_t warp, lane;
+  uint32_t phase = 0;  // parity bit of each of this warp's ring barriers
+  bool dead = false;
+
+  __device__ __forceinline__ uint32_t* misc_u32() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
+  // misc: [0] dead flag, [1..2] amax bits per vector, [4..4+2W) partial ids, then 8-byte aligned XInfo and
+  // reduction scratch
+  __device__ __forceinline__ volatile uint32_t* dead_flag() { return misc_u32(); }
+  __device__ __forceinline__ uint32_t* part_ids() { return misc_u32() + 4; }
+  __device__ __forceinline__ XInfo* xinfo() { return reinterpret_cast<XInfo*>(smem + L.misc + 192); }
+  __device__ __forceinline__ long long* sum_scratch() { return reinterpret_cast<long long*>(smem + L.misc + 256); }
+
+  __device__ __forceinline__ uint32_t bar_addr(uint32_t slot) { return tbl_addr + L.bar + (warp * kSlots + slot) * 8u; }
+
+  // ---- activation vectors -> digit columns in shared memory --------------------------------
+  __device__ void prepare_x(const tq_tiles_desc& d) {
+    const uint32_t tid = threadIdx.x;
+    const uint32_t G = d.cols >> 2;
+    uint32_t* xs = reinterpret_cast<uint32_t*>(smem + L.x);
+    const uint2* xg = reinterpret_cast<const uint2*>(d.x);
+    if (tid < 2) misc_u32()[1 + tid] = 0u;
+    if (tid < 2 * NB) sum_scratch()[tid] = 0;
+    __syncthreads();
+    // largest magnitude, on the bf16 bit patterns (monotonic; Inf and NaN sort last)
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      uint32_t m = 0;
+      for (uint32_t g = tid; g < G; g += kThreads) {
+        const uint2 v = __ldg(xg + (size_t)b * G + g);
+        const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu;
+        m = max(max(m, a0 & 0xFFFFu), max(a0 >> 16, max(a1 & 0xFFFFu, a1 >> 16)));
+      }
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) m = max(m, __shfl_xor_sync(kFull, m, s));
+      if (lane == 0) atomicMax(&misc_u32()[1 + b], m);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      const uint32_t mb = misc_u32()[1 + b];
+      const bool finite = mb < 0x7F80u;
+      int e = (int)(mb >> 7) - 126;  // max |x| < 2^e
+      e = max(e, -100);
+      const float in_scale = __uint_as_float((uint32_t)(127 + 22 - e) << 23);  // 2^(22-e), e in [-100, 128]
+      long long sum = 0;
+      for (uint32_t g = tid; g < G; g += kThreads) {
+        const uint2 v = __ldg(xg + (size_t)b * G + g);
+        const uint32_t h[4] = {v.x << 16, v.x & 0xFFFF0000u, v.y << 16, v.y & 0xFFFF0000u};
+        uint32_t w0 = 0, w1 = 0, w2 = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          int X = finite ? __float2int_rn(__uint_as_float(h[i]) * in_scale) : 0;
+          sum += X;
+          const int d0 = (int)(signed char)(X & 0xFF);
+          X = (X - d0) >> 8;
+          const int d1 = (int)(signed char)(X & 0xFF);
+          const int d2 = (X - d1) >> 8;
+          w0 |= (uint32_t)(d0 & 0xFF) << (8 * i);
+          w1 |= (uint32_t)(d1 & 0xFF) << (8 * i);
+          w2 |= (uint32_t)(d2 & 0xFF) << (8 * i);
+        }
+        xs[(3 * b + 0) * xstride + g] = w0;
+        xs[(3 * b + 1) * xstride + g] = w1;
+        xs[(3 * b + 2) * xstride + g] = w2;
+      }
+      if (d.has_zero) {
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) sum += __shfl_xor_sync(kFull, sum, s);
+        if (lane == 0) atomicAdd(reinterpret_cast<unsigned long long*>(&sum_scratch()[b]), (unsigned long long)sum);
+      }
+      if (tid == 0) {
+        // 2^(e-22) as a double, built from its exponent field
+        const double os = __longlong_as_double((long long)(1023 + e - 22) << 52);
+        xinfo()->out_scale[b] = finite ? os : __longlong_as_double(0x7FF8000000000000ll);
+      }
+    }
+    __syncthreads();
+    if (tid < NB) xinfo()->sum_x[tid] = xinfo()->out_scale[tid] * (double)sum_scratch()[tid];
+    // digit words of the groups between G and the end of the last tile are never initialised: they
+    // only ever multiply the zero bytes that token 0 decodes to, and integers have no NaN.
+  }
+
+  // ---- results ----------------------------------------------------------------------------
+  // Turns the 16 x 8 accumulator tile (MMA fragment layout) of row block rb into y.
+  __device__ __forceinline__ void finalize(const tq_tiles_desc& d, uint32_t rb, const int (&c)[4]) {
+    int* st = reinterpret_cast<int*>(smem + L.stage + warp * 512u);
+    const uint32_t g = lane >> 2, t = lane & 3u;
+    st[g * 8 + 2 * t] = c[0];
+    st[g * 8 + 2 * t + 1] = c[1];
+    st[(g + 8) * 8 + 2 * t] = c[2];
+    st[(g + 8) * 8 + 2 * t + 1] = c[3];
+    __syncwarp();
+    const uint32_t row = lane & 15u, b = lane >> 4;
+    const uint32_t r = rb * 16u + row;
+    if (b < (uint32_t)NB && r < d.rows) {
+      const long long Y = (long long)st[row * 8 + 3 * b] + 256ll * st[row * 8 + 3 * b + 1] +
+                          65536ll * st[row * 8 + 3 * b + 2];
+      const XInfo* xi = xinfo();
+      double v = (double)Y * xi->out_scale[b];
+      if (d.has_zero) v -= (double)d.zero[r] * xi->sum_x[b];
+      d.y[(size_t)b * d.rows + r] = (float)((double)d.scale[r] * v);
+    }
+    __syncwarp();
+  }
+
+  __device__ __forceinline__ void store_partial(uint32_t slot, uint32_t rb, const int (&c)[4]) {
+    int4* p = reinterpret_cast<int4*>(smem + L.part + (2u * warp + slot) * 512u);
+    p[lane] = make_int4(c[0], c[1], c[2], c[3]);
+    if (lane == 0) part_ids()[2 * warp + slot] = rb;
+  }
+
+  // ---- raw ring ---------------------------------------------------------------------------
+  __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t chunk) {
+    if (lane == 0) {
+      const uint32_t slot = chunk & (kSlots - 1u);
+      const uint32_t bar = bar_addr(slot);
+      mbar_expect_tx(bar, kChunkWords * 4u);
+      bulk_g2s(tbl_addr + L.ring + (warp * kRingWords + slot * kChunkWords) * 4u, raw + (size_t)chunk * kChunkWords,
+               kChunkWords * 4u, bar);
+    }
+  }
+  __device__ __forceinline__ bool wait_chunk(uint32_t chunk) {
+    const uint32_t slot = chunk & (kSlots - 1u);
+    const uint32_t bar = bar_addr(slot);
+    const uint32_t par = (phase >> slot) & 1u;
+    bool ok = mbar_try(bar, par);
+    if (!ok) {  // bounded both in attempts and in time (about 2 s)
+      const uint64_t t_start = global_ns();
+      for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try(bar, par)) { ok = true; break; }
+        if ((i & 63u) == 63u && (*dead_flag() || global_ns() - t_start > 2000000000ull)) break;
+      }
+    }
+    ok = __all_sync(kFull, ok);
+    phase ^= 1u << slot;
+    return ok;
+  }
+
+  // ---- one warp, tiles [t0, t1) of matrix d -------------------------------------------------
+  __device__ void run_tiles(const tq_tiles_desc& d, uint32_t t0, uint32_t t1) {
+    const uint32_t S = d.steps;
+    const uint32_t g = lane >> 2, t = lane & 3u;
+    const uint32_t ring_idx = (L.ring >> 2) + warp * kRingWords;
+    const uint32_t* xs = reinterpret_cast<const uint32_t*>(smem + L.x);
+    const bool has_b = g < (uint32_t)NCOL;
+    const uint32_t x_lane = g * xstride + 8u * t;
+
+    uint32_t rd = __ldg(d.tile_raw + t0);
+    const uint32_t rd_end = __ldg(d.tile_raw + t1);
+    uint32_t c_issue = rd / kChunkWords, c_wait = c_issue;
+    const uint32_t c_stop = rd_end > rd ? (rd_end - 1u) / kChunkWords + 1u : c_issue;  // one past the last chunk needed
+    for (int k = 0; k < kSlots && c_issue < c_stop; ++k) issue_chunk(d.raw, c_issue++);
+
+    uint4 q[kPrefetch][2];
+#pragma unroll
+    for (int k = 0; k < kPrefetch; ++k) {
+      q[k][0] = ldg_stream(d.tokens + (size_t)(t0 + k) * 64u + lane);
+      q[k][1] = ldg_stream(d.tokens + (size_t)(t0 + k) * 64u + 32u + lane);
+    }
+
+    uint32_t s = t0 % S, rb = t0 / S;
+    bool from_start = s == 0;
+    bool used_first = false;
+    int acc[4] = {0, 0, 0, 0};
+    uint32_t wc[16] = {};
+    bool pending = false;
+    uint32_t pend_s = 0;
+
+    auto consume = [&]() {
+      uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = xa;
+      if (has_b) {
+        const uint4* xp = reinterpret_cast<const uint4*>(xs + x_lane + 32u * pend_s);
+        xa = xp[0];
+        xb = xp[1];
+      }
+      mma_s8<SIGNED>(acc, wc[0], wc[8], wc[1], wc[9], xa.x, xa.y);
+      mma_s8<SIGNED>(acc, wc[2], wc[10], wc[3], wc[11], xa.z, xa.w);
+      mma_s8<SIGNED>(acc, wc[4], wc[12], wc[5], wc[13], xb.x, xb.y);
+      mma_s8<SIGNED>(acc, wc[6], wc[14], wc[7], wc[15], xb.z, xb.w);
+      if (pend_s == S - 1u) {
+        if (from_start) {
+          finalize(d, rb, acc);
+        } else {
+          store_partial(0, rb, acc);
+          used_first = true;
+        }
+        acc[0] = acc[1] = acc[2] = acc[3] = 0;
+        from_start = true;
+        ++rb;
+      }
+    };
+
+    for (uint32_t tile = t0; tile < t1; ++tile) {
+      const uint4 ca = q[0][0], cb = q[0][1];
+#pragma unroll
+      for (int k = 0; k + 1 < kPrefetch; ++k) {
+        q[k][0] = q[k + 1][0];
+        q[k][1] = q[k + 1][1];
+      }
+      q[kPrefetch - 1][0] = ldg_stream(d.tokens + (size_t)(tile + kPrefetch) * 64u + lane);
+      q[kPrefetch - 1][1] = ldg_stream(d.tokens + (size_t)(tile + kPrefetch) * 64u + 32u + lane);
+
+      const uint32_t R[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+      uint32_t tk[16];
+      uint32_t n = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        tk[2 * k] = R[k] & 0xFFFFu;
+        tk[2 * k + 1] = R[k] >> 16;
+        n += (tk[2 * k] == 0xFFFFu) + (tk[2 * k + 1] == 0xFFFFu);
+      }
+      uint32_t incl = n;
+#pragma unroll
+      for (int sft = 1; sft < 32; sft <<= 1) {
+        const uint32_t v = __shfl_up_sync(kFull, incl, sft);
+        if (lane >= (uint32_t)sft) incl += v;
+      }
+      const uint32_t total = __shfl_sync(kFull, incl, 31);
+      uint32_t cursor = rd + incl - n;
+      rd += total;
+      // the chunks holding this tile's raw words
+      const uint32_t c_need = total ? (rd - 1u) / kChunkWords + 1u : c_wait;
+      while (c_wait < c_need) {
+        if (!wait_chunk(c_wait)) { dead = true; break; }
+        ++c_wait;
+      }
+      if (dead) break;
+
+      uint32_t wn[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) wn[j] = lookup(tk[j], cursor, tbl_addr, ring_idx, KS, gtable);
+
+      if (pending) consume();
+#pragma unroll
+      for (int j = 0; j < 16; ++j) wc[j] = wn[j];
+      pending = true;
+      pend_s = s;
+      if (++s == S) s = 0;
+
+      // every lane has finished reading the chunks below rd (the MMAs above consumed the previous
+      // tile's words; this tile's loads are ordered before the refill by the warp barrier)
+      __syncwarp();
+      const uint32_t c_free = rd / kChunkWords;  // chunks below this index are fully consumed
+      while (c_issue < c_stop && c_issue < c_free + kSlots) issue_chunk(d.raw, c_issue++);
+    }
+    if (pending && !dead) {
+      consume();
+      if (pend_s != S - 1u) {  // the run ended inside a row block
+        if (!from_start && !used_first) store_partial(0, rb, acc);
+        else store_partial(1, rb, acc);
+      }
+    }
+    if (dead) {
+      *dead_flag() = 1u;
+      if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
+    } else {
+      while (c_wait < c_issue) {  // nothing may still be landing when the ring is reused
+        if (!wait_chunk(c_wait)) { dead = true; *dead_flag() = 1u; break; }
+        ++c_wait;
+      }
+    }
+  }
+
+  // ---- one segment: row blocks [rb0, rb1) of matrix d, all warps ----------------------------
+  __device__ void run_segment(const tq_tiles_desc& d, uint32_t rb0, uint32_t rb1) {
+    __syncthreads();  // the previous segment is done with x, the partials and the staging tiles
+    prepare_x(d);
+    if (lane < 2) part_ids()[2 * warp + lane] = kNoBlock;
+    __syncthreads();
+    const uint64_t T = (uint64_t)(rb1 - rb0) * d.steps;
+    const uint32_t t0 = rb0 * d.steps + (uint32_t)(T * warp / W);
+    const uint32_t t1 = rb0 * d.steps + (uint32_t)(T * (warp + 1) / W);
+    if (t0 < t1 && !dead && !*dead_flag()) run_tiles(d, t0, t1);
+    __syncthreads();
+    // partial row blocks: entries of the same block are adjacent (warp order = tile order)
+    if (warp == 0 && !*dead_flag()) {
+      uint32_t cur = kNoBlock;
+      int sum[4] = {0, 0, 0, 0};
+      for (uint32_t e = 0; e < 2u * W; ++e) {
+        const uint32_t id = part_ids()[e];
+        if (id == kNoBlock) continue;
+        if (id != cur) {
+          if (cur != kNoBlock) finalize(d, cur, sum);
+          cur = id;
+          sum[0] = sum[1] = sum[2] = sum[3] = 0;
+        }
+        const int4 v = reinterpret_cast<const int4*>(smem + L.part + e * 512u)[lane];
+        sum[0] += v.x;
+        sum[1] += v.y;
+        sum[2] += v.z;
+        sum[3] += v.w;
+      }
+      if (cur != kNoBlock) finalize(d, cur, sum);
+    }
+  }
+};
+
+template <int W, int NB, bool SIGNED>
+__global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams p) {
+  extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
+  TilesCta<W, NB, SIGNED> cta;
+  cta.smem = tiles_smem_raw;
+  cta.L = tiles_smem(p.KS, 3u * NB * p.xstride, W);
+  cta.tbl_addr = smem_u32(tiles_smem_raw);
+  cta.KS = p.KS;
+  cta.xstride = p.xstride;
+  cta.gtable = p.table;
+  cta.warp = threadIdx.x >> 5;
+  cta.lane = threadIdx.x & 31u;
+
+  if (threadIdx.x < W * kSlots) mbar_init(cta.tbl_addr + cta.L.bar + threadIdx.x * 8u, 1u);
+  if (threadIdx.x == 0) *cta.dead_flag() = 0u;
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(p.table);
+    uint4* dst = reinterpret_cast<uint4*>(tiles_smem_raw);
+    for (uint32_t i = threadIdx.x; i < p.KS / 4u; i += W * 32) dst[i] = __ldg(src + i);
+  }
+  __syncthreads();
+
+  if (p.mats == nullptr) {
+    const uint32_t nrb = p.one.row_blocks;
+    const uint32_t rb0 = (uint32_t)((uint64_t)nrb * blockIdx.x / gridDim.x);
+    const uint32_t rb1 = (uint32_t)((uint64_t)nrb * (blockIdx.x + 1) / gridDim.x);
+    if (rb0 < rb1) cta.run_segment(p.one, rb0, rb1);
+  } else {
+    for (uint32_t si = p.cta_seg[blockIdx.x]; si < p.cta_seg[blockIdx.x + 1]; ++si) {
+      const TilesSeg sg = p.segs[si];
+      const tq_tiles_desc d = p.mats[sg.mat];
+      cta.run_segment(d, sg.rb_begin, sg.rb_end);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Decompress: one warp per tile, table and raw words read from global memory.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+decompress_tiles_kernel(const tq_tiles_desc d, const uint32_t* __restrict__ table, uint32_t K,
+                        uint32_t* __restrict__ out) {
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
+  const uint32_t n_tiles = d.steps * d.row_blocks;
+  const uint32_t g = lane >> 2, t = lane & 3u;
+  const uint32_t gpr = d.cols >> 2;
+  uint32_t bad = 0;
+  for (uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; tile < n_tiles; tile += warps) {
+    const uint32_t rb = tile / d.steps, s = tile % d.steps;
+    const uint4 a = ldg_stream(d.tokens + (size_t)tile * 64u + lane);
+    const uint4 b = ldg_stream(d.tokens + (size_t)tile * 64u + 32u + lane);
+    const uint32_t R[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t tk[16], n = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      tk[2 * k] = R[k] & 0xFFFFu;
+      tk[2 * k + 1] = R[k] >> 16;
+      n += (tk[2 * k] == 0xFFFFu) + (tk[2 * k + 1] == 0xFFFFu);
+    }
+    uint32_t incl = n;
+#pragma unroll
+    for (int sft = 1; sft < 32; sft <<= 1) {
+      const uint32_t v = __shfl_up_sync(kFull, incl, sft);
+      if (lane >= (uint32_t)sft) incl += v;
+    }
+    const uint32_t* rp = d.raw + __ldg(d.tile_raw + tile) + (incl - n);
+    uint32_t w[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      if (tk[j] == 0xFFFFu) {
+        w[j] = __ldg(rp++);
+      } else {
+        const uint32_t cl = min(tk[j], K);
+        bad |= tk[j] ^ cl;
+        w[j] = __ldg(table + cl);
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint32_t r = rb * 16u + g + 8u * h;
+      const uint32_t g0 = 32u * s + 8u * t;
+      if (r >= d.rows || g0 >= gpr) continue;
+      uint32_t* o = out + (size_t)r * gpr + g0;
+      if (g0 + 8u <= gpr && ((gpr & 3u) == 0u)) {
+        reinterpret_cast<uint4*>(o)[0] = make_uint4(w[8 * h], w[8 * h + 1], w[8 * h + 2], w[8 * h + 3]);
+        reinterpret_cast<uint4*>(o)[1] = make_uint4(w[8 * h + 4], w[8 * h + 5], w[8 * h + 6], w[8 * h + 7]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (g0 + i < gpr) o[i] = w[8 * h + i];
+      }
+    }
+  }
+  if (bad) atomicOr(d.status, TQ_STATUS_BAD_CODE);
+}
+
+int sm_count_tiles() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  return n;
+}
+
+constexpr int kTilesWarps = 8;
+constexpr uint32_t kSmemLimit = 232448u;  // 227 KB per CTA
+
+// Largest table prefix (multiple of 1024 words) that fits beside everything else.
+uint32_t pick_ks(uint32_t x_words, int warps, uint32_t K) {
+  const TilesSmem fixed = tiles_smem(0, x_words, warps);
+  if (fixed.total > kSmemLimit) return 0xFFFFFFFFu;
+  uint32_t ks = (kSmemLimit - fixed.total) / 4096u * 1024u;
+  ks = std::min<uint32_t>(ks, 65536u);
+  ks = std::min<uint32_t>(ks, align_up_u32(K + 1u, 1024u));
+  return ks;
+}
+
+template <int NB, bool SIGNED>
+int launch_tiles(const TilesParams& p, uint32_t grid, size_t smem, cudaStream_t st) {
+  auto kern = gemv_tiles_kernel<kTilesWarps, NB, SIGNED>;
+  static size_t configured = 0;
+  if (smem > configured) {
+    if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+                                "gemv(tiles): raising the dynamic shared memory limit"))
+      return rc;
+    configured = smem;
+  }
+  kern<<<grid, kTilesWarps * 32, smem, st>>>(p);
+  return tq_cuda_status((int)cudaGetLastError(), "gemv(tiles) launch");
+}
+
+}  // namespace
+
+// x: bf16 [nb][cols], y: fp32 [nb][rows], nb in 1..2.
+int tq_tiles_gemv(const tq_dmat* m, const void* x, int nb, float* y, void* cuda_stream) {
+  TilesParams p{};
+  p.one = m->tiles;
+  p.one.x = x;
+  p.one.y = y;
+  p.table = m->dict->d_table;
+  p.xstride = m->tiles.steps * 32u + 4u;
+  p.KS = pick_ks(3u * nb * p.xstride, kTilesWarps, m->dict->K);
+  if (p.KS == 0xFFFFFFFFu) return TQ_ERR_UNSUPPORTED_SHAPE;
+  const TilesSmem L = tiles_smem(p.KS, 3u * nb * p.xstride, kTilesWarps);
+  const uint32_t grid = std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count_tiles());
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const bool sg = m->info.levels_signed != 0;
+  if (nb == 1) return sg ? launch_tiles<1, true>(p, grid, L.total, st) : launch_tiles<1, false>(p, grid, L.total, st);
+  return sg ? launch_tiles<2, true>(p, grid, L.total, st) : launch_tiles<2, false>(p, grid, L.total, st);
+}
+
+int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
+  const uint32_t n_tiles = m->tiles.steps * m->tiles.row_blocks;
+  const uint32_t grid = std::min<uint32_t>((n_tiles + 7u) / 8u, (uint32_t)sm_count_tiles() * 8u);
+  decompress_tiles_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(m->tiles, m->dict->d_table, m->dict->K,
+                                                                       reinterpret_cast<uint32_t*>(d_codes));
+  return tq_cuda_status((int)cudaGetLastError(), "decompress(tiles) launch");
+}

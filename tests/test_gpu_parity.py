@@ -18,10 +18,10 @@ def tq():
     return binding
 
 
-LAYOUTS = [0, 1]  # TQ_LAYOUT_STREAM, TQ_LAYOUT_PLANES
+LAYOUTS = [0, 1, 2]  # TQ_LAYOUT_STREAM, TQ_LAYOUT_PLANES, TQ_LAYOUT_TILES
 
 
-@pytest.fixture(params=LAYOUTS, ids=["stream", "planes"])
+@pytest.fixture(params=LAYOUTS, ids=["stream", "planes", "tiles"])
 def layout(request):
     return request.param
 

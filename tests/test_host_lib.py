@@ -185,3 +185,50 @@ def _rank_main(rank, world):
         assert cover[0][0] == 0 and cover[-1][1] == rows and all(a[1] == b[0] for a, b in zip(cover, cover[1:]))
     finally:
         dist.destroy_process_group()
+
+
+def _decode_tiles_image(img, offs, steps, row_blocks, rows, cols, entries):
+    """Walks a TQ_LAYOUT_TILES image the way the layout is documented and returns the levels."""
+    n_tiles = steps * row_blocks
+    tile_raw = img[offs["tile_raw"]:offs["tile_raw"] + 4 * (n_tiles + 1)].view(np.uint32)
+    tokens = img[offs["tokens"]:offs["tokens"] + 1024 * n_tiles].view(np.uint16).reshape(n_tiles, 2, 32, 8)
+    raw = img[offs["raw"]:].view(np.uint32)
+    table = np.zeros((65536, 4), dtype=np.uint8)
+    table[1:1 + len(entries)] = entries
+    out = np.zeros((row_blocks * 16, steps * 128), dtype=np.uint8)
+    for tile in range(n_tiles):
+        rb, s = divmod(tile, steps)
+        nxt = int(tile_raw[tile])
+        for lane in range(32):
+            g, t = lane >> 2, lane & 3
+            for h in range(2):
+                for i in range(8):
+                    tk = int(tokens[tile, h, lane, i])
+                    if tk == 0xFFFF:
+                        w = np.array([raw[nxt]], dtype=np.uint32).view(np.uint8)
+                        nxt += 1
+                    else:
+                        w = table[tk]
+                    c0 = 4 * (32 * s + 8 * t + i)
+                    out[rb * 16 + g + 8 * h, c0:c0 + 4] = w
+        assert nxt == int(tile_raw[tile + 1])
+    assert not out[rows:].any() and not out[:, cols:].any()  # padding decodes to zeros
+    return out[:rows, :cols]
+
+
+@pytest.mark.parametrize("rows,cols,top_k", [(16, 128, 50), (37, 516, 300), (5, 4, 10), (48, 1280, 0), (33, 260, 65535)])
+def test_tiles_image_decodes_to_the_original_levels(rows, cols, top_k):
+    rng = np.random.default_rng(rows * 7 + cols)
+    q = np.clip(np.rint(rng.standard_t(5, size=(rows, cols)) * 3), -127, 127).astype(np.int8)
+    d = oracle.Dictionary.build([q], top_k=top_k)
+    stream = d.encode(q)[0]
+    s = (rng.random(rows) + 0.5).astype(np.float32)
+    z = rng.integers(0, 9, rows).astype(np.float32)
+    img, offs, steps, row_blocks = tq.tq_tiles_image_host(stream, rows, cols, d.K, s, z)
+    assert steps == -(-cols // 128) and row_blocks == -(-rows // 16)
+    got = _decode_tiles_image(img, offs, steps, row_blocks, rows, cols, d.entries)
+    assert np.array_equal(got, q.view(np.uint8))
+    assert np.array_equal(img[offs["scale"]:offs["scale"] + 4 * rows].view(np.float32), s)
+    assert np.array_equal(img[offs["zero"]:offs["zero"] + 4 * rows].view(np.float32), z)
+    n_miss = int(np.count_nonzero(stream == 0xFFFF))
+    assert int(img[offs["tile_raw"]:].view(np.uint32)[steps * row_blocks]) == n_miss
