@@ -126,9 +126,17 @@ void tq_ddict_free(tq_ddict* d); /* host handle only */
 #define TQ_LAYOUT_TILES 2  /* the PLANES content ordered for the integer tensor-core GEMV: tokens in 1 KB
                               tiles of 16 rows x 32 groups laid out in the register order of an 8-bit
                               mma (so a looked-up word is an operand as it stands), raw words in one
-                              stream in the order a warp meets the markers.  Same bytes per group as
+                              stream, each addressed by the token that replaces its marker.  Same bytes per group as
                               PLANES.  tq_decompress and tq_fused_gemv accept it; tq_fused_gemm does not.
-                              Requires cols <= 65536. */
+                              Requires cols <= TQ_TILES_MAX_COLS.  The kernels hold the table they index in shared
+                              memory, which has room for TQ_TILES_TABLE_WORDS words: a group whose code is
+                              beyond that is stored as Listing 3 stores a group that is not in the table
+                              (marker + its 4 bytes), i.e. the image is the stream Listing 3 produces with
+                              top_k = TQ_TILES_TABLE_WORDS - 1.  Same decoded bytes, 4 more bytes per such
+                              group (tq_dmat_info.n_raw_words counts them). */
+#define TQ_TILES_TABLE_WORDS 43008u
+#define TQ_TILES_MAX_COLS 8704u /* table + one activation vector as 3 digit bytes per column must fit 227 KB */
+#define TQ_TILES_RING_WORDS 1024u /* a miss token of the image is 0xFC00 + (index of its raw word mod 1024) */
 
 /* Bytes of DEVICE memory the layout of this stream needs.  stream: HOST.  Requires cols % 4 == 0
  * (no aligned group straddles two rows; true of every LLaMA shape), else TQ_ERR_UNSUPPORTED_SHAPE. */
@@ -149,13 +157,13 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
 
 /* The TQ_LAYOUT_TILES image exactly as tq_upload would place it in device memory, built in HOST
  * memory instead (for inspection, or to prepare images ahead of time).  out == NULL only queries
- * *out_bytes.  K is the table size the codes are checked against.  offsets[5] receives the byte
- * offsets of: row scales, row zero points, the tile_raw index (tiles + 1 uint32), the token tiles
- * (1 KB each), the raw words; dims[2] receives tiles per row block and row blocks.  Tile layout:
- * see TQ_LAYOUT_TILES; inside a tile, lane l = 4*g + t holds at byte h*512 + l*16 the 8 tokens of
- * row 16*row_block + g + 8*h, groups 32*step + 8*t .. + 7. */
-int tq_tiles_image_host(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
-                        uint32_t K, const float* row_scale, const float* row_zero, uint8_t* out,
+ * *out_bytes.  offsets[5] receives the byte offsets of: row scales, row zero points, the tile_raw
+ * index (tiles + 1 uint32), the token tiles (1 KB each), the raw words; dims[2] receives tiles per
+ * row block and row blocks.  Tile layout: see TQ_LAYOUT_TILES; inside a tile, lane l = 4*g + t
+ * holds at byte h*512 + l*16 the 8 tokens of row 16*row_block + g + 8*h, groups
+ * 32*step + 8*t .. + 7. */
+int tq_tiles_image_host(const tq_dict* d, const uint16_t* stream, uint64_t stream_len, uint32_t rows,
+                        uint32_t cols, const float* row_scale, const float* row_zero, uint8_t* out,
                         uint64_t out_cap, uint64_t* out_bytes, uint64_t* offsets, uint32_t* dims);
 
 typedef struct tq_dmat_info {
@@ -166,6 +174,8 @@ typedef struct tq_dmat_info {
   uint64_t payload_bytes;    /* bytes a kernel reads per pass: token segments with their
                                 padding + per-row index + scales                              */
   uint64_t device_bytes;     /* whole footprint in the caller's buffer                         */
+  uint64_t n_raw_words;      /* 4-byte raw words in the device layout: n_miss, plus for
+                                TQ_LAYOUT_TILES the groups coded beyond TQ_TILES_TABLE_WORDS     */
 } tq_dmat_info;
 int tq_dmat_get_info(const tq_dmat* m, tq_dmat_info* info);
 

@@ -25,6 +25,8 @@ TQ_ERR_NOMEM = -7
 TQ_LAYOUT_STREAM = 0
 TQ_LAYOUT_PLANES = 1
 TQ_LAYOUT_TILES = 2
+TQ_TILES_TABLE_WORDS = 43008
+TQ_TILES_MAX_COLS = 8704
 TQ_STATUS_BAD_CODE = 1
 TQ_STATUS_BAD_ROW = 2
 TQ_STATUS_WAIT_EXPIRED = 4
@@ -50,7 +52,7 @@ class _Info(C.Structure):
     _fields_ = [("rows", C.c_uint32), ("cols", C.c_uint32), ("K", C.c_uint32),
                 ("layout", C.c_int32), ("levels_signed", C.c_int32),
                 ("n_hits", C.c_uint64), ("n_miss", C.c_uint64), ("stream_bytes", C.c_uint64),
-                ("payload_bytes", C.c_uint64), ("device_bytes", C.c_uint64)]
+                ("payload_bytes", C.c_uint64), ("device_bytes", C.c_uint64), ("n_raw_words", C.c_uint64)]
 
 
 def _load() -> C.CDLL:
@@ -76,7 +78,7 @@ def _load() -> C.CDLL:
         "tq_upload_size": (C.c_int, [u16p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_int, u64p]),
         "tq_upload": (C.c_int, [vp, u16p, C.c_uint64, C.c_uint32, C.c_uint32, f32p, f32p, C.c_int,
                                 C.c_int, vp, C.c_uint64, vp, C.POINTER(vp)]),
-        "tq_tiles_image_host": (C.c_int, [u16p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, f32p, f32p, u8p,
+        "tq_tiles_image_host": (C.c_int, [vp, u16p, C.c_uint64, C.c_uint32, C.c_uint32, f32p, f32p, u8p,
                                           C.c_uint64, u64p, u64p, u32p]),
         "tq_dmat_get_info": (C.c_int, [vp, C.POINTER(_Info)]),
         "tq_decompress": (C.c_int, [vp, vp, vp]),
@@ -241,6 +243,7 @@ class MatInfo:
     stream_bytes: int
     payload_bytes: int
     device_bytes: int
+    n_raw_words: int
 
 
 class DeviceMatrix:
@@ -289,7 +292,7 @@ def tq_upload(ddict: DeviceDict, stream: np.ndarray, rows: int, cols: int, row_s
     return DeviceMatrix(out.value, buf, ddict)
 
 
-def tq_tiles_image_host(stream: np.ndarray, rows: int, cols: int, K: int, row_scale: np.ndarray, row_zero=None):
+def tq_tiles_image_host(d: Dict, stream: np.ndarray, rows: int, cols: int, row_scale: np.ndarray, row_zero=None):
     """-> (image uint8, dict of byte offsets, tiles per row block, row blocks)"""
     s = np.ascontiguousarray(stream, dtype=np.uint16)
     sc = np.ascontiguousarray(row_scale, dtype=np.float32)
@@ -298,12 +301,12 @@ def tq_tiles_image_host(stream: np.ndarray, rows: int, cols: int, K: int, row_sc
         zr = np.ascontiguousarray(row_zero, dtype=np.float32)
         zp = _np_ptr(zr, C.c_float)
     need = C.c_uint64()
-    _check(_lib.tq_tiles_image_host(_np_ptr(s, C.c_uint16), s.size, rows, cols, K, None, None, None, 0,
+    _check(_lib.tq_tiles_image_host(d._h, _np_ptr(s, C.c_uint16), s.size, rows, cols, None, None, None, 0,
                                     C.byref(need), None, None), "tq_tiles_image_host")
     out = np.zeros(need.value, dtype=np.uint8)
     offs = (C.c_uint64 * 5)()
     dims = (C.c_uint32 * 2)()
-    _check(_lib.tq_tiles_image_host(_np_ptr(s, C.c_uint16), s.size, rows, cols, K, _np_ptr(sc, C.c_float), zp,
+    _check(_lib.tq_tiles_image_host(d._h, _np_ptr(s, C.c_uint16), s.size, rows, cols, _np_ptr(sc, C.c_float), zp,
                                     _np_ptr(out, C.c_uint8), out.size, C.byref(need), offs, dims), "tq_tiles_image_host")
     names = ("scale", "zero", "tile_raw", "tokens", "raw")
     return out, dict(zip(names, (int(o) for o in offs))), int(dims[0]), int(dims[1])

@@ -13,6 +13,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <cstring>
 #include <mutex>
 #include <new>
 
@@ -577,6 +578,13 @@ int tq_dict_upload(const tq_dict* d, void* d_buf, uint64_t d_buf_bytes, void* cu
   if (!dd) return TQ_ERR_NOMEM;
   dd->K = d->K;
   dd->d_table = static_cast<const uint32_t*>(d_buf);
+  try {
+    dd->h_table.assign((size_t)d->K + 1, 0u);
+  } catch (const std::bad_alloc&) {
+    delete dd;
+    return TQ_ERR_NOMEM;
+  }
+  if (d->K) std::memcpy(dd->h_table.data() + 1, d->entries.data(), (size_t)d->K * 4);
   *out = dd;
   return TQ_OK;
 }
@@ -591,7 +599,7 @@ int tq_upload_size(const uint16_t* stream, uint64_t stream_len, uint32_t rows, u
   if (layout == TQ_LAYOUT_PLANES)
     return tq_build_planes_image(stream, stream_len, rows, cols, 0xFFFFFFFFu, nullptr, nullptr, device_bytes, nullptr);
   if (layout == TQ_LAYOUT_TILES)
-    return tq_build_tiles_image(stream, stream_len, rows, cols, 0xFFFFFFFFu, nullptr, nullptr, device_bytes, nullptr);
+    return tq_build_tiles_image(stream, stream_len, rows, cols, 0xFFFFFFFFu, nullptr, nullptr, nullptr, device_bytes, nullptr);
   return TQ_ERR_INVALID_ARG;
 }
 
@@ -626,7 +634,7 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
     m->info.payload_bytes = img.token_chunks * 16 + (uint64_t)rows * (sizeof(tq_rowseg) + 4 + (row_zero ? 4 : 0));
   } else if (layout == TQ_LAYOUT_TILES) {
     tq_tiles_image img;
-    rc = tq_build_tiles_image(stream, stream_len, rows, cols, dict->K, row_scale, row_zero, &need, &img);
+    rc = tq_build_tiles_image(stream, stream_len, rows, cols, dict->K, dict->h_table.data(), row_scale, row_zero, &need, &img);
     if (rc == TQ_OK && d_buf_bytes < need) rc = TQ_ERR_BUFFER_TOO_SMALL;
     if (rc == TQ_OK) rc = cuda_ok(cudaMemcpyAsync(d_buf, img.blob.data(), img.blob.size(), cudaMemcpyHostToDevice, st), "upload");
     if (rc == TQ_OK) rc = cuda_ok(cudaStreamSynchronize(st), "upload");
@@ -646,10 +654,12 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
     t.steps = img.steps;
     t.row_blocks = img.row_blocks;
     t.has_zero = row_zero != nullptr;
+    t.table_words = TQ_TILES_TABLE_WORDS;
     n_hits = img.n_hits;
     n_miss = img.n_miss;
     const uint64_t n_tiles = (uint64_t)img.steps * img.row_blocks;
-    m->info.payload_bytes = n_tiles * 1024 + n_miss * 4 + (n_tiles + 1) * 4 + (uint64_t)rows * (4 + (row_zero ? 4 : 0));
+    m->info.payload_bytes = n_tiles * 1024 + img.n_raw * 4 + (n_tiles + 1) * 4 + (uint64_t)rows * (4 + (row_zero ? 4 : 0));
+    m->info.n_raw_words = img.n_raw;
   } else {
     tq_planes_image img;
     rc = tq_build_planes_image(stream, stream_len, rows, cols, dict->K, row_scale, row_zero, &need, &img);
@@ -680,6 +690,7 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
   m->info.n_hits = n_hits;
   m->info.n_miss = n_miss;
   m->info.stream_bytes = 2 * (n_hits + 5 * n_miss);
+  if (layout != TQ_LAYOUT_TILES) m->info.n_raw_words = n_miss;
   m->info.device_bytes = need;
   *out = m;
   return TQ_OK;
@@ -715,9 +726,11 @@ int tq_fused_gemv(const tq_dmat* m, const void* d_x_bf16, int B, float* d_y, voi
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(d_x_bf16);
   const uint32_t rows = m->info.rows, cols = m->info.cols;
-  if (m->info.layout == TQ_LAYOUT_TILES) {  // two batch columns per pass of the integer-MMA kernel
-    for (int b0 = 0; b0 < B; b0 += 2) {
-      if (int rc = tq_tiles_gemv(m, x + (size_t)b0 * cols, std::min(2, B - b0), d_y + (size_t)b0 * rows, cuda_stream))
+  if (m->info.layout == TQ_LAYOUT_TILES) {  // up to two batch columns per pass of the integer-MMA kernel
+    const int per_pass = tq_tiles_max_nb(m);
+    if (per_pass < 1) return TQ_ERR_UNSUPPORTED_SHAPE;
+    for (int b0 = 0; b0 < B; b0 += per_pass) {
+      if (int rc = tq_tiles_gemv(m, x + (size_t)b0 * cols, std::min(per_pass, B - b0), d_y + (size_t)b0 * rows, cuda_stream))
         return rc;
     }
     return TQ_OK;

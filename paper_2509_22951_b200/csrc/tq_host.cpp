@@ -695,26 +695,37 @@ int tq_build_planes_image(const uint16_t* stream, uint64_t stream_len, uint32_t 
 }
 
 // ---------------------------------------------------------------------------------------------
-// TILES layout: the same tokens and raw words as PLANES, ordered for a warp that decodes 16 rows
-// at a time straight into the operand registers of an 8-bit tensor-core MMA.  A tile covers a row
-// block of 16 rows and a step of 32 groups (128 columns) and is 1 KB of tokens: lane l = 4*g + t
-// of the warp owns, for h = 0, 1, the 8 tokens of row 16*rb + g + 8*h, groups 32*s + 8*t .. + 7,
-// stored at byte h*512 + l*16 of the tile (one 128-bit load per lane and half).  Tiles are stored
-// row block by row block, step by step.  Rows past the matrix and groups past the row hold token
-// 0, which decodes to four zero bytes.  The 4 raw bytes behind each marker are packed into one
-// word of a single raw stream that follows the order in which the warp meets the markers: tile
-// by tile, inside a tile lane by lane, inside a lane h = 0 before h = 1, group order.  tile_raw[i]
-// is the index of tile i's first raw word, so any tile can be the start of a walk.
+// TILES layout: the content of PLANES, ordered for a warp that decodes 16 rows at a time straight
+// into the operand registers of an 8-bit tensor-core MMA.  A tile covers a row block of 16 rows and
+// a step of 32 groups (128 columns) and is 1 KB of tokens: lane l = 4*g + t of the warp owns, for
+// h = 0, 1, the 8 tokens of row 16*rb + g + 8*h, groups 32*s + 8*t .. + 7, stored at byte
+// h*512 + l*16 of the tile (one 128-bit load per lane and half).  Tiles are stored row block by
+// row block, step by step.  Rows past the matrix and groups past the row hold token 0, which
+// decodes to four zero bytes.  The 4 raw bytes behind each marker are packed into one word of a
+// single raw stream, tile by tile; tile_raw[i] is the index of tile i's first raw word.  In place
+// of the marker 0xFFFF the token of such a group is 0xFC00 + (p mod 1024), p being the index of
+// its raw word in that stream: the kernels stage the stream through a ring of
+// TQ_TILES_RING_WORDS = 1024 words in which word p sits in slot p mod 1024, so the token is the
+// address of its word and no marker counting is needed.  (A tile holds at most 512 raw words, so
+// p is recovered from tile_raw[i] and the token.)
+//
+// The kernels keep the whole table they index in shared memory, which holds TQ_TILES_TABLE_WORDS
+// words.  A group whose code is beyond that is therefore stored the way Listing 3 stores a group
+// that is not in the table -- marker in the token tile, its 4 bytes (taken from the table) in the
+// raw stream -- which is the stream Listing 3 would have produced with top_k =
+// TQ_TILES_TABLE_WORDS - 1, since the table is ranked and a shorter one is a prefix of it.
+// Decoding gives the same bytes; the image is 4 bytes larger per such group.
 // ---------------------------------------------------------------------------------------------
 int tq_build_tiles_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
-                         uint32_t K, const float* row_scale, const float* row_zero,
+                         uint32_t K, const uint32_t* table, const float* row_scale, const float* row_zero,
                          uint64_t* device_bytes, tq_tiles_image* img) {
   std::vector<uint64_t> row_start;
   uint64_t H = 0, M = 0;
   int rc = scan_stream(stream, stream_len, rows, cols, K, row_start, H, M);
   if (rc != TQ_OK) return rc;
   if (M >= (1ull << 32) - 65536) return TQ_ERR_UNSUPPORTED_SHAPE;
-  if (cols > 65536u) return TQ_ERR_UNSUPPORTED_SHAPE;  // 32-bit accumulators of the integer MMA
+  // the activation digits of a whole row (3 bytes per column) share the CTA's shared memory with the table
+  if (cols > TQ_TILES_MAX_COLS) return TQ_ERR_UNSUPPORTED_SHAPE;
 
   const uint32_t gpr = cols / 4;
   const uint32_t steps = (gpr + 31u) / 32u;
@@ -722,18 +733,57 @@ int tq_build_tiles_image(const uint16_t* stream, uint64_t stream_len, uint32_t r
   const uint64_t n_tiles = (uint64_t)steps * row_blocks;
   if (n_tiles >= (1ull << 31)) return TQ_ERR_UNSUPPORTED_SHAPE;
   const uint64_t rows_pad = (uint64_t)row_blocks * 16;
+  const uint32_t limit = TQ_TILES_TABLE_WORDS;
+  const uint32_t miss_base = 0x10000u - TQ_TILES_RING_WORDS;
+  static_assert(TQ_TILES_TABLE_WORDS <= 0x10000u - TQ_TILES_RING_WORDS, "codes and miss tokens must not overlap");
+
+  // pass 1: raw words per tile (markers and codes beyond the shared-memory table)
+  std::vector<uint32_t> tile_raw_v;
+  try {
+    tile_raw_v.assign(n_tiles + 1, 0);
+  } catch (const std::bad_alloc&) {
+    return TQ_ERR_NOMEM;
+  }
+  const int T = (int)std::min<uint64_t>(tq_num_threads(), row_blocks);
+  parallel_run(T, [&](int t) {
+    const uint32_t b0 = (uint32_t)((uint64_t)row_blocks * t / T), b1 = (uint32_t)((uint64_t)row_blocks * (t + 1) / T);
+    for (uint32_t rb = b0; rb < b1; ++rb) {
+      uint32_t* cnt = tile_raw_v.data() + (uint64_t)rb * steps + 1;  // shifted by one: becomes the prefix sum below
+      for (uint32_t i = 0; i < 16; ++i) {
+        const uint32_t r = rb * 16 + i;
+        if (r >= rows) break;
+        const uint16_t* s = stream + row_start[r];
+        for (uint32_t g = 0; g < gpr; ++g) {
+          const uint16_t v = *s;
+          if (v == TQ_ESCAPE) {
+            ++cnt[g >> 5];
+            s += 5;
+          } else {
+            if (v >= limit) ++cnt[g >> 5];
+            ++s;
+          }
+        }
+      }
+    }
+  });
+  uint64_t n_raw = 0;
+  for (uint64_t i = 0; i < n_tiles; ++i) {
+    n_raw += tile_raw_v[i + 1];
+    if (n_raw >= (1ull << 32) - 65536) return TQ_ERR_UNSUPPORTED_SHAPE;
+    tile_raw_v[i + 1] = (uint32_t)n_raw;
+  }
 
   const uint64_t off_status = 0;
   const uint64_t off_scale = 256;
   const uint64_t off_zero = align_up(off_scale + rows_pad * 4, 256);
   const uint64_t off_tile_raw = align_up(off_zero + rows_pad * 4, 256);
-  const uint64_t off_tokens = align_up(off_tile_raw + (n_tiles + 1) * 4, 1024);
-  // 4 KB of token padding and 16 KB of raw padding: prefetches past the last tile stay inside the buffer
-  const uint64_t off_raw = align_up(off_tokens + n_tiles * 1024 + 4096, 1024);
-  const uint64_t total = align_up(off_raw + M * 4 + 16384, 256);
+  const uint64_t off_tokens = align_up(off_tile_raw + (n_tiles + 1 + 8) * 4, 1024);
+  // 8 KB of token padding and 16 KB of raw padding: prefetches past the last tile stay inside the buffer
+  const uint64_t off_raw = align_up(off_tokens + n_tiles * 1024 + 8192, 1024);
+  const uint64_t total = align_up(off_raw + n_raw * 4 + 16384, 256);
   if (device_bytes) *device_bytes = total;
   if (!img) return TQ_OK;
-  if (!row_scale) return TQ_ERR_INVALID_ARG;
+  if (!row_scale || !table) return TQ_ERR_INVALID_ARG;
   try {
     img->blob.assign(total, 0);
   } catch (const std::bad_alloc&) {
@@ -749,62 +799,64 @@ int tq_build_tiles_image(const uint16_t* stream, uint64_t stream_len, uint32_t r
   img->row_blocks = row_blocks;
   img->n_hits = H;
   img->n_miss = M;
+  img->n_raw = n_raw;
   uint8_t* base = img->blob.data();
   std::memcpy(base + off_scale, row_scale, (size_t)rows * 4);
   if (row_zero) std::memcpy(base + off_zero, row_zero, (size_t)rows * 4);
   uint32_t* tile_raw = reinterpret_cast<uint32_t*>(base + off_tile_raw);
+  std::memcpy(tile_raw, tile_raw_v.data(), (n_tiles + 1) * 4);
+  for (int i = 1; i <= 8; ++i) tile_raw[n_tiles + i] = (uint32_t)n_raw;  // read ahead by the kernels, never used
   uint16_t* tokens = reinterpret_cast<uint16_t*>(base + off_tokens);
   uint32_t* raw = reinterpret_cast<uint32_t*>(base + off_raw);
 
-  // pass 1: markers per tile
-  const int T = (int)std::min<uint64_t>(tq_num_threads(), row_blocks);
-  parallel_run(T, [&](int t) {
-    const uint32_t b0 = (uint32_t)((uint64_t)row_blocks * t / T), b1 = (uint32_t)((uint64_t)row_blocks * (t + 1) / T);
-    for (uint32_t rb = b0; rb < b1; ++rb) {
-      uint32_t* cnt = tile_raw + (uint64_t)rb * steps + 1;  // shifted by one: becomes the prefix sum below
-      for (uint32_t i = 0; i < 16; ++i) {
-        const uint32_t r = rb * 16 + i;
-        if (r >= rows) break;
-        const uint16_t* s = stream + row_start[r];
-        for (uint32_t g = 0; g < gpr; ++g) {
-          if (*s == TQ_ESCAPE) {
-            ++cnt[g >> 5];
-            s += 5;
-          } else {
-            ++s;
-          }
-        }
-      }
-    }
-  });
-  for (uint64_t i = 0; i < n_tiles; ++i) tile_raw[i + 1] += tile_raw[i];
-
   // pass 2: tokens and raw words in tile order.  A row's groups are met in ascending order, so one
-  // cursor per row is enough.
+  // cursor per row is enough.  Inside a tile the raw words are numbered slot by slot (slot j = 8h + i
+  // of every lane, lanes ascending), so the words one lookup instruction of the warp reads are
+  // neighbours in shared memory.
   parallel_run(T, [&](int t) {
     const uint32_t b0 = (uint32_t)((uint64_t)row_blocks * t / T), b1 = (uint32_t)((uint64_t)row_blocks * (t + 1) / T);
+    uint32_t word[32][16];
+    bool is_raw[32][16];
     for (uint32_t rb = b0; rb < b1; ++rb) {
       const uint16_t* cur[16];
       for (uint32_t i = 0; i < 16; ++i) cur[i] = rb * 16 + i < rows ? stream + row_start[rb * 16 + i] : nullptr;
       for (uint32_t s = 0; s < steps; ++s) {
         const uint64_t tile = (uint64_t)rb * steps + s;
         uint16_t* tk = tokens + tile * 512;
-        uint32_t* rw = raw + tile_raw[tile];
         for (uint32_t lane = 0; lane < 32; ++lane) {
           const uint32_t g = lane >> 2, q = lane & 3u;
           for (uint32_t h = 0; h < 2; ++h) {
             const uint16_t*& c = cur[g + 8 * h];
-            uint16_t* out = tk + h * 256 + lane * 8;
             for (uint32_t i = 0; i < 8; ++i) {
-              const uint32_t grp = 32 * s + 8 * q + i;
-              if (!c || grp >= gpr) continue;  // stays token 0
+              const uint32_t grp = 32 * s + 8 * q + i, j = 8 * h + i;
+              is_raw[lane][j] = false;
+              word[lane][j] = 0;  // token 0: four zero bytes
+              if (!c || grp >= gpr) continue;
               const uint16_t v = *c++;
-              out[i] = v;
               if (v == TQ_ESCAPE) {
-                *rw++ = (uint32_t)(c[0] & 0xFF) | ((uint32_t)(c[1] & 0xFF) << 8) | ((uint32_t)(c[2] & 0xFF) << 16) |
-                        ((uint32_t)(c[3] & 0xFF) << 24);
+                is_raw[lane][j] = true;
+                word[lane][j] = (uint32_t)(c[0] & 0xFF) | ((uint32_t)(c[1] & 0xFF) << 8) |
+                                ((uint32_t)(c[2] & 0xFF) << 16) | ((uint32_t)(c[3] & 0xFF) << 24);
                 c += 4;
+              } else if (v >= limit) {
+                is_raw[lane][j] = true;
+                word[lane][j] = table[v];
+              } else {
+                word[lane][j] = v;
               }
+            }
+          }
+        }
+        uint32_t pos = tile_raw[tile];
+        for (uint32_t j = 0; j < 16; ++j) {
+          for (uint32_t lane = 0; lane < 32; ++lane) {
+            uint16_t* out = tk + (j >> 3) * 256 + lane * 8 + (j & 7u);
+            if (is_raw[lane][j]) {
+              raw[pos] = word[lane][j];
+              *out = (uint16_t)(miss_base | (pos & (TQ_TILES_RING_WORDS - 1u)));
+              ++pos;
+            } else {
+              *out = (uint16_t)word[lane][j];
             }
           }
         }
@@ -814,14 +866,16 @@ int tq_build_tiles_image(const uint16_t* stream, uint64_t stream_len, uint32_t r
   return TQ_OK;
 }
 
-extern "C" int tq_tiles_image_host(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
-                                   uint32_t K, const float* row_scale, const float* row_zero, uint8_t* out,
+extern "C" int tq_tiles_image_host(const tq_dict* d, const uint16_t* stream, uint64_t stream_len, uint32_t rows,
+                                   uint32_t cols, const float* row_scale, const float* row_zero, uint8_t* out,
                                    uint64_t out_cap, uint64_t* out_bytes, uint64_t* offsets, uint32_t* dims) {
-  if (!out_bytes) return TQ_ERR_INVALID_ARG;
-  if (!out) return tq_build_tiles_image(stream, stream_len, rows, cols, K, nullptr, nullptr, out_bytes, nullptr);
+  if (!d || !out_bytes) return TQ_ERR_INVALID_ARG;
+  if (!out) return tq_build_tiles_image(stream, stream_len, rows, cols, d->K, nullptr, nullptr, nullptr, out_bytes, nullptr);
   if (!offsets || !dims) return TQ_ERR_INVALID_ARG;
+  std::vector<uint32_t> table((size_t)d->K + 1, 0);
+  if (d->K) std::memcpy(table.data() + 1, d->entries.data(), (size_t)d->K * 4);
   tq_tiles_image img;
-  int rc = tq_build_tiles_image(stream, stream_len, rows, cols, K, row_scale, row_zero, out_bytes, &img);
+  int rc = tq_build_tiles_image(stream, stream_len, rows, cols, d->K, table.data(), row_scale, row_zero, out_bytes, &img);
   if (rc != TQ_OK) return rc;
   if (out_cap < img.blob.size()) return TQ_ERR_BUFFER_TOO_SMALL;
   std::memcpy(out, img.blob.data(), img.blob.size());

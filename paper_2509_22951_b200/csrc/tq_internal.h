@@ -25,6 +25,7 @@ struct tq_ddict {
   // DEVICE: K + 1 words indexed by code; word 0 is zero (token 0 = padding), word c holds entry
   // c - 1 with byte i of the window in bits 8i..8i+7
   const uint32_t* d_table = nullptr;
+  std::vector<uint32_t> h_table;  // HOST copy of the same K + 1 words
 };
 
 // Row descriptor of the STREAM layout: where the row's token segment starts (in 16-byte units
@@ -48,7 +49,7 @@ struct tq_tiles_desc {
   uint32_t steps;            // tiles per row block = ceil(cols / 128)
   uint32_t row_blocks;       // ceil(rows / 16)
   uint32_t has_zero;
-  uint32_t pad_;
+  uint32_t table_words;      // tokens are < table_words or the marker
 };
 
 struct tq_dmat {
@@ -90,7 +91,8 @@ struct tq_tiles_image {
   std::vector<uint8_t> blob;
   uint64_t off_status = 0, off_scale = 0, off_zero = 0, off_tile_raw = 0, off_tokens = 0, off_raw = 0;
   uint32_t steps = 0, row_blocks = 0;
-  uint64_t n_hits = 0, n_miss = 0;
+  uint64_t n_hits = 0, n_miss = 0;  // of the paper's stream
+  uint64_t n_raw = 0;               // raw words of the image: n_miss + the groups whose code is >= table_words
 };
 
 int tq_num_threads();
@@ -103,13 +105,15 @@ int tq_cuda_status(int cuda_error, const char* what);
 int tq_build_stream_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
                           uint32_t K, const float* row_scale, const float* row_zero,
                           uint64_t* device_bytes, tq_host_image* img);
+// table: HOST, K + 1 words indexed by code (needed only when img != nullptr).
 int tq_build_tiles_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
-                         uint32_t K, const float* row_scale, const float* row_zero,
+                         uint32_t K, const uint32_t* table, const float* row_scale, const float* row_zero,
                          uint64_t* device_bytes, tq_tiles_image* img);
 int tq_build_planes_image(const uint16_t* stream, uint64_t stream_len, uint32_t rows, uint32_t cols,
                           uint32_t K, const float* row_scale, const float* row_zero,
                           uint64_t* device_bytes, tq_planes_image* img);
 
-// TILES layout entry points (tq_tiles.cu).  x: bf16 [nb][cols], nb in 1..2; y: fp32 [nb][rows].
+// TILES layout entry points (tq_tiles.cu).  x: bf16 [nb][cols], nb in 1..tq_tiles_max_nb(m); y: fp32 [nb][rows].
+int tq_tiles_max_nb(const tq_dmat* m);
 int tq_tiles_gemv(const tq_dmat* m, const void* x, int nb, float* y, void* cuda_stream);
 int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream);

@@ -14,12 +14,13 @@
 // (bf16 carries 8), far inside the fp32-accumulation tolerance, and is independent of how the
 // columns are split among warps.  Two batch columns fit one MMA (6 of 8 B columns).
 //
-// Data movement.  One persistent CTA per SM keeps the first KS words of the table in shared
-// memory (lookups there are bank-conflict limited, not tag limited like divergent global loads);
-// codes >= KS are read from the full table in global memory.  Each warp walks a contiguous run of
-// tiles: token tiles come through registers three tiles ahead; raw words come through a per-warp
-// ring in shared memory that a single lane keeps filled with 512-byte bulk copies
-// (cp.async.bulk + mbarrier), so neither stream sits on the dependent path.
+// Data movement.  One persistent CTA per SM keeps the table (TQ_TILES_TABLE_WORDS words) in shared
+// memory: lookups there are bank-conflict limited, not tag limited like divergent global loads.
+// Each warp walks a contiguous run of tiles.  Token tiles come through registers, four tiles
+// ahead.  Raw words come through a per-warp ring of TQ_TILES_RING_WORDS words in shared memory
+// that one lane keeps filled with 512-byte bulk copies (cp.async.bulk + mbarrier); raw word p of
+// the matrix always sits in ring slot p mod ring size, and that slot number is what a miss token
+// carries, so a lookup is: token -> (token >= 0xFC00 ? ring : table)[token] -> MMA operand.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -31,27 +32,27 @@
 namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kRingWords = TQ_TILES_RING_WORDS;     // 4 KB per warp
 constexpr int kChunkWords = 128;                    // one bulk copy: 512 bytes of raw words
-constexpr int kSlots = 8;                           // chunks per ring
-constexpr int kRingWords = kChunkWords * kSlots;    // 4 KB per warp
-constexpr int kPrefetch = 3;                        // token tiles in flight per warp
+constexpr int kSlots = kRingWords / kChunkWords;    // chunks per ring
+constexpr int kPrefetch = 4;                        // token tiles in flight per warp (even: two word buffers alternate)
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr uint32_t kNoBlock = 0xFFFFFFFFu;
+constexpr uint32_t kMissBase = 0x10000u - TQ_TILES_RING_WORDS;  // first miss token
+static_assert(kSlots == 8 && (kRingWords & (kRingWords - 1)) == 0, "ring geometry");
 
 __host__ __device__ inline uint32_t align_up_u32(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 
 // Shared-memory plan, identical on host and device.
 struct TilesSmem {
-  uint32_t ring, x, bar, part, stage, misc, total;
+  uint32_t ring, x, bar, misc, total;
 };
-__host__ __device__ inline TilesSmem tiles_smem(uint32_t KS, uint32_t x_words, int warps) {
+__host__ __device__ inline TilesSmem tiles_smem(uint32_t table_words, uint32_t x_words, int warps) {
   TilesSmem L;
-  L.ring = align_up_u32(KS * 4u, 4096u);  // rings start on a multiple of their size from the table base
+  L.ring = align_up_u32(table_words * 4u, 16u);
   L.x = L.ring + (uint32_t)warps * kRingWords * 4u;
   L.bar = align_up_u32(L.x + x_words * 4u, 16u);
-  L.part = L.bar + (uint32_t)warps * kSlots * 8u;
-  L.stage = L.part + 2u * warps * 512u;
-  L.misc = L.stage + (uint32_t)warps * 512u;
+  L.misc = L.bar + (uint32_t)warps * kSlots * 8u;
   L.total = L.misc + 512u;
   return L;
 }
@@ -66,7 +67,7 @@ struct TilesParams {
   const uint32_t* cta_seg;    // stack mode: gridDim.x + 1 offsets into segs
   tq_tiles_desc one;          // single-matrix mode
   const uint32_t* table;      // 65536 words, zero past the last entry
-  uint32_t KS;                // table words kept in shared memory (multiple of 1024)
+  uint32_t table_words;       // words of it kept in shared memory
   uint32_t xstride;           // words per digit column in shared memory
 };
 
@@ -77,6 +78,11 @@ __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
   asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
   return v;
 }
 
@@ -108,25 +114,6 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                : "memory");
 }
 
-// One decoded word: from the table in shared memory (code < KS), from the warp's raw ring (marker;
-// `cursor` is the lane's next raw word and moves on), or from the table in global memory.
-__device__ __forceinline__ uint32_t lookup(uint32_t tk, uint32_t& cursor, uint32_t tbl_addr, uint32_t ring_idx,
-                                           uint32_t KS, const uint32_t* __restrict__ gtable) {
-  const bool mk = tk == 0xFFFFu;
-  const uint32_t idx = mk ? (ring_idx | (cursor & (kRingWords - 1u))) : tk;
-  cursor += mk ? 1u : 0u;
-  const uint32_t far = (tk >= KS && !mk) ? 1u : 0u;
-  uint32_t w;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.u32 p, %1, 0;\n\t"
-      "@p ld.global.nc.u32 %0, [%2];\n\t"
-      "@!p ld.shared.u32 %0, [%3];\n\t}"
-      : "=r"(w)
-      : "r"(far), "l"(gtable + tk), "r"(tbl_addr + idx * 4u));
-  return w;
-}
-
 template <bool SIGNED>
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
@@ -155,8 +142,7 @@ struct TilesCta {
   uint8_t* smem;
   TilesSmem L;
   uint32_t tbl_addr;
-  uint32_t KS, xstride;
-  const uint32_t* gtable;
+  uint32_t xstride;
   uint32_t warp, lane;
   uint32_t phase = 0;  // parity bit of each of this warp's ring barriers
   bool dead = false;
@@ -240,30 +226,34 @@ struct TilesCta {
   }
 
   // ---- results ----------------------------------------------------------------------------
-  // Turns the 16 x 8 accumulator tile (MMA fragment layout) of row block rb into y.
+  // Turns the 16 x 8 accumulator tile (MMA fragment layout: lane 4g+t holds rows g, g+8 and
+  // columns 2t, 2t+1) of row block rb into y.  Lane L gathers the three digit sums of row L & 15,
+  // batch column L >> 4 with shuffles.
   __device__ __forceinline__ void finalize(const tq_tiles_desc& d, uint32_t rb, const int (&c)[4]) {
-    int* st = reinterpret_cast<int*>(smem + L.stage + warp * 512u);
-    const uint32_t g = lane >> 2, t = lane & 3u;
-    st[g * 8 + 2 * t] = c[0];
-    st[g * 8 + 2 * t + 1] = c[1];
-    st[(g + 8) * 8 + 2 * t] = c[2];
-    st[(g + 8) * 8 + 2 * t + 1] = c[3];
-    __syncwarp();
     const uint32_t row = lane & 15u, b = lane >> 4;
+    long long Y = 0;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+      const uint32_t col = min(3u * b + k, 7u);
+      const uint32_t src = (row & 7u) * 4u + (col >> 1);
+      const int v0 = __shfl_sync(kFull, c[0], src), v1 = __shfl_sync(kFull, c[1], src);
+      const int v2 = __shfl_sync(kFull, c[2], src), v3 = __shfl_sync(kFull, c[3], src);
+      const int lo = (col & 1u) ? v1 : v0, hi = (col & 1u) ? v3 : v2;
+      Y += (long long)((row & 8u) ? hi : lo) << (8 * k);
+    }
     const uint32_t r = rb * 16u + row;
     if (b < (uint32_t)NB && r < d.rows) {
-      const long long Y = (long long)st[row * 8 + 3 * b] + 256ll * st[row * 8 + 3 * b + 1] +
-                          65536ll * st[row * 8 + 3 * b + 2];
       const XInfo* xi = xinfo();
       double v = (double)Y * xi->out_scale[b];
       if (d.has_zero) v -= (double)d.zero[r] * xi->sum_x[b];
       d.y[(size_t)b * d.rows + r] = (float)((double)d.scale[r] * v);
     }
-    __syncwarp();
   }
 
+  // Partial sums of a row block shared with a neighbouring warp; parked in the warp's own ring,
+  // which is idle by then.
   __device__ __forceinline__ void store_partial(uint32_t slot, uint32_t rb, const int (&c)[4]) {
-    int4* p = reinterpret_cast<int4*>(smem + L.part + (2u * warp + slot) * 512u);
+    int4* p = reinterpret_cast<int4*>(smem + L.ring + warp * (kRingWords * 4u) + slot * 512u);
     p[lane] = make_int4(c[0], c[1], c[2], c[3]);
     if (lane == 0) part_ids()[2 * warp + slot] = rb;
   }
@@ -296,10 +286,15 @@ struct TilesCta {
   }
 
   // ---- one warp, tiles [t0, t1) of matrix d -------------------------------------------------
+  // The tile loop is unrolled by kPrefetch so that every buffer has a fixed register name: token
+  // loads land in the registers of the tile they replace, and the words looked up for tile i
+  // (buffer i & 1) are consumed by the MMAs one tile later -- no register is copied while a load
+  // into it is still in flight.
   __device__ void run_tiles(const tq_tiles_desc& d, uint32_t t0, uint32_t t1) {
     const uint32_t S = d.steps;
     const uint32_t g = lane >> 2, t = lane & 3u;
-    const uint32_t ring_idx = (L.ring >> 2) + warp * kRingWords;
+    // a miss token m (>= kMissBase) addresses word m - kMissBase of this warp's ring
+    const uint32_t miss_adj = (L.ring >> 2) + warp * kRingWords - kMissBase;
     const uint32_t* xs = reinterpret_cast<const uint32_t*>(smem + L.x);
     const bool has_b = g < (uint32_t)NCOL;
     const uint32_t x_lane = g * xstride + 8u * t;
@@ -310,22 +305,29 @@ struct TilesCta {
     const uint32_t c_stop = rd_end > rd ? (rd_end - 1u) / kChunkWords + 1u : c_issue;  // one past the last chunk needed
     for (int k = 0; k < kSlots && c_issue < c_stop; ++k) issue_chunk(d.raw, c_issue++);
 
+    const uint4* tok = d.tokens + (size_t)t0 * 64u + lane;
+    const uint32_t* trp = d.tile_raw + t0 + 1;
     uint4 q[kPrefetch][2];
+    uint32_t tr[kPrefetch];  // tile_raw[tile + 1]: where the tile's raw words end
 #pragma unroll
     for (int k = 0; k < kPrefetch; ++k) {
-      q[k][0] = ldg_stream(d.tokens + (size_t)(t0 + k) * 64u + lane);
-      q[k][1] = ldg_stream(d.tokens + (size_t)(t0 + k) * 64u + 32u + lane);
+      q[k][0] = ldg_stream(tok + k * 64);
+      q[k][1] = ldg_stream(tok + k * 64 + 32);
+      tr[k] = __ldg(trp + k);
     }
+    tok += kPrefetch * 64;
+    trp += kPrefetch;
 
     uint32_t s = t0 % S, rb = t0 / S;
     bool from_start = s == 0;
-    bool used_first = false;
+    uint32_t first_rb = kNoBlock;
+    int first_acc[4] = {0, 0, 0, 0};
     int acc[4] = {0, 0, 0, 0};
-    uint32_t wc[16] = {};
+    uint32_t wbuf[2][16] = {};
     bool pending = false;
     uint32_t pend_s = 0;
 
-    auto consume = [&]() {
+    auto consume = [&](const uint32_t (&wc)[16]) {
       uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = xa;
       if (has_b) {
         const uint4* xp = reinterpret_cast<const uint4*>(xs + x_lane + 32u * pend_s);
@@ -339,9 +341,10 @@ struct TilesCta {
       if (pend_s == S - 1u) {
         if (from_start) {
           finalize(d, rb, acc);
-        } else {
-          store_partial(0, rb, acc);
-          used_first = true;
+        } else {  // the run began inside this row block: keep its sums for the merge
+          first_rb = rb;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) first_acc[i] = acc[i];
         }
         acc[0] = acc[1] = acc[2] = acc[3] = 0;
         from_start = true;
@@ -349,80 +352,76 @@ struct TilesCta {
       }
     };
 
-    for (uint32_t tile = t0; tile < t1; ++tile) {
-      const uint4 ca = q[0][0], cb = q[0][1];
+    for (uint32_t tile = t0; tile < t1 && !dead; tile += kPrefetch) {
 #pragma unroll
-      for (int k = 0; k + 1 < kPrefetch; ++k) {
-        q[k][0] = q[k + 1][0];
-        q[k][1] = q[k + 1][1];
-      }
-      q[kPrefetch - 1][0] = ldg_stream(d.tokens + (size_t)(tile + kPrefetch) * 64u + lane);
-      q[kPrefetch - 1][1] = ldg_stream(d.tokens + (size_t)(tile + kPrefetch) * 64u + 32u + lane);
+      for (int k = 0; k < kPrefetch; ++k) {
+        if (tile + k < t1 && !dead) {
+          const uint32_t R[8] = {q[k][0].x, q[k][0].y, q[k][0].z, q[k][0].w, q[k][1].x, q[k][1].y, q[k][1].z, q[k][1].w};
+          const uint32_t rd_next = tr[k];
+          uint32_t tk[16];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            tk[2 * i] = R[i] & 0xFFFFu;
+            tk[2 * i + 1] = R[i] >> 16;
+          }
+          q[k][0] = ldg_stream(tok);
+          q[k][1] = ldg_stream(tok + 32);
+          tr[k] = __ldg(trp);
+          tok += 64;
+          ++trp;
 
-      const uint32_t R[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
-      uint32_t tk[16];
-      uint32_t n = 0;
+          // the chunks holding this tile's raw words [rd, rd_next)
+          const uint32_t c_need = rd_next > rd ? (rd_next - 1u) / kChunkWords + 1u : c_wait;
+          while (c_wait < c_need) {
+            if (!wait_chunk(c_wait)) { dead = true; break; }
+            ++c_wait;
+          }
+          rd = rd_next;
+          if (!dead) {
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        tk[2 * k] = R[k] & 0xFFFFu;
-        tk[2 * k + 1] = R[k] >> 16;
-        n += (tk[2 * k] == 0xFFFFu) + (tk[2 * k + 1] == 0xFFFFu);
-      }
-      uint32_t incl = n;
-#pragma unroll
-      for (int sft = 1; sft < 32; sft <<= 1) {
-        const uint32_t v = __shfl_up_sync(kFull, incl, sft);
-        if (lane >= (uint32_t)sft) incl += v;
-      }
-      const uint32_t total = __shfl_sync(kFull, incl, 31);
-      uint32_t cursor = rd + incl - n;
-      rd += total;
-      // the chunks holding this tile's raw words
-      const uint32_t c_need = total ? (rd - 1u) / kChunkWords + 1u : c_wait;
-      while (c_wait < c_need) {
-        if (!wait_chunk(c_wait)) { dead = true; break; }
-        ++c_wait;
-      }
-      if (dead) break;
-
-      uint32_t wn[16];
-#pragma unroll
-      for (int j = 0; j < 16; ++j) wn[j] = lookup(tk[j], cursor, tbl_addr, ring_idx, KS, gtable);
-
-      if (pending) consume();
-#pragma unroll
-      for (int j = 0; j < 16; ++j) wc[j] = wn[j];
-      pending = true;
-      pend_s = s;
-      if (++s == S) s = 0;
-
-      // every lane has finished reading the chunks below rd (the MMAs above consumed the previous
-      // tile's words; this tile's loads are ordered before the refill by the warp barrier)
-      __syncwarp();
-      const uint32_t c_free = rd / kChunkWords;  // chunks below this index are fully consumed
-      while (c_issue < c_stop && c_issue < c_free + kSlots) issue_chunk(d.raw, c_issue++);
-    }
-    if (pending && !dead) {
-      consume();
-      if (pend_s != S - 1u) {  // the run ended inside a row block
-        if (!from_start && !used_first) store_partial(0, rb, acc);
-        else store_partial(1, rb, acc);
+            for (int j = 0; j < 16; ++j) {
+              const uint32_t idx = tk[j] + (tk[j] >= kMissBase ? miss_adj : 0u);
+              wbuf[k & 1][j] = lds_u32(tbl_addr + idx * 4u);
+            }
+            if (pending) consume(wbuf[(k + 1) & 1]);
+            pending = true;
+            pend_s = s;
+            if (++s == S) s = 0;
+            // every lane has issued its reads of the chunks below rd; the warp barrier orders them
+            // before the refill that may overwrite those chunks
+            __syncwarp();
+            const uint32_t c_free = rd / kChunkWords;  // chunks below this index are fully consumed
+            while (c_issue < c_stop && c_issue < c_free + kSlots) issue_chunk(d.raw, c_issue++);
+          }
+        }
       }
     }
     if (dead) {
       *dead_flag() = 1u;
       if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
+      return;
+    }
+    if (pending) {
+      // the last tile's words sit in buffer (t1 - t0 - 1) & 1
+      if ((t1 - t0 - 1u) & 1u) consume(wbuf[1]);
+      else consume(wbuf[0]);
+    }
+    while (c_wait < c_issue) {  // nothing may still be landing when the ring is reused
+      if (!wait_chunk(c_wait)) { dead = true; *dead_flag() = 1u; return; }
+      ++c_wait;
+    }
+    __syncwarp();
+    if (!from_start) {
+      store_partial(0, rb, acc);  // the whole run lies inside one row block
     } else {
-      while (c_wait < c_issue) {  // nothing may still be landing when the ring is reused
-        if (!wait_chunk(c_wait)) { dead = true; *dead_flag() = 1u; break; }
-        ++c_wait;
-      }
+      if (first_rb != kNoBlock) store_partial(0, first_rb, first_acc);
+      if (pend_s != S - 1u) store_partial(1, rb, acc);  // the run ended inside a row block
     }
   }
 
   // ---- one segment: row blocks [rb0, rb1) of matrix d, all warps ----------------------------
   __device__ void run_segment(const tq_tiles_desc& d, uint32_t rb0, uint32_t rb1) {
-    __syncthreads();  // the previous segment is done with x, the partials and the staging tiles
+    __syncthreads();  // the previous segment is done with x and with the partials in the rings
     prepare_x(d);
     if (lane < 2) part_ids()[2 * warp + lane] = kNoBlock;
     __syncthreads();
@@ -443,7 +442,7 @@ struct TilesCta {
           cur = id;
           sum[0] = sum[1] = sum[2] = sum[3] = 0;
         }
-        const int4 v = reinterpret_cast<const int4*>(smem + L.part + e * 512u)[lane];
+        const int4 v = reinterpret_cast<const int4*>(smem + L.ring + (e >> 1) * (kRingWords * 4u) + (e & 1u) * 512u)[lane];
         sum[0] += v.x;
         sum[1] += v.y;
         sum[2] += v.z;
@@ -459,11 +458,9 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
   extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
   TilesCta<W, NB, SIGNED> cta;
   cta.smem = tiles_smem_raw;
-  cta.L = tiles_smem(p.KS, 3u * NB * p.xstride, W);
+  cta.L = tiles_smem(p.table_words, 3u * NB * p.xstride, W);
   cta.tbl_addr = smem_u32(tiles_smem_raw);
-  cta.KS = p.KS;
   cta.xstride = p.xstride;
-  cta.gtable = p.table;
   cta.warp = threadIdx.x >> 5;
   cta.lane = threadIdx.x & 31u;
 
@@ -474,7 +471,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
   {
     const uint4* src = reinterpret_cast<const uint4*>(p.table);
     uint4* dst = reinterpret_cast<uint4*>(tiles_smem_raw);
-    for (uint32_t i = threadIdx.x; i < p.KS / 4u; i += W * 32) dst[i] = __ldg(src + i);
+    for (uint32_t i = threadIdx.x; i < p.table_words / 4u; i += W * 32) dst[i] = __ldg(src + i);
   }
   __syncthreads();
 
@@ -496,8 +493,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
 // Decompress: one warp per tile, table and raw words read from global memory.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-decompress_tiles_kernel(const tq_tiles_desc d, const uint32_t* __restrict__ table, uint32_t K,
-                        uint32_t* __restrict__ out) {
+decompress_tiles_kernel(const tq_tiles_desc d, const uint32_t* __restrict__ table, uint32_t* __restrict__ out) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
   const uint32_t n_tiles = d.steps * d.row_blocks;
@@ -508,30 +504,18 @@ decompress_tiles_kernel(const tq_tiles_desc d, const uint32_t* __restrict__ tabl
     const uint32_t rb = tile / d.steps, s = tile % d.steps;
     const uint4 a = ldg_stream(d.tokens + (size_t)tile * 64u + lane);
     const uint4 b = ldg_stream(d.tokens + (size_t)tile * 64u + 32u + lane);
+    const uint32_t rd = __ldg(d.tile_raw + tile);
     const uint32_t R[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    uint32_t tk[16], n = 0;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      tk[2 * k] = R[k] & 0xFFFFu;
-      tk[2 * k + 1] = R[k] >> 16;
-      n += (tk[2 * k] == 0xFFFFu) + (tk[2 * k + 1] == 0xFFFFu);
-    }
-    uint32_t incl = n;
-#pragma unroll
-    for (int sft = 1; sft < 32; sft <<= 1) {
-      const uint32_t v = __shfl_up_sync(kFull, incl, sft);
-      if (lane >= (uint32_t)sft) incl += v;
-    }
-    const uint32_t* rp = d.raw + __ldg(d.tile_raw + tile) + (incl - n);
     uint32_t w[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      if (tk[j] == 0xFFFFu) {
-        w[j] = __ldg(rp++);
+      const uint32_t tk = (j & 1) ? (R[j >> 1] >> 16) : (R[j >> 1] & 0xFFFFu);
+      if (tk >= kMissBase) {
+        // the token names the ring slot of its raw word: its position modulo the ring size
+        w[j] = __ldg(d.raw + rd + ((tk - rd) & (kRingWords - 1u)));
       } else {
-        const uint32_t cl = min(tk[j], K);
-        bad |= tk[j] ^ cl;
-        w[j] = __ldg(table + cl);
+        bad |= tk >= d.table_words;
+        w[j] = __ldg(table + tk);
       }
     }
 #pragma unroll
@@ -563,16 +547,6 @@ int sm_count_tiles() {
 constexpr int kTilesWarps = 8;
 constexpr uint32_t kSmemLimit = 232448u;  // 227 KB per CTA
 
-// Largest table prefix (multiple of 1024 words) that fits beside everything else.
-uint32_t pick_ks(uint32_t x_words, int warps, uint32_t K) {
-  const TilesSmem fixed = tiles_smem(0, x_words, warps);
-  if (fixed.total > kSmemLimit) return 0xFFFFFFFFu;
-  uint32_t ks = (kSmemLimit - fixed.total) / 4096u * 1024u;
-  ks = std::min<uint32_t>(ks, 65536u);
-  ks = std::min<uint32_t>(ks, align_up_u32(K + 1u, 1024u));
-  return ks;
-}
-
 template <int NB, bool SIGNED>
 int launch_tiles(const TilesParams& p, uint32_t grid, size_t smem, cudaStream_t st) {
   auto kern = gemv_tiles_kernel<kTilesWarps, NB, SIGNED>;
@@ -589,17 +563,25 @@ int launch_tiles(const TilesParams& p, uint32_t grid, size_t smem, cudaStream_t 
 
 }  // namespace
 
-// x: bf16 [nb][cols], y: fp32 [nb][rows], nb in 1..2.
+// Batch columns one launch can take for this matrix (2, 1, or 0 if even one does not fit).
+int tq_tiles_max_nb(const tq_dmat* m) {
+  const uint32_t xstride = m->tiles.steps * 32u + 4u;
+  for (int nb = 2; nb >= 1; --nb)
+    if (tiles_smem(m->tiles.table_words, 3u * nb * xstride, kTilesWarps).total <= kSmemLimit) return nb;
+  return 0;
+}
+
+// x: bf16 [nb][cols], y: fp32 [nb][rows], nb in 1..tq_tiles_max_nb(m).
 int tq_tiles_gemv(const tq_dmat* m, const void* x, int nb, float* y, void* cuda_stream) {
   TilesParams p{};
   p.one = m->tiles;
   p.one.x = x;
   p.one.y = y;
   p.table = m->dict->d_table;
+  p.table_words = m->tiles.table_words;
   p.xstride = m->tiles.steps * 32u + 4u;
-  p.KS = pick_ks(3u * nb * p.xstride, kTilesWarps, m->dict->K);
-  if (p.KS == 0xFFFFFFFFu) return TQ_ERR_UNSUPPORTED_SHAPE;
-  const TilesSmem L = tiles_smem(p.KS, 3u * nb * p.xstride, kTilesWarps);
+  const TilesSmem L = tiles_smem(p.table_words, 3u * nb * p.xstride, kTilesWarps);
+  if (nb < 1 || nb > 2 || L.total > kSmemLimit) return TQ_ERR_UNSUPPORTED_SHAPE;
   const uint32_t grid = std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count_tiles());
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const bool sg = m->info.levels_signed != 0;
@@ -610,7 +592,7 @@ int tq_tiles_gemv(const tq_dmat* m, const void* x, int nb, float* y, void* cuda_
 int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
   const uint32_t n_tiles = m->tiles.steps * m->tiles.row_blocks;
   const uint32_t grid = std::min<uint32_t>((n_tiles + 7u) / 8u, (uint32_t)sm_count_tiles() * 8u);
-  decompress_tiles_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(m->tiles, m->dict->d_table, m->dict->K,
+  decompress_tiles_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(m->tiles, m->dict->d_table,
                                                                        reinterpret_cast<uint32_t*>(d_codes));
   return tq_cuda_status((int)cudaGetLastError(), "decompress(tiles) launch");
 }

@@ -73,6 +73,11 @@ def test_config0_layer_2048x2048(tq, layout):
 
 @pytest.mark.parametrize("rows,cols", [(1, 4), (3, 8), (7, 260), (8, 256), (9, 1028), (33, 2052), (17, 8192), (5, 12288), (40, 4 * 300)])
 def test_ragged_shapes(tq, rows, cols, layout):
+    if layout == 2 and cols > tq.TQ_TILES_MAX_COLS:
+        with pytest.raises(tq.TqError) as e:
+            tq.tq_upload_size(np.zeros(rows * cols // 4, dtype=np.uint16) + 1, rows, cols, layout)
+        assert e.value.status == tq.TQ_ERR_UNSUPPORTED_SHAPE
+        return
     rng = np.random.default_rng(rows * 1000 + cols)
     q = np.clip(np.rint(rng.standard_t(5, size=(rows, cols)) * 3), -127, 127).astype(np.int8)
     s = (rng.random(rows) + 0.5).astype(np.float32)

@@ -198,20 +198,24 @@ def _decode_tiles_image(img, offs, steps, row_blocks, rows, cols, entries):
     out = np.zeros((row_blocks * 16, steps * 128), dtype=np.uint8)
     for tile in range(n_tiles):
         rb, s = divmod(tile, steps)
-        nxt = int(tile_raw[tile])
+        first, end = int(tile_raw[tile]), int(tile_raw[tile + 1])
+        used = set()
         for lane in range(32):
             g, t = lane >> 2, lane & 3
             for h in range(2):
                 for i in range(8):
                     tk = int(tokens[tile, h, lane, i])
-                    if tk == 0xFFFF:
-                        w = np.array([raw[nxt]], dtype=np.uint32).view(np.uint8)
-                        nxt += 1
+                    if tk >= 0xFC00:  # miss: the token is the ring slot of its raw word
+                        p = first + ((tk - first) & 1023)
+                        assert first <= p < end and p not in used
+                        used.add(p)
+                        w = np.array([raw[p]], dtype=np.uint32).view(np.uint8)
                     else:
+                        assert tk < tq.TQ_TILES_TABLE_WORDS
                         w = table[tk]
                     c0 = 4 * (32 * s + 8 * t + i)
                     out[rb * 16 + g + 8 * h, c0:c0 + 4] = w
-        assert nxt == int(tile_raw[tile + 1])
+        assert len(used) == end - first
     assert not out[rows:].any() and not out[:, cols:].any()  # padding decodes to zeros
     return out[:rows, :cols]
 
@@ -224,7 +228,8 @@ def test_tiles_image_decodes_to_the_original_levels(rows, cols, top_k):
     stream = d.encode(q)[0]
     s = (rng.random(rows) + 0.5).astype(np.float32)
     z = rng.integers(0, 9, rows).astype(np.float32)
-    img, offs, steps, row_blocks = tq.tq_tiles_image_host(stream, rows, cols, d.K, s, z)
+    hd = tq.tq_dict_from_entries(d.entries)
+    img, offs, steps, row_blocks = tq.tq_tiles_image_host(hd, stream, rows, cols, s, z)
     assert steps == -(-cols // 128) and row_blocks == -(-rows // 16)
     got = _decode_tiles_image(img, offs, steps, row_blocks, rows, cols, d.entries)
     assert np.array_equal(got, q.view(np.uint8))
@@ -232,3 +237,30 @@ def test_tiles_image_decodes_to_the_original_levels(rows, cols, top_k):
     assert np.array_equal(img[offs["zero"]:offs["zero"] + 4 * rows].view(np.float32), z)
     n_miss = int(np.count_nonzero(stream == 0xFFFF))
     assert int(img[offs["tile_raw"]:].view(np.uint32)[steps * row_blocks]) == n_miss
+
+
+def test_tiles_image_stores_codes_beyond_the_shared_memory_table_as_raw_words():
+    # a table with 65534 entries: groups coded at or beyond TQ_TILES_TABLE_WORDS become raw words
+    rng = np.random.default_rng(77)
+    q = rng.integers(-20, 21, size=(64, 2048)).astype(np.int8)
+    d = oracle.Dictionary.build([q])
+    assert d.K == 65534
+    stream = d.encode(q)[0]
+    far = int(np.count_nonzero((stream >= tq.TQ_TILES_TABLE_WORDS) & (stream != 0xFFFF) & _code_slots(stream)))
+    assert far > 0
+    s = np.ones(64, dtype=np.float32)
+    hd = tq.tq_dict_from_entries(d.entries)
+    img, offs, steps, row_blocks = tq.tq_tiles_image_host(hd, stream, 64, 2048, s)
+    got = _decode_tiles_image(img, offs, steps, row_blocks, 64, 2048, d.entries)
+    assert np.array_equal(got, q.view(np.uint8))
+    n_miss = int(np.count_nonzero(stream == 0xFFFF))
+    assert int(img[offs["tile_raw"]:].view(np.uint32)[steps * row_blocks]) == n_miss + far
+
+
+def _code_slots(stream):
+    """True at the slots of a token stream that hold a code or a marker (not a raw value)."""
+    esc = np.flatnonzero(stream == 0xFFFF)
+    mask = np.ones(stream.size, dtype=bool)
+    for k in range(1, 5):
+        mask[esc + k] = False
+    return mask
