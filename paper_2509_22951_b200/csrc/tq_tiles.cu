@@ -18,7 +18,7 @@
 // memory: lookups there are bank-conflict limited, not tag limited like divergent global loads.
 // Each warp walks a contiguous run of tiles.  Token tiles come through registers, four tiles
 // ahead.  Raw words come through a per-warp ring of TQ_TILES_RING_WORDS words in shared memory
-// that one lane keeps filled with 512-byte bulk copies (cp.async.bulk + mbarrier); raw word p of
+// that one lane keeps filled with 1 KB bulk copies (cp.async.bulk + mbarrier); raw word p of
 // the matrix always sits in ring slot p mod ring size, and that slot number is what a miss token
 // carries, so a lookup is: token -> (token >= 0xFC00 ? ring : table)[token] -> MMA operand.
 #include <cuda_bf16.h>
@@ -33,13 +33,13 @@ namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kRingWords = TQ_TILES_RING_WORDS;     // 4 KB per warp
-constexpr int kChunkWords = 128;                    // one bulk copy: 512 bytes of raw words
+constexpr int kChunkWords = 256;                    // one bulk copy: 1 KB of raw words
 constexpr int kSlots = kRingWords / kChunkWords;    // chunks per ring
 constexpr int kPrefetch = 4;                        // token tiles in flight per warp (even: two word buffers alternate)
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr uint32_t kNoBlock = 0xFFFFFFFFu;
 constexpr uint32_t kMissBase = 0x10000u - TQ_TILES_RING_WORDS;  // first miss token
-static_assert(kSlots == 8 && (kRingWords & (kRingWords - 1)) == 0, "ring geometry");
+static_assert(kSlots == 4 && (kRingWords & (kRingWords - 1)) == 0, "ring geometry");
 
 __host__ __device__ inline uint32_t align_up_u32(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 
@@ -155,8 +155,6 @@ struct TilesCta {
   __device__ __forceinline__ XInfo* xinfo() { return reinterpret_cast<XInfo*>(smem + L.misc + 192); }
   __device__ __forceinline__ long long* sum_scratch() { return reinterpret_cast<long long*>(smem + L.misc + 256); }
 
-  __device__ __forceinline__ uint32_t bar_addr(uint32_t slot) { return tbl_addr + L.bar + (warp * kSlots + slot) * 8u; }
-
   // ---- activation vectors -> digit columns in shared memory --------------------------------
   __device__ void prepare_x(const tq_tiles_desc& d) {
     const uint32_t tid = threadIdx.x;
@@ -259,30 +257,31 @@ struct TilesCta {
   }
 
   // ---- raw ring ---------------------------------------------------------------------------
+  uint32_t ring_addr, bar_base;  // shared addresses of this warp's ring and of its first barrier
+
   __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t chunk) {
     if (lane == 0) {
       const uint32_t slot = chunk & (kSlots - 1u);
-      const uint32_t bar = bar_addr(slot);
-      mbar_expect_tx(bar, kChunkWords * 4u);
-      bulk_g2s(tbl_addr + L.ring + (warp * kRingWords + slot * kChunkWords) * 4u, raw + (size_t)chunk * kChunkWords,
-               kChunkWords * 4u, bar);
+      mbar_expect_tx(bar_base + slot * 8u, kChunkWords * 4u);
+      bulk_g2s(ring_addr + slot * (kChunkWords * 4u), raw + (size_t)chunk * kChunkWords, kChunkWords * 4u,
+               bar_base + slot * 8u);
     }
+  }
+  __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t par) {  // bounded in attempts and in time (about 2 s)
+    const uint64_t t_start = global_ns();
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+      if (mbar_try(bar, par)) return true;
+      if ((i & 63u) == 63u && (*dead_flag() || global_ns() - t_start > 2000000000ull)) break;
+    }
+    return false;
   }
   __device__ __forceinline__ bool wait_chunk(uint32_t chunk) {
     const uint32_t slot = chunk & (kSlots - 1u);
-    const uint32_t bar = bar_addr(slot);
+    const uint32_t bar = bar_base + slot * 8u;
     const uint32_t par = (phase >> slot) & 1u;
-    bool ok = mbar_try(bar, par);
-    if (!ok) {  // bounded both in attempts and in time (about 2 s)
-      const uint64_t t_start = global_ns();
-      for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try(bar, par)) { ok = true; break; }
-        if ((i & 63u) == 63u && (*dead_flag() || global_ns() - t_start > 2000000000ull)) break;
-      }
-    }
-    ok = __all_sync(kFull, ok);
     phase ^= 1u << slot;
-    return ok;
+    if (mbar_try(bar, par)) return true;
+    return __all_sync(kFull, wait_slow(bar, par));
   }
 
   // ---- one warp, tiles [t0, t1) of matrix d -------------------------------------------------
@@ -294,7 +293,7 @@ struct TilesCta {
     const uint32_t S = d.steps;
     const uint32_t g = lane >> 2, t = lane & 3u;
     // a miss token m (>= kMissBase) addresses word m - kMissBase of this warp's ring
-    const uint32_t miss_adj = (L.ring >> 2) + warp * kRingWords - kMissBase;
+    const uint32_t miss_adj4 = ring_addr - 4u * kMissBase;
     const uint32_t* xs = reinterpret_cast<const uint32_t*>(smem + L.x);
     const bool has_b = g < (uint32_t)NCOL;
     const uint32_t x_lane = g * xstride + 8u * t;
@@ -322,7 +321,7 @@ struct TilesCta {
     bool from_start = s == 0;
     uint32_t first_rb = kNoBlock;
     int first_acc[4] = {0, 0, 0, 0};
-    int acc[4] = {0, 0, 0, 0};
+    int acc[4] = {0, 0, 0, 0}, acc2[4] = {0, 0, 0, 0};  // two chains of MMAs, summed at the end of a row block
     uint32_t wbuf[2][16] = {};
     bool pending = false;
     uint32_t pend_s = 0;
@@ -335,10 +334,15 @@ struct TilesCta {
         xb = xp[1];
       }
       mma_s8<SIGNED>(acc, wc[0], wc[8], wc[1], wc[9], xa.x, xa.y);
-      mma_s8<SIGNED>(acc, wc[2], wc[10], wc[3], wc[11], xa.z, xa.w);
+      mma_s8<SIGNED>(acc2, wc[2], wc[10], wc[3], wc[11], xa.z, xa.w);
       mma_s8<SIGNED>(acc, wc[4], wc[12], wc[5], wc[13], xb.x, xb.y);
-      mma_s8<SIGNED>(acc, wc[6], wc[14], wc[7], wc[15], xb.z, xb.w);
+      mma_s8<SIGNED>(acc2, wc[6], wc[14], wc[7], wc[15], xb.z, xb.w);
       if (pend_s == S - 1u) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          acc[i] += acc2[i];
+          acc2[i] = 0;
+        }
         if (from_start) {
           finalize(d, rb, acc);
         } else {  // the run began inside this row block: keep its sums for the merge
@@ -358,11 +362,11 @@ struct TilesCta {
         if (tile + k < t1 && !dead) {
           const uint32_t R[8] = {q[k][0].x, q[k][0].y, q[k][0].z, q[k][0].w, q[k][1].x, q[k][1].y, q[k][1].z, q[k][1].w};
           const uint32_t rd_next = tr[k];
-          uint32_t tk[16];
+          uint32_t tk4[16];  // token * 4: byte offset into the table
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            tk[2 * i] = R[i] & 0xFFFFu;
-            tk[2 * i + 1] = R[i] >> 16;
+            tk4[2 * i] = (R[i] << 2) & 0x3FFFCu;
+            tk4[2 * i + 1] = (R[i] >> 14) & 0x3FFFCu;
           }
           q[k][0] = ldg_stream(tok);
           q[k][1] = ldg_stream(tok + 32);
@@ -380,8 +384,8 @@ struct TilesCta {
           if (!dead) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const uint32_t idx = tk[j] + (tk[j] >= kMissBase ? miss_adj : 0u);
-              wbuf[k & 1][j] = lds_u32(tbl_addr + idx * 4u);
+              const uint32_t a = tk4[j] + (tk4[j] >= 4u * kMissBase ? miss_adj4 : tbl_addr);
+              wbuf[k & 1][j] = lds_u32(a);
             }
             if (pending) consume(wbuf[(k + 1) & 1]);
             pending = true;
@@ -411,6 +415,8 @@ struct TilesCta {
       ++c_wait;
     }
     __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] += acc2[i];
     if (!from_start) {
       store_partial(0, rb, acc);  // the whole run lies inside one row block
     } else {
@@ -463,6 +469,8 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
   cta.xstride = p.xstride;
   cta.warp = threadIdx.x >> 5;
   cta.lane = threadIdx.x & 31u;
+  cta.ring_addr = cta.tbl_addr + cta.L.ring + cta.warp * (kRingWords * 4u);
+  cta.bar_base = cta.tbl_addr + cta.L.bar + cta.warp * (kSlots * 8u);
 
   if (threadIdx.x < W * kSlots) mbar_init(cta.tbl_addr + cta.L.bar + threadIdx.x * 8u, 1u);
   if (threadIdx.x == 0) *cta.dead_flag() = 0u;
