@@ -16,7 +16,7 @@
 //
 // Data movement.  One persistent CTA per SM keeps the table (TQ_TILES_TABLE_WORDS words) in shared
 // memory: lookups there are bank-conflict limited, not tag limited like divergent global loads.
-// Each warp walks a contiguous run of tiles.  Token tiles come through registers, four tiles
+// Each warp walks a contiguous run of tiles.  Token tiles come through registers, two tiles
 // ahead.  Raw words come through a per-warp ring of TQ_TILES_RING_WORDS words in shared memory
 // that one lane keeps filled with 1 KB bulk copies (cp.async.bulk + mbarrier); raw word p of
 // the matrix always sits in ring slot p mod ring size, and that slot number is what a miss token
@@ -35,7 +35,7 @@ constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kRingWords = TQ_TILES_RING_WORDS;     // 4 KB per warp
 constexpr int kChunkWords = 256;                    // one bulk copy: 1 KB of raw words
 constexpr int kSlots = kRingWords / kChunkWords;    // chunks per ring
-constexpr int kPrefetch = 4;                        // token tiles in flight per warp (even: two word buffers alternate)
+constexpr int kL2Ahead = 8;                         // token tiles prefetched into L2 ahead of their use (<= 8: padding)
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr uint32_t kNoBlock = 0xFFFFFFFFu;
 constexpr uint32_t kMissBase = 0x10000u - TQ_TILES_RING_WORDS;  // first miss token
@@ -103,6 +103,9 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -134,6 +137,45 @@ struct XInfo {
   double sum_x[2];      // out_scale * sum_c X[c]
 };
 
+// Bounded in attempts and in time (about 2 s).  Kept out of line and free of references so that the
+// caller's state stays in registers.
+__device__ __noinline__ bool tiles_wait_slow(uint32_t bar, uint32_t par, volatile uint32_t* dead_flag) {
+  const uint64_t t_start = global_ns();
+  bool ok = false;
+  for (uint32_t i = 0; i < kSpinLimit && !ok; ++i) {
+    ok = mbar_try(bar, par);
+    if ((i & 63u) == 63u && (*dead_flag || global_ns() - t_start > 2000000000ull)) break;
+  }
+  return __all_sync(kFull, ok);
+}
+
+// Turns the 16 x 8 accumulator tile (MMA fragment layout: lane 4g+t holds rows g, g+8 and columns
+// 2t, 2t+1) of row block rb into y.  Lane L gathers the three digit sums of row L & 15, batch
+// column L >> 4 with shuffles.
+template <int NB>
+__device__ __noinline__ void tiles_finalize(const float* __restrict__ scale, const float* __restrict__ zero,
+                                            float* __restrict__ y, uint32_t rows, uint32_t has_zero, const XInfo* xi,
+                                            uint32_t rb, int c0, int c1, int c2, int c3) {
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t row = lane & 15u, b = lane >> 4;
+  long long Y = 0;
+#pragma unroll
+  for (int k = 0; k < 3; ++k) {
+    const uint32_t col = min(3u * b + k, 7u);
+    const uint32_t src = (row & 7u) * 4u + (col >> 1);
+    const int v0 = __shfl_sync(kFull, c0, src), v1 = __shfl_sync(kFull, c1, src);
+    const int v2 = __shfl_sync(kFull, c2, src), v3 = __shfl_sync(kFull, c3, src);
+    const int lo = (col & 1u) ? v1 : v0, hi = (col & 1u) ? v3 : v2;
+    Y += (long long)((row & 8u) ? hi : lo) << (8 * k);
+  }
+  const uint32_t r = rb * 16u + row;
+  if (b < (uint32_t)NB && r < rows) {
+    double v = (double)Y * xi->out_scale[b];
+    if (has_zero) v -= (double)zero[r] * xi->sum_x[b];
+    y[(size_t)b * rows + r] = (float)((double)scale[r] * v);
+  }
+}
+
 template <int W, int NB, bool SIGNED>
 struct TilesCta {
   static constexpr int kThreads = W * 32;
@@ -144,7 +186,6 @@ struct TilesCta {
   uint32_t tbl_addr;
   uint32_t xstride;
   uint32_t warp, lane;
-  uint32_t phase = 0;  // parity bit of each of this warp's ring barriers
   bool dead = false;
 
   __device__ __forceinline__ uint32_t* misc_u32() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
@@ -224,28 +265,8 @@ struct TilesCta {
   }
 
   // ---- results ----------------------------------------------------------------------------
-  // Turns the 16 x 8 accumulator tile (MMA fragment layout: lane 4g+t holds rows g, g+8 and
-  // columns 2t, 2t+1) of row block rb into y.  Lane L gathers the three digit sums of row L & 15,
-  // batch column L >> 4 with shuffles.
-  __device__ __forceinline__ void finalize(const tq_tiles_desc& d, uint32_t rb, const int (&c)[4]) {
-    const uint32_t row = lane & 15u, b = lane >> 4;
-    long long Y = 0;
-#pragma unroll
-    for (int k = 0; k < 3; ++k) {
-      const uint32_t col = min(3u * b + k, 7u);
-      const uint32_t src = (row & 7u) * 4u + (col >> 1);
-      const int v0 = __shfl_sync(kFull, c[0], src), v1 = __shfl_sync(kFull, c[1], src);
-      const int v2 = __shfl_sync(kFull, c[2], src), v3 = __shfl_sync(kFull, c[3], src);
-      const int lo = (col & 1u) ? v1 : v0, hi = (col & 1u) ? v3 : v2;
-      Y += (long long)((row & 8u) ? hi : lo) << (8 * k);
-    }
-    const uint32_t r = rb * 16u + row;
-    if (b < (uint32_t)NB && r < d.rows) {
-      const XInfo* xi = xinfo();
-      double v = (double)Y * xi->out_scale[b];
-      if (d.has_zero) v -= (double)d.zero[r] * xi->sum_x[b];
-      d.y[(size_t)b * d.rows + r] = (float)((double)d.scale[r] * v);
-    }
+  __device__ __forceinline__ void finalize(const tq_tiles_desc& d, uint32_t rb, int c0, int c1, int c2, int c3) {
+    tiles_finalize<NB>(d.scale, d.zero, d.y, d.rows, d.has_zero, xinfo(), rb, c0, c1, c2, c3);
   }
 
   // Partial sums of a row block shared with a neighbouring warp; parked in the warp's own ring,
@@ -257,171 +278,165 @@ struct TilesCta {
   }
 
   // ---- raw ring ---------------------------------------------------------------------------
+  // Chunk c of the raw stream (words 256c .. 256c+255) always lands at ring offset (c mod 4) KB, the
+  // place its tokens point to.  The barriers are used round robin in issue order, which is also the
+  // order of the waits: use number n takes barrier n mod 4 and completes its phase (n / 4) mod 2.
   uint32_t ring_addr, bar_base;  // shared addresses of this warp's ring and of its first barrier
+  uint32_t n_issued = 0, n_waited = 0;
 
-  __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t chunk) {
+  __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t pos) {  // pos: first word, multiple of 256
     if (lane == 0) {
-      const uint32_t slot = chunk & (kSlots - 1u);
-      mbar_expect_tx(bar_base + slot * 8u, kChunkWords * 4u);
-      bulk_g2s(ring_addr + slot * (kChunkWords * 4u), raw + (size_t)chunk * kChunkWords, kChunkWords * 4u,
-               bar_base + slot * 8u);
+      const uint32_t bar = bar_base + (n_issued & (kSlots - 1u)) * 8u;
+      mbar_expect_tx(bar, kChunkWords * 4u);
+      bulk_g2s(ring_addr + ((pos * 4u) & (kRingWords * 4u - 1u)), raw + pos, kChunkWords * 4u, bar);
     }
+    ++n_issued;
   }
-  __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t par) {  // bounded in attempts and in time (about 2 s)
-    const uint64_t t_start = global_ns();
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-      if (mbar_try(bar, par)) return true;
-      if ((i & 63u) == 63u && (*dead_flag() || global_ns() - t_start > 2000000000ull)) break;
-    }
-    return false;
-  }
-  __device__ __forceinline__ bool wait_chunk(uint32_t chunk) {
-    const uint32_t slot = chunk & (kSlots - 1u);
-    const uint32_t bar = bar_base + slot * 8u;
-    const uint32_t par = (phase >> slot) & 1u;
-    phase ^= 1u << slot;
+  __device__ __forceinline__ bool wait_chunk() {
+    const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
+    const uint32_t par = (n_waited >> 2) & 1u;
+    ++n_waited;
     if (mbar_try(bar, par)) return true;
-    return __all_sync(kFull, wait_slow(bar, par));
+    return tiles_wait_slow(bar, par, dead_flag());
   }
 
   // ---- one warp, tiles [t0, t1) of matrix d -------------------------------------------------
-  // The tile loop is unrolled by kPrefetch so that every buffer has a fixed register name: token
-  // loads land in the registers of the tile they replace, and the words looked up for tile i
-  // (buffer i & 1) are consumed by the MMAs one tile later -- no register is copied while a load
-  // into it is still in flight.
+  // Tile i of the run uses token registers q[i & 1] and word buffer i & 1; its words are consumed
+  // by the MMAs while tile i + 1 is being looked up, and its token registers are reloaded (two
+  // tiles ahead) only after the last use, so no register is copied while a load into it is in
+  // flight.
   __device__ void run_tiles(const tq_tiles_desc& d, uint32_t t0, uint32_t t1) {
     const uint32_t S = d.steps;
     const uint32_t g = lane >> 2, t = lane & 3u;
     // a miss token m (>= kMissBase) addresses word m - kMissBase of this warp's ring
     const uint32_t miss_adj4 = ring_addr - 4u * kMissBase;
-    const uint32_t* xs = reinterpret_cast<const uint32_t*>(smem + L.x);
-    const bool has_b = g < (uint32_t)NCOL;
-    const uint32_t x_lane = g * xstride + 8u * t;
+    // lanes whose B column is not in use read the last used column: what they feed the MMA only
+    // reaches accumulator columns nobody reads
+    const uint32_t x_lane = tbl_addr + L.x + (min(g, (uint32_t)NCOL - 1u) * xstride + 8u * t) * 4u;
 
     uint32_t rd = __ldg(d.tile_raw + t0);
-    const uint32_t rd_end = __ldg(d.tile_raw + t1);
-    uint32_t c_issue = rd / kChunkWords, c_wait = c_issue;
-    const uint32_t c_stop = rd_end > rd ? (rd_end - 1u) / kChunkWords + 1u : c_issue;  // one past the last chunk needed
-    for (int k = 0; k < kSlots && c_issue < c_stop; ++k) issue_chunk(d.raw, c_issue++);
+    const uint32_t stop_pos = __ldg(d.tile_raw + t1);          // raw words of the run end here
+    uint32_t w_pos = rd & ~(uint32_t)(kChunkWords - 1);        // first word of the next chunk to wait for
+    uint32_t i_pos = w_pos;                                    // first word of the next chunk to issue
+    for (int k = 0; k < kSlots && i_pos < stop_pos; ++k, i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
 
     const uint4* tok = d.tokens + (size_t)t0 * 64u + lane;
+    const uint4* tok_end = d.tokens + (size_t)t1 * 64u;  // lane 0's view of the end of the run
     const uint32_t* trp = d.tile_raw + t0 + 1;
-    uint4 q[kPrefetch][2];
-    uint32_t tr[kPrefetch];  // tile_raw[tile + 1]: where the tile's raw words end
+    uint4 q[2][2];
+    uint32_t tr[2];  // tile_raw[tile + 1]: where the tile's raw words end
 #pragma unroll
-    for (int k = 0; k < kPrefetch; ++k) {
+    for (int k = 0; k < 2; ++k) {
       q[k][0] = ldg_stream(tok + k * 64);
       q[k][1] = ldg_stream(tok + k * 64 + 32);
       tr[k] = __ldg(trp + k);
     }
-    tok += kPrefetch * 64;
-    trp += kPrefetch;
+    tok += 2 * 64;
+    trp += 2;
 
-    uint32_t s = t0 % S, rb = t0 / S;
-    bool from_start = s == 0;
+    uint32_t s_p = t0 % S, rb = t0 / S;  // step and row block of the tile whose words await the MMAs
+    bool from_start = s_p == 0;
     uint32_t first_rb = kNoBlock;
     int first_acc[4] = {0, 0, 0, 0};
     int acc[4] = {0, 0, 0, 0}, acc2[4] = {0, 0, 0, 0};  // two chains of MMAs, summed at the end of a row block
-    uint32_t wbuf[2][16] = {};
-    bool pending = false;
-    uint32_t pend_s = 0;
+    uint32_t wbuf[2][16];
 
-    auto consume = [&](const uint32_t (&wc)[16]) {
-      uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = xa;
-      if (has_b) {
-        const uint4* xp = reinterpret_cast<const uint4*>(xs + x_lane + 32u * pend_s);
-        xa = xp[0];
-        xb = xp[1];
+    auto lookups = [&](int k) -> bool {  // tile words -> wbuf[k], then reload q[k] two tiles ahead
+      const uint32_t rd_next = tr[k];
+      while (rd_next > w_pos) {  // the chunks holding this tile's raw words [rd, rd_next)
+        if (!wait_chunk()) return false;
+        w_pos += kChunkWords;
       }
+      const uint32_t R[8] = {q[k][0].x, q[k][0].y, q[k][0].z, q[k][0].w, q[k][1].x, q[k][1].y, q[k][1].z, q[k][1].w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t lo4 = (R[i] << 2) & 0x3FFFCu, hi4 = (R[i] >> 14) & 0x3FFFCu;  // token * 4
+        wbuf[k][2 * i] = lds_u32(lo4 + (lo4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
+        wbuf[k][2 * i + 1] = lds_u32(hi4 + (hi4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
+      }
+      q[k][0] = ldg_stream(tok);
+      q[k][1] = ldg_stream(tok + 32);
+      tr[k] = __ldg(trp);
+      tok += 64;
+      ++trp;
+      rd = rd_next;
+      return true;
+    };
+    auto refill = [&]() {
+      // every lane has issued its reads of the chunks below rd; the warp barrier orders them before
+      // the copies that overwrite those chunks
+      __syncwarp();
+      const uint32_t lim = min(stop_pos, (rd & ~(uint32_t)(kChunkWords - 1)) + kRingWords);
+      for (; i_pos < lim; i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
+      // the token tile kL2Ahead tiles further on: brought into L2 now, so that the register load two
+      // tiles ahead of its use finds it there (tok already points two tiles ahead)
+      if (lane == 0 && tok + (kL2Ahead - 2) * 64 < tok_end) bulk_prefetch_l2(tok + (kL2Ahead - 2) * 64, 1024u);
+    };
+    auto consume = [&](const uint32_t (&wc)[16]) {
+      uint4 xa, xb;
+      const uint32_t xp = x_lane + 128u * s_p;
+      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(xa.x), "=r"(xa.y), "=r"(xa.z), "=r"(xa.w) : "r"(xp));
+      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+16];" : "=r"(xb.x), "=r"(xb.y), "=r"(xb.z), "=r"(xb.w) : "r"(xp));
       mma_s8<SIGNED>(acc, wc[0], wc[8], wc[1], wc[9], xa.x, xa.y);
       mma_s8<SIGNED>(acc2, wc[2], wc[10], wc[3], wc[11], xa.z, xa.w);
       mma_s8<SIGNED>(acc, wc[4], wc[12], wc[5], wc[13], xb.x, xb.y);
       mma_s8<SIGNED>(acc2, wc[6], wc[14], wc[7], wc[15], xb.z, xb.w);
-      if (pend_s == S - 1u) {
+      if (++s_p == S) {  // the row block is complete
+        s_p = 0;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          acc[i] += acc2[i];
-          acc2[i] = 0;
-        }
+        for (int i = 0; i < 4; ++i) acc[i] += acc2[i];
         if (from_start) {
-          finalize(d, rb, acc);
+          finalize(d, rb, acc[0], acc[1], acc[2], acc[3]);
         } else {  // the run began inside this row block: keep its sums for the merge
           first_rb = rb;
 #pragma unroll
           for (int i = 0; i < 4; ++i) first_acc[i] = acc[i];
         }
-        acc[0] = acc[1] = acc[2] = acc[3] = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[i] = acc2[i] = 0;
         from_start = true;
         ++rb;
       }
     };
 
-    for (uint32_t tile = t0; tile < t1 && !dead; tile += kPrefetch) {
-#pragma unroll
-      for (int k = 0; k < kPrefetch; ++k) {
-        if (tile + k < t1 && !dead) {
-          const uint32_t R[8] = {q[k][0].x, q[k][0].y, q[k][0].z, q[k][0].w, q[k][1].x, q[k][1].y, q[k][1].z, q[k][1].w};
-          const uint32_t rd_next = tr[k];
-          uint32_t tk4[16];  // token * 4: byte offset into the table
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            tk4[2 * i] = (R[i] << 2) & 0x3FFFCu;
-            tk4[2 * i + 1] = (R[i] >> 14) & 0x3FFFCu;
-          }
-          q[k][0] = ldg_stream(tok);
-          q[k][1] = ldg_stream(tok + 32);
-          tr[k] = __ldg(trp);
-          tok += 64;
-          ++trp;
-
-          // the chunks holding this tile's raw words [rd, rd_next)
-          const uint32_t c_need = rd_next > rd ? (rd_next - 1u) / kChunkWords + 1u : c_wait;
-          while (c_wait < c_need) {
-            if (!wait_chunk(c_wait)) { dead = true; break; }
-            ++c_wait;
-          }
-          rd = rd_next;
-          if (!dead) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const uint32_t a = tk4[j] + (tk4[j] >= 4u * kMissBase ? miss_adj4 : tbl_addr);
-              wbuf[k & 1][j] = lds_u32(a);
-            }
-            if (pending) consume(wbuf[(k + 1) & 1]);
-            pending = true;
-            pend_s = s;
-            if (++s == S) s = 0;
-            // every lane has issued its reads of the chunks below rd; the warp barrier orders them
-            // before the refill that may overwrite those chunks
-            __syncwarp();
-            const uint32_t c_free = rd / kChunkWords;  // chunks below this index are fully consumed
-            while (c_issue < c_stop && c_issue < c_free + kSlots) issue_chunk(d.raw, c_issue++);
-          }
-        }
-      }
+    const uint32_t n = t1 - t0;
+    bool ok = lookups(0);
+    if (ok) refill();
+    uint32_t i = 1;
+    for (; ok && i + 1 < n; i += 2) {
+      ok = lookups(1);
+      if (!ok) break;
+      consume(wbuf[0]);
+      refill();
+      ok = lookups(0);
+      if (!ok) break;
+      consume(wbuf[1]);
+      refill();
     }
-    if (dead) {
+    if (ok && i < n) {
+      ok = lookups(1);
+      if (ok) {
+        consume(wbuf[0]);
+        consume(wbuf[1]);
+      }
+    } else if (ok) {
+      consume(wbuf[0]);
+    }
+    while (ok && n_waited < n_issued) ok = wait_chunk();  // nothing may still be landing when the ring is reused
+    if (!ok) {
+      dead = true;
       *dead_flag() = 1u;
       if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
       return;
     }
-    if (pending) {
-      // the last tile's words sit in buffer (t1 - t0 - 1) & 1
-      if ((t1 - t0 - 1u) & 1u) consume(wbuf[1]);
-      else consume(wbuf[0]);
-    }
-    while (c_wait < c_issue) {  // nothing may still be landing when the ring is reused
-      if (!wait_chunk(c_wait)) { dead = true; *dead_flag() = 1u; return; }
-      ++c_wait;
-    }
     __syncwarp();
 #pragma unroll
-    for (int i = 0; i < 4; ++i) acc[i] += acc2[i];
+    for (int k = 0; k < 4; ++k) acc[k] += acc2[k];
     if (!from_start) {
       store_partial(0, rb, acc);  // the whole run lies inside one row block
     } else {
       if (first_rb != kNoBlock) store_partial(0, first_rb, first_acc);
-      if (pend_s != S - 1u) store_partial(1, rb, acc);  // the run ended inside a row block
+      if (s_p != 0) store_partial(1, rb, acc);  // the run ended inside a row block
     }
   }
 
@@ -444,7 +459,7 @@ struct TilesCta {
         const uint32_t id = part_ids()[e];
         if (id == kNoBlock) continue;
         if (id != cur) {
-          if (cur != kNoBlock) finalize(d, cur, sum);
+          if (cur != kNoBlock) finalize(d, cur, sum[0], sum[1], sum[2], sum[3]);
           cur = id;
           sum[0] = sum[1] = sum[2] = sum[3] = 0;
         }
@@ -454,7 +469,7 @@ struct TilesCta {
         sum[2] += v.z;
         sum[3] += v.w;
       }
-      if (cur != kNoBlock) finalize(d, cur, sum);
+      if (cur != kNoBlock) finalize(d, cur, sum[0], sum[1], sum[2], sum[3]);
     }
   }
 };
@@ -552,7 +567,7 @@ int sm_count_tiles() {
   return n;
 }
 
-constexpr int kTilesWarps = 8;
+constexpr int kTilesWarps = 16;
 constexpr uint32_t kSmemLimit = 232448u;  // 227 KB per CTA
 
 template <int NB, bool SIGNED>
