@@ -218,6 +218,26 @@ int tq_fused_gemv_host_static(const tq_dmat* m, const void* h_x_bf16, int B, flo
  * d_X_bf16: DEVICE [M][cols] bf16, 16-byte aligned; d_Y: DEVICE [M][rows] fp32. */
 int tq_fused_gemm(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, void* cuda_stream);
 
+/* A stack: several TQ_LAYOUT_TILES matrices that share one table (for instance every linear layer
+ * of a decoder, Section 2.3: the weights are expanded layer by layer), bound to their operands and
+ * executed by ONE persistent launch in which every SM loads the table into shared memory once and
+ * then streams its share of the row blocks of all the matrices.  The products are independent of
+ * one another: a caller whose layers feed each other makes one stack per group of layers that can
+ * run together (q/k/v; gate/up; ...).  d_x[i]: DEVICE bf16 [B][cols_i], 16-byte aligned; d_y[i]:
+ * DEVICE fp32 [B][rows_i]; B in 1..32 (one launch per two batch columns, or per column when the
+ * widest matrix leaves no room for two).  mats, d_x, d_y: HOST arrays of n_mats entries.  The
+ * work split and the operand addresses are written to the caller's DEVICE buffer d_buf (256-byte
+ * aligned, tq_stack_size bytes), which must outlive the handle, as must the matrices.
+ * TQ_ERR_UNSUPPORTED_SHAPE if the matrices do not share table, level type and layout.
+ * tq_stack_create synchronises cuda_stream; tq_fused_gemv_stack is asynchronous. */
+typedef struct tq_stack tq_stack;
+int tq_stack_size(int n_mats, uint64_t* device_bytes);
+int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* const* d_y, int n_mats,
+                    int B, void* d_buf, uint64_t d_buf_bytes, void* cuda_stream, tq_stack** out);
+int tq_fused_gemv_stack(const tq_stack* s, void* cuda_stream);
+int tq_stack_launches(const tq_stack* s); /* kernel launches one tq_fused_gemv_stack call makes */
+void tq_stack_free(tq_stack* s);
+
 /* Read and clear the matrix's device status word (TQ_STATUS_* bits); synchronises cuda_stream. */
 int tq_device_status(const tq_dmat* m, void* cuda_stream, uint32_t* status);
 

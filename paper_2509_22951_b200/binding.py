@@ -36,7 +36,8 @@ EXPORTS = [
     "tq_quantize_rows_device", "tq_build_dictionary", "tq_dict_from_entries", "tq_dict_entries",
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
-    "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_device_status", "tq_dmat_free",
+    "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_stack_size", "tq_stack_create",
+    "tq_fused_gemv_stack", "tq_stack_launches", "tq_stack_free", "tq_device_status", "tq_dmat_free",
 ]
 
 
@@ -86,6 +87,12 @@ def _load() -> C.CDLL:
         "tq_fused_gemv_host": (C.c_int, [vp, vp, C.c_int, vp, vp, vp, vp]),
         "tq_fused_gemv_host_static": (C.c_int, [vp, vp, C.c_int, vp, vp]),
         "tq_fused_gemm": (C.c_int, [vp, vp, C.c_int, vp, vp]),
+        "tq_stack_size": (C.c_int, [C.c_int, u64p]),
+        "tq_stack_create": (C.c_int, [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int, C.c_int, vp, C.c_uint64, vp,
+                                      C.POINTER(vp)]),
+        "tq_fused_gemv_stack": (C.c_int, [vp, vp]),
+        "tq_stack_launches": (C.c_int, [vp]),
+        "tq_stack_free": (None, [vp]),
         "tq_device_status": (C.c_int, [vp, vp, u32p]),
         "tq_dmat_free": (None, [vp]),
     }
@@ -366,6 +373,49 @@ def tq_fused_gemm(m: DeviceMatrix, X: torch.Tensor, Y: torch.Tensor | None = Non
     assert Y.is_cuda and Y.dtype == torch.float32 and Y.is_contiguous() and Y.numel() == M * m.info.rows
     _check(_lib.tq_fused_gemm(m._h, X2.data_ptr(), M, Y.data_ptr(), _stream_ptr(stream)), "tq_fused_gemm")
     return Y
+
+
+class Stack:
+    """Several TILES matrices bound to their operands for one persistent launch.  Keeps the
+    matrices, the operand tensors and its own device buffer alive."""
+
+    def __init__(self, handle: int, buf: torch.Tensor, mats, xs, ys, B: int):
+        self._h = C.c_void_p(handle)
+        self.buf, self.mats, self.xs, self.ys, self.B = buf, list(mats), list(xs), list(ys), B
+
+    @property
+    def launches(self) -> int:
+        return _lib.tq_stack_launches(self._h)
+
+    def __del__(self):
+        if getattr(self, "_h", None) and _lib is not None:
+            _lib.tq_stack_free(self._h)
+            self._h = None
+
+
+def tq_stack_create(mats, xs, ys, stream=None) -> Stack:
+    """mats: DeviceMatrix list (TILES layout, one table); xs[i]: CUDA bf16 [B][cols_i]; ys[i]: CUDA fp32 [B][rows_i]."""
+    n = len(mats)
+    assert n >= 1 and len(xs) == n and len(ys) == n
+    B = xs[0].numel() // mats[0].info.cols
+    for m, x, y in zip(mats, xs, ys):
+        assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.numel() == B * m.info.cols
+        assert y.is_cuda and y.dtype == torch.float32 and y.is_contiguous() and y.numel() == B * m.info.rows
+    need = C.c_uint64()
+    _check(_lib.tq_stack_size(n, C.byref(need)), "tq_stack_size")
+    buf = torch.empty(need.value, dtype=torch.uint8, device=mats[0].buf.device)
+    hm = (C.c_void_p * n)(*[m._h for m in mats])
+    hx = (C.c_void_p * n)(*[x.data_ptr() for x in xs])
+    hy = (C.c_void_p * n)(*[y.data_ptr() for y in ys])
+    out = C.c_void_p()
+    with torch.cuda.device(buf.device):
+        _check(_lib.tq_stack_create(hm, hx, hy, n, B, buf.data_ptr(), buf.numel(), _stream_ptr(stream), C.byref(out)),
+               "tq_stack_create")
+    return Stack(out.value, buf, mats, xs, ys, B)
+
+
+def tq_fused_gemv_stack(s: Stack, stream=None) -> None:
+    _check(_lib.tq_fused_gemv_stack(s._h, _stream_ptr(stream)), "tq_fused_gemv_stack")
 
 
 def tq_device_status(m: DeviceMatrix, stream=None) -> int:

@@ -655,6 +655,7 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
     t.row_blocks = img.row_blocks;
     t.has_zero = row_zero != nullptr;
     t.table_words = TQ_TILES_TABLE_WORDS;
+    m->rb_raw = std::move(img.rb_raw);
     n_hits = img.n_hits;
     n_miss = img.n_miss;
     const uint64_t n_tiles = (uint64_t)img.steps * img.row_blocks;

@@ -800,6 +800,8 @@ int tq_build_tiles_image(const uint16_t* stream, uint64_t stream_len, uint32_t r
   img->n_hits = H;
   img->n_miss = M;
   img->n_raw = n_raw;
+  img->rb_raw.resize((size_t)row_blocks + 1);
+  for (uint32_t rb = 0; rb <= row_blocks; ++rb) img->rb_raw[rb] = tile_raw_v[(uint64_t)rb * steps];
   uint8_t* base = img->blob.data();
   std::memcpy(base + off_scale, row_scale, (size_t)rows * 4);
   if (row_zero) std::memcpy(base + off_zero, row_zero, (size_t)rows * 4);

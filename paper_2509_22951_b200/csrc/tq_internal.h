@@ -70,6 +70,7 @@ struct tq_dmat {
   uint32_t gpr_pad = 0, nidx_pad = 0;
   // TILES layout
   tq_tiles_desc tiles{};
+  std::vector<uint32_t> rb_raw;  // HOST: row_blocks + 1, index of each row block's first raw word
 };
 
 // Host-side image of a matrix in the STREAM layout, ready for one cudaMemcpy.
@@ -93,6 +94,7 @@ struct tq_tiles_image {
   uint32_t steps = 0, row_blocks = 0;
   uint64_t n_hits = 0, n_miss = 0;  // of the paper's stream
   uint64_t n_raw = 0;               // raw words of the image: n_miss + the groups whose code is >= table_words
+  std::vector<uint32_t> rb_raw;     // row_blocks + 1, index of each row block's first raw word
 };
 
 int tq_num_threads();
@@ -117,3 +119,17 @@ int tq_build_planes_image(const uint16_t* stream, uint64_t stream_len, uint32_t 
 int tq_tiles_max_nb(const tq_dmat* m);
 int tq_tiles_gemv(const tq_dmat* m, const void* x, int nb, float* y, void* cuda_stream);
 int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream);
+
+// A set of TILES matrices bound to their operands, with the work split among the CTAs of one
+// persistent launch (tq_tiles.cu).
+struct tq_stack {
+  int n = 0, B = 0;
+  int levels_signed = 0;
+  uint32_t grid = 0, xstride = 0, table_words = 0;
+  const uint32_t* d_table = nullptr;
+  const tq_tiles_desc* d_descs = nullptr;  // DEVICE
+  const void* d_segs = nullptr;            // DEVICE
+  const uint32_t* d_cta_seg = nullptr;     // DEVICE
+  uint32_t n_segs = 0;
+  uint64_t x_bytes = 0, y_bytes = 0;       // sizes of the operand arenas when bound with tq_stack_create_arena
+};

@@ -26,6 +26,8 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <new>
+#include <vector>
 
 #include "tq_internal.h"
 
@@ -69,6 +71,7 @@ struct TilesParams {
   const uint32_t* table;      // 65536 words, zero past the last entry
   uint32_t table_words;       // words of it kept in shared memory
   uint32_t xstride;           // words per digit column in shared memory
+  uint32_t b0;                // stack mode: first batch column of this pass
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -506,7 +509,9 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
   } else {
     for (uint32_t si = p.cta_seg[blockIdx.x]; si < p.cta_seg[blockIdx.x + 1]; ++si) {
       const TilesSeg sg = p.segs[si];
-      const tq_tiles_desc d = p.mats[sg.mat];
+      tq_tiles_desc d = p.mats[sg.mat];
+      d.x = static_cast<const __nv_bfloat16*>(d.x) + (size_t)p.b0 * d.cols;
+      d.y += (size_t)p.b0 * d.rows;
       cta.run_segment(d, sg.rb_begin, sg.rb_end);
     }
   }
@@ -619,3 +624,159 @@ int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
                                                                        reinterpret_cast<uint32_t*>(d_codes));
   return tq_cuda_status((int)cudaGetLastError(), "decompress(tiles) launch");
 }
+
+// ---------------------------------------------------------------------------------------------
+// Stack: many matrices, one persistent launch.
+// ---------------------------------------------------------------------------------------------
+namespace {
+// Cost of a segment start (table of activations rebuilt, pipelines refilled), in bytes of stream.
+constexpr uint64_t kSegmentOverheadBytes = 96 * 1024;
+
+struct StackPlan {
+  std::vector<TilesSeg> segs;
+  std::vector<uint32_t> cta_seg;
+};
+
+// Row blocks in matrix order, cut into `grid` consecutive shares of equal cost (bytes streamed plus
+// a fixed charge per segment start).
+StackPlan plan_stack(const tq_dmat* const* mats, int n, uint32_t grid) {
+  auto rb_cost = [&](const tq_dmat* m, uint32_t rb) -> uint64_t {
+    return (uint64_t)m->tiles.steps * 1024 + (uint64_t)(m->rb_raw[rb + 1] - m->rb_raw[rb]) * 4;
+  };
+  uint64_t total = 0;
+  for (int i = 0; i < n; ++i) {
+    const tq_dmat* m = mats[i];
+    total += (uint64_t)m->tiles.steps * 1024 * m->tiles.row_blocks + (uint64_t)m->rb_raw[m->tiles.row_blocks] * 4;
+  }
+  total += kSegmentOverheadBytes * ((uint64_t)n + grid);
+  const uint64_t share = total / grid + 1;
+  StackPlan pl;
+  pl.cta_seg.push_back(0);
+  uint64_t acc = 0;  // cost given to the current CTA
+  for (int i = 0; i < n; ++i) {
+    const tq_dmat* m = mats[i];
+    uint32_t rb = 0;
+    while (rb < m->tiles.row_blocks) {
+      if (acc + kSegmentOverheadBytes >= share && pl.cta_seg.size() < grid) {  // no room for a useful segment
+        pl.cta_seg.push_back((uint32_t)pl.segs.size());
+        acc = 0;
+      }
+      acc += kSegmentOverheadBytes;
+      const uint32_t begin = rb;
+      const bool last_cta = pl.cta_seg.size() >= grid;
+      while (rb < m->tiles.row_blocks && (last_cta || acc < share)) acc += rb_cost(m, rb++);
+      pl.segs.push_back(TilesSeg{(uint32_t)i, begin, rb});
+      if (acc >= share && !last_cta) {
+        pl.cta_seg.push_back((uint32_t)pl.segs.size());
+        acc = 0;
+      }
+    }
+  }
+  while (pl.cta_seg.size() < (size_t)grid + 1) pl.cta_seg.push_back((uint32_t)pl.segs.size());
+  return pl;
+}
+
+inline uint64_t align256(uint64_t v) { return (v + 255) / 256 * 256; }
+}  // namespace
+
+extern "C" {
+
+int tq_stack_size(int n_mats, uint64_t* device_bytes) {
+  if (n_mats < 1 || !device_bytes) return TQ_ERR_INVALID_ARG;
+  const uint64_t grid = (uint64_t)sm_count_tiles();
+  *device_bytes = align256((uint64_t)n_mats * sizeof(tq_tiles_desc)) + align256(((uint64_t)n_mats + grid) * sizeof(TilesSeg)) +
+                  align256((grid + 1) * 4);
+  return TQ_OK;
+}
+
+int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* const* d_y, int n_mats, int B,
+                    void* d_buf, uint64_t d_buf_bytes, void* cuda_stream, tq_stack** out) {
+  if (!mats || !d_x || !d_y || n_mats < 1 || B < 1 || B > 32 || !d_buf || !out || ((uintptr_t)d_buf & 255))
+    return TQ_ERR_INVALID_ARG;
+  uint64_t need = 0;
+  tq_stack_size(n_mats, &need);
+  if (d_buf_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
+  uint32_t max_steps = 0;
+  for (int i = 0; i < n_mats; ++i) {
+    const tq_dmat* m = mats[i];
+    if (!m || !d_x[i] || !d_y[i] || ((uintptr_t)d_x[i] & 15)) return TQ_ERR_INVALID_ARG;
+    if (m->info.layout != TQ_LAYOUT_TILES || m->dict != mats[0]->dict ||
+        m->info.levels_signed != mats[0]->info.levels_signed)
+      return TQ_ERR_UNSUPPORTED_SHAPE;  // one table, one kind of level, TILES layout
+    max_steps = std::max(max_steps, m->tiles.steps);
+  }
+  tq_stack* s = new (std::nothrow) tq_stack();
+  if (!s) return TQ_ERR_NOMEM;
+  s->n = n_mats;
+  s->B = B;
+  s->levels_signed = mats[0]->info.levels_signed;
+  s->grid = (uint32_t)sm_count_tiles();
+  s->xstride = max_steps * 32u + 4u;
+  s->table_words = mats[0]->tiles.table_words;
+  s->d_table = mats[0]->dict->d_table;
+  if (tiles_smem(s->table_words, 3u * s->xstride, kTilesWarps).total > kSmemLimit) {
+    delete s;
+    return TQ_ERR_UNSUPPORTED_SHAPE;
+  }
+  const StackPlan pl = plan_stack(mats, n_mats, s->grid);
+  std::vector<tq_tiles_desc> descs((size_t)n_mats);
+  for (int i = 0; i < n_mats; ++i) {
+    descs[i] = mats[i]->tiles;
+    descs[i].x = d_x[i];
+    descs[i].y = d_y[i];
+  }
+  uint8_t* base = static_cast<uint8_t*>(d_buf);
+  const uint64_t off_segs = align256((uint64_t)n_mats * sizeof(tq_tiles_desc));
+  const uint64_t off_cta = off_segs + align256(((uint64_t)n_mats + s->grid) * sizeof(TilesSeg));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int rc = tq_cuda_status((int)cudaMemcpyAsync(base, descs.data(), descs.size() * sizeof(tq_tiles_desc), cudaMemcpyHostToDevice, st), "stack upload");
+  if (rc == TQ_OK)
+    rc = tq_cuda_status((int)cudaMemcpyAsync(base + off_segs, pl.segs.data(), pl.segs.size() * sizeof(TilesSeg), cudaMemcpyHostToDevice, st), "stack upload");
+  if (rc == TQ_OK)
+    rc = tq_cuda_status((int)cudaMemcpyAsync(base + off_cta, pl.cta_seg.data(), pl.cta_seg.size() * 4, cudaMemcpyHostToDevice, st), "stack upload");
+  if (rc == TQ_OK) rc = tq_cuda_status((int)cudaStreamSynchronize(st), "stack upload");
+  if (rc != TQ_OK) {
+    delete s;
+    return rc;
+  }
+  s->d_descs = reinterpret_cast<const tq_tiles_desc*>(base);
+  s->d_segs = base + off_segs;
+  s->d_cta_seg = reinterpret_cast<const uint32_t*>(base + off_cta);
+  s->n_segs = (uint32_t)pl.segs.size();
+  *out = s;
+  return TQ_OK;
+}
+
+int tq_fused_gemv_stack(const tq_stack* s, void* cuda_stream) {
+  if (!s) return TQ_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  TilesParams p{};
+  p.mats = s->d_descs;
+  p.segs = static_cast<const TilesSeg*>(s->d_segs);
+  p.cta_seg = s->d_cta_seg;
+  p.table = s->d_table;
+  p.table_words = s->table_words;
+  p.xstride = s->xstride;
+  const bool two = tiles_smem(s->table_words, 6u * s->xstride, kTilesWarps).total <= kSmemLimit;
+  for (int b0 = 0; b0 < s->B;) {
+    const int nb = (two && s->B - b0 >= 2) ? 2 : 1;
+    p.b0 = (uint32_t)b0;
+    const TilesSmem L = tiles_smem(p.table_words, 3u * nb * p.xstride, kTilesWarps);
+    int rc;
+    if (nb == 1) rc = s->levels_signed ? launch_tiles<1, true>(p, s->grid, L.total, st) : launch_tiles<1, false>(p, s->grid, L.total, st);
+    else rc = s->levels_signed ? launch_tiles<2, true>(p, s->grid, L.total, st) : launch_tiles<2, false>(p, s->grid, L.total, st);
+    if (rc != TQ_OK) return rc;
+    b0 += nb;
+  }
+  return TQ_OK;
+}
+
+int tq_stack_launches(const tq_stack* s) {
+  if (!s) return TQ_ERR_INVALID_ARG;
+  const bool two = tiles_smem(s->table_words, 6u * s->xstride, kTilesWarps).total <= kSmemLimit;
+  return two ? (s->B + 1) / 2 : s->B;
+}
+
+void tq_stack_free(tq_stack* s) { delete s; }
+
+}  // extern "C"

@@ -213,3 +213,51 @@ def test_fused_gemm_agrees_with_fused_gemv(tq):
     a = tq.tq_fused_gemm(m, X)
     b = tq.tq_fused_gemv(m, X)
     assert float((a - b).abs().max() / b.abs().max()) < 1e-5
+
+
+# ------------------------------------------------------------------ stack: one persistent launch
+@pytest.mark.parametrize("B", [1, 2, 3])
+def test_stack_matches_oracle_and_single_calls(tq, B):
+    """Several matrices of different shapes behind one table, one launch.  The integer sums make
+    the result independent of how row blocks and columns are split among CTAs and warps, so the
+    stack must reproduce the single-matrix calls bit for bit, and both must match the oracle."""
+    shapes = [(300, 1024), (17, 8192), (1024, 3072), (16, 128), (530, 2052), (2048, 512)]
+    rng = np.random.default_rng(100 + B)
+    qs = [np.clip(np.rint(rng.standard_t(5, size=s) * 4), -127, 127).astype(np.int8) for s in shapes]
+    ss = [(rng.random(r) + 0.5).astype(np.float32) for r, _ in shapes]
+    d, streams = _oracle_pack(qs)
+    dd = tq.tq_dict_upload(tq.tq_dict_from_entries(d.entries))
+    mats = [tq.tq_upload(dd, st, r, c, s, layout=tq.TQ_LAYOUT_TILES) for st, (r, c), s in zip(streams, shapes, ss)]
+    xs = [synth.activations(B, c, 300 + i).cuda() for i, (_, c) in enumerate(shapes)]
+    ys = [torch.full((B, r), float("nan"), dtype=torch.float32, device="cuda") for r, _ in shapes]
+    stack = tq.tq_stack_create(mats, xs, ys)
+    assert stack.launches == (B + 1) // 2 or stack.launches == B
+    for _ in range(2):  # a second launch reuses everything the first left behind
+        for y in ys:
+            y.fill_(float("nan"))
+        tq.tq_fused_gemv_stack(stack)
+        torch.cuda.synchronize()
+        for m, q, s, x, y in zip(mats, qs, ss, xs, ys):
+            single = tq.tq_fused_gemv(m, x)
+            assert torch.equal(single, y)
+            yref = oracle.layer_forward(q, s, x.cpu().double().numpy())
+            assert _rel_err(y.cpu().numpy().astype(np.float64), yref) <= TOL
+            assert tq.tq_device_status(m) == 0
+
+
+def test_stack_rejects_mixed_tables_and_layouts(tq):
+    rng = np.random.default_rng(9)
+    q = rng.integers(-3, 4, size=(32, 256)).astype(np.int8)
+    s = np.ones(32, dtype=np.float32)
+    d, (stream,) = _oracle_pack([q])
+    dd1 = tq.tq_dict_upload(tq.tq_dict_from_entries(d.entries))
+    dd2 = tq.tq_dict_upload(tq.tq_dict_from_entries(d.entries))
+    a = tq.tq_upload(dd1, stream, 32, 256, s, layout=tq.TQ_LAYOUT_TILES)
+    b = tq.tq_upload(dd2, stream, 32, 256, s, layout=tq.TQ_LAYOUT_TILES)
+    c = tq.tq_upload(dd1, stream, 32, 256, s, layout=tq.TQ_LAYOUT_PLANES)
+    x = synth.activations(1, 256, 1).cuda()
+    y = torch.empty((1, 32), dtype=torch.float32, device="cuda")
+    for pair in ([a, b], [a, c]):
+        with pytest.raises(tq.TqError) as e:
+            tq.tq_stack_create(pair, [x, x], [y, y.clone()])
+        assert e.value.status == tq.TQ_ERR_UNSUPPORTED_SHAPE
