@@ -103,6 +103,11 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the ncu capture
+# summarised under profiles/ (None: not captured for that launch shape, or kernel changed since).
+TRAFFIC = {}
+
+
 def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout=1):
     """Generate, quantize (GPU), build the table and encode (host), upload.  Returns
     (matrices, xs, ys, table, stats)."""
@@ -126,19 +131,34 @@ def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout
         mats.append(tq.tq_upload(dd, stream, rows, cols, scales[i], layout=layout))
         del stream
     t3 = time.time()
-    xs = [synth.activations(batch, cols, 7000 + i, device=device) for i, (_, rows, cols) in enumerate(shapes)]
-    ys = [torch.empty((batch, rows), dtype=torch.float32, device=device) for (_, rows, cols) in shapes]
+    # all x in one arena and all y in another (16-byte aligned pieces), so that the end-to-end
+    # path moves each with one copy
+    xoff, yoff, xo, yo = [], [], 0, 0
+    for (_, rows, cols) in shapes:
+        xoff.append(xo)
+        yoff.append(yo)
+        xo += -(-batch * cols // 8) * 8
+        yo += -(-batch * rows // 4) * 4
+    x_arena = torch.zeros(xo, dtype=torch.bfloat16, device=device)
+    y_arena = torch.zeros(yo, dtype=torch.float32, device=device)
+    xs, ys = [], []
+    for i, (_, rows, cols) in enumerate(shapes):
+        x = x_arena[xoff[i]: xoff[i] + batch * cols].view(batch, cols)
+        x.copy_(synth.activations(batch, cols, 7000 + i, device=device))
+        xs.append(x)
+        ys.append(y_arena[yoff[i]: yoff[i] + batch * rows].view(batch, rows))
     stats = {"gen_quant_s": t1 - t0, "table_s": t2 - t1, "encode_upload_s": t3 - t2, "K": hd.K}
-    return mats, xs, ys, hd, q_host, scales, stats
+    return mats, xs, ys, hd, q_host, scales, stats, x_arena, y_arena, dd
 
 
 def algorithmic_bytes(info, batch):
-    """Bytes the method has to move for one call: the tokens of the layout in use, an 8-byte row
-    index, the row scale, x and y.  Padding is not counted."""
+    """Bytes the method has to move for one call: the tokens and raw words of the layout in use
+    (for tiles: with the table limited to what shared memory holds), its index, the row scale, x
+    and y.  Padding is not counted."""
     if info.layout == 0:   # paper stream: 2 bytes per code, 10 per escaped group
         tokens = info.stream_bytes
-    else:                  # planes: one 2-byte token per group + one 4-byte word per escaped group
-        tokens = 2 * (info.n_hits + info.n_miss) + 4 * info.n_miss
+    else:                  # planes / tiles: one 2-byte token per group + one 4-byte word per raw group
+        tokens = 2 * (info.n_hits + info.n_miss) + 4 * info.n_raw_words
     if info.layout == 2:   # tiles: a 4-byte raw-stream index per tile of 16 rows x 128 columns
         index = 4 * (-(-info.rows // 16) * -(-info.cols // 128) + 1)
     else:
@@ -168,7 +188,7 @@ def oracle_sample_run(hd_entries, q_host, scales, shapes, batch, sample_idx, rep
     return total, times
 
 
-def time_extras(tq, mats, infos, shapes, args, device, stream):
+def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
     """Standalone tq_decompress of the whole weight set and the prefill product (tq_fused_gemm) at
     M tokens, timed with CUDA events on the launching stream (3 warm-ups, inputs far larger than L2)."""
     out = {}
@@ -197,7 +217,14 @@ def time_extras(tq, mats, infos, shapes, args, device, stream):
     out["decompress"] = {"ms": ms, "GB_per_s": (rd + n_weights) / (ms * 1e-3) / 1e9,
                          "bytes": {"read": rd, "written": n_weights},
                          "frac_of_measured_hbm": (rd + n_weights) / (ms * 1e-3) / 1e9 / measured_peaks()[0]}
-    if args.layout == "planes":
+    if args.layout != "stream":
+        if args.layout != "planes":  # the tensor-core product reads the PLANES layout: upload it beside the other
+            gemm_mats = []
+            for i, (name, rows, cols) in enumerate(shapes):
+                stream_i, _, _ = tq.tq_encode(extra["hd"], extra["q_host"][i])
+                gemm_mats.append(tq.tq_upload(extra["dd"], stream_i, rows, cols, extra["scales"][i], layout=1))
+                del stream_i
+            mats = gemm_mats
         M = args.prefill_tokens
         max_rows = max(i.rows for i in infos)
         Y = torch.empty(M * max_rows, dtype=torch.float32, device=device)
@@ -241,7 +268,8 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="decoder layers to build (default: all)")
     ap.add_argument("--no-lm-head", action="store_true")
     ap.add_argument("--shapes", default=None, help="custom workload, e.g. 32768x3072,3072x8192 (profiling cases)")
-    ap.add_argument("--layout", default="planes", choices=["stream", "planes", "tiles"])
+    ap.add_argument("--layout", default="tiles", choices=["stream", "planes", "tiles"])
+    ap.add_argument("--per-layer", action="store_true", help="tiles layout: one launch per matrix instead of one persistent launch for the stack")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -295,7 +323,7 @@ def main():
         dist.broadcast(ent, 0)
         table_entries = ent.cpu().numpy()
 
-    mats, xs, ys, hd, q_host, scales, stats = build_model(tq, shapes, args.batch, device, threads, table_entries, layout={"stream": 0, "planes": 1, "tiles": 2}[args.layout])
+    mats, xs, ys, hd, q_host, scales, stats, x_arena, y_arena, dd = build_model(tq, shapes, args.batch, device, threads, table_entries, layout={"stream": 0, "planes": 1, "tiles": 2}[args.layout])
     infos = [m.info for m in mats]
     hits = sum(i.n_hits for i in infos)
     miss = sum(i.n_miss for i in infos)
@@ -306,11 +334,21 @@ def main():
         f"stream {stream_bytes/1e9:.3f} GB, setup {stats}")
 
     stream = torch.cuda.Stream(device)
-    launches_per_step = len(mats) * ((args.batch + 3) // 4)
+    use_stack = args.layout == "tiles" and not args.per_layer
+    hit_rate_device = 1.0 - sum(i.n_raw_words for i in infos) / (hits + miss)
+    if use_stack:
+        stack = tq.tq_stack_create(mats, xs, ys)
+        launches_per_step = stack.launches
 
-    def step_plain():
-        for m, x, y in zip(mats, xs, ys):
-            tq.tq_fused_gemv(m, x, y)
+        def step_plain():
+            tq.tq_fused_gemv_stack(stack)
+    else:
+        per_pass = 4 if args.layout != "tiles" else 2
+        launches_per_step = len(mats) * (-(-args.batch // per_pass))
+
+        def step_plain():
+            for m, x, y in zip(mats, xs, ys):
+                tq.tq_fused_gemv(m, x, y)
 
     with torch.cuda.stream(stream):
         step_plain()  # sets kernel attributes before any capture
@@ -369,9 +407,16 @@ def main():
             hy = [torch.empty(y.shape, dtype=torch.float32).pin_memory() for y in ys]
             e_steps = max(3, min(args.steps, 10))
 
-            def step_e2e():
-                for m, a, b, dx, dy in zip(mats, hx, hy, xs, ys):
-                    tq.tq_fused_gemv_host(m, a, b, dx, dy)
+            if use_stack:
+                hxa = x_arena.cpu().pin_memory()
+                hya = torch.empty(y_arena.shape, dtype=torch.float32).pin_memory()
+
+                def step_e2e():
+                    tq.tq_fused_gemv_stack_host(stack, hxa, x_arena, hya, y_arena)
+            else:
+                def step_e2e():
+                    for m, a, b, dx, dy in zip(mats, hx, hy, xs, ys):
+                        tq.tq_fused_gemv_host(m, a, b, dx, dy)
 
             for _ in range(3):
                 step_e2e()
@@ -394,7 +439,8 @@ def main():
         # ---- the other device calls on the same resident model (single GPU only) ----
         extras = {}
         if not args.no_extras and world == 1:
-            extras = time_extras(tq, mats, infos, shapes, args, device, stream)
+            extras = time_extras(tq, mats, infos, shapes, args, device, stream,
+                                 {"hd": hd, "dd": dd, "q_host": q_host, "scales": scales})
 
     ms_step = ms_total / args.steps
     if world > 1:
@@ -420,9 +466,14 @@ def main():
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8 weights x bf16 activations, fp32 accumulate",
         "data": "synthetic",
-        "config": {"workload": workload, "n_weights": n_weights, "hit_rate": hits / (hits + miss), "K": stats["K"],
+        "config": {"workload": workload, "n_weights": n_weights, "hit_rate": hits / (hits + miss),
+                   "hit_rate_device_layout": hit_rate_device, "K": stats["K"],
+                   "launch": ("one persistent launch over all matrices (tq_fused_gemv_stack)" if use_stack
+                              else "one launch per matrix (tq_fused_gemv)"),
                    "layout": {"stream": "paper token stream, per-row segments", "planes": "two planes: fixed-stride tokens + packed raw words",
-                              "tiles": "1 KB token tiles of 16 rows x 32 groups in integer-MMA operand order + one raw-word stream"}[args.layout], "cuda_graph": graph is not None,
+                              "tiles": "1 KB token tiles of 16 rows x 32 groups in integer-MMA operand order + one raw-word stream; "
+                                       "table limited to the %d words shared memory holds" % tq.TQ_TILES_TABLE_WORDS}[args.layout],
+                   "cuda_graph": graph is not None,
                    "l2": "inputs larger than L2: each step streams %.2f GB" % (payload_bytes / 1e9),
                    "multi_gpu": "independent replicas, no data-path collective" if world > 1 else "single GPU"},
         "us_per_token": ms_step * 1e3 / args.batch,
@@ -432,8 +483,10 @@ def main():
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
-                     "traffic": None, "kernel": "gemv_kernel", "peak_source": peak_src,
-                     "note": "achieved = algorithmic bytes of the %d launches of a step / step time (launch gaps included)" % launches_per_step},
+                     "traffic": TRAFFIC.get(args.layout if not use_stack else "tiles_stack"),
+                     "kernel": {"stream": "gemv_kernel", "planes": "gemv_planes_kernel", "tiles": "gemv_tiles_kernel"}[args.layout],
+                     "peak_source": peak_src,
+                     "note": "achieved = algorithmic bytes of the %d launch(es) of a step / step time (launch gaps included)" % launches_per_step},
         "setup_s": stats,
     }
     out.update(extras)

@@ -235,6 +235,11 @@ int tq_stack_size(int n_mats, uint64_t* device_bytes);
 int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* const* d_y, int n_mats,
                     int B, void* d_buf, uint64_t d_buf_bytes, void* cuda_stream, tq_stack** out);
 int tq_fused_gemv_stack(const tq_stack* s, void* cuda_stream);
+/* The same call with HOST operands, for a stack whose d_x[i] all lie in one DEVICE arena of x_bytes
+ * and whose d_y[i] all lie in one DEVICE arena of y_bytes: copies h_x (the arena's image, HOST) in,
+ * runs the stack, copies the y arena out to h_y, all on cuda_stream, without synchronising. */
+int tq_fused_gemv_stack_host(const tq_stack* s, const void* h_x, void* d_x_arena, uint64_t x_bytes,
+                             float* h_y, const float* d_y_arena, uint64_t y_bytes, void* cuda_stream);
 int tq_stack_launches(const tq_stack* s); /* kernel launches one tq_fused_gemv_stack call makes */
 void tq_stack_free(tq_stack* s);
 

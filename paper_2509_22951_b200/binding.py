@@ -37,7 +37,7 @@ EXPORTS = [
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
     "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_stack_size", "tq_stack_create",
-    "tq_fused_gemv_stack", "tq_stack_launches", "tq_stack_free", "tq_device_status", "tq_dmat_free",
+    "tq_fused_gemv_stack", "tq_fused_gemv_stack_host", "tq_stack_launches", "tq_stack_free", "tq_device_status", "tq_dmat_free",
 ]
 
 
@@ -91,6 +91,7 @@ def _load() -> C.CDLL:
         "tq_stack_create": (C.c_int, [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int, C.c_int, vp, C.c_uint64, vp,
                                       C.POINTER(vp)]),
         "tq_fused_gemv_stack": (C.c_int, [vp, vp]),
+        "tq_fused_gemv_stack_host": (C.c_int, [vp, vp, vp, C.c_uint64, vp, vp, C.c_uint64, vp]),
         "tq_stack_launches": (C.c_int, [vp]),
         "tq_stack_free": (None, [vp]),
         "tq_device_status": (C.c_int, [vp, vp, u32p]),
@@ -416,6 +417,17 @@ def tq_stack_create(mats, xs, ys, stream=None) -> Stack:
 
 def tq_fused_gemv_stack(s: Stack, stream=None) -> None:
     _check(_lib.tq_fused_gemv_stack(s._h, _stream_ptr(stream)), "tq_fused_gemv_stack")
+
+
+def tq_fused_gemv_stack_host(s: Stack, h_x: torch.Tensor, d_x_arena: torch.Tensor, h_y: torch.Tensor,
+                             d_y_arena: torch.Tensor, stream=None) -> None:
+    """h_x / h_y: CPU (pinned) images of the x / y arenas the stack's operands live in."""
+    assert (not h_x.is_cuda) and (not h_y.is_cuda) and d_x_arena.is_cuda and d_y_arena.is_cuda
+    xb = d_x_arena.numel() * d_x_arena.element_size()
+    yb = d_y_arena.numel() * d_y_arena.element_size()
+    assert h_x.numel() * h_x.element_size() == xb and h_y.numel() * h_y.element_size() == yb
+    _check(_lib.tq_fused_gemv_stack_host(s._h, h_x.data_ptr(), d_x_arena.data_ptr(), xb, h_y.data_ptr(),
+                                         d_y_arena.data_ptr(), yb, _stream_ptr(stream)), "tq_fused_gemv_stack_host")
 
 
 def tq_device_status(m: DeviceMatrix, stream=None) -> int:

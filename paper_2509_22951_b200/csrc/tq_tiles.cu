@@ -771,6 +771,16 @@ int tq_fused_gemv_stack(const tq_stack* s, void* cuda_stream) {
   return TQ_OK;
 }
 
+int tq_fused_gemv_stack_host(const tq_stack* s, const void* h_x, void* d_x_arena, uint64_t x_bytes, float* h_y,
+                             const float* d_y_arena, uint64_t y_bytes, void* cuda_stream) {
+  if (!s || !h_x || !d_x_arena || !h_y || !d_y_arena) return TQ_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (int rc = tq_cuda_status((int)cudaMemcpyAsync(d_x_arena, h_x, x_bytes, cudaMemcpyHostToDevice, st), "stack: copy of x"))
+    return rc;
+  if (int rc = tq_fused_gemv_stack(s, cuda_stream)) return rc;
+  return tq_cuda_status((int)cudaMemcpyAsync(h_y, d_y_arena, y_bytes, cudaMemcpyDeviceToHost, st), "stack: copy of y");
+}
+
 int tq_stack_launches(const tq_stack* s) {
   if (!s) return TQ_ERR_INVALID_ARG;
   const bool two = tiles_smem(s->table_words, 6u * s->xstride, kTilesWarps).total <= kSmemLimit;

@@ -261,3 +261,41 @@ def test_stack_rejects_mixed_tables_and_layouts(tq):
         with pytest.raises(tq.TqError) as e:
             tq.tq_stack_create(pair, [x, x], [y, y.clone()])
         assert e.value.status == tq.TQ_ERR_UNSUPPORTED_SHAPE
+
+
+# ------------------------------------------------------------------ full size, as benchmarked
+def test_full_3b_stack_as_benchmarked_on_sampled_rows(tq):
+    """The whole LLaMA-3.2-3B linear stack (197 matrices, 3.2 G weights) built by the benchmark's
+    own builder and run in the launch configuration the benchmark times (one persistent launch,
+    batch 1).  The oracle regenerates sampled rows, quantizes them itself and computes their
+    outputs one by one; decoded levels of those rows must match bit for bit."""
+    import bench
+
+    shapes = synth.llama32_linear_shapes("3b")
+    device = torch.device("cuda", 0)
+    mats, xs, ys, hd, q_host, scales, stats, x_arena, y_arena, dd = bench.build_model(
+        tq, shapes, 1, device, 0, None, layout=tq.TQ_LAYOUT_TILES)
+    stack = tq.tq_stack_create(mats, xs, ys)
+    y_arena.fill_(float("nan"))
+    tq.tq_fused_gemv_stack(stack)
+    torch.cuda.synchronize()
+    assert not torch.isnan(y_arena).any()
+    rng = np.random.default_rng(2025)
+    picks = [0, 1, 2, 3, 4, 5, 6, 97, 100, 103, 190, 195, 196]  # every kind of layer, first/middle/last, lm_head
+    for i in picks:
+        name, rows, cols = shapes[i]
+        sample = np.sort(rng.choice(rows, 24, replace=False))
+        sample[0], sample[-1] = 0, rows - 1
+        w = synth.weight(rows, cols, synth.matrix_seed(i), device=device)[torch.from_numpy(sample).to(device)].cpu().numpy()
+        qo, so = oracle.quantize_rows(w)
+        assert np.array_equal(qo, q_host[i][sample]) and np.array_equal(so, scales[i][sample])
+        x = xs[i].cpu().double().numpy()
+        yref = oracle.layer_forward(qo, so, x)
+        y = ys[i][:, torch.from_numpy(sample).to(device)].cpu().numpy().astype(np.float64)
+        err = np.max(np.abs(y - yref), axis=1) / np.max(np.abs(yref), axis=1)
+        assert float(err.max()) <= TOL, (name, err)
+        assert tq.tq_device_status(mats[i]) == 0
+    # decoded levels of one mid-sized matrix, whole, against the levels that were encoded
+    i = 6
+    got = tq.tq_decompress(mats[i])
+    assert np.array_equal(got.cpu().numpy().view(np.int8), q_host[i])
