@@ -727,15 +727,7 @@ int tq_fused_gemv(const tq_dmat* m, const void* d_x_bf16, int B, float* d_y, voi
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(d_x_bf16);
   const uint32_t rows = m->info.rows, cols = m->info.cols;
-  if (m->info.layout == TQ_LAYOUT_TILES) {  // up to two batch columns per pass of the integer-MMA kernel
-    const int per_pass = tq_tiles_max_nb(m);
-    if (per_pass < 1) return TQ_ERR_UNSUPPORTED_SHAPE;
-    for (int b0 = 0; b0 < B; b0 += per_pass) {
-      if (int rc = tq_tiles_gemv(m, x + (size_t)b0 * cols, std::min(per_pass, B - b0), d_y + (size_t)b0 * rows, cuda_stream))
-        return rc;
-    }
-    return TQ_OK;
-  }
+  if (m->info.layout == TQ_LAYOUT_TILES) return tq_tiles_gemv(m, x, B, d_y, cuda_stream);
   // fp32 x for up to 4 batch columns must fit the 227 KB of shared memory
   const bool planes = m->info.layout == TQ_LAYOUT_PLANES;
   const size_t xcols = planes ? ((((size_t)m->gpr_pad + 255) >> 8) << 10) : cols;  // staged columns per batch column

@@ -115,7 +115,7 @@ int tq_build_planes_image(const uint16_t* stream, uint64_t stream_len, uint32_t 
                           uint32_t K, const float* row_scale, const float* row_zero,
                           uint64_t* device_bytes, tq_planes_image* img);
 
-// TILES layout entry points (tq_tiles.cu).  x: bf16 [nb][cols], nb in 1..tq_tiles_max_nb(m); y: fp32 [nb][rows].
+// TILES layout entry points (tq_tiles.cu).  x: bf16 [B][cols], y: fp32 [B][rows], any B >= 1.
 int tq_tiles_max_nb(const tq_dmat* m);
 int tq_tiles_gemv(const tq_dmat* m, const void* x, int nb, float* y, void* cuda_stream);
 int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream);

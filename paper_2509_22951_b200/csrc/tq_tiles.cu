@@ -72,6 +72,7 @@ struct TilesParams {
   uint32_t table_words;       // words of it kept in shared memory
   uint32_t xstride;           // words per digit column in shared memory
   uint32_t b0;                // stack mode: first batch column of this pass
+  uint32_t nb_valid;          // wide passes: vectors present (<= the kernel's NB)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -517,6 +518,336 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Wide batches (3..8 activation vectors per pass): the digit columns of all vectors no longer fit
+// shared memory for a whole row, so the CTA works in column panels of kPanelSteps tiles.  Every warp
+// owns whole row blocks and all warps walk their blocks in step (tile i of every warp covers the
+// same 128 columns), so one panel of digits -- double buffered, rebuilt by all threads while the
+// previous one is in use, one CTA barrier per panel -- serves all 16 warps.  Up to 24 digit columns
+// = three 8-column MMA tiles per decoded word.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPanelSteps = 4;
+constexpr int kPanelStride = kPanelSteps * 32 + 4;  // words per digit column of one panel buffer
+
+struct XInfo8 {
+  double out_scale[8];
+  double sum_x[8];
+};
+
+// Lane L ends up with all digit sums of row L & 15; lanes 0-15 write the even batch columns, lanes
+// 16-31 the odd ones.
+template <int NB, int NT>
+__device__ __noinline__ void panel_finalize(const float* __restrict__ scale, const float* __restrict__ zero,
+                                            float* __restrict__ y, uint32_t rows, uint32_t has_zero, const XInfo8* xi,
+                                            uint32_t nb_valid, uint32_t rb, const int (&c)[NT][4]) {
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t row = lane & 15u, half = lane >> 4;
+  const uint32_t r = rb * 16u + row;
+  int dsum[3 * NB];
+#pragma unroll
+  for (int col = 0; col < 3 * NB; ++col) {
+    const int nt = col >> 3, w = col & 7;
+    const uint32_t src = (row & 7u) * 4u + (uint32_t)(w >> 1);
+    const int lo = __shfl_sync(kFull, c[nt][w & 1], src), hi = __shfl_sync(kFull, c[nt][2 + (w & 1)], src);
+    dsum[col] = (row & 8u) ? hi : lo;
+  }
+#pragma unroll
+  for (int b = 0; b < NB; ++b) {
+    if ((uint32_t)(b & 1) == half && (uint32_t)b < nb_valid && r < rows) {
+      const long long Y = (long long)dsum[3 * b] + 256ll * dsum[3 * b + 1] + 65536ll * dsum[3 * b + 2];
+      double v = (double)Y * xi->out_scale[b];
+      if (has_zero) v -= (double)zero[r] * xi->sum_x[b];
+      y[(size_t)b * rows + r] = (float)((double)scale[r] * v);
+    }
+  }
+}
+
+template <int W, int NB, bool SIGNED>
+struct PanelCta {
+  static constexpr int kThreads = W * 32;
+  static constexpr int NCOL = 3 * NB;
+  static constexpr int NT = (NCOL + 7) / 8;
+  static constexpr int kBufWords = 8 * NT * kPanelStride;  // one panel buffer: whole MMA tiles of columns
+
+  uint8_t* smem;
+  TilesSmem L;
+  uint32_t tbl_addr, warp, lane, nb_valid;
+  uint32_t ring_addr, bar_base;
+  uint32_t n_issued = 0, n_waited = 0;
+
+  // misc: [0] dead flag, +16 amax bits[8], +64 in_scale[8], +128 XInfo8, +256 sums[8]
+  __device__ __forceinline__ volatile uint32_t* dead_flag() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
+  __device__ __forceinline__ uint32_t* amax_bits() { return reinterpret_cast<uint32_t*>(smem + L.misc + 16); }
+  __device__ __forceinline__ float* in_scale() { return reinterpret_cast<float*>(smem + L.misc + 64); }
+  __device__ __forceinline__ XInfo8* xinfo() { return reinterpret_cast<XInfo8*>(smem + L.misc + 128); }
+  __device__ __forceinline__ long long* sums() { return reinterpret_cast<long long*>(smem + L.misc + 256); }
+
+  __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t pos) {
+    if (lane == 0) {
+      const uint32_t bar = bar_base + (n_issued & (kSlots - 1u)) * 8u;
+      mbar_expect_tx(bar, kChunkWords * 4u);
+      bulk_g2s(ring_addr + ((pos * 4u) & (kRingWords * 4u - 1u)), raw + pos, kChunkWords * 4u, bar);
+    }
+    ++n_issued;
+  }
+  __device__ __forceinline__ bool wait_chunk() {
+    const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
+    const uint32_t par = (n_waited >> 2) & 1u;
+    ++n_waited;
+    if (mbar_try(bar, par)) return true;
+    return tiles_wait_slow(bar, par, dead_flag());
+  }
+
+  // digits of one activation group (4 columns) -> three words
+  static __device__ __forceinline__ void digits(uint2 v, float scale, bool finite, uint32_t& w0, uint32_t& w1,
+                                                uint32_t& w2, long long* sum) {
+    const uint32_t h[4] = {v.x << 16, v.x & 0xFFFF0000u, v.y << 16, v.y & 0xFFFF0000u};
+    w0 = w1 = w2 = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      int X = finite ? __float2int_rn(__uint_as_float(h[i]) * scale) : 0;
+      if (sum) *sum += X;
+      const int d0 = (int)(signed char)(X & 0xFF);
+      X = (X - d0) >> 8;
+      const int d1 = (int)(signed char)(X & 0xFF);
+      const int d2 = (X - d1) >> 8;
+      w0 |= (uint32_t)(d0 & 0xFF) << (8 * i);
+      w1 |= (uint32_t)(d1 & 0xFF) << (8 * i);
+      w2 |= (uint32_t)(d2 & 0xFF) << (8 * i);
+    }
+  }
+
+  // Per-vector scales (and, with zero points, the sum of each vector's fixed-point values).
+  __device__ void prepare_scales(const tq_tiles_desc& d) {
+    const uint32_t tid = threadIdx.x;
+    const uint32_t G = d.cols >> 2;
+    const uint2* xg = reinterpret_cast<const uint2*>(d.x);
+    if (tid < 8) {
+      amax_bits()[tid] = 0u;
+      sums()[tid] = 0;
+    }
+    __syncthreads();
+    for (uint32_t b = 0; b < nb_valid; ++b) {
+      uint32_t m = 0;
+      for (uint32_t g = tid; g < G; g += kThreads) {
+        const uint2 v = __ldg(xg + (size_t)b * G + g);
+        const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu;
+        m = max(max(m, a0 & 0xFFFFu), max(a0 >> 16, max(a1 & 0xFFFFu, a1 >> 16)));
+      }
+#pragma unroll
+      for (int sft = 16; sft > 0; sft >>= 1) m = max(m, __shfl_xor_sync(kFull, m, sft));
+      if (lane == 0) atomicMax(&amax_bits()[b], m);
+    }
+    __syncthreads();
+    if (tid < 8) {
+      const uint32_t mb = amax_bits()[tid];
+      const bool finite = mb < 0x7F80u;
+      const int e = max((int)(mb >> 7) - 126, -100);
+      // a non-finite vector: scale 0 (all digits zero) and a NaN output scale
+      in_scale()[tid] = finite ? __uint_as_float((uint32_t)(127 + 22 - e) << 23) : 0.f;
+      xinfo()->out_scale[tid] = finite ? __longlong_as_double((long long)(1023 + e - 22) << 52)
+                                       : __longlong_as_double(0x7FF8000000000000ll);
+    }
+    __syncthreads();
+    if (d.has_zero) {
+      for (uint32_t b = 0; b < nb_valid; ++b) {
+        const float sc = in_scale()[b];
+        long long sum = 0;
+        for (uint32_t g = tid; g < G; g += kThreads) {
+          uint32_t w0, w1, w2;
+          digits(__ldg(xg + (size_t)b * G + g), sc, true, w0, w1, w2, &sum);
+        }
+#pragma unroll
+        for (int sft = 16; sft > 0; sft >>= 1) sum += __shfl_xor_sync(kFull, sum, sft);
+        if (lane == 0) atomicAdd(reinterpret_cast<unsigned long long*>(&sums()[b]), (unsigned long long)sum);
+      }
+      __syncthreads();
+      if (tid < 8) xinfo()->sum_x[tid] = xinfo()->out_scale[tid] * (double)sums()[tid];
+    }
+  }
+
+  // Digits of step panel P (steps P*kPanelSteps ..) of all vectors into buffer `buf`.
+  __device__ __forceinline__ void fill_panel(const tq_tiles_desc& d, uint32_t P, uint32_t buf) {
+    const uint32_t G = d.cols >> 2;
+    const uint2* xg = reinterpret_cast<const uint2*>(d.x);
+    uint32_t* xs = reinterpret_cast<uint32_t*>(smem + L.x) + buf * kBufWords;
+    constexpr uint32_t kGroups = kPanelSteps * 32;
+    for (uint32_t idx = threadIdx.x; idx < kGroups * NB; idx += kThreads) {
+      const uint32_t gl = idx % kGroups, b = idx / kGroups;
+      const uint32_t g = P * kGroups + gl;
+      uint32_t w0 = 0, w1 = 0, w2 = 0;
+      if (g < G && b < nb_valid) digits(__ldg(xg + (size_t)b * G + g), in_scale()[b], true, w0, w1, w2, nullptr);
+      xs[(3 * b + 0) * kPanelStride + gl] = w0;
+      xs[(3 * b + 1) * kPanelStride + gl] = w1;
+      xs[(3 * b + 2) * kPanelStride + gl] = w2;
+    }
+  }
+
+  // Row blocks [rb0, rb1) of matrix d: warp w takes the w-th share of whole row blocks; every warp
+  // runs `n_iter` iterations so that all meet at the panel barriers.
+  __device__ void run_segment(const tq_tiles_desc& d, uint32_t rb0, uint32_t rb1) {
+    __syncthreads();  // the previous segment is done with the panel buffers and the scales
+    prepare_scales(d);
+    const uint32_t S = d.steps;
+    const uint32_t NP = (S + kPanelSteps - 1) / kPanelSteps;  // panels per row block
+    const uint32_t R = (rb1 - rb0 + W - 1) / W;               // row blocks per warp
+    const uint32_t my0 = min(rb1, rb0 + warp * R), my1 = min(rb1, my0 + R);
+    const uint32_t t0 = my0 * S, t1 = my1 * S;
+    const uint32_t n_real = t1 - t0, n_iter = R * S;
+    fill_panel(d, 0, 0);
+    fill_panel(d, 1 % NP, 1);
+    __syncthreads();
+
+    const uint32_t g = lane >> 2, t = lane & 3u;
+    const uint32_t miss_adj4 = ring_addr - 4u * kMissBase;
+    const uint32_t x_lane = tbl_addr + L.x + (g * kPanelStride + 8u * t) * 4u;
+
+    uint32_t rd = 0, stop_pos = 0, w_pos = 0, i_pos = 0;
+    const uint4* tok = d.tokens + (size_t)t0 * 64u + lane;
+    const uint4* tok_end = d.tokens + (size_t)t1 * 64u;
+    const uint32_t* trp = d.tile_raw + t0 + 1;
+    uint4 q[2][2] = {};
+    uint32_t tr[2] = {0, 0};
+    if (n_real) {
+      rd = __ldg(d.tile_raw + t0);
+      stop_pos = __ldg(d.tile_raw + t1);
+      w_pos = i_pos = rd & ~(uint32_t)(kChunkWords - 1);
+      for (int k = 0; k < kSlots && i_pos < stop_pos; ++k, i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        q[k][0] = ldg_stream(tok + k * 64);
+        q[k][1] = ldg_stream(tok + k * 64 + 32);
+        tr[k] = __ldg(trp + k);
+      }
+      tok += 2 * 64;
+      trp += 2;
+    }
+
+    uint32_t s_p = 0, s_local = 0, rb = my0;  // step, step inside the panel, row block of the tile awaiting the MMAs
+    uint32_t panels_done = 0;                  // index, in the endless panel sequence, of the panel in use
+    int acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0;
+    uint32_t wbuf[2][16];
+    bool ok = true;
+
+    auto lookups = [&](int k) {
+      const uint32_t rd_next = tr[k];
+      while (ok && rd_next > w_pos) {
+        ok = wait_chunk();
+        w_pos += kChunkWords;
+      }
+      if (!ok) return;
+      const uint32_t Rg[8] = {q[k][0].x, q[k][0].y, q[k][0].z, q[k][0].w, q[k][1].x, q[k][1].y, q[k][1].z, q[k][1].w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t lo4 = (Rg[i] << 2) & 0x3FFFCu, hi4 = (Rg[i] >> 14) & 0x3FFFCu;
+        wbuf[k][2 * i] = lds_u32(lo4 + (lo4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
+        wbuf[k][2 * i + 1] = lds_u32(hi4 + (hi4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
+      }
+      q[k][0] = ldg_stream(tok);
+      q[k][1] = ldg_stream(tok + 32);
+      tr[k] = __ldg(trp);
+      tok += 64;
+      ++trp;
+      rd = rd_next;
+      __syncwarp();
+      const uint32_t lim = min(stop_pos, (rd & ~(uint32_t)(kChunkWords - 1)) + kRingWords);
+      for (; i_pos < lim; i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
+      if (lane == 0 && tok + (kL2Ahead - 2) * 64 < tok_end) bulk_prefetch_l2(tok + (kL2Ahead - 2) * 64, 1024u);
+    };
+    // MMAs of one tile (real == false: the warp has no tile in this iteration but keeps step with the others)
+    auto consume = [&](const uint32_t (&wc)[16], bool real) {
+      if (real) {
+        const uint32_t xp = x_lane + (panels_done & 1u) * (kBufWords * 4u) + 128u * s_local;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          uint4 xa, xb;
+          const uint32_t a = xp + (uint32_t)nt * (8u * kPanelStride * 4u);
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(xa.x), "=r"(xa.y), "=r"(xa.z), "=r"(xa.w) : "r"(a));
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+16];" : "=r"(xb.x), "=r"(xb.y), "=r"(xb.z), "=r"(xb.w) : "r"(a));
+          mma_s8<SIGNED>(acc[nt], wc[0], wc[8], wc[1], wc[9], xa.x, xa.y);
+          mma_s8<SIGNED>(acc[nt], wc[2], wc[10], wc[3], wc[11], xa.z, xa.w);
+          mma_s8<SIGNED>(acc[nt], wc[4], wc[12], wc[5], wc[13], xb.x, xb.y);
+          mma_s8<SIGNED>(acc[nt], wc[6], wc[14], wc[7], wc[15], xb.z, xb.w);
+        }
+      }
+      ++s_local;
+      if (++s_p == S) {  // the row block is complete
+        s_p = 0;
+        if (real) {
+          panel_finalize<NB, NT>(d.scale, d.zero, d.y, d.rows, d.has_zero, xinfo(), nb_valid, rb, acc);
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0;
+        }
+        ++rb;
+        s_local = kPanelSteps;  // a row block ends its last panel, full or not
+      }
+      if (s_local == kPanelSteps) {  // panel finished by every warp: its buffer takes the panel after next
+        s_local = 0;
+        ++panels_done;
+        __syncthreads();
+        fill_panel(d, (panels_done + 1u) % NP, (panels_done + 1u) & 1u);
+      }
+    };
+
+    // when NCOL is not a multiple of 8 the last MMA tile has columns nobody fills or reads back:
+    // whatever the buffer holds there only reaches accumulator columns that are never used
+    for (uint32_t i = 0; i <= n_iter; i += 2) {
+      if (i < n_real && ok) lookups(0);
+      if (i >= 1 && i - 1 < n_iter) consume(wbuf[1], i - 1 < n_real && ok);
+      if (i + 1 < n_real && ok) lookups(1);
+      if (i < n_iter) consume(wbuf[0], i < n_real && ok);
+    }
+    while (ok && n_waited < n_issued) ok = wait_chunk();
+    if (!ok) {
+      *dead_flag() = 1u;
+      if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
+    }
+  }
+};
+
+template <int W, int NB, bool SIGNED>
+__global__ void __launch_bounds__(W * 32, 1) gemv_tiles_panel_kernel(const TilesParams p) {
+  extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
+  PanelCta<W, NB, SIGNED> cta;
+  cta.smem = tiles_smem_raw;
+  cta.L = tiles_smem(p.table_words, 2u * PanelCta<W, NB, SIGNED>::kBufWords, W);
+  cta.tbl_addr = smem_u32(tiles_smem_raw);
+  cta.warp = threadIdx.x >> 5;
+  cta.lane = threadIdx.x & 31u;
+  cta.nb_valid = p.nb_valid;
+  cta.ring_addr = cta.tbl_addr + cta.L.ring + cta.warp * (kRingWords * 4u);
+  cta.bar_base = cta.tbl_addr + cta.L.bar + cta.warp * (kSlots * 8u);
+
+  if (threadIdx.x < W * kSlots) mbar_init(cta.tbl_addr + cta.L.bar + threadIdx.x * 8u, 1u);
+  if (threadIdx.x == 0) *cta.dead_flag() = 0u;
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(p.table);
+    uint4* dst = reinterpret_cast<uint4*>(tiles_smem_raw);
+    for (uint32_t i = threadIdx.x; i < p.table_words / 4u; i += W * 32) dst[i] = __ldg(src + i);
+  }
+  __syncthreads();
+
+  if (p.mats == nullptr) {
+    const uint32_t nrb = p.one.row_blocks;
+    const uint32_t rb0 = (uint32_t)((uint64_t)nrb * blockIdx.x / gridDim.x);
+    const uint32_t rb1 = (uint32_t)((uint64_t)nrb * (blockIdx.x + 1) / gridDim.x);
+    if (rb0 < rb1) cta.run_segment(p.one, rb0, rb1);
+  } else {
+    for (uint32_t si = p.cta_seg[blockIdx.x]; si < p.cta_seg[blockIdx.x + 1]; ++si) {
+      const TilesSeg sg = p.segs[si];
+      tq_tiles_desc d = p.mats[sg.mat];
+      d.x = static_cast<const __nv_bfloat16*>(d.x) + (size_t)p.b0 * d.cols;
+      d.y += (size_t)p.b0 * d.rows;
+      cta.run_segment(d, sg.rb_begin, sg.rb_end);
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Decompress: one warp per tile, table and raw words read from global memory.
 // ---------------------------------------------------------------------------------------------
@@ -589,6 +920,43 @@ int launch_tiles(const TilesParams& p, uint32_t grid, size_t smem, cudaStream_t 
   return tq_cuda_status((int)cudaGetLastError(), "gemv(tiles) launch");
 }
 
+template <int NB, bool SIGNED>
+int launch_panel(const TilesParams& p, uint32_t grid, cudaStream_t st) {
+  auto kern = gemv_tiles_panel_kernel<kTilesWarps, NB, SIGNED>;
+  const size_t smem = tiles_smem(p.table_words, 2u * PanelCta<kTilesWarps, NB, SIGNED>::kBufWords, kTilesWarps).total;
+  if (smem > kSmemLimit) return TQ_ERR_UNSUPPORTED_SHAPE;
+  static size_t configured = 0;
+  if (smem > configured) {
+    if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+                                "gemv(tiles, wide): raising the dynamic shared memory limit"))
+      return rc;
+    configured = smem;
+  }
+  kern<<<grid, kTilesWarps * 32, smem, st>>>(p);
+  return tq_cuda_status((int)cudaGetLastError(), "gemv(tiles, wide) launch");
+}
+
+// One pass over nb batch columns (1..8) with the kernel that fits: p.one / p.mats describe the work.
+int launch_pass(TilesParams& p, int nb, bool narrow_two, bool sg, uint32_t grid, cudaStream_t st) {
+  if (nb <= 2 && (nb == 1 || narrow_two)) {
+    const TilesSmem L = tiles_smem(p.table_words, 3u * nb * p.xstride, kTilesWarps);
+    if (L.total > kSmemLimit) return TQ_ERR_UNSUPPORTED_SHAPE;
+    if (nb == 1) return sg ? launch_tiles<1, true>(p, grid, L.total, st) : launch_tiles<1, false>(p, grid, L.total, st);
+    return sg ? launch_tiles<2, true>(p, grid, L.total, st) : launch_tiles<2, false>(p, grid, L.total, st);
+  }
+  p.nb_valid = (uint32_t)nb;
+  if (nb <= 4) return sg ? launch_panel<4, true>(p, grid, st) : launch_panel<4, false>(p, grid, st);
+  return sg ? launch_panel<8, true>(p, grid, st) : launch_panel<8, false>(p, grid, st);
+}
+
+// Batch columns of the next pass when `left` remain: 8 at a time; a remainder of one column (or of
+// two where two fit the narrow kernel) goes to the narrow kernel, which has no panel barriers.
+int next_pass(int left, bool narrow_two) {
+  if (left >= 8) return 8;
+  if (left == 2 && !narrow_two) return 2;  // wide kernel with two columns
+  return left;
+}
+
 }  // namespace
 
 // Batch columns one launch can take for this matrix (2, 1, or 0 if even one does not fit).
@@ -599,22 +967,25 @@ int tq_tiles_max_nb(const tq_dmat* m) {
   return 0;
 }
 
-// x: bf16 [nb][cols], y: fp32 [nb][rows], nb in 1..tq_tiles_max_nb(m).
-int tq_tiles_gemv(const tq_dmat* m, const void* x, int nb, float* y, void* cuda_stream) {
+// x: bf16 [B][cols], y: fp32 [B][rows], any B >= 1: passes of up to 8 batch columns.
+int tq_tiles_gemv(const tq_dmat* m, const void* x, int B, float* y, void* cuda_stream) {
   TilesParams p{};
   p.one = m->tiles;
-  p.one.x = x;
-  p.one.y = y;
   p.table = m->dict->d_table;
   p.table_words = m->tiles.table_words;
   p.xstride = m->tiles.steps * 32u + 4u;
-  const TilesSmem L = tiles_smem(p.table_words, 3u * nb * p.xstride, kTilesWarps);
-  if (nb < 1 || nb > 2 || L.total > kSmemLimit) return TQ_ERR_UNSUPPORTED_SHAPE;
+  const bool narrow_two = tq_tiles_max_nb(m) >= 2;
   const uint32_t grid = std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count_tiles());
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const bool sg = m->info.levels_signed != 0;
-  if (nb == 1) return sg ? launch_tiles<1, true>(p, grid, L.total, st) : launch_tiles<1, false>(p, grid, L.total, st);
-  return sg ? launch_tiles<2, true>(p, grid, L.total, st) : launch_tiles<2, false>(p, grid, L.total, st);
+  for (int b0 = 0; b0 < B;) {
+    const int nb = next_pass(B - b0, narrow_two);
+    p.one.x = static_cast<const __nv_bfloat16*>(x) + (size_t)b0 * m->info.cols;
+    p.one.y = y + (size_t)b0 * m->info.rows;
+    if (int rc = launch_pass(p, nb, narrow_two, sg, grid, st)) return rc;
+    b0 += nb;
+  }
+  return TQ_OK;
 }
 
 int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
@@ -759,13 +1130,9 @@ int tq_fused_gemv_stack(const tq_stack* s, void* cuda_stream) {
   p.xstride = s->xstride;
   const bool two = tiles_smem(s->table_words, 6u * s->xstride, kTilesWarps).total <= kSmemLimit;
   for (int b0 = 0; b0 < s->B;) {
-    const int nb = (two && s->B - b0 >= 2) ? 2 : 1;
+    const int nb = next_pass(s->B - b0, two);
     p.b0 = (uint32_t)b0;
-    const TilesSmem L = tiles_smem(p.table_words, 3u * nb * p.xstride, kTilesWarps);
-    int rc;
-    if (nb == 1) rc = s->levels_signed ? launch_tiles<1, true>(p, s->grid, L.total, st) : launch_tiles<1, false>(p, s->grid, L.total, st);
-    else rc = s->levels_signed ? launch_tiles<2, true>(p, s->grid, L.total, st) : launch_tiles<2, false>(p, s->grid, L.total, st);
-    if (rc != TQ_OK) return rc;
+    if (int rc = launch_pass(p, nb, two, s->levels_signed != 0, s->grid, st)) return rc;
     b0 += nb;
   }
   return TQ_OK;
@@ -784,7 +1151,9 @@ int tq_fused_gemv_stack_host(const tq_stack* s, const void* h_x, void* d_x_arena
 int tq_stack_launches(const tq_stack* s) {
   if (!s) return TQ_ERR_INVALID_ARG;
   const bool two = tiles_smem(s->table_words, 6u * s->xstride, kTilesWarps).total <= kSmemLimit;
-  return two ? (s->B + 1) / 2 : s->B;
+  int n = 0;
+  for (int b0 = 0; b0 < s->B; ++n) b0 += next_pass(s->B - b0, two);
+  return n;
 }
 
 void tq_stack_free(tq_stack* s) { delete s; }
