@@ -196,9 +196,21 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
     max_elems = max(i.rows * i.cols for i in infos)
     buf = torch.empty(max_elems, dtype=torch.uint8, device=device)
 
-    def run_dec():
-        for m in mats:
-            tq.tq_decompress(m, buf[: m.info.rows * m.info.cols])
+    if args.layout == "tiles" and not args.per_layer:  # one persistent launch, every matrix to its own buffer
+        del buf
+        big = torch.empty(n_weights, dtype=torch.uint8, device=device)
+        outs, o = [], 0
+        for i in infos:
+            outs.append(big[o: o + i.rows * i.cols])
+            o += i.rows * i.cols
+        dstack = tq.tq_stack_create(mats)
+
+        def run_dec():
+            tq.tq_decompress_stack(dstack, outs)
+    else:
+        def run_dec():
+            for m in mats:
+                tq.tq_decompress(m, buf[: m.info.rows * m.info.cols])
 
     def timed(fn, reps):
         for _ in range(3):
@@ -215,6 +227,8 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
     ms = timed(run_dec, 10)
     rd = sum(algorithmic_bytes(i, 0) for i in infos)
     out["decompress"] = {"ms": ms, "GB_per_s": (rd + n_weights) / (ms * 1e-3) / 1e9,
+                         "launch": "one persistent launch (tq_decompress_stack)" if args.layout == "tiles" and not args.per_layer
+                         else "one launch per matrix (tq_decompress)",
                          "bytes": {"read": rd, "written": n_weights},
                          "frac_of_measured_hbm": (rd + n_weights) / (ms * 1e-3) / 1e9 / measured_peaks()[0]}
     if args.layout != "stream":

@@ -241,6 +241,10 @@ int tq_fused_gemv_stack(const tq_stack* s, void* cuda_stream);
 int tq_fused_gemv_stack_host(const tq_stack* s, const void* h_x, void* d_x_arena, uint64_t x_bytes,
                              float* h_y, const float* d_y_arena, uint64_t y_bytes, void* cuda_stream);
 int tq_stack_launches(const tq_stack* s); /* kernel launches one tq_fused_gemv_stack call makes */
+/* tq_decompress of every matrix of the stack in one persistent launch.  d_out_ptrs: DEVICE array of
+ * n_mats DEVICE pointers, each 16-byte aligned with room for rows_i * cols_i bytes.  A stack made
+ * with d_x == d_y == NULL (B ignored) serves this call only. */
+int tq_decompress_stack(const tq_stack* s, uint8_t* const* d_out_ptrs, void* cuda_stream);
 void tq_stack_free(tq_stack* s);
 
 /* Read and clear the matrix's device status word (TQ_STATUS_* bits); synchronises cuda_stream. */

@@ -37,7 +37,7 @@ EXPORTS = [
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
     "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_stack_size", "tq_stack_create",
-    "tq_fused_gemv_stack", "tq_fused_gemv_stack_host", "tq_stack_launches", "tq_stack_free", "tq_device_status", "tq_dmat_free",
+    "tq_fused_gemv_stack", "tq_fused_gemv_stack_host", "tq_stack_launches", "tq_decompress_stack", "tq_stack_free", "tq_device_status", "tq_dmat_free",
 ]
 
 
@@ -93,6 +93,7 @@ def _load() -> C.CDLL:
         "tq_fused_gemv_stack": (C.c_int, [vp, vp]),
         "tq_fused_gemv_stack_host": (C.c_int, [vp, vp, vp, C.c_uint64, vp, vp, C.c_uint64, vp]),
         "tq_stack_launches": (C.c_int, [vp]),
+        "tq_decompress_stack": (C.c_int, [vp, vp, vp]),
         "tq_stack_free": (None, [vp]),
         "tq_device_status": (C.c_int, [vp, vp, u32p]),
         "tq_dmat_free": (None, [vp]),
@@ -394,25 +395,39 @@ class Stack:
             self._h = None
 
 
-def tq_stack_create(mats, xs, ys, stream=None) -> Stack:
-    """mats: DeviceMatrix list (TILES layout, one table); xs[i]: CUDA bf16 [B][cols_i]; ys[i]: CUDA fp32 [B][rows_i]."""
+def tq_stack_create(mats, xs=None, ys=None, stream=None) -> Stack:
+    """mats: DeviceMatrix list (TILES layout, one table); xs[i]: CUDA bf16 [B][cols_i]; ys[i]: CUDA fp32 [B][rows_i].
+    Without xs / ys the stack serves tq_decompress_stack only."""
     n = len(mats)
-    assert n >= 1 and len(xs) == n and len(ys) == n
-    B = xs[0].numel() // mats[0].info.cols
-    for m, x, y in zip(mats, xs, ys):
-        assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.numel() == B * m.info.cols
-        assert y.is_cuda and y.dtype == torch.float32 and y.is_contiguous() and y.numel() == B * m.info.rows
+    assert n >= 1 and (xs is None) == (ys is None)
     need = C.c_uint64()
     _check(_lib.tq_stack_size(n, C.byref(need)), "tq_stack_size")
     buf = torch.empty(need.value, dtype=torch.uint8, device=mats[0].buf.device)
     hm = (C.c_void_p * n)(*[m._h for m in mats])
-    hx = (C.c_void_p * n)(*[x.data_ptr() for x in xs])
-    hy = (C.c_void_p * n)(*[y.data_ptr() for y in ys])
+    B, hx, hy = 0, None, None
+    if xs is not None:
+        assert len(xs) == n and len(ys) == n
+        B = xs[0].numel() // mats[0].info.cols
+        for m, x, y in zip(mats, xs, ys):
+            assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.numel() == B * m.info.cols
+            assert y.is_cuda and y.dtype == torch.float32 and y.is_contiguous() and y.numel() == B * m.info.rows
+        hx = (C.c_void_p * n)(*[x.data_ptr() for x in xs])
+        hy = (C.c_void_p * n)(*[y.data_ptr() for y in ys])
     out = C.c_void_p()
     with torch.cuda.device(buf.device):
         _check(_lib.tq_stack_create(hm, hx, hy, n, B, buf.data_ptr(), buf.numel(), _stream_ptr(stream), C.byref(out)),
                "tq_stack_create")
-    return Stack(out.value, buf, mats, xs, ys, B)
+    return Stack(out.value, buf, mats, xs or [], ys or [], B)
+
+
+def tq_decompress_stack(s: Stack, outs, stream=None) -> None:
+    """outs[i]: CUDA 1-byte tensor with rows_i * cols_i elements."""
+    assert len(outs) == len(s.mats)
+    for m, o in zip(s.mats, outs):
+        assert o.is_cuda and o.is_contiguous() and o.element_size() == 1 and o.numel() == m.info.rows * m.info.cols
+    ptrs = torch.tensor([o.data_ptr() for o in outs], dtype=torch.int64).to(s.buf.device)
+    _check(_lib.tq_decompress_stack(s._h, ptrs.data_ptr(), _stream_ptr(stream)), "tq_decompress_stack")
+    s._out_ptrs = ptrs  # keep the pointer array alive until the stream has used it
 
 
 def tq_fused_gemv_stack(s: Stack, stream=None) -> None:

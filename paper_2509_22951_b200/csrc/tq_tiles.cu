@@ -906,6 +906,194 @@ int sm_count_tiles() {
 constexpr int kTilesWarps = 16;
 constexpr uint32_t kSmemLimit = 232448u;  // 227 KB per CTA
 
+// ---------------------------------------------------------------------------------------------
+// Decompress for large inputs: the data path of the GEMV kernel (table in shared memory, raw words
+// through the ring, two-tile register pipeline) with the MMAs replaced by 32-byte stores.  A lane
+// holds, per tile and half, the 8 words of one row = 32 consecutive bytes of the output row; the 4
+// lanes of a quad cover 128 consecutive bytes.
+// ---------------------------------------------------------------------------------------------
+struct DecompParams {
+  const tq_tiles_desc* mats;   // stack mode: DEVICE array; nullptr in single-matrix mode
+  const TilesSeg* segs;
+  const uint32_t* cta_seg;
+  uint8_t* const* outs;        // stack mode: DEVICE array of output pointers, one per matrix
+  tq_tiles_desc one;           // single-matrix mode
+  uint8_t* out_one;
+  const uint32_t* table;
+  uint32_t table_words;
+};
+
+template <int W>
+struct DecompCta {
+  uint8_t* smem;
+  TilesSmem L;
+  uint32_t tbl_addr, warp, lane;
+  uint32_t ring_addr, bar_base;
+  uint32_t n_issued = 0, n_waited = 0;
+
+  __device__ __forceinline__ volatile uint32_t* dead_flag() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
+  __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t pos) {
+    if (lane == 0) {
+      const uint32_t bar = bar_base + (n_issued & (kSlots - 1u)) * 8u;
+      mbar_expect_tx(bar, kChunkWords * 4u);
+      bulk_g2s(ring_addr + ((pos * 4u) & (kRingWords * 4u - 1u)), raw + pos, kChunkWords * 4u, bar);
+    }
+    ++n_issued;
+  }
+  __device__ __forceinline__ bool wait_chunk() {
+    const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
+    const uint32_t par = (n_waited >> 2) & 1u;
+    ++n_waited;
+    if (mbar_try(bar, par)) return true;
+    return tiles_wait_slow(bar, par, dead_flag());
+  }
+
+  // tiles [t0, t1) of matrix d -> out (rows x cols bytes, row-major)
+  __device__ void run_tiles(const tq_tiles_desc& d, uint32_t* __restrict__ out, uint32_t t0, uint32_t t1) {
+    const uint32_t S = d.steps, gpr = d.cols >> 2;
+    const uint32_t g = lane >> 2, t = lane & 3u;
+    const uint32_t miss_adj4 = ring_addr - 4u * kMissBase;
+    const bool vec_ok = (gpr & 3u) == 0u;  // every row starts on a 16-byte boundary
+
+    uint32_t rd = __ldg(d.tile_raw + t0);
+    const uint32_t stop_pos = __ldg(d.tile_raw + t1);
+    uint32_t w_pos = rd & ~(uint32_t)(kChunkWords - 1), i_pos = w_pos;
+    for (int k = 0; k < kSlots && i_pos < stop_pos; ++k, i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
+    const uint4* tok = d.tokens + (size_t)t0 * 64u + lane;
+    const uint4* tok_end = d.tokens + (size_t)t1 * 64u;
+    const uint32_t* trp = d.tile_raw + t0 + 1;
+    uint4 q[2][2];
+    uint32_t tr[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      q[k][0] = ldg_stream(tok + k * 64);
+      q[k][1] = ldg_stream(tok + k * 64 + 32);
+      tr[k] = __ldg(trp + k);
+    }
+    tok += 2 * 64;
+    trp += 2;
+    uint32_t s = t0 % S, rb = t0 / S;
+    bool ok = true;
+
+    auto step = [&](int k) {
+      const uint32_t rd_next = tr[k];
+      while (ok && rd_next > w_pos) {
+        ok = wait_chunk();
+        w_pos += kChunkWords;
+      }
+      if (!ok) return;
+      const uint32_t Rg[8] = {q[k][0].x, q[k][0].y, q[k][0].z, q[k][0].w, q[k][1].x, q[k][1].y, q[k][1].z, q[k][1].w};
+      uint32_t w[16];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t lo4 = (Rg[i] << 2) & 0x3FFFCu, hi4 = (Rg[i] >> 14) & 0x3FFFCu;
+        w[2 * i] = lds_u32(lo4 + (lo4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
+        w[2 * i + 1] = lds_u32(hi4 + (hi4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
+      }
+      q[k][0] = ldg_stream(tok);
+      q[k][1] = ldg_stream(tok + 32);
+      tr[k] = __ldg(trp);
+      tok += 64;
+      ++trp;
+      rd = rd_next;
+      const uint32_t g0 = 32u * s + 8u * t;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const uint32_t r = rb * 16u + g + 8u * h;
+        if (r < d.rows && g0 < gpr) {
+          uint32_t* o = out + (size_t)r * gpr + g0;
+          if (vec_ok && g0 + 8u <= gpr) {
+            asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(o), "r"(w[8 * h]), "r"(w[8 * h + 1]),
+                         "r"(w[8 * h + 2]), "r"(w[8 * h + 3])
+                         : "memory");
+            asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(o + 4), "r"(w[8 * h + 4]), "r"(w[8 * h + 5]),
+                         "r"(w[8 * h + 6]), "r"(w[8 * h + 7])
+                         : "memory");
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              if (g0 + i < gpr) o[i] = w[8 * h + i];
+          }
+        }
+      }
+      if (++s == S) {
+        s = 0;
+        ++rb;
+      }
+      __syncwarp();
+      const uint32_t lim = min(stop_pos, (rd & ~(uint32_t)(kChunkWords - 1)) + kRingWords);
+      for (; i_pos < lim; i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
+      if (lane == 0 && tok + (kL2Ahead - 2) * 64 < tok_end) bulk_prefetch_l2(tok + (kL2Ahead - 2) * 64, 1024u);
+    };
+
+    for (uint32_t i = t0; i < t1 && ok; i += 2) {
+      step(0);
+      if (i + 1 < t1 && ok) step(1);
+    }
+    while (ok && n_waited < n_issued) ok = wait_chunk();
+    if (!ok) {
+      *dead_flag() = 1u;
+      if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
+    }
+  }
+
+  __device__ void run_segment(const tq_tiles_desc& d, uint8_t* out, uint32_t rb0, uint32_t rb1) {
+    const uint64_t T = (uint64_t)(rb1 - rb0) * d.steps;
+    const uint32_t t0 = rb0 * d.steps + (uint32_t)(T * warp / W);
+    const uint32_t t1 = rb0 * d.steps + (uint32_t)(T * (warp + 1) / W);
+    if (t0 < t1 && !*dead_flag()) run_tiles(d, reinterpret_cast<uint32_t*>(out), t0, t1);
+  }
+};
+
+template <int W>
+__global__ void __launch_bounds__(W * 32, 1) decompress_tiles_smem_kernel(const DecompParams p) {
+  extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
+  DecompCta<W> cta;
+  cta.smem = tiles_smem_raw;
+  cta.L = tiles_smem(p.table_words, 0u, W);
+  cta.tbl_addr = smem_u32(tiles_smem_raw);
+  cta.warp = threadIdx.x >> 5;
+  cta.lane = threadIdx.x & 31u;
+  cta.ring_addr = cta.tbl_addr + cta.L.ring + cta.warp * (kRingWords * 4u);
+  cta.bar_base = cta.tbl_addr + cta.L.bar + cta.warp * (kSlots * 8u);
+  if (threadIdx.x < W * kSlots) mbar_init(cta.tbl_addr + cta.L.bar + threadIdx.x * 8u, 1u);
+  if (threadIdx.x == 0) *cta.dead_flag() = 0u;
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(p.table);
+    uint4* dst = reinterpret_cast<uint4*>(tiles_smem_raw);
+    for (uint32_t i = threadIdx.x; i < p.table_words / 4u; i += W * 32) dst[i] = __ldg(src + i);
+  }
+  __syncthreads();
+  if (p.mats == nullptr) {
+    const uint32_t nrb = p.one.row_blocks;
+    const uint32_t rb0 = (uint32_t)((uint64_t)nrb * blockIdx.x / gridDim.x);
+    const uint32_t rb1 = (uint32_t)((uint64_t)nrb * (blockIdx.x + 1) / gridDim.x);
+    if (rb0 < rb1) cta.run_segment(p.one, p.out_one, rb0, rb1);
+  } else {
+    for (uint32_t si = p.cta_seg[blockIdx.x]; si < p.cta_seg[blockIdx.x + 1]; ++si) {
+      const TilesSeg sg = p.segs[si];
+      const tq_tiles_desc d = p.mats[sg.mat];
+      cta.run_segment(d, p.outs[sg.mat], sg.rb_begin, sg.rb_end);
+    }
+  }
+}
+
+int launch_decomp(const DecompParams& p, uint32_t grid, cudaStream_t st) {
+  auto kern = decompress_tiles_smem_kernel<kTilesWarps>;
+  const size_t smem = tiles_smem(p.table_words, 0u, kTilesWarps).total;
+  static bool configured = false;
+  if (!configured) {
+    if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+                                "decompress(tiles): raising the dynamic shared memory limit"))
+      return rc;
+    configured = true;
+  }
+  kern<<<grid, kTilesWarps * 32, smem, st>>>(p);
+  return tq_cuda_status((int)cudaGetLastError(), "decompress(tiles) launch");
+}
+
 template <int NB, bool SIGNED>
 int launch_tiles(const TilesParams& p, uint32_t grid, size_t smem, cudaStream_t st) {
   auto kern = gemv_tiles_kernel<kTilesWarps, NB, SIGNED>;
@@ -990,6 +1178,15 @@ int tq_tiles_gemv(const tq_dmat* m, const void* x, int B, float* y, void* cuda_s
 
 int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
   const uint32_t n_tiles = m->tiles.steps * m->tiles.row_blocks;
+  // loading the table into every SM's shared memory pays off from a few thousand tiles per SM on
+  if ((uint64_t)n_tiles >= 64ull * (uint64_t)sm_count_tiles()) {
+    DecompParams p{};
+    p.one = m->tiles;
+    p.out_one = d_codes;
+    p.table = m->dict->d_table;
+    p.table_words = m->tiles.table_words;
+    return launch_decomp(p, std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count_tiles()), (cudaStream_t)cuda_stream);
+  }
   const uint32_t grid = std::min<uint32_t>((n_tiles + 7u) / 8u, (uint32_t)sm_count_tiles() * 8u);
   decompress_tiles_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(m->tiles, m->dict->d_table,
                                                                        reinterpret_cast<uint32_t*>(d_codes));
@@ -1062,7 +1259,9 @@ int tq_stack_size(int n_mats, uint64_t* device_bytes) {
 
 int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* const* d_y, int n_mats, int B,
                     void* d_buf, uint64_t d_buf_bytes, void* cuda_stream, tq_stack** out) {
-  if (!mats || !d_x || !d_y || n_mats < 1 || B < 1 || B > 32 || !d_buf || !out || ((uintptr_t)d_buf & 255))
+  const bool bound = d_x && d_y;  // without operands the stack serves tq_decompress_stack only
+  if (!mats || (!bound && (d_x || d_y)) || n_mats < 1 || (bound && (B < 1 || B > 32)) || !d_buf || !out ||
+      ((uintptr_t)d_buf & 255))
     return TQ_ERR_INVALID_ARG;
   uint64_t need = 0;
   tq_stack_size(n_mats, &need);
@@ -1070,7 +1269,7 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   uint32_t max_steps = 0;
   for (int i = 0; i < n_mats; ++i) {
     const tq_dmat* m = mats[i];
-    if (!m || !d_x[i] || !d_y[i] || ((uintptr_t)d_x[i] & 15)) return TQ_ERR_INVALID_ARG;
+    if (!m || (bound && (!d_x[i] || !d_y[i] || ((uintptr_t)d_x[i] & 15)))) return TQ_ERR_INVALID_ARG;
     if (m->info.layout != TQ_LAYOUT_TILES || m->dict != mats[0]->dict ||
         m->info.levels_signed != mats[0]->info.levels_signed)
       return TQ_ERR_UNSUPPORTED_SHAPE;  // one table, one kind of level, TILES layout
@@ -1079,7 +1278,7 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   tq_stack* s = new (std::nothrow) tq_stack();
   if (!s) return TQ_ERR_NOMEM;
   s->n = n_mats;
-  s->B = B;
+  s->B = bound ? B : 0;
   s->levels_signed = mats[0]->info.levels_signed;
   s->grid = (uint32_t)sm_count_tiles();
   s->xstride = max_steps * 32u + 4u;
@@ -1093,8 +1292,8 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   std::vector<tq_tiles_desc> descs((size_t)n_mats);
   for (int i = 0; i < n_mats; ++i) {
     descs[i] = mats[i]->tiles;
-    descs[i].x = d_x[i];
-    descs[i].y = d_y[i];
+    descs[i].x = bound ? d_x[i] : nullptr;
+    descs[i].y = bound ? d_y[i] : nullptr;
   }
   uint8_t* base = static_cast<uint8_t*>(d_buf);
   const uint64_t off_segs = align256((uint64_t)n_mats * sizeof(tq_tiles_desc));
@@ -1119,7 +1318,7 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
 }
 
 int tq_fused_gemv_stack(const tq_stack* s, void* cuda_stream) {
-  if (!s) return TQ_ERR_INVALID_ARG;
+  if (!s || s->B < 1) return TQ_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   TilesParams p{};
   p.mats = s->d_descs;
@@ -1146,6 +1345,18 @@ int tq_fused_gemv_stack_host(const tq_stack* s, const void* h_x, void* d_x_arena
     return rc;
   if (int rc = tq_fused_gemv_stack(s, cuda_stream)) return rc;
   return tq_cuda_status((int)cudaMemcpyAsync(h_y, d_y_arena, y_bytes, cudaMemcpyDeviceToHost, st), "stack: copy of y");
+}
+
+int tq_decompress_stack(const tq_stack* s, uint8_t* const* d_out_ptrs, void* cuda_stream) {
+  if (!s || !d_out_ptrs) return TQ_ERR_INVALID_ARG;
+  DecompParams p{};
+  p.mats = s->d_descs;
+  p.segs = static_cast<const TilesSeg*>(s->d_segs);
+  p.cta_seg = s->d_cta_seg;
+  p.outs = d_out_ptrs;
+  p.table = s->d_table;
+  p.table_words = s->table_words;
+  return launch_decomp(p, s->grid, (cudaStream_t)cuda_stream);
 }
 
 int tq_stack_launches(const tq_stack* s) {

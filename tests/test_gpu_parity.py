@@ -245,6 +245,32 @@ def test_stack_matches_oracle_and_single_calls(tq, B):
             assert tq.tq_device_status(m) == 0
 
 
+def test_decompress_stack_bit_exact(tq):
+    """One persistent launch decompresses every matrix of a stack (ragged shapes, a table larger
+    than the shared-memory limit so that some groups are stored raw); a stack may be made without
+    operands for this purpose."""
+    shapes = [(300, 1024), (17, 8192), (1000, 3072), (16, 128), (530, 2052), (1, 4)]
+    rng = np.random.default_rng(41)
+    qs = [rng.integers(-20, 21, size=s).astype(np.int8) for s in shapes]
+    d, streams = _oracle_pack(qs)
+    assert d.K > tq.TQ_TILES_TABLE_WORDS
+    dd = tq.tq_dict_upload(tq.tq_dict_from_entries(d.entries))
+    ones = [np.ones(r, dtype=np.float32) for r, _ in shapes]
+    mats = [tq.tq_upload(dd, st, r, c, s, layout=tq.TQ_LAYOUT_TILES) for st, (r, c), s in zip(streams, shapes, ones)]
+    assert sum(m.info.n_raw_words - m.info.n_miss for m in mats) > 0
+    stack = tq.tq_stack_create(mats)
+    outs = [torch.full((r * c,), 0x55, dtype=torch.uint8, device="cuda") for r, c in shapes]
+    for _ in range(2):
+        tq.tq_decompress_stack(stack, outs)
+        torch.cuda.synchronize()
+        for o, q, m, st in zip(outs, qs, mats, streams):
+            assert np.array_equal(o.cpu().numpy().reshape(q.shape), d.decode(st).reshape(q.shape))
+            assert np.array_equal(o.cpu().numpy().reshape(q.shape), q.view(np.uint8))
+            assert tq.tq_device_status(m) == 0
+    with pytest.raises(tq.TqError):
+        tq.tq_fused_gemv_stack(stack)  # no operands were bound
+
+
 def test_stack_rejects_mixed_tables_and_layouts(tq):
     rng = np.random.default_rng(9)
     q = rng.integers(-3, 4, size=(32, 256)).astype(np.int8)
@@ -295,7 +321,8 @@ def test_full_3b_stack_as_benchmarked_on_sampled_rows(tq):
         err = np.max(np.abs(y - yref), axis=1) / np.max(np.abs(yref), axis=1)
         assert float(err.max()) <= TOL, (name, err)
         assert tq.tq_device_status(mats[i]) == 0
-    # decoded levels of one mid-sized matrix, whole, against the levels that were encoded
-    i = 6
-    got = tq.tq_decompress(mats[i])
-    assert np.array_equal(got.cpu().numpy().view(np.int8), q_host[i])
+    # decoded levels of two matrices, whole, against the levels that were encoded
+    for i in (6, 196):
+        got = tq.tq_decompress(mats[i])
+        assert np.array_equal(got.cpu().numpy().view(np.int8), q_host[i])
+        del got
