@@ -232,27 +232,28 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
                          "bytes": {"read": rd, "written": n_weights},
                          "frac_of_measured_hbm": (rd + n_weights) / (ms * 1e-3) / 1e9 / measured_peaks()[0]}
     if args.layout != "stream":
-        if args.layout != "planes":  # the tensor-core product reads the PLANES layout: upload it beside the other
-            gemm_mats = []
-            for i, (name, rows, cols) in enumerate(shapes):
-                stream_i, _, _ = tq.tq_encode(extra["hd"], extra["q_host"][i])
-                gemm_mats.append(tq.tq_upload(extra["dd"], stream_i, rows, cols, extra["scales"][i], layout=1))
-                del stream_i
-            mats = gemm_mats
         M = args.prefill_tokens
         max_rows = max(i.rows for i in infos)
         Y = torch.empty(M * max_rows, dtype=torch.float32, device=device)
         Xs = {c: synth.activations(M, c, 99, device=device) for c in sorted({i.cols for i in infos})}
+        if args.layout == "tiles":  # decode once per layer into a workspace, then the TMA-fed tensor-core product
+            ws = torch.empty(max(tq.tq_gemm_workspace_size(m) for m in mats), dtype=torch.uint8, device=device)
 
-        def run_gemm():
-            for m in mats:
-                tq.tq_fused_gemm(m, Xs[m.info.cols], Y[: M * m.info.rows].view(M, m.info.rows))
+            def run_gemm():
+                for m in mats:
+                    tq.tq_fused_gemm_ws(m, Xs[m.info.cols], ws, Y[: M * m.info.rows].view(M, m.info.rows))
+        else:
+            def run_gemm():
+                for m in mats:
+                    tq.tq_fused_gemm(m, Xs[m.info.cols], Y[: M * m.info.rows].view(M, m.info.rows))
 
         ms = timed(run_gemm, 3)
         flops = 2.0 * M * n_weights
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
         pk = float(peaks.get("bf16_tflops_sustained", 1400.0))
-        out["prefill"] = {"tokens": M, "ms": ms, "TFLOP_per_s": flops / (ms * 1e-3) / 1e12,
+        out["prefill"] = {"tokens": M, "ms": ms,
+                          "call": "tq_fused_gemm_ws (decode to a bf16 workspace + TMA-fed tcgen05 GEMM, per layer)" if args.layout == "tiles"
+                          else "tq_fused_gemm (decode inside the GEMM)", "TFLOP_per_s": flops / (ms * 1e-3) / 1e12,
                           "frac_of_measured_bf16_sustained": flops / (ms * 1e-3) / 1e12 / pk, "peak_TFLOP_per_s": pk}
         status = 0
         for m in mats:

@@ -218,6 +218,16 @@ int tq_fused_gemv_host_static(const tq_dmat* m, const void* h_x_bf16, int B, flo
  * d_X_bf16: DEVICE [M][cols] bf16, 16-byte aligned; d_Y: DEVICE [M][rows] fp32. */
 int tq_fused_gemm(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, void* cuda_stream);
 
+/* The prefill-sized product for a TQ_LAYOUT_TILES matrix, in two phases on cuda_stream that share a
+ * caller-provided DEVICE workspace (256-byte aligned, tq_gemm_workspace_size bytes = the matrix as
+ * bf16, padded to whole tiles): the layer is decompressed once into the workspace as bf16
+ * (level - zero point: exact for integer zero points), then a persistent tcgen05 GEMM reads both
+ * operands by TMA and applies the row scale in fp32.  Same result definition, argument layout and
+ * alignment as tq_fused_gemm; the workspace may be reused by the next call on the same stream. */
+int tq_gemm_workspace_size(const tq_dmat* m, uint64_t* bytes);
+int tq_fused_gemm_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, void* d_workspace,
+                     uint64_t workspace_bytes, void* cuda_stream);
+
 /* A stack: several TQ_LAYOUT_TILES matrices that share one table (for instance every linear layer
  * of a decoder, Section 2.3: the weights are expanded layer by layer), bound to their operands and
  * executed by ONE persistent launch in which every SM loads the table into shared memory once and

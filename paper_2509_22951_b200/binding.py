@@ -36,7 +36,8 @@ EXPORTS = [
     "tq_quantize_rows_device", "tq_build_dictionary", "tq_dict_from_entries", "tq_dict_entries",
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
-    "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_stack_size", "tq_stack_create",
+    "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_gemm_workspace_size",
+    "tq_fused_gemm_ws", "tq_stack_size", "tq_stack_create",
     "tq_fused_gemv_stack", "tq_fused_gemv_stack_host", "tq_stack_launches", "tq_decompress_stack", "tq_stack_free", "tq_device_status", "tq_dmat_free",
 ]
 
@@ -87,6 +88,8 @@ def _load() -> C.CDLL:
         "tq_fused_gemv_host": (C.c_int, [vp, vp, C.c_int, vp, vp, vp, vp]),
         "tq_fused_gemv_host_static": (C.c_int, [vp, vp, C.c_int, vp, vp]),
         "tq_fused_gemm": (C.c_int, [vp, vp, C.c_int, vp, vp]),
+        "tq_gemm_workspace_size": (C.c_int, [vp, u64p]),
+        "tq_fused_gemm_ws": (C.c_int, [vp, vp, C.c_int, vp, vp, C.c_uint64, vp]),
         "tq_stack_size": (C.c_int, [C.c_int, u64p]),
         "tq_stack_create": (C.c_int, [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int, C.c_int, vp, C.c_uint64, vp,
                                       C.POINTER(vp)]),
@@ -374,6 +377,26 @@ def tq_fused_gemm(m: DeviceMatrix, X: torch.Tensor, Y: torch.Tensor | None = Non
         Y = torch.empty((M, m.info.rows), dtype=torch.float32, device=X.device)
     assert Y.is_cuda and Y.dtype == torch.float32 and Y.is_contiguous() and Y.numel() == M * m.info.rows
     _check(_lib.tq_fused_gemm(m._h, X2.data_ptr(), M, Y.data_ptr(), _stream_ptr(stream)), "tq_fused_gemm")
+    return Y
+
+
+def tq_gemm_workspace_size(m: DeviceMatrix) -> int:
+    need = C.c_uint64()
+    _check(_lib.tq_gemm_workspace_size(m._h, C.byref(need)), "tq_gemm_workspace_size")
+    return need.value
+
+
+def tq_fused_gemm_ws(m: DeviceMatrix, X: torch.Tensor, workspace: torch.Tensor, Y: torch.Tensor | None = None,
+                     stream=None) -> torch.Tensor:
+    """Two-phase prefill product for the TILES layout; workspace: CUDA tensor of >= tq_gemm_workspace_size(m) bytes."""
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.is_contiguous() and workspace.is_cuda
+    X2 = X.view(-1, m.info.cols)
+    M = X2.shape[0]
+    if Y is None:
+        Y = torch.empty((M, m.info.rows), dtype=torch.float32, device=X.device)
+    assert Y.is_cuda and Y.dtype == torch.float32 and Y.is_contiguous() and Y.numel() == M * m.info.rows
+    _check(_lib.tq_fused_gemm_ws(m._h, X2.data_ptr(), M, Y.data_ptr(), workspace.data_ptr(),
+                                 workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "tq_fused_gemm_ws")
     return Y
 
 

@@ -119,6 +119,8 @@ int tq_build_planes_image(const uint16_t* stream, uint64_t stream_len, uint32_t 
 int tq_tiles_max_nb(const tq_dmat* m);
 int tq_tiles_gemv(const tq_dmat* m, const void* x, int nb, float* y, void* cuda_stream);
 int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream);
+// bf16 (level - zero point) in whole tiles: row_blocks * 16 rows, row pitch steps * 128 columns
+int tq_tiles_decode_bf16(const tq_dmat* m, void* d_out, void* cuda_stream);
 
 // A set of TILES matrices bound to their operands, with the work split among the CTAs of one
 // persistent launch (tq_tiles.cu).

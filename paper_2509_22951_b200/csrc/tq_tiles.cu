@@ -921,14 +921,15 @@ struct DecompParams {
   uint8_t* out_one;
   const uint32_t* table;
   uint32_t table_words;
+  uint32_t levels_signed;      // bf16 output: how to read a level byte
 };
 
-template <int W>
+template <int W, bool BF16>
 struct DecompCta {
   uint8_t* smem;
   TilesSmem L;
   uint32_t tbl_addr, warp, lane;
-  uint32_t ring_addr, bar_base;
+  uint32_t ring_addr, bar_base, levels_signed;
   uint32_t n_issued = 0, n_waited = 0;
 
   __device__ __forceinline__ volatile uint32_t* dead_flag() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
@@ -948,12 +949,14 @@ struct DecompCta {
     return tiles_wait_slow(bar, par, dead_flag());
   }
 
-  // tiles [t0, t1) of matrix d -> out (rows x cols bytes, row-major)
+  // tiles [t0, t1) of matrix d -> out (rows x cols bytes, row-major; or whole tiles of bf16)
   __device__ void run_tiles(const tq_tiles_desc& d, uint32_t* __restrict__ out, uint32_t t0, uint32_t t1) {
     const uint32_t S = d.steps, gpr = d.cols >> 2;
     const uint32_t g = lane >> 2, t = lane & 3u;
     const uint32_t miss_adj4 = ring_addr - 4u * kMissBase;
     const bool vec_ok = (gpr & 3u) == 0u;  // every row starts on a 16-byte boundary
+    const uint32_t xor_mask = levels_signed ? 0x80808080u : 0u;          // int8 bit pattern -> biased byte
+    const float magic = levels_signed ? 8388736.0f : 8388608.0f;         // 2^23 (+ 128): as_float(0x4B000000 | byte) - magic = level
 
     uint32_t rd = __ldg(d.tile_raw + t0);
     const uint32_t stop_pos = __ldg(d.tile_raw + t1);
@@ -997,8 +1000,34 @@ struct DecompCta {
       ++trp;
       rd = rd_next;
       const uint32_t g0 = 32u * s + 8u * t;
+      if (BF16) {
+        // level - zero point as bf16 into whole tiles (row pitch S * 128 columns): no bounds to check
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t r = rb * 16u + g + 8u * h;
+          const float off = magic + (d.has_zero ? __ldg(d.zero + r) : 0.f);
+          uint32_t* o = out + ((size_t)r * (S * 32u) + g0) * 2u;  // 2 words of bf16 per group
+#pragma unroll
+          for (int i = 0; i < 8; i += 2) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const uint32_t v = w[8 * h + i + e] ^ xor_mask;
+              const float f0 = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7540)) - off;
+              const float f1 = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7541)) - off;
+              const float f2 = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7542)) - off;
+              const float f3 = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7543)) - off;
+              const __nv_bfloat162 lo = __floats2bfloat162_rn(f0, f1), hi = __floats2bfloat162_rn(f2, f3);
+              pk[2 * e] = *reinterpret_cast<const uint32_t*>(&lo);
+              pk[2 * e + 1] = *reinterpret_cast<const uint32_t*>(&hi);
+            }
+            asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(o + 2 * i), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3])
+                         : "memory");
+          }
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < 2 && !BF16; ++h) {
         const uint32_t r = rb * 16u + g + 8u * h;
         if (r < d.rows && g0 < gpr) {
           uint32_t* o = out + (size_t)r * gpr + g0;
@@ -1045,10 +1074,11 @@ struct DecompCta {
   }
 };
 
-template <int W>
+template <int W, bool BF16>
 __global__ void __launch_bounds__(W * 32, 1) decompress_tiles_smem_kernel(const DecompParams p) {
   extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
-  DecompCta<W> cta;
+  DecompCta<W, BF16> cta;
+  cta.levels_signed = p.levels_signed;
   cta.smem = tiles_smem_raw;
   cta.L = tiles_smem(p.table_words, 0u, W);
   cta.tbl_addr = smem_u32(tiles_smem_raw);
@@ -1080,8 +1110,9 @@ __global__ void __launch_bounds__(W * 32, 1) decompress_tiles_smem_kernel(const 
   }
 }
 
+template <bool BF16>
 int launch_decomp(const DecompParams& p, uint32_t grid, cudaStream_t st) {
-  auto kern = decompress_tiles_smem_kernel<kTilesWarps>;
+  auto kern = decompress_tiles_smem_kernel<kTilesWarps, BF16>;
   const size_t smem = tiles_smem(p.table_words, 0u, kTilesWarps).total;
   static bool configured = false;
   if (!configured) {
@@ -1185,12 +1216,23 @@ int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
     p.out_one = d_codes;
     p.table = m->dict->d_table;
     p.table_words = m->tiles.table_words;
-    return launch_decomp(p, std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count_tiles()), (cudaStream_t)cuda_stream);
+    return launch_decomp<false>(p, std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count_tiles()), (cudaStream_t)cuda_stream);
   }
   const uint32_t grid = std::min<uint32_t>((n_tiles + 7u) / 8u, (uint32_t)sm_count_tiles() * 8u);
   decompress_tiles_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(m->tiles, m->dict->d_table,
                                                                        reinterpret_cast<uint32_t*>(d_codes));
   return tq_cuda_status((int)cudaGetLastError(), "decompress(tiles) launch");
+}
+
+// The matrix as bf16 (level - zero point) in whole tiles: row_blocks * 16 rows of steps * 128 columns.
+int tq_tiles_decode_bf16(const tq_dmat* m, void* d_out, void* cuda_stream) {
+  DecompParams p{};
+  p.one = m->tiles;
+  p.out_one = static_cast<uint8_t*>(d_out);
+  p.table = m->dict->d_table;
+  p.table_words = m->tiles.table_words;
+  p.levels_signed = m->info.levels_signed != 0;
+  return launch_decomp<true>(p, std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count_tiles()), (cudaStream_t)cuda_stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1356,7 +1398,7 @@ int tq_decompress_stack(const tq_stack* s, uint8_t* const* d_out_ptrs, void* cud
   p.outs = d_out_ptrs;
   p.table = s->d_table;
   p.table_words = s->table_words;
-  return launch_decomp(p, s->grid, (cudaStream_t)cuda_stream);
+  return launch_decomp<false>(p, s->grid, (cudaStream_t)cuda_stream);
 }
 
 int tq_stack_launches(const tq_stack* s) {

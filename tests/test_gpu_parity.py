@@ -215,6 +215,57 @@ def test_fused_gemm_agrees_with_fused_gemv(tq):
     assert float((a - b).abs().max() / b.abs().max()) < 1e-5
 
 
+# ------------------------------------------------------------------ prefill product, two phases (TILES)
+@pytest.mark.parametrize("rows,cols,M", [(128, 128, 256), (256, 512, 300), (130, 264, 1), (384, 3072, 2048),
+                                         (100, 1024, 77), (1000, 8192, 513), (17, 8, 5)])
+def test_fused_gemm_ws_matches_oracle(tq, rows, cols, M):
+    """Decode once to bf16 in a workspace, then the TMA-fed tcgen05 GEMM: ragged rows, columns and
+    token counts (tiles of 128 rows x 256 tokens x 64 columns), several tiles per CTA at M = 2048."""
+    rng = np.random.default_rng(rows + cols + M)
+    q = np.clip(np.rint(rng.standard_t(5, size=(rows, cols)) * 6), -127, 127).astype(np.int8)
+    s = (rng.random(rows) + 0.5).astype(np.float32)
+    d, (stream,) = _oracle_pack([q], top_k=3000)
+    m = _upload_from_oracle(tq, d, stream, rows, cols, s, layout=2)
+    ws = torch.full((tq.tq_gemm_workspace_size(m),), 0x7F, dtype=torch.uint8, device="cuda")  # NaN-ish garbage
+    X = synth.activations(M, cols, 123)
+    for _ in range(2):
+        Y = tq.tq_fused_gemm_ws(m, X.cuda(), ws).cpu().numpy().astype(np.float64)
+    assert tq.tq_device_status(m) == 0
+    sample = np.arange(M) if M <= 300 else np.sort(rng.choice(M, 64, replace=False))
+    Yref = oracle.layer_forward(q, s, X[sample].double().numpy())
+    assert Y.shape == (M, rows)
+    assert _rel_err(Y[sample], Yref) <= TOL
+
+
+def test_fused_gemm_ws_unsigned_levels_with_zero_point(tq):
+    w = synth.weight(256, 512, synth.matrix_seed(21)).numpy()
+    qu, sc, zp = oracle.quantize_paper(w)
+    qu = qu.reshape(256, 512)
+    s = np.full(256, sc, dtype=np.float32)
+    z = np.full(256, zp, dtype=np.float32)
+    d, (stream,) = _oracle_pack([qu])
+    m = _upload_from_oracle(tq, d, stream, 256, 512, s, zero=z, signed=False, layout=2)
+    ws = torch.empty(tq.tq_gemm_workspace_size(m), dtype=torch.uint8, device="cuda")
+    X = synth.activations(64, 512, 9)
+    Y = tq.tq_fused_gemm_ws(m, X.cuda(), ws).cpu().numpy().astype(np.float64)
+    Yref = oracle.layer_forward(qu, s, X.double().numpy(), zero=z)
+    assert _rel_err(Y, Yref) <= TOL
+    assert tq.tq_device_status(m) == 0
+
+
+def test_fused_gemm_ws_agrees_with_fused_gemv(tq):
+    rng = np.random.default_rng(78)
+    q = np.clip(np.rint(rng.standard_t(5, size=(512, 2048)) * 8), -127, 127).astype(np.int8)
+    s = (rng.random(512) + 0.5).astype(np.float32)
+    d, (stream,) = _oracle_pack([q])
+    m = _upload_from_oracle(tq, d, stream, 512, 2048, s, layout=2)
+    ws = torch.empty(tq.tq_gemm_workspace_size(m), dtype=torch.uint8, device="cuda")
+    X = synth.activations(8, 2048, 5).cuda()
+    a = tq.tq_fused_gemm_ws(m, X, ws)
+    b = tq.tq_fused_gemv(m, X)
+    assert float((a - b).abs().max() / b.abs().max()) < 1e-5
+
+
 # ------------------------------------------------------------------ stack: one persistent launch
 @pytest.mark.parametrize("B", [1, 2, 3, 8, 11])
 def test_stack_matches_oracle_and_single_calls(tq, B):
