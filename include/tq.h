@@ -227,6 +227,13 @@ int tq_fused_gemm(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, voi
 int tq_gemm_workspace_size(const tq_dmat* m, uint64_t* bytes);
 int tq_fused_gemm_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, void* d_workspace,
                      uint64_t workspace_bytes, void* cuda_stream);
+/* The two phases on their own: a layer's weights do not depend on the activations, so phase 1 may run
+ * ahead of time, and tq_decode_bf16_stack (declared with the stack calls below) runs it for every
+ * matrix of a stack in one launch.  tq_gemm_bf16_ws multiplies by a workspace that one of them
+ * filled for this matrix. */
+int tq_decode_bf16(const tq_dmat* m, void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
+int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, const void* d_workspace,
+                    void* cuda_stream);
 
 /* A stack: several TQ_LAYOUT_TILES matrices that share one table (for instance every linear layer
  * of a decoder, Section 2.3: the weights are expanded layer by layer), bound to their operands and
@@ -255,6 +262,10 @@ int tq_stack_launches(const tq_stack* s); /* kernel launches one tq_fused_gemv_s
  * n_mats DEVICE pointers, each 16-byte aligned with room for rows_i * cols_i bytes.  A stack made
  * with d_x == d_y == NULL (B ignored) serves this call only. */
 int tq_decompress_stack(const tq_stack* s, uint8_t* const* d_out_ptrs, void* cuda_stream);
+/* Phase 1 of tq_fused_gemm_ws for every matrix of the stack in one persistent launch.
+ * d_workspace_ptrs: DEVICE array of n_mats DEVICE pointers (256-byte aligned, tq_gemm_workspace_size
+ * bytes each). */
+int tq_decode_bf16_stack(const tq_stack* s, void* const* d_workspace_ptrs, void* cuda_stream);
 void tq_stack_free(tq_stack* s);
 
 /* Read and clear the matrix's device status word (TQ_STATUS_* bits); synchronises cuda_stream. */

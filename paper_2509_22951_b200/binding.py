@@ -37,7 +37,7 @@ EXPORTS = [
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
     "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_gemm_workspace_size",
-    "tq_fused_gemm_ws", "tq_stack_size", "tq_stack_create",
+    "tq_fused_gemm_ws", "tq_decode_bf16", "tq_gemm_bf16_ws", "tq_decode_bf16_stack", "tq_stack_size", "tq_stack_create",
     "tq_fused_gemv_stack", "tq_fused_gemv_stack_host", "tq_stack_launches", "tq_decompress_stack", "tq_stack_free", "tq_device_status", "tq_dmat_free",
 ]
 
@@ -90,6 +90,9 @@ def _load() -> C.CDLL:
         "tq_fused_gemm": (C.c_int, [vp, vp, C.c_int, vp, vp]),
         "tq_gemm_workspace_size": (C.c_int, [vp, u64p]),
         "tq_fused_gemm_ws": (C.c_int, [vp, vp, C.c_int, vp, vp, C.c_uint64, vp]),
+        "tq_decode_bf16": (C.c_int, [vp, vp, C.c_uint64, vp]),
+        "tq_gemm_bf16_ws": (C.c_int, [vp, vp, C.c_int, vp, vp, vp]),
+        "tq_decode_bf16_stack": (C.c_int, [vp, vp, vp]),
         "tq_stack_size": (C.c_int, [C.c_int, u64p]),
         "tq_stack_create": (C.c_int, [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int, C.c_int, vp, C.c_uint64, vp,
                                       C.POINTER(vp)]),
@@ -400,6 +403,27 @@ def tq_fused_gemm_ws(m: DeviceMatrix, X: torch.Tensor, workspace: torch.Tensor, 
     return Y
 
 
+def tq_decode_bf16(m: DeviceMatrix, workspace: torch.Tensor, stream=None) -> None:
+    assert workspace.is_cuda
+    _check(_lib.tq_decode_bf16(m._h, workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                               _stream_ptr(stream)), "tq_decode_bf16")
+
+
+def tq_gemm_bf16_ws(m: DeviceMatrix, X: torch.Tensor, workspace: torch.Tensor, Y: torch.Tensor | None = None,
+                    stream=None) -> torch.Tensor:
+    """Phase 2 alone: workspace was filled for m by tq_decode_bf16 or tq_decode_bf16_stack."""
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.is_contiguous() and workspace.is_cuda
+    assert workspace.numel() * workspace.element_size() >= tq_gemm_workspace_size(m)
+    X2 = X.view(-1, m.info.cols)
+    M = X2.shape[0]
+    if Y is None:
+        Y = torch.empty((M, m.info.rows), dtype=torch.float32, device=X.device)
+    assert Y.is_cuda and Y.dtype == torch.float32 and Y.is_contiguous() and Y.numel() == M * m.info.rows
+    _check(_lib.tq_gemm_bf16_ws(m._h, X2.data_ptr(), M, Y.data_ptr(), workspace.data_ptr(), _stream_ptr(stream)),
+           "tq_gemm_bf16_ws")
+    return Y
+
+
 class Stack:
     """Several TILES matrices bound to their operands for one persistent launch.  Keeps the
     matrices, the operand tensors and its own device buffer alive."""
@@ -451,6 +475,16 @@ def tq_decompress_stack(s: Stack, outs, stream=None) -> None:
     ptrs = torch.tensor([o.data_ptr() for o in outs], dtype=torch.int64).to(s.buf.device)
     _check(_lib.tq_decompress_stack(s._h, ptrs.data_ptr(), _stream_ptr(stream)), "tq_decompress_stack")
     s._out_ptrs = ptrs  # keep the pointer array alive until the stream has used it
+
+
+def tq_decode_bf16_stack(s: Stack, workspaces, stream=None) -> None:
+    """workspaces[i]: CUDA tensor of >= tq_gemm_workspace_size(mats[i]) bytes, 256-byte aligned."""
+    assert len(workspaces) == len(s.mats)
+    for m, w in zip(s.mats, workspaces):
+        assert w.is_cuda and w.numel() * w.element_size() >= tq_gemm_workspace_size(m) and w.data_ptr() % 256 == 0
+    ptrs = torch.tensor([w.data_ptr() for w in workspaces], dtype=torch.int64).to(s.buf.device)
+    _check(_lib.tq_decode_bf16_stack(s._h, ptrs.data_ptr(), _stream_ptr(stream)), "tq_decode_bf16_stack")
+    s._ws_ptrs = ptrs  # keep the pointer array alive until the stream has used it
 
 
 def tq_fused_gemv_stack(s: Stack, stream=None) -> None:

@@ -22,14 +22,17 @@
 namespace {
 
 constexpr int BM = 128;   // weight rows per tile (MMA M)
-constexpr int BN = 256;   // tokens per tile (MMA N)
+// tokens per tile (MMA N) is a template parameter: 256, or 128 where that fills the SMs better
 constexpr int BK = 64;    // columns per stage: one 128-byte swizzle atom of bf16
 constexpr int kStages = 4;
 constexpr uint32_t A_BYTES = BM * BK * 2;  // 16 KB
-constexpr uint32_t B_BYTES = BN * BK * 2;  // 32 KB
-constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int kThreads = 6 * 32;  // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
-constexpr uint32_t SMEM_BYTES = kStages * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+template <int BN>
+struct Geo {
+  static constexpr uint32_t B_BYTES = BN * BK * 2;  // 32 or 16 KB
+  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr uint32_t SMEM_BYTES = kStages * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+};
 constexpr uint32_t kSpinLimit = 1u << 26;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -99,8 +102,10 @@ struct GemmWsParams {
   uint32_t row_tiles, token_tiles;
 };
 
+template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, const GemmWsParams p) {
+  constexpr uint32_t STAGE_BYTES = Geo<BN>::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // operand tiles need 1024-byte alignment
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -267,48 +272,41 @@ int tq_gemm_workspace_size(const tq_dmat* m, uint64_t* bytes) {
   return TQ_OK;
 }
 
+int tq_decode_bf16(const tq_dmat* m, void* d_workspace, uint64_t workspace_bytes, void* cuda_stream) {
+  if (!m || !d_workspace || ((uintptr_t)d_workspace & 255)) return TQ_ERR_INVALID_ARG;
+  if (m->info.layout != TQ_LAYOUT_TILES) return TQ_ERR_UNSUPPORTED_SHAPE;
+  uint64_t need = 0;
+  tq_gemm_workspace_size(m, &need);
+  if (workspace_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
+  return tq_tiles_decode_bf16(m, d_workspace, cuda_stream);
+}
+
 int tq_fused_gemm_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, void* d_workspace,
                      uint64_t workspace_bytes, void* cuda_stream) {
+  if (!d_X_bf16 || !d_Y || M < 1) return TQ_ERR_INVALID_ARG;
+  if (int rc = tq_decode_bf16(m, d_workspace, workspace_bytes, cuda_stream)) return rc;
+  return tq_gemm_bf16_ws(m, d_X_bf16, M, d_Y, d_workspace, cuda_stream);
+}
+
+int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, const void* d_workspace,
+                    void* cuda_stream) {
   if (!m || !d_X_bf16 || !d_Y || !d_workspace || M < 1 || ((uintptr_t)d_X_bf16 & 15) || ((uintptr_t)d_workspace & 255))
     return TQ_ERR_INVALID_ARG;
   if (m->info.layout != TQ_LAYOUT_TILES) return TQ_ERR_UNSUPPORTED_SHAPE;
   if ((m->info.cols * 2u) % 16u != 0) return TQ_ERR_UNSUPPORTED_SHAPE;  // TMA row pitch must be a multiple of 16 bytes
-  uint64_t need = 0;
-  tq_gemm_workspace_size(m, &need);
-  if (workspace_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return tq_cuda_status((int)cudaErrorUnknown, "gemm: cuTensorMapEncodeTiled not available");
 
-  // phase 1: the layer as bf16 (level - zero point), whole tiles, row pitch = steps * 128 columns
-  if (int rc = tq_tiles_decode_bf16(m, d_workspace, cuda_stream)) return rc;
-
-  // phase 2
   const uint32_t rows_pad = m->tiles.row_blocks * 16u, pitch = m->tiles.steps * 128u;
-  CUtensorMap tmap_w, tmap_x;
+  CUtensorMap tmap_w;
   const cuuint32_t estr[2] = {1, 1};
   {
     const cuuint64_t gdim[2] = {m->info.cols, rows_pad};
     const cuuint64_t gstride[1] = {(cuuint64_t)pitch * 2};
     const cuuint32_t box[2] = {BK, BM};
-    if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_workspace, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d_workspace), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return tq_cuda_status((int)cudaErrorInvalidValue, "gemm: tensor map of the weights");
-  }
-  {
-    const cuuint64_t gdim[2] = {m->info.cols, (cuuint64_t)M};
-    const cuuint64_t gstride[1] = {(cuuint64_t)m->info.cols * 2};
-    const cuuint32_t box[2] = {BK, BN};
-    if (enc(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d_X_bf16), gdim, gstride, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return tq_cuda_status((int)cudaErrorInvalidValue, "gemm: tensor map of the activations");
-  }
-  static bool configured = false;
-  if (!configured) {
-    if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(gemm_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES),
-                                "gemm: raising the dynamic shared memory limit"))
-      return rc;
-    configured = true;
   }
   GemmWsParams p;
   p.scale = m->d_scale;
@@ -318,9 +316,42 @@ int tq_fused_gemm_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, 
   p.cols = m->info.cols;
   p.M = (uint32_t)M;
   p.row_tiles = (m->info.rows + BM - 1) / BM;
-  p.token_tiles = ((uint32_t)M + BN - 1) / BN;
-  const uint32_t grid = std::min<uint32_t>(p.row_tiles * p.token_tiles, (uint32_t)sm_count_ws());
-  gemm_ws_kernel<<<grid, kThreads, SMEM_BYTES, (cudaStream_t)cuda_stream>>>(tmap_w, tmap_x, p);
+  // 256-token tiles halve the operand traffic per flop; 128-token tiles where they leave fewer SMs idle
+  const uint32_t sms = (uint32_t)sm_count_ws();
+  auto fill = [&](uint32_t bn) {
+    const uint32_t tiles = p.row_tiles * (((uint32_t)M + bn - 1) / bn);
+    return (double)tiles / (double)(((tiles + sms - 1) / sms) * sms);
+  };
+  // (measured: at M = 2048 the narrow tile loses more to operand traffic than it gains in SM fill, so it
+  // is kept for token counts that leave half of a 256-token tile empty)
+  const bool narrow = (uint32_t)M <= 128u && fill(128) >= fill(256);
+  const uint32_t bn = narrow ? 128u : 256u;
+  p.token_tiles = ((uint32_t)M + bn - 1) / bn;
+  CUtensorMap tmap_x;
+  {
+    const cuuint64_t gdim[2] = {m->info.cols, (cuuint64_t)M};
+    const cuuint64_t gstride[1] = {(cuuint64_t)m->info.cols * 2};
+    const cuuint32_t box[2] = {BK, bn};
+    if (enc(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d_X_bf16), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return tq_cuda_status((int)cudaErrorInvalidValue, "gemm: tensor map of the activations");
+  }
+  const uint32_t grid = std::min<uint32_t>(p.row_tiles * p.token_tiles, sms);
+  static bool configured = false;
+  if (!configured) {
+    int rc = tq_cuda_status((int)cudaFuncSetAttribute(gemm_ws_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                      (int)Geo<256>::SMEM_BYTES), "gemm: raising the dynamic shared memory limit");
+    if (rc == TQ_OK)
+      rc = tq_cuda_status((int)cudaFuncSetAttribute(gemm_ws_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    (int)Geo<128>::SMEM_BYTES), "gemm: raising the dynamic shared memory limit");
+    if (rc != TQ_OK) return rc;
+    configured = true;
+  }
+  if (narrow)
+    gemm_ws_kernel<128><<<grid, kThreads, Geo<128>::SMEM_BYTES, (cudaStream_t)cuda_stream>>>(tmap_w, tmap_x, p);
+  else
+    gemm_ws_kernel<256><<<grid, kThreads, Geo<256>::SMEM_BYTES, (cudaStream_t)cuda_stream>>>(tmap_w, tmap_x, p);
   return tq_cuda_status((int)cudaGetLastError(), "gemm launch");
 }
 

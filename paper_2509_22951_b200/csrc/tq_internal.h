@@ -135,3 +135,7 @@ struct tq_stack {
   uint32_t n_segs = 0;
   uint64_t x_bytes = 0, y_bytes = 0;       // sizes of the operand arenas when bound with tq_stack_create_arena
 };
+
+// Phase 2 of the workspace GEMM (tq_gemm_ws.cu), declared here for tq_fused_gemm_ws.
+extern "C" int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, const void* d_workspace,
+                               void* cuda_stream);

@@ -1401,6 +1401,19 @@ int tq_decompress_stack(const tq_stack* s, uint8_t* const* d_out_ptrs, void* cud
   return launch_decomp<false>(p, s->grid, (cudaStream_t)cuda_stream);
 }
 
+int tq_decode_bf16_stack(const tq_stack* s, void* const* d_workspace_ptrs, void* cuda_stream) {
+  if (!s || !d_workspace_ptrs) return TQ_ERR_INVALID_ARG;
+  DecompParams p{};
+  p.mats = s->d_descs;
+  p.segs = static_cast<const TilesSeg*>(s->d_segs);
+  p.cta_seg = s->d_cta_seg;
+  p.outs = reinterpret_cast<uint8_t* const*>(d_workspace_ptrs);
+  p.table = s->d_table;
+  p.table_words = s->table_words;
+  p.levels_signed = s->levels_signed != 0;
+  return launch_decomp<true>(p, s->grid, (cudaStream_t)cuda_stream);
+}
+
 int tq_stack_launches(const tq_stack* s) {
   if (!s) return TQ_ERR_INVALID_ARG;
   const bool two = tiles_smem(s->table_words, 6u * s->xstride, kTilesWarps).total <= kSmemLimit;

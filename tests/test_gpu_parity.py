@@ -322,6 +322,30 @@ def test_decompress_stack_bit_exact(tq):
         tq.tq_fused_gemv_stack(stack)  # no operands were bound
 
 
+def test_decode_bf16_stack_then_gemm(tq):
+    """Phase 1 of the prefill product for all matrices of a stack in one launch, phase 2 per matrix."""
+    shapes = [(300, 1024), (130, 8192), (1000, 3072), (16, 128)]
+    rng = np.random.default_rng(43)
+    qs = [np.clip(np.rint(rng.standard_t(5, size=s) * 5), -127, 127).astype(np.int8) for s in shapes]
+    ss = [(rng.random(r) + 0.5).astype(np.float32) for r, _ in shapes]
+    d, streams = _oracle_pack(qs)
+    dd = tq.tq_dict_upload(tq.tq_dict_from_entries(d.entries))
+    mats = [tq.tq_upload(dd, st, r, c, s, layout=tq.TQ_LAYOUT_TILES) for st, (r, c), s in zip(streams, shapes, ss)]
+    stack = tq.tq_stack_create(mats)
+    wss = [torch.full((tq.tq_gemm_workspace_size(m),), 0x7F, dtype=torch.uint8, device="cuda") for m in mats]
+    tq.tq_decode_bf16_stack(stack, wss)
+    M = 70
+    for m, q, s, w, (r, c) in zip(mats, qs, ss, wss, shapes):
+        X = synth.activations(M, c, 17)
+        Y = tq.tq_gemm_bf16_ws(m, X.cuda(), w).cpu().numpy().astype(np.float64)
+        assert _rel_err(Y, oracle.layer_forward(q, s, X.double().numpy())) <= TOL
+        # the workspace holds the levels themselves as bf16, in whole tiles
+        rows_pad, pitch = -(-r // 16) * 16, -(-c // 128) * 128
+        wb = w.view(torch.bfloat16)[: rows_pad * pitch].view(rows_pad, pitch)[:r, :c].float().cpu().numpy()
+        assert np.array_equal(wb, q.astype(np.float32))
+        assert tq.tq_device_status(m) == 0
+
+
 def test_stack_rejects_mixed_tables_and_layouts(tq):
     rng = np.random.default_rng(9)
     q = rng.integers(-3, 4, size=(32, 256)).astype(np.int8)
