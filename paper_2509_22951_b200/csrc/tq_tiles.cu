@@ -667,21 +667,42 @@ struct PanelCta {
     }
   }
 
-  // Digits of step panel P (steps P*kPanelSteps ..) of all vectors into buffer `buf`.
-  __device__ __forceinline__ void fill_panel(const tq_tiles_desc& d, uint32_t P, uint32_t buf) {
+  static constexpr int kItems = (kPanelSteps * 32 * NB + kThreads - 1) / kThreads;  // activation groups per thread and panel
+  // Loads of step panel P (steps P*kPanelSteps ..) of all vectors; fill_store turns them into digits.
+  __device__ __forceinline__ void fill_load(const tq_tiles_desc& d, uint32_t P, uint2 (&v)[kItems]) {
     const uint32_t G = d.cols >> 2;
     const uint2* xg = reinterpret_cast<const uint2*>(d.x);
-    uint32_t* xs = reinterpret_cast<uint32_t*>(smem + L.x) + buf * kBufWords;
     constexpr uint32_t kGroups = kPanelSteps * 32;
-    for (uint32_t idx = threadIdx.x; idx < kGroups * NB; idx += kThreads) {
+#pragma unroll
+    for (int it = 0; it < kItems; ++it) {
+      const uint32_t idx = threadIdx.x + (uint32_t)it * kThreads;
       const uint32_t gl = idx % kGroups, b = idx / kGroups;
       const uint32_t g = P * kGroups + gl;
-      uint32_t w0 = 0, w1 = 0, w2 = 0;
-      if (g < G && b < nb_valid) digits(__ldg(xg + (size_t)b * G + g), in_scale()[b], true, w0, w1, w2, nullptr);
-      xs[(3 * b + 0) * kPanelStride + gl] = w0;
-      xs[(3 * b + 1) * kPanelStride + gl] = w1;
-      xs[(3 * b + 2) * kPanelStride + gl] = w2;
+      v[it] = make_uint2(0u, 0u);  // absent groups: zero bits, zero digits
+      if (idx < kGroups * NB && g < G && b < nb_valid) v[it] = __ldg(xg + (size_t)b * G + g);
     }
+  }
+  __device__ __forceinline__ void fill_store(uint32_t buf, const uint2 (&v)[kItems]) {
+    uint32_t* xs = reinterpret_cast<uint32_t*>(smem + L.x) + buf * kBufWords;
+    constexpr uint32_t kGroups = kPanelSteps * 32;
+#pragma unroll
+    for (int it = 0; it < kItems; ++it) {
+      const uint32_t idx = threadIdx.x + (uint32_t)it * kThreads;
+      const uint32_t gl = idx % kGroups, b = idx / kGroups;
+      if (idx < kGroups * NB) {
+        uint32_t w0, w1, w2;
+        digits(v[it], b < nb_valid ? in_scale()[b] : 0.f, true, w0, w1, w2, nullptr);
+        xs[(3 * b + 0) * kPanelStride + gl] = w0;
+        xs[(3 * b + 1) * kPanelStride + gl] = w1;
+        xs[(3 * b + 2) * kPanelStride + gl] = w2;
+      }
+    }
+  }
+  // Digits of step panel P of all vectors into buffer `buf`.
+  __device__ __forceinline__ void fill_panel(const tq_tiles_desc& d, uint32_t P, uint32_t buf) {
+    uint2 v[kItems];
+    fill_load(d, P, v);
+    fill_store(buf, v);
   }
 
   // Row blocks [rb0, rb1) of matrix d: warp w takes the w-th share of whole row blocks; every warp
@@ -787,8 +808,10 @@ struct PanelCta {
       if (s_local == kPanelSteps) {  // panel finished by every warp: its buffer takes the panel after next
         s_local = 0;
         ++panels_done;
+        uint2 v[kItems];
+        fill_load(d, (panels_done + 1u) % NP, v);  // in flight while the warps gather at the barrier
         __syncthreads();
-        fill_panel(d, (panels_done + 1u) % NP, (panels_done + 1u) & 1u);
+        fill_store((panels_done + 1u) & 1u, v);
       }
     };
 
