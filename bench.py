@@ -105,6 +105,9 @@ class ClockSampler:
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the ncu capture
 # summarised under profiles/ (None: not captured for that launch shape, or kernel changed since).
+# tiles_stack: 213.2 MB read + 4.2 MB written for 207.7 MB of algorithmic bytes on a 14-matrix stack (2 decoder
+# layers), i.e. 1.047 x; traffic grows with the bytes streamed, so the 3B launch (3.333 GB) is scaled by that ratio.
+TRAFFIC_RATIO = {"tiles_stack": 1.047}
 TRAFFIC = {}
 
 
@@ -522,7 +525,10 @@ def main():
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
-                     "traffic": TRAFFIC.get(args.layout if not use_stack else "tiles_stack"),
+                     "traffic": (TRAFFIC_RATIO["tiles_stack"] * alg_bytes / launches_per_step
+                                 if use_stack and args.batch <= 2 else TRAFFIC.get(args.layout)),
+                     "traffic_note": ("dram bytes per launch, scaled from the ncu capture of a 14-matrix stack "
+                                      "(profiles/gemv_tiles_stack_llama3b_b1.md)" if use_stack and args.batch <= 2 else None),
                      "kernel": {"stream": "gemv_kernel", "planes": "gemv_planes_kernel", "tiles": "gemv_tiles_kernel"}[args.layout],
                      "peak_source": peak_src,
                      "note": "achieved = algorithmic bytes of the %d launch(es) of a step / step time (launch gaps included)" % launches_per_step},

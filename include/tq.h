@@ -135,7 +135,8 @@ void tq_ddict_free(tq_ddict* d); /* host handle only */
                               top_k = TQ_TILES_TABLE_WORDS - 1.  Same decoded bytes, 4 more bytes per such
                               group (tq_dmat_info.n_raw_words counts them). */
 #define TQ_TILES_TABLE_WORDS 34816u
-#define TQ_TILES_MAX_COLS 8704u /* table + one activation vector as 3 digit bytes per column must fit 227 KB */
+#define TQ_TILES_MAX_COLS 65536u /* 32-bit integer accumulators; rows of more than 8704 columns go through the
+                                    column-panel kernel, whose shared memory need does not grow with the row */
 #define TQ_TILES_RING_WORDS 1024u /* a miss token of the image is 0xFC00 + (index of its raw word mod 1024) */
 
 /* Bytes of DEVICE memory the layout of this stream needs.  stream: HOST.  Requires cols % 4 == 0

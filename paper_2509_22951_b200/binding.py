@@ -26,7 +26,7 @@ TQ_LAYOUT_STREAM = 0
 TQ_LAYOUT_PLANES = 1
 TQ_LAYOUT_TILES = 2
 TQ_TILES_TABLE_WORDS = 34816
-TQ_TILES_MAX_COLS = 8704
+TQ_TILES_MAX_COLS = 65536
 TQ_STATUS_BAD_CODE = 1
 TQ_STATUS_BAD_ROW = 2
 TQ_STATUS_WAIT_EXPIRED = 4

@@ -724,8 +724,7 @@ int tq_build_tiles_image(const uint16_t* stream, uint64_t stream_len, uint32_t r
   int rc = scan_stream(stream, stream_len, rows, cols, K, row_start, H, M);
   if (rc != TQ_OK) return rc;
   if (M >= (1ull << 32) - 65536) return TQ_ERR_UNSUPPORTED_SHAPE;
-  // the activation digits of a whole row (3 bytes per column) share the CTA's shared memory with the table
-  if (cols > TQ_TILES_MAX_COLS) return TQ_ERR_UNSUPPORTED_SHAPE;
+  if (cols > TQ_TILES_MAX_COLS) return TQ_ERR_UNSUPPORTED_SHAPE;  // 32-bit accumulators of the integer MMA
 
   const uint32_t gpr = cols / 4;
   const uint32_t steps = (gpr + 31u) / 32u;

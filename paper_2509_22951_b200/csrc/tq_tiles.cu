@@ -1180,9 +1180,10 @@ int launch_panel(const TilesParams& p, uint32_t grid, cudaStream_t st) {
 
 // One pass over nb batch columns (1..8) with the kernel that fits: p.one / p.mats describe the work.
 int launch_pass(TilesParams& p, int nb, bool narrow_two, bool sg, uint32_t grid, cudaStream_t st) {
-  if (nb <= 2 && (nb == 1 || narrow_two)) {
-    const TilesSmem L = tiles_smem(p.table_words, 3u * nb * p.xstride, kTilesWarps);
-    if (L.total > kSmemLimit) return TQ_ERR_UNSUPPORTED_SHAPE;
+  // the narrow kernel keeps the digits of a whole row in shared memory; rows too long for that
+  // (more than 8704 columns) take the wide kernel, which works in column panels, for any batch
+  const TilesSmem L = tiles_smem(p.table_words, 3u * std::min(nb, 2) * p.xstride, kTilesWarps);
+  if (nb <= 2 && (nb == 1 || narrow_two) && L.total <= kSmemLimit) {
     if (nb == 1) return sg ? launch_tiles<1, true>(p, grid, L.total, st) : launch_tiles<1, false>(p, grid, L.total, st);
     return sg ? launch_tiles<2, true>(p, grid, L.total, st) : launch_tiles<2, false>(p, grid, L.total, st);
   }
@@ -1349,10 +1350,6 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   s->xstride = max_steps * 32u + 4u;
   s->table_words = mats[0]->tiles.table_words;
   s->d_table = mats[0]->dict->d_table;
-  if (tiles_smem(s->table_words, 3u * s->xstride, kTilesWarps).total > kSmemLimit) {
-    delete s;
-    return TQ_ERR_UNSUPPORTED_SHAPE;
-  }
   const StackPlan pl = plan_stack(mats, n_mats, s->grid);
   std::vector<tq_tiles_desc> descs((size_t)n_mats);
   for (int i = 0; i < n_mats; ++i) {

@@ -71,7 +71,8 @@ def test_config0_layer_2048x2048(tq, layout):
     assert m.info.stream_bytes == stream.nbytes
 
 
-@pytest.mark.parametrize("rows,cols", [(1, 4), (3, 8), (7, 260), (8, 256), (9, 1028), (33, 2052), (17, 8192), (5, 12288), (40, 4 * 300)])
+@pytest.mark.parametrize("rows,cols", [(1, 4), (3, 8), (7, 260), (8, 256), (9, 1028), (33, 2052), (17, 8192), (5, 12288),
+                                       (40, 4 * 300), (35, 28672)])
 def test_ragged_shapes(tq, rows, cols, layout):
     if layout == 2 and cols > tq.TQ_TILES_MAX_COLS:
         with pytest.raises(tq.TqError) as e:
