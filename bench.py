@@ -234,6 +234,40 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
                          else "one launch per matrix (tq_decompress)",
                          "bytes": {"read": rd, "written": n_weights},
                          "frac_of_measured_hbm": (rd + n_weights) / (ms * 1e-3) / 1e9 / measured_peaks()[0]}
+    if args.layout == "tiles" and not args.per_layer and not args.shapes and "xs" in extra:
+        # The same products launched the way a decoder with real data dependencies could launch them:
+        # one stack per set of layers that may run together ({q,k,v}, {o}, {gate,up}, {down} per decoder
+        # layer, then the output head), replayed as one CUDA graph.  Every launch reloads the table.
+        names = [n.split(".")[-1] for n, _, _ in shapes]
+        sets, cur, last = [], [], None
+        kind = {"q": 0, "k": 0, "v": 0, "o": 1, "gate": 2, "up": 2, "down": 3, "lm_head": 4}
+        for i, n in enumerate(names):
+            k = kind.get(n, 5)
+            if cur and k != last:
+                sets.append(cur)
+                cur = []
+            cur.append(i)
+            last = k
+        sets.append(cur)
+        dep_stacks = [tq.tq_stack_create([mats[i] for i in g], [extra["xs"][i] for i in g], [extra["ys"][i] for i in g])
+                      for g in sets]
+
+        def run_dep():
+            for st in dep_stacks:
+                tq.tq_fused_gemv_stack(st)
+
+        run_dep()
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            run_dep()
+        ms = timed(g.replay, 20)
+        alg = sum(algorithmic_bytes(i, args.batch) for i in infos)
+        out["dependent_launches"] = {"launches_per_token": sum(s_.launches for s_ in dep_stacks), "ms": ms,
+                                     "GB_per_s": alg / (ms * 1e-3) / 1e9,
+                                     "frac_of_measured_hbm": alg / (ms * 1e-3) / 1e9 / measured_peaks()[0],
+                                     "grouping": "{q,k,v} {o} {gate,up} {down} per decoder layer, then the output head"}
+        del dep_stacks, g
     if args.layout != "stream":
         M = args.prefill_tokens
         max_rows = max(i.rows for i in infos)
@@ -482,7 +516,7 @@ def main():
         extras = {}
         if not args.no_extras and world == 1:
             extras = time_extras(tq, mats, infos, shapes, args, device, stream,
-                                 {"hd": hd, "dd": dd, "q_host": q_host, "scales": scales})
+                                 {"hd": hd, "dd": dd, "q_host": q_host, "scales": scales, "xs": xs, "ys": ys})
 
     ms_step = ms_total / args.steps
     if world > 1:

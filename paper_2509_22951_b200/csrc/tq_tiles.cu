@@ -121,6 +121,16 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                : "memory");
 }
 
+// The table into shared memory with bulk copies (one thread issues them; nothing waits until the
+// first lookup, so the activation set-up and the first loads of the streams overlap the copy).
+constexpr uint32_t kTableBarOffset = 400u;  // inside the misc area of the shared-memory plan
+__device__ __forceinline__ void table_load_async(uint32_t tbl_addr, uint32_t bar, const uint32_t* table, uint32_t words) {
+  const uint32_t bytes = words * 4u;
+  mbar_expect_tx(bar, bytes);
+  for (uint32_t off = 0; off < bytes; off += 8192u)
+    bulk_g2s(tbl_addr + off, reinterpret_cast<const uint8_t*>(table) + off, min(8192u, bytes - off), bar);
+}
+
 template <bool SIGNED>
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
@@ -190,7 +200,7 @@ struct TilesCta {
   uint32_t tbl_addr;
   uint32_t xstride;
   uint32_t warp, lane;
-  bool dead = false;
+  bool dead = false, table_ready = false;
 
   __device__ __forceinline__ uint32_t* misc_u32() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
   // misc: [0] dead flag, [1..2] amax bits per vector, [4..4+2W) partial ids, then 8-byte aligned XInfo and
@@ -300,7 +310,7 @@ struct TilesCta {
     const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
     const uint32_t par = (n_waited >> 2) & 1u;
     ++n_waited;
-    if (mbar_try(bar, par)) return true;
+    if (__all_sync(kFull, mbar_try(bar, par))) return true;  // one answer per warp: the slow path votes too
     return tiles_wait_slow(bar, par, dead_flag());
   }
 
@@ -310,6 +320,15 @@ struct TilesCta {
   // tiles ahead) only after the last use, so no register is copied while a load into it is in
   // flight.
   __device__ void run_tiles(const tq_tiles_desc& d, uint32_t t0, uint32_t t1) {
+    if (!table_ready) {  // the table copy started with the kernel; its first use is here
+      if (!__all_sync(kFull, mbar_try(tbl_addr + L.misc + kTableBarOffset, 0u)) &&
+          !tiles_wait_slow(tbl_addr + L.misc + kTableBarOffset, 0u, dead_flag())) {
+        dead = true;
+        if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
+        return;
+      }
+      table_ready = true;
+    }
     const uint32_t S = d.steps;
     const uint32_t g = lane >> 2, t = lane & 3u;
     // a miss token m (>= kMissBase) addresses word m - kMissBase of this warp's ring
@@ -493,13 +512,10 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
 
   if (threadIdx.x < W * kSlots) mbar_init(cta.tbl_addr + cta.L.bar + threadIdx.x * 8u, 1u);
   if (threadIdx.x == 0) *cta.dead_flag() = 0u;
+  if (threadIdx.x == 0) mbar_init(cta.tbl_addr + cta.L.misc + kTableBarOffset, 1u);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(p.table);
-    uint4* dst = reinterpret_cast<uint4*>(tiles_smem_raw);
-    for (uint32_t i = threadIdx.x; i < p.table_words / 4u; i += W * 32) dst[i] = __ldg(src + i);
-  }
+  if (threadIdx.x == 0) table_load_async(cta.tbl_addr, cta.tbl_addr + cta.L.misc + kTableBarOffset, p.table, p.table_words);
   __syncthreads();
 
   if (p.mats == nullptr) {
@@ -575,6 +591,7 @@ struct PanelCta {
   uint32_t tbl_addr, warp, lane, nb_valid;
   uint32_t ring_addr, bar_base;
   uint32_t n_issued = 0, n_waited = 0;
+  bool table_ready = false;
 
   // misc: [0] dead flag, +16 amax bits[8], +64 in_scale[8], +128 XInfo8, +256 sums[8]
   __device__ __forceinline__ volatile uint32_t* dead_flag() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
@@ -595,7 +612,7 @@ struct PanelCta {
     const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
     const uint32_t par = (n_waited >> 2) & 1u;
     ++n_waited;
-    if (mbar_try(bar, par)) return true;
+    if (__all_sync(kFull, mbar_try(bar, par))) return true;  // one answer per warp: the slow path votes too
     return tiles_wait_slow(bar, par, dead_flag());
   }
 
@@ -710,6 +727,12 @@ struct PanelCta {
   __device__ void run_segment(const tq_tiles_desc& d, uint32_t rb0, uint32_t rb1) {
     __syncthreads();  // the previous segment is done with the panel buffers and the scales
     prepare_scales(d);
+    bool table_ok = true;
+    if (!table_ready) {  // the table copy started with the kernel; its first use is below
+      table_ok = __all_sync(kFull, mbar_try(tbl_addr + L.misc + kTableBarOffset, 0u)) ||
+                 tiles_wait_slow(tbl_addr + L.misc + kTableBarOffset, 0u, dead_flag());
+      table_ready = true;
+    }
     const uint32_t S = d.steps;
     const uint32_t NP = (S + kPanelSteps - 1) / kPanelSteps;  // panels per row block
     const uint32_t R = (rb1 - rb0 + W - 1) / W;               // row blocks per warp
@@ -751,7 +774,7 @@ struct PanelCta {
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0;
     uint32_t wbuf[2][16];
-    bool ok = true;
+    bool ok = table_ok;
 
     auto lookups = [&](int k) {
       const uint32_t rd_next = tr[k];
@@ -846,13 +869,10 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_panel_kernel(const Tiles
 
   if (threadIdx.x < W * kSlots) mbar_init(cta.tbl_addr + cta.L.bar + threadIdx.x * 8u, 1u);
   if (threadIdx.x == 0) *cta.dead_flag() = 0u;
+  if (threadIdx.x == 0) mbar_init(cta.tbl_addr + cta.L.misc + kTableBarOffset, 1u);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(p.table);
-    uint4* dst = reinterpret_cast<uint4*>(tiles_smem_raw);
-    for (uint32_t i = threadIdx.x; i < p.table_words / 4u; i += W * 32) dst[i] = __ldg(src + i);
-  }
+  if (threadIdx.x == 0) table_load_async(cta.tbl_addr, cta.tbl_addr + cta.L.misc + kTableBarOffset, p.table, p.table_words);
   __syncthreads();
 
   if (p.mats == nullptr) {
@@ -954,6 +974,7 @@ struct DecompCta {
   uint32_t tbl_addr, warp, lane;
   uint32_t ring_addr, bar_base, levels_signed;
   uint32_t n_issued = 0, n_waited = 0;
+  bool table_ready = false;
 
   __device__ __forceinline__ volatile uint32_t* dead_flag() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
   __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t pos) {
@@ -968,12 +989,20 @@ struct DecompCta {
     const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
     const uint32_t par = (n_waited >> 2) & 1u;
     ++n_waited;
-    if (mbar_try(bar, par)) return true;
+    if (__all_sync(kFull, mbar_try(bar, par))) return true;  // one answer per warp: the slow path votes too
     return tiles_wait_slow(bar, par, dead_flag());
   }
 
   // tiles [t0, t1) of matrix d -> out (rows x cols bytes, row-major; or whole tiles of bf16)
   __device__ void run_tiles(const tq_tiles_desc& d, uint32_t* __restrict__ out, uint32_t t0, uint32_t t1) {
+    if (!table_ready) {  // the table copy started with the kernel; its first use is here
+      if (!__all_sync(kFull, mbar_try(tbl_addr + L.misc + kTableBarOffset, 0u)) &&
+          !tiles_wait_slow(tbl_addr + L.misc + kTableBarOffset, 0u, dead_flag())) {
+        if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
+        return;
+      }
+      table_ready = true;
+    }
     const uint32_t S = d.steps, gpr = d.cols >> 2;
     const uint32_t g = lane >> 2, t = lane & 3u;
     const uint32_t miss_adj4 = ring_addr - 4u * kMissBase;
@@ -1111,13 +1140,10 @@ __global__ void __launch_bounds__(W * 32, 1) decompress_tiles_smem_kernel(const 
   cta.bar_base = cta.tbl_addr + cta.L.bar + cta.warp * (kSlots * 8u);
   if (threadIdx.x < W * kSlots) mbar_init(cta.tbl_addr + cta.L.bar + threadIdx.x * 8u, 1u);
   if (threadIdx.x == 0) *cta.dead_flag() = 0u;
+  if (threadIdx.x == 0) mbar_init(cta.tbl_addr + cta.L.misc + kTableBarOffset, 1u);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(p.table);
-    uint4* dst = reinterpret_cast<uint4*>(tiles_smem_raw);
-    for (uint32_t i = threadIdx.x; i < p.table_words / 4u; i += W * 32) dst[i] = __ldg(src + i);
-  }
+  if (threadIdx.x == 0) table_load_async(cta.tbl_addr, cta.tbl_addr + cta.L.misc + kTableBarOffset, p.table, p.table_words);
   __syncthreads();
   if (p.mats == nullptr) {
     const uint32_t nrb = p.one.row_blocks;
