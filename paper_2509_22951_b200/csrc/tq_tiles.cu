@@ -190,22 +190,91 @@ __device__ __noinline__ void tiles_finalize(const float* __restrict__ scale, con
   }
 }
 
+// What every CTA of these kernels carries: the shared-memory plan, the table and this warp's raw ring.
+//
+// Raw ring: chunk c of a matrix's raw stream (words 256c .. 256c+255) always lands at ring offset
+// (c mod 4) KB, the place its tokens point to.  The barriers are used round robin in issue order,
+// which is also the order of the waits: use number n takes barrier n mod 4 and completes its phase
+// (n / 4) mod 2.
+struct CtaBase {
+  uint8_t* smem;
+  TilesSmem L;
+  uint32_t tbl_addr;             // shared address of the table (start of dynamic shared memory)
+  uint32_t warp, lane;
+  uint32_t ring_addr, bar_base;  // shared addresses of this warp's ring and of its first barrier
+  uint32_t n_issued = 0, n_waited = 0;
+  bool table_ready = false;
+
+  __device__ __forceinline__ volatile uint32_t* dead_flag() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
+
+  // Barriers, table copy (asynchronous: wait_table() before the first lookup), one CTA barrier.
+  __device__ __forceinline__ void setup(uint8_t* smem_raw, const TilesSmem& plan, int warps, const uint32_t* table,
+                                        uint32_t table_words) {
+    smem = smem_raw;
+    L = plan;
+    tbl_addr = smem_u32(smem_raw);
+    warp = threadIdx.x >> 5;
+    lane = threadIdx.x & 31u;
+    ring_addr = tbl_addr + L.ring + warp * (kRingWords * 4u);
+    bar_base = tbl_addr + L.bar + warp * (kSlots * 8u);
+    if (threadIdx.x < (uint32_t)warps * kSlots) mbar_init(tbl_addr + L.bar + threadIdx.x * 8u, 1u);
+    if (threadIdx.x == 0) {
+      *dead_flag() = 0u;
+      mbar_init(tbl_addr + L.misc + kTableBarOffset, 1u);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (threadIdx.x == 0) table_load_async(tbl_addr, tbl_addr + L.misc + kTableBarOffset, table, table_words);
+    __syncthreads();
+  }
+  // False if the bounded wait ran out.
+  __device__ __forceinline__ bool wait_table() {
+    if (table_ready) return true;
+    const uint32_t bar = tbl_addr + L.misc + kTableBarOffset;
+    if (!__all_sync(kFull, mbar_try(bar, 0u)) && !tiles_wait_slow(bar, 0u, dead_flag())) return false;
+    table_ready = true;
+    return true;
+  }
+  __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t pos) {  // pos: first word, multiple of 256
+    if (lane == 0) {
+      const uint32_t bar = bar_base + (n_issued & (kSlots - 1u)) * 8u;
+      mbar_expect_tx(bar, kChunkWords * 4u);
+      bulk_g2s(ring_addr + ((pos * 4u) & (kRingWords * 4u - 1u)), raw + pos, kChunkWords * 4u, bar);
+    }
+    ++n_issued;
+  }
+  __device__ __forceinline__ bool wait_chunk() {
+    const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
+    const uint32_t par = (n_waited >> 2) & 1u;
+    ++n_waited;
+    if (__all_sync(kFull, mbar_try(bar, par))) return true;  // one answer per warp: the slow path votes too
+    return tiles_wait_slow(bar, par, dead_flag());
+  }
+  // The 16 words of this lane's tokens: a token below kMissBase indexes the table, any other names
+  // the ring slot of its raw word.
+  __device__ __forceinline__ void lookup16(const uint4 (&q)[2], uint32_t (&w)[16]) const {
+    const uint32_t miss_adj4 = ring_addr - 4u * kMissBase;
+    const uint32_t R[8] = {q[0].x, q[0].y, q[0].z, q[0].w, q[1].x, q[1].y, q[1].z, q[1].w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const uint32_t lo4 = (R[i] << 2) & 0x3FFFCu, hi4 = (R[i] >> 14) & 0x3FFFCu;  // token * 4
+      w[2 * i] = lds_u32(lo4 + (lo4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
+      w[2 * i + 1] = lds_u32(hi4 + (hi4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
+    }
+  }
+};
+
 template <int W, int NB, bool SIGNED>
-struct TilesCta {
+struct TilesCta : CtaBase {
   static constexpr int kThreads = W * 32;
   static constexpr int NCOL = 3 * NB;
 
-  uint8_t* smem;
-  TilesSmem L;
-  uint32_t tbl_addr;
   uint32_t xstride;
-  uint32_t warp, lane;
-  bool dead = false, table_ready = false;
+  bool dead = false;
 
   __device__ __forceinline__ uint32_t* misc_u32() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
   // misc: [0] dead flag, [1..2] amax bits per vector, [4..4+2W) partial ids, then 8-byte aligned XInfo and
   // reduction scratch
-  __device__ __forceinline__ volatile uint32_t* dead_flag() { return misc_u32(); }
   __device__ __forceinline__ uint32_t* part_ids() { return misc_u32() + 4; }
   __device__ __forceinline__ XInfo* xinfo() { return reinterpret_cast<XInfo*>(smem + L.misc + 192); }
   __device__ __forceinline__ long long* sum_scratch() { return reinterpret_cast<long long*>(smem + L.misc + 256); }
@@ -291,48 +360,19 @@ struct TilesCta {
     if (lane == 0) part_ids()[2 * warp + slot] = rb;
   }
 
-  // ---- raw ring ---------------------------------------------------------------------------
-  // Chunk c of the raw stream (words 256c .. 256c+255) always lands at ring offset (c mod 4) KB, the
-  // place its tokens point to.  The barriers are used round robin in issue order, which is also the
-  // order of the waits: use number n takes barrier n mod 4 and completes its phase (n / 4) mod 2.
-  uint32_t ring_addr, bar_base;  // shared addresses of this warp's ring and of its first barrier
-  uint32_t n_issued = 0, n_waited = 0;
-
-  __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t pos) {  // pos: first word, multiple of 256
-    if (lane == 0) {
-      const uint32_t bar = bar_base + (n_issued & (kSlots - 1u)) * 8u;
-      mbar_expect_tx(bar, kChunkWords * 4u);
-      bulk_g2s(ring_addr + ((pos * 4u) & (kRingWords * 4u - 1u)), raw + pos, kChunkWords * 4u, bar);
-    }
-    ++n_issued;
-  }
-  __device__ __forceinline__ bool wait_chunk() {
-    const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
-    const uint32_t par = (n_waited >> 2) & 1u;
-    ++n_waited;
-    if (__all_sync(kFull, mbar_try(bar, par))) return true;  // one answer per warp: the slow path votes too
-    return tiles_wait_slow(bar, par, dead_flag());
-  }
-
   // ---- one warp, tiles [t0, t1) of matrix d -------------------------------------------------
   // Tile i of the run uses token registers q[i & 1] and word buffer i & 1; its words are consumed
   // by the MMAs while tile i + 1 is being looked up, and its token registers are reloaded (two
   // tiles ahead) only after the last use, so no register is copied while a load into it is in
   // flight.
   __device__ void run_tiles(const tq_tiles_desc& d, uint32_t t0, uint32_t t1) {
-    if (!table_ready) {  // the table copy started with the kernel; its first use is here
-      if (!__all_sync(kFull, mbar_try(tbl_addr + L.misc + kTableBarOffset, 0u)) &&
-          !tiles_wait_slow(tbl_addr + L.misc + kTableBarOffset, 0u, dead_flag())) {
-        dead = true;
-        if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
-        return;
-      }
-      table_ready = true;
+    if (!wait_table()) {  // the table copy started with the kernel; its first use is here
+      dead = true;
+      if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
+      return;
     }
     const uint32_t S = d.steps;
     const uint32_t g = lane >> 2, t = lane & 3u;
-    // a miss token m (>= kMissBase) addresses word m - kMissBase of this warp's ring
-    const uint32_t miss_adj4 = ring_addr - 4u * kMissBase;
     // lanes whose B column is not in use read the last used column: what they feed the MMA only
     // reaches accumulator columns nobody reads
     const uint32_t x_lane = tbl_addr + L.x + (min(g, (uint32_t)NCOL - 1u) * xstride + 8u * t) * 4u;
@@ -370,13 +410,7 @@ struct TilesCta {
         if (!wait_chunk()) return false;
         w_pos += kChunkWords;
       }
-      const uint32_t R[8] = {q[k][0].x, q[k][0].y, q[k][0].z, q[k][0].w, q[k][1].x, q[k][1].y, q[k][1].z, q[k][1].w};
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const uint32_t lo4 = (R[i] << 2) & 0x3FFFCu, hi4 = (R[i] >> 14) & 0x3FFFCu;  // token * 4
-        wbuf[k][2 * i] = lds_u32(lo4 + (lo4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
-        wbuf[k][2 * i + 1] = lds_u32(hi4 + (hi4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
-      }
+      lookup16(q[k], wbuf[k]);
       q[k][0] = ldg_stream(tok);
       q[k][1] = ldg_stream(tok + 32);
       tr[k] = __ldg(trp);
@@ -501,22 +535,8 @@ template <int W, int NB, bool SIGNED>
 __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams p) {
   extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
   TilesCta<W, NB, SIGNED> cta;
-  cta.smem = tiles_smem_raw;
-  cta.L = tiles_smem(p.table_words, 3u * NB * p.xstride, W);
-  cta.tbl_addr = smem_u32(tiles_smem_raw);
+  cta.setup(tiles_smem_raw, tiles_smem(p.table_words, 3u * NB * p.xstride, W), W, p.table, p.table_words);
   cta.xstride = p.xstride;
-  cta.warp = threadIdx.x >> 5;
-  cta.lane = threadIdx.x & 31u;
-  cta.ring_addr = cta.tbl_addr + cta.L.ring + cta.warp * (kRingWords * 4u);
-  cta.bar_base = cta.tbl_addr + cta.L.bar + cta.warp * (kSlots * 8u);
-
-  if (threadIdx.x < W * kSlots) mbar_init(cta.tbl_addr + cta.L.bar + threadIdx.x * 8u, 1u);
-  if (threadIdx.x == 0) *cta.dead_flag() = 0u;
-  if (threadIdx.x == 0) mbar_init(cta.tbl_addr + cta.L.misc + kTableBarOffset, 1u);
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  if (threadIdx.x == 0) table_load_async(cta.tbl_addr, cta.tbl_addr + cta.L.misc + kTableBarOffset, p.table, p.table_words);
-  __syncthreads();
 
   if (p.mats == nullptr) {
     const uint32_t nrb = p.one.row_blocks;
@@ -580,41 +600,19 @@ __device__ __noinline__ void panel_finalize(const float* __restrict__ scale, con
 }
 
 template <int W, int NB, bool SIGNED>
-struct PanelCta {
+struct PanelCta : CtaBase {
   static constexpr int kThreads = W * 32;
   static constexpr int NCOL = 3 * NB;
   static constexpr int NT = (NCOL + 7) / 8;
   static constexpr int kBufWords = 8 * NT * kPanelStride;  // one panel buffer: whole MMA tiles of columns
 
-  uint8_t* smem;
-  TilesSmem L;
-  uint32_t tbl_addr, warp, lane, nb_valid;
-  uint32_t ring_addr, bar_base;
-  uint32_t n_issued = 0, n_waited = 0;
-  bool table_ready = false;
+  uint32_t nb_valid;
 
   // misc: [0] dead flag, +16 amax bits[8], +64 in_scale[8], +128 XInfo8, +256 sums[8]
-  __device__ __forceinline__ volatile uint32_t* dead_flag() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
   __device__ __forceinline__ uint32_t* amax_bits() { return reinterpret_cast<uint32_t*>(smem + L.misc + 16); }
   __device__ __forceinline__ float* in_scale() { return reinterpret_cast<float*>(smem + L.misc + 64); }
   __device__ __forceinline__ XInfo8* xinfo() { return reinterpret_cast<XInfo8*>(smem + L.misc + 128); }
   __device__ __forceinline__ long long* sums() { return reinterpret_cast<long long*>(smem + L.misc + 256); }
-
-  __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t pos) {
-    if (lane == 0) {
-      const uint32_t bar = bar_base + (n_issued & (kSlots - 1u)) * 8u;
-      mbar_expect_tx(bar, kChunkWords * 4u);
-      bulk_g2s(ring_addr + ((pos * 4u) & (kRingWords * 4u - 1u)), raw + pos, kChunkWords * 4u, bar);
-    }
-    ++n_issued;
-  }
-  __device__ __forceinline__ bool wait_chunk() {
-    const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
-    const uint32_t par = (n_waited >> 2) & 1u;
-    ++n_waited;
-    if (__all_sync(kFull, mbar_try(bar, par))) return true;  // one answer per warp: the slow path votes too
-    return tiles_wait_slow(bar, par, dead_flag());
-  }
 
   // digits of one activation group (4 columns) -> three words
   static __device__ __forceinline__ void digits(uint2 v, float scale, bool finite, uint32_t& w0, uint32_t& w1,
@@ -727,12 +725,7 @@ struct PanelCta {
   __device__ void run_segment(const tq_tiles_desc& d, uint32_t rb0, uint32_t rb1) {
     __syncthreads();  // the previous segment is done with the panel buffers and the scales
     prepare_scales(d);
-    bool table_ok = true;
-    if (!table_ready) {  // the table copy started with the kernel; its first use is below
-      table_ok = __all_sync(kFull, mbar_try(tbl_addr + L.misc + kTableBarOffset, 0u)) ||
-                 tiles_wait_slow(tbl_addr + L.misc + kTableBarOffset, 0u, dead_flag());
-      table_ready = true;
-    }
+    const bool table_ok = wait_table();  // the table copy started with the kernel; its first use is below
     const uint32_t S = d.steps;
     const uint32_t NP = (S + kPanelSteps - 1) / kPanelSteps;  // panels per row block
     const uint32_t R = (rb1 - rb0 + W - 1) / W;               // row blocks per warp
@@ -744,7 +737,6 @@ struct PanelCta {
     __syncthreads();
 
     const uint32_t g = lane >> 2, t = lane & 3u;
-    const uint32_t miss_adj4 = ring_addr - 4u * kMissBase;
     const uint32_t x_lane = tbl_addr + L.x + (g * kPanelStride + 8u * t) * 4u;
 
     uint32_t rd = 0, stop_pos = 0, w_pos = 0, i_pos = 0;
@@ -783,13 +775,7 @@ struct PanelCta {
         w_pos += kChunkWords;
       }
       if (!ok) return;
-      const uint32_t Rg[8] = {q[k][0].x, q[k][0].y, q[k][0].z, q[k][0].w, q[k][1].x, q[k][1].y, q[k][1].z, q[k][1].w};
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const uint32_t lo4 = (Rg[i] << 2) & 0x3FFFCu, hi4 = (Rg[i] >> 14) & 0x3FFFCu;
-        wbuf[k][2 * i] = lds_u32(lo4 + (lo4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
-        wbuf[k][2 * i + 1] = lds_u32(hi4 + (hi4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
-      }
+      lookup16(q[k], wbuf[k]);
       q[k][0] = ldg_stream(tok);
       q[k][1] = ldg_stream(tok + 32);
       tr[k] = __ldg(trp);
@@ -858,22 +844,8 @@ template <int W, int NB, bool SIGNED>
 __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_panel_kernel(const TilesParams p) {
   extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
   PanelCta<W, NB, SIGNED> cta;
-  cta.smem = tiles_smem_raw;
-  cta.L = tiles_smem(p.table_words, 2u * PanelCta<W, NB, SIGNED>::kBufWords, W);
-  cta.tbl_addr = smem_u32(tiles_smem_raw);
-  cta.warp = threadIdx.x >> 5;
-  cta.lane = threadIdx.x & 31u;
+  cta.setup(tiles_smem_raw, tiles_smem(p.table_words, 2u * PanelCta<W, NB, SIGNED>::kBufWords, W), W, p.table, p.table_words);
   cta.nb_valid = p.nb_valid;
-  cta.ring_addr = cta.tbl_addr + cta.L.ring + cta.warp * (kRingWords * 4u);
-  cta.bar_base = cta.tbl_addr + cta.L.bar + cta.warp * (kSlots * 8u);
-
-  if (threadIdx.x < W * kSlots) mbar_init(cta.tbl_addr + cta.L.bar + threadIdx.x * 8u, 1u);
-  if (threadIdx.x == 0) *cta.dead_flag() = 0u;
-  if (threadIdx.x == 0) mbar_init(cta.tbl_addr + cta.L.misc + kTableBarOffset, 1u);
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  if (threadIdx.x == 0) table_load_async(cta.tbl_addr, cta.tbl_addr + cta.L.misc + kTableBarOffset, p.table, p.table_words);
-  __syncthreads();
 
   if (p.mats == nullptr) {
     const uint32_t nrb = p.one.row_blocks;
@@ -968,44 +940,17 @@ struct DecompParams {
 };
 
 template <int W, bool BF16>
-struct DecompCta {
-  uint8_t* smem;
-  TilesSmem L;
-  uint32_t tbl_addr, warp, lane;
-  uint32_t ring_addr, bar_base, levels_signed;
-  uint32_t n_issued = 0, n_waited = 0;
-  bool table_ready = false;
-
-  __device__ __forceinline__ volatile uint32_t* dead_flag() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
-  __device__ __forceinline__ void issue_chunk(const uint32_t* raw, uint32_t pos) {
-    if (lane == 0) {
-      const uint32_t bar = bar_base + (n_issued & (kSlots - 1u)) * 8u;
-      mbar_expect_tx(bar, kChunkWords * 4u);
-      bulk_g2s(ring_addr + ((pos * 4u) & (kRingWords * 4u - 1u)), raw + pos, kChunkWords * 4u, bar);
-    }
-    ++n_issued;
-  }
-  __device__ __forceinline__ bool wait_chunk() {
-    const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
-    const uint32_t par = (n_waited >> 2) & 1u;
-    ++n_waited;
-    if (__all_sync(kFull, mbar_try(bar, par))) return true;  // one answer per warp: the slow path votes too
-    return tiles_wait_slow(bar, par, dead_flag());
-  }
+struct DecompCta : CtaBase {
+  uint32_t levels_signed;
 
   // tiles [t0, t1) of matrix d -> out (rows x cols bytes, row-major; or whole tiles of bf16)
   __device__ void run_tiles(const tq_tiles_desc& d, uint32_t* __restrict__ out, uint32_t t0, uint32_t t1) {
-    if (!table_ready) {  // the table copy started with the kernel; its first use is here
-      if (!__all_sync(kFull, mbar_try(tbl_addr + L.misc + kTableBarOffset, 0u)) &&
-          !tiles_wait_slow(tbl_addr + L.misc + kTableBarOffset, 0u, dead_flag())) {
-        if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
-        return;
-      }
-      table_ready = true;
+    if (!wait_table()) {  // the table copy started with the kernel; its first use is here
+      if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
+      return;
     }
     const uint32_t S = d.steps, gpr = d.cols >> 2;
     const uint32_t g = lane >> 2, t = lane & 3u;
-    const uint32_t miss_adj4 = ring_addr - 4u * kMissBase;
     const bool vec_ok = (gpr & 3u) == 0u;  // every row starts on a 16-byte boundary
     const uint32_t xor_mask = levels_signed ? 0x80808080u : 0u;          // int8 bit pattern -> biased byte
     const float magic = levels_signed ? 8388736.0f : 8388608.0f;         // 2^23 (+ 128): as_float(0x4B000000 | byte) - magic = level
@@ -1037,14 +982,8 @@ struct DecompCta {
         w_pos += kChunkWords;
       }
       if (!ok) return;
-      const uint32_t Rg[8] = {q[k][0].x, q[k][0].y, q[k][0].z, q[k][0].w, q[k][1].x, q[k][1].y, q[k][1].z, q[k][1].w};
       uint32_t w[16];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const uint32_t lo4 = (Rg[i] << 2) & 0x3FFFCu, hi4 = (Rg[i] >> 14) & 0x3FFFCu;
-        w[2 * i] = lds_u32(lo4 + (lo4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
-        w[2 * i + 1] = lds_u32(hi4 + (hi4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
-      }
+      lookup16(q[k], w);
       q[k][0] = ldg_stream(tok);
       q[k][1] = ldg_stream(tok + 32);
       tr[k] = __ldg(trp);
@@ -1130,21 +1069,8 @@ template <int W, bool BF16>
 __global__ void __launch_bounds__(W * 32, 1) decompress_tiles_smem_kernel(const DecompParams p) {
   extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
   DecompCta<W, BF16> cta;
+  cta.setup(tiles_smem_raw, tiles_smem(p.table_words, 0u, W), W, p.table, p.table_words);
   cta.levels_signed = p.levels_signed;
-  cta.smem = tiles_smem_raw;
-  cta.L = tiles_smem(p.table_words, 0u, W);
-  cta.tbl_addr = smem_u32(tiles_smem_raw);
-  cta.warp = threadIdx.x >> 5;
-  cta.lane = threadIdx.x & 31u;
-  cta.ring_addr = cta.tbl_addr + cta.L.ring + cta.warp * (kRingWords * 4u);
-  cta.bar_base = cta.tbl_addr + cta.L.bar + cta.warp * (kSlots * 8u);
-  if (threadIdx.x < W * kSlots) mbar_init(cta.tbl_addr + cta.L.bar + threadIdx.x * 8u, 1u);
-  if (threadIdx.x == 0) *cta.dead_flag() = 0u;
-  if (threadIdx.x == 0) mbar_init(cta.tbl_addr + cta.L.misc + kTableBarOffset, 1u);
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  if (threadIdx.x == 0) table_load_async(cta.tbl_addr, cta.tbl_addr + cta.L.misc + kTableBarOffset, p.table, p.table_words);
-  __syncthreads();
   if (p.mats == nullptr) {
     const uint32_t nrb = p.one.row_blocks;
     const uint32_t rb0 = (uint32_t)((uint64_t)nrb * blockIdx.x / gridDim.x);
