@@ -250,6 +250,16 @@ int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, c
  * tq_stack_create synchronises cuda_stream; tq_fused_gemv_stack is asynchronous. */
 typedef struct tq_stack tq_stack;
 int tq_stack_size(int n_mats, uint64_t* device_bytes);
+/* The work split tq_stack_create computes, as a host-only call (no device needed): the row blocks
+ * (16 rows) of the matrices, in order, are cut into n_ctas consecutive shares of about equal cost
+ * (bytes streamed plus a fixed charge per segment); a share is a list of segments (matrix, first
+ * row block, one past the last).  steps[i] = ceil(cols_i / 128), row_blocks[i] = ceil(rows_i / 16),
+ * rb_raw[i] = HOST array of row_blocks[i] + 1 prefix counts of raw words per row block.  segs
+ * receives 3 values per segment (at most n_mats + n_ctas segments), *n_segs their number,
+ * cta_seg[n_ctas + 1] the first segment of each share. */
+int tq_stack_plan_host(int n_mats, const uint32_t* steps, const uint32_t* row_blocks,
+                       const uint32_t* const* rb_raw, uint32_t n_ctas, uint32_t* segs, uint32_t segs_cap,
+                       uint32_t* n_segs, uint32_t* cta_seg);
 int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* const* d_y, int n_mats,
                     int B, void* d_buf, uint64_t d_buf_bytes, void* cuda_stream, tq_stack** out);
 int tq_fused_gemv_stack(const tq_stack* s, void* cuda_stream);

@@ -37,7 +37,7 @@ EXPORTS = [
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
     "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_gemm_workspace_size",
-    "tq_fused_gemm_ws", "tq_decode_bf16", "tq_gemm_bf16_ws", "tq_decode_bf16_stack", "tq_stack_size", "tq_stack_create",
+    "tq_fused_gemm_ws", "tq_decode_bf16", "tq_gemm_bf16_ws", "tq_decode_bf16_stack", "tq_stack_size", "tq_stack_plan_host", "tq_stack_create",
     "tq_fused_gemv_stack", "tq_fused_gemv_stack_host", "tq_stack_launches", "tq_decompress_stack", "tq_stack_free", "tq_device_status", "tq_dmat_free",
 ]
 
@@ -94,6 +94,7 @@ def _load() -> C.CDLL:
         "tq_gemm_bf16_ws": (C.c_int, [vp, vp, C.c_int, vp, vp, vp]),
         "tq_decode_bf16_stack": (C.c_int, [vp, vp, vp]),
         "tq_stack_size": (C.c_int, [C.c_int, u64p]),
+        "tq_stack_plan_host": (C.c_int, [C.c_int, u32p, u32p, C.POINTER(u32p), C.c_uint32, u32p, C.c_uint32, u32p, u32p]),
         "tq_stack_create": (C.c_int, [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int, C.c_int, vp, C.c_uint64, vp,
                                       C.POINTER(vp)]),
         "tq_fused_gemv_stack": (C.c_int, [vp, vp]),
@@ -422,6 +423,22 @@ def tq_gemm_bf16_ws(m: DeviceMatrix, X: torch.Tensor, workspace: torch.Tensor, Y
     _check(_lib.tq_gemm_bf16_ws(m._h, X2.data_ptr(), M, Y.data_ptr(), workspace.data_ptr(), _stream_ptr(stream)),
            "tq_gemm_bf16_ws")
     return Y
+
+
+def tq_stack_plan_host(steps, row_blocks, rb_raw, n_ctas: int):
+    """-> (segments [(matrix, first row block, end row block)], cta_seg): the work split of a stack, computed on the host."""
+    n = len(steps)
+    st = np.ascontiguousarray(steps, dtype=np.uint32)
+    rbk = np.ascontiguousarray(row_blocks, dtype=np.uint32)
+    raws = [np.ascontiguousarray(r, dtype=np.uint32) for r in rb_raw]
+    ptrs = (C.POINTER(C.c_uint32) * n)(*[_np_ptr(r, C.c_uint32) for r in raws])
+    cap = n + n_ctas
+    segs = np.zeros(3 * cap, dtype=np.uint32)
+    cta = np.zeros(n_ctas + 1, dtype=np.uint32)
+    ns = C.c_uint32()
+    _check(_lib.tq_stack_plan_host(n, _np_ptr(st, C.c_uint32), _np_ptr(rbk, C.c_uint32), ptrs, n_ctas,
+                                   _np_ptr(segs, C.c_uint32), cap, C.byref(ns), _np_ptr(cta, C.c_uint32)), "tq_stack_plan_host")
+    return [tuple(int(v) for v in segs[3 * i: 3 * i + 3]) for i in range(ns.value)], cta.tolist()
 
 
 class Stack:

@@ -1225,24 +1225,27 @@ struct StackPlan {
 
 // Row blocks in matrix order, cut into `grid` consecutive shares of equal cost (bytes streamed plus
 // a fixed charge per segment start).
-StackPlan plan_stack(const tq_dmat* const* mats, int n, uint32_t grid) {
-  auto rb_cost = [&](const tq_dmat* m, uint32_t rb) -> uint64_t {
-    return (uint64_t)m->tiles.steps * 1024 + (uint64_t)(m->rb_raw[rb + 1] - m->rb_raw[rb]) * 4;
+struct PlanMat {
+  uint32_t steps, row_blocks;
+  const uint32_t* rb_raw;  // row_blocks + 1: index of each row block's first raw word
+};
+
+StackPlan plan_stack(const PlanMat* mats, int n, uint32_t grid) {
+  auto rb_cost = [&](const PlanMat& m, uint32_t rb) -> uint64_t {
+    return (uint64_t)m.steps * 1024 + (uint64_t)(m.rb_raw[rb + 1] - m.rb_raw[rb]) * 4;
   };
   uint64_t total = 0;
-  for (int i = 0; i < n; ++i) {
-    const tq_dmat* m = mats[i];
-    total += (uint64_t)m->tiles.steps * 1024 * m->tiles.row_blocks + (uint64_t)m->rb_raw[m->tiles.row_blocks] * 4;
-  }
+  for (int i = 0; i < n; ++i)
+    total += (uint64_t)mats[i].steps * 1024 * mats[i].row_blocks + (uint64_t)mats[i].rb_raw[mats[i].row_blocks] * 4;
   total += kSegmentOverheadBytes * ((uint64_t)n + grid);
   const uint64_t share = total / grid + 1;
   StackPlan pl;
   pl.cta_seg.push_back(0);
   uint64_t acc = 0;  // cost given to the current CTA
   for (int i = 0; i < n; ++i) {
-    const tq_dmat* m = mats[i];
+    const PlanMat& m = mats[i];
     uint32_t rb = 0;
-    while (rb < m->tiles.row_blocks) {
+    while (rb < m.row_blocks) {
       if (acc + kSegmentOverheadBytes >= share && pl.cta_seg.size() < grid) {  // no room for a useful segment
         pl.cta_seg.push_back((uint32_t)pl.segs.size());
         acc = 0;
@@ -1250,7 +1253,7 @@ StackPlan plan_stack(const tq_dmat* const* mats, int n, uint32_t grid) {
       acc += kSegmentOverheadBytes;
       const uint32_t begin = rb;
       const bool last_cta = pl.cta_seg.size() >= grid;
-      while (rb < m->tiles.row_blocks && (last_cta || acc < share)) acc += rb_cost(m, rb++);
+      while (rb < m.row_blocks && (last_cta || acc < share)) acc += rb_cost(m, rb++);
       pl.segs.push_back(TilesSeg{(uint32_t)i, begin, rb});
       if (acc >= share && !last_cta) {
         pl.cta_seg.push_back((uint32_t)pl.segs.size());
@@ -1266,6 +1269,26 @@ inline uint64_t align256(uint64_t v) { return (v + 255) / 256 * 256; }
 }  // namespace
 
 extern "C" {
+
+int tq_stack_plan_host(int n_mats, const uint32_t* steps, const uint32_t* row_blocks, const uint32_t* const* rb_raw,
+                       uint32_t n_ctas, uint32_t* segs, uint32_t segs_cap, uint32_t* n_segs, uint32_t* cta_seg) {
+  if (n_mats < 1 || !steps || !row_blocks || !rb_raw || n_ctas < 1 || !segs || !n_segs || !cta_seg) return TQ_ERR_INVALID_ARG;
+  std::vector<PlanMat> pm((size_t)n_mats);
+  for (int i = 0; i < n_mats; ++i) {
+    if (!rb_raw[i] || steps[i] == 0 || row_blocks[i] == 0) return TQ_ERR_INVALID_ARG;
+    pm[i] = PlanMat{steps[i], row_blocks[i], rb_raw[i]};
+  }
+  const StackPlan pl = plan_stack(pm.data(), n_mats, n_ctas);
+  *n_segs = (uint32_t)pl.segs.size();
+  if (pl.segs.size() > segs_cap) return TQ_ERR_BUFFER_TOO_SMALL;
+  for (size_t i = 0; i < pl.segs.size(); ++i) {
+    segs[3 * i] = pl.segs[i].mat;
+    segs[3 * i + 1] = pl.segs[i].rb_begin;
+    segs[3 * i + 2] = pl.segs[i].rb_end;
+  }
+  for (uint32_t c = 0; c <= n_ctas; ++c) cta_seg[c] = pl.cta_seg[c];
+  return TQ_OK;
+}
 
 int tq_stack_size(int n_mats, uint64_t* device_bytes) {
   if (n_mats < 1 || !device_bytes) return TQ_ERR_INVALID_ARG;
@@ -1302,7 +1325,9 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   s->xstride = max_steps * 32u + 4u;
   s->table_words = mats[0]->tiles.table_words;
   s->d_table = mats[0]->dict->d_table;
-  const StackPlan pl = plan_stack(mats, n_mats, s->grid);
+  std::vector<PlanMat> pm((size_t)n_mats);
+  for (int i = 0; i < n_mats; ++i) pm[i] = PlanMat{mats[i]->tiles.steps, mats[i]->tiles.row_blocks, mats[i]->rb_raw.data()};
+  const StackPlan pl = plan_stack(pm.data(), n_mats, s->grid);
   std::vector<tq_tiles_desc> descs((size_t)n_mats);
   for (int i = 0; i < n_mats; ++i) {
     descs[i] = mats[i]->tiles;

@@ -264,3 +264,38 @@ def _code_slots(stream):
     for k in range(1, 5):
         mask[esc + k] = False
     return mask
+
+
+@pytest.mark.parametrize("n_ctas", [1, 7, 148])
+def test_stack_plan_covers_every_row_block_once_and_balances_cost(n_ctas):
+    """The persistent kernels trust this split: every row block of every matrix must fall in exactly
+    one segment, segments must come in matrix order, and the shares must cost about the same."""
+    rng = np.random.default_rng(n_ctas)
+    shapes = [(3072, 3072), (1024, 3072), (1024, 3072), (3072, 3072), (8192, 3072), (8192, 3072), (3072, 8192)] * 4
+    shapes += [(128256, 3072), (17, 4), (16, 128)]
+    steps = [-(-c // 128) for _, c in shapes]
+    row_blocks = [-(-r // 16) for r, _ in shapes]
+    rb_raw = []
+    for s_, nrb in zip(steps, row_blocks):  # raw words per row block: about 55 % of the 512 groups of a tile
+        per = rng.binomial(512 * s_, 0.55, size=nrb).astype(np.uint64)
+        rb_raw.append(np.concatenate([[0], np.cumsum(per)]).astype(np.uint32))
+    segs, cta_seg = tq.tq_stack_plan_host(steps, row_blocks, rb_raw, n_ctas)
+    assert len(cta_seg) == n_ctas + 1 and cta_seg[0] == 0 and cta_seg[-1] == len(segs)
+    assert all(a <= b for a, b in zip(cta_seg, cta_seg[1:]))
+    nxt = [0] * len(shapes)
+    order = []
+    for m, b, e in segs:
+        assert b == nxt[m] and b < e <= row_blocks[m]
+        nxt[m] = e
+        order.append(m)
+    assert nxt == row_blocks and order == sorted(order)
+
+    def cost(m, b, e):
+        return (e - b) * steps[m] * 1024 + 4 * (int(rb_raw[m][e]) - int(rb_raw[m][b]))
+
+    share = [sum(cost(*segs[i]) for i in range(cta_seg[c], cta_seg[c + 1])) for c in range(n_ctas)]
+    total = sum(share)
+    assert total == sum(cost(m, 0, row_blocks[m]) for m in range(len(shapes)))
+    if n_ctas > 1:
+        biggest_block = max(cost(m, 0, 1) for m in range(len(shapes))) * 2
+        assert max(share) <= total / n_ctas + biggest_block + (len(shapes) + n_ctas) * 96 * 1024 / n_ctas + 96 * 1024 * 3
