@@ -111,18 +111,26 @@ TRAFFIC_RATIO = {"tiles_stack": 1.047}
 TRAFFIC = {}
 
 
-def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout=1):
-    """Generate, quantize (GPU), build the table and encode (host), upload.  Returns
-    (matrices, xs, ys, table, stats)."""
+def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout=1, quantizer="rows"):
+    """Generate, quantize, build the table and encode (host), upload.  quantizer "rows": per-row
+    symmetric int8 on the GPU (the workload definition); "paper": Listing 1, one scale and zero point
+    per tensor, unsigned levels (host).  Returns (matrices, xs, ys, table, ...)."""
     t0 = time.time()
     if threads:
         tq.tq_set_num_threads(threads)
-    q_host, scales = [], []
+    q_host, scales, zeros = [], [], []
     for i, (name, rows, cols) in enumerate(shapes):
         w = synth.weight(rows, cols, synth.matrix_seed(i), device=device)
-        q, s = tq.tq_quantize_rows_device(w)
-        q_host.append(q.cpu().numpy())
-        scales.append(s.cpu().numpy())
+        if quantizer == "paper":
+            q, s, z = tq.tq_quantize_tensor(w.cpu().numpy())
+            q_host.append(q.reshape(rows, cols))
+            scales.append(np.full(rows, s, dtype=np.float32))
+            zeros.append(np.full(rows, z, dtype=np.float32))
+        else:
+            q, s = tq.tq_quantize_rows_device(w)
+            q_host.append(q.cpu().numpy())
+            scales.append(s.cpu().numpy())
+            zeros.append(None)
         del w, q, s
     t1 = time.time()
     hd = tq.tq_build_dictionary(q_host) if table_entries is None else tq.tq_dict_from_entries(table_entries)
@@ -131,7 +139,8 @@ def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout
     mats = []
     for i, (name, rows, cols) in enumerate(shapes):
         stream, h, m = tq.tq_encode(hd, q_host[i])
-        mats.append(tq.tq_upload(dd, stream, rows, cols, scales[i], layout=layout))
+        mats.append(tq.tq_upload(dd, stream, rows, cols, scales[i], zeros[i], levels_signed=(quantizer != "paper"),
+                                 layout=layout))
         del stream
     t3 = time.time()
     # all x in one arena and all y in another (16-byte aligned pieces), so that the end-to-end
@@ -339,7 +348,10 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="tq", choices=["tq", "reference"])
-    ap.add_argument("--model", default="3b", choices=["1b", "3b"])
+    ap.add_argument("--model", default="3b", choices=["1b", "3b", "11b"])
+    ap.add_argument("--quantizer", default="rows", choices=["rows", "paper"],
+                    help="rows: per-row symmetric int8 (the workload definition); paper: Listing 1, per tensor, unsigned levels "
+                         "with a zero point (a regime where nearly every group is in the table); single GPU, no CPU baseline")
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--layers", type=int, default=None, help="decoder layers to build (default: all)")
     ap.add_argument("--no-lm-head", action="store_true")
@@ -358,6 +370,9 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     shapes = synth.llama32_linear_shapes(args.model, args.layers, lm_head=not args.no_lm_head)
     workload = f"llama3.2-{args.model} linear stack ({len(shapes)} matrices), batch {args.batch}"
+    if args.quantizer == "paper":
+        workload += ", per-tensor quantizer of Listing 1"
+        assert int(os.environ.get("WORLD_SIZE", "1")) == 1 and not args.per_layer
     if args.shapes:
         shapes = [(f"m{i}", int(t.split("x")[0]), int(t.split("x")[1])) for i, t in enumerate(args.shapes.split(","))]
         workload = f"custom shapes {args.shapes}, batch {args.batch}"
@@ -399,7 +414,7 @@ def main():
         dist.broadcast(ent, 0)
         table_entries = ent.cpu().numpy()
 
-    mats, xs, ys, hd, q_host, scales, stats, x_arena, y_arena, dd = build_model(tq, shapes, args.batch, device, threads, table_entries, layout={"stream": 0, "planes": 1, "tiles": 2}[args.layout])
+    mats, xs, ys, hd, q_host, scales, stats, x_arena, y_arena, dd = build_model(tq, shapes, args.batch, device, threads, table_entries, layout={"stream": 0, "planes": 1, "tiles": 2}[args.layout], quantizer=args.quantizer)
     infos = [m.info for m in mats]
     hits = sum(i.n_hits for i in infos)
     miss = sum(i.n_miss for i in infos)
@@ -574,7 +589,7 @@ def main():
                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                       "ms_per_step": e2e["ms_per_step"], "steps": e2e["steps"]}
 
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and args.quantizer == "rows":
         sample = pick_sample(shapes, 3_300_000_000)  # ~13 s of single-thread oracle work for the 3B stack
         total, times = oracle_sample_run(hd.entries, q_host, scales, shapes, args.batch, sample, reps=1)
         best = min(times)

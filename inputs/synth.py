@@ -16,7 +16,7 @@ Recipe
   from the same seed are bit-identical.
 * Activations: the same sampler with a standard-normal quantile table, rounded
   to bf16 (round to nearest even).
-* Shapes: the linear layers of LLaMA-3.2-1B / 3B (q, k, v, o, gate, up, down per
+* Shapes: the linear layers of LLaMA-3.2-1B / 3B / 11B (q, k, v, o, gate, up, down per
   decoder layer, then lm_head), in that order.
 """
 from __future__ import annotations
@@ -129,6 +129,8 @@ def llama32_linear_shapes(model: str, n_layers: int | None = None, lm_head: bool
     cfg = {
         "1b": dict(h=2048, kv=512, ffn=8192, layers=16, vocab=128256),
         "3b": dict(h=3072, kv=1024, ffn=8192, layers=28, vocab=128256),
+        # text decoder of LLaMA-3.2-11B-Vision (its self-attention layers): a second workload with long rows
+        "11b": dict(h=4096, kv=1024, ffn=14336, layers=32, vocab=128256),
     }[model.lower()]
     L = cfg["layers"] if n_layers is None else n_layers
     out = []

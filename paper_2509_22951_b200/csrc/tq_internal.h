@@ -124,16 +124,23 @@ int tq_tiles_decode_bf16(const tq_dmat* m, void* d_out, void* cuda_stream);
 
 // A set of TILES matrices bound to their operands, with the work split among the CTAs of one
 // persistent launch (tq_tiles.cu).
+// One split of (a subset of) a stack's matrices among the CTAs.
+struct tq_stack_plan {
+  const void* d_segs = nullptr;         // DEVICE: segments, grouped by CTA
+  const uint32_t* d_cta_seg = nullptr;  // DEVICE: grid + 1 offsets into the segments
+  uint32_t n_segs = 0, n_mats = 0;
+  uint32_t xstride = 0;                 // words per digit column a whole row of its longest matrix needs
+};
+
 struct tq_stack {
   int n = 0, B = 0;
   int levels_signed = 0;
-  uint32_t grid = 0, xstride = 0, table_words = 0;
+  uint32_t grid = 0, table_words = 0;
   const uint32_t* d_table = nullptr;
   const tq_tiles_desc* d_descs = nullptr;  // DEVICE
-  const void* d_segs = nullptr;            // DEVICE
-  const uint32_t* d_cta_seg = nullptr;     // DEVICE
-  uint32_t n_segs = 0;
-  uint64_t x_bytes = 0, y_bytes = 0;       // sizes of the operand arenas when bound with tq_stack_create_arena
+  // [0] all matrices; [1] those whose rows are short enough for the kernel that keeps a whole row of
+  // activation digits in shared memory; [2] the others (column-panel kernel)
+  tq_stack_plan plan[3];
 };
 
 // Phase 2 of the workspace GEMM (tq_gemm_ws.cu), declared here for tq_fused_gemm_ws.

@@ -1131,11 +1131,11 @@ int launch_panel(const TilesParams& p, uint32_t grid, cudaStream_t st) {
 }
 
 // One pass over nb batch columns (1..8) with the kernel that fits: p.one / p.mats describe the work.
-int launch_pass(TilesParams& p, int nb, bool narrow_two, bool sg, uint32_t grid, cudaStream_t st) {
+int launch_pass(TilesParams& p, int nb, bool narrow_two, bool sg, uint32_t grid, cudaStream_t st, bool wide = false) {
   // the narrow kernel keeps the digits of a whole row in shared memory; rows too long for that
   // (more than 8704 columns) take the wide kernel, which works in column panels, for any batch
   const TilesSmem L = tiles_smem(p.table_words, 3u * std::min(nb, 2) * p.xstride, kTilesWarps);
-  if (nb <= 2 && (nb == 1 || narrow_two) && L.total <= kSmemLimit) {
+  if (!wide && nb <= 2 && (nb == 1 || narrow_two) && L.total <= kSmemLimit) {
     if (nb == 1) return sg ? launch_tiles<1, true>(p, grid, L.total, st) : launch_tiles<1, false>(p, grid, L.total, st);
     return sg ? launch_tiles<2, true>(p, grid, L.total, st) : launch_tiles<2, false>(p, grid, L.total, st);
   }
@@ -1230,7 +1230,8 @@ struct PlanMat {
   const uint32_t* rb_raw;  // row_blocks + 1: index of each row block's first raw word
 };
 
-StackPlan plan_stack(const PlanMat* mats, int n, uint32_t grid) {
+// mats[0..n): the matrices to split; ids[i] is the index recorded in the segments for mats[i].
+StackPlan plan_stack(const PlanMat* mats, const uint32_t* ids, int n, uint32_t grid) {
   auto rb_cost = [&](const PlanMat& m, uint32_t rb) -> uint64_t {
     return (uint64_t)m.steps * 1024 + (uint64_t)(m.rb_raw[rb + 1] - m.rb_raw[rb]) * 4;
   };
@@ -1254,7 +1255,7 @@ StackPlan plan_stack(const PlanMat* mats, int n, uint32_t grid) {
       const uint32_t begin = rb;
       const bool last_cta = pl.cta_seg.size() >= grid;
       while (rb < m.row_blocks && (last_cta || acc < share)) acc += rb_cost(m, rb++);
-      pl.segs.push_back(TilesSeg{(uint32_t)i, begin, rb});
+      pl.segs.push_back(TilesSeg{ids[i], begin, rb});
       if (acc >= share && !last_cta) {
         pl.cta_seg.push_back((uint32_t)pl.segs.size());
         acc = 0;
@@ -1278,7 +1279,9 @@ int tq_stack_plan_host(int n_mats, const uint32_t* steps, const uint32_t* row_bl
     if (!rb_raw[i] || steps[i] == 0 || row_blocks[i] == 0) return TQ_ERR_INVALID_ARG;
     pm[i] = PlanMat{steps[i], row_blocks[i], rb_raw[i]};
   }
-  const StackPlan pl = plan_stack(pm.data(), n_mats, n_ctas);
+  std::vector<uint32_t> ids((size_t)n_mats);
+  for (int i = 0; i < n_mats; ++i) ids[i] = (uint32_t)i;
+  const StackPlan pl = plan_stack(pm.data(), ids.data(), n_mats, n_ctas);
   *n_segs = (uint32_t)pl.segs.size();
   if (pl.segs.size() > segs_cap) return TQ_ERR_BUFFER_TOO_SMALL;
   for (size_t i = 0; i < pl.segs.size(); ++i) {
@@ -1293,8 +1296,8 @@ int tq_stack_plan_host(int n_mats, const uint32_t* steps, const uint32_t* row_bl
 int tq_stack_size(int n_mats, uint64_t* device_bytes) {
   if (n_mats < 1 || !device_bytes) return TQ_ERR_INVALID_ARG;
   const uint64_t grid = (uint64_t)sm_count_tiles();
-  *device_bytes = align256((uint64_t)n_mats * sizeof(tq_tiles_desc)) + align256(((uint64_t)n_mats + grid) * sizeof(TilesSeg)) +
-                  align256((grid + 1) * 4);
+  *device_bytes = align256((uint64_t)n_mats * sizeof(tq_tiles_desc)) +
+                  3 * (align256(((uint64_t)n_mats + grid) * sizeof(TilesSeg)) + align256((grid + 1) * 4));
   return TQ_OK;
 }
 
@@ -1307,14 +1310,12 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   uint64_t need = 0;
   tq_stack_size(n_mats, &need);
   if (d_buf_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
-  uint32_t max_steps = 0;
   for (int i = 0; i < n_mats; ++i) {
     const tq_dmat* m = mats[i];
     if (!m || (bound && (!d_x[i] || !d_y[i] || ((uintptr_t)d_x[i] & 15)))) return TQ_ERR_INVALID_ARG;
     if (m->info.layout != TQ_LAYOUT_TILES || m->dict != mats[0]->dict ||
         m->info.levels_signed != mats[0]->info.levels_signed)
       return TQ_ERR_UNSUPPORTED_SHAPE;  // one table, one kind of level, TILES layout
-    max_steps = std::max(max_steps, m->tiles.steps);
   }
   tq_stack* s = new (std::nothrow) tq_stack();
   if (!s) return TQ_ERR_NOMEM;
@@ -1322,12 +1323,9 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   s->B = bound ? B : 0;
   s->levels_signed = mats[0]->info.levels_signed;
   s->grid = (uint32_t)sm_count_tiles();
-  s->xstride = max_steps * 32u + 4u;
   s->table_words = mats[0]->tiles.table_words;
   s->d_table = mats[0]->dict->d_table;
-  std::vector<PlanMat> pm((size_t)n_mats);
-  for (int i = 0; i < n_mats; ++i) pm[i] = PlanMat{mats[i]->tiles.steps, mats[i]->tiles.row_blocks, mats[i]->rb_raw.data()};
-  const StackPlan pl = plan_stack(pm.data(), n_mats, s->grid);
+
   std::vector<tq_tiles_desc> descs((size_t)n_mats);
   for (int i = 0; i < n_mats; ++i) {
     descs[i] = mats[i]->tiles;
@@ -1335,42 +1333,87 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
     descs[i].y = bound ? d_y[i] : nullptr;
   }
   uint8_t* base = static_cast<uint8_t*>(d_buf);
-  const uint64_t off_segs = align256((uint64_t)n_mats * sizeof(tq_tiles_desc));
-  const uint64_t off_cta = off_segs + align256(((uint64_t)n_mats + s->grid) * sizeof(TilesSeg));
+  const uint64_t segs_bytes = align256(((uint64_t)n_mats + s->grid) * sizeof(TilesSeg));
+  const uint64_t plan_bytes = segs_bytes + align256((s->grid + 1) * 4);
+  const uint64_t off_plans = align256((uint64_t)n_mats * sizeof(tq_tiles_desc));
   cudaStream_t st = (cudaStream_t)cuda_stream;
   int rc = tq_cuda_status((int)cudaMemcpyAsync(base, descs.data(), descs.size() * sizeof(tq_tiles_desc), cudaMemcpyHostToDevice, st), "stack upload");
-  if (rc == TQ_OK)
-    rc = tq_cuda_status((int)cudaMemcpyAsync(base + off_segs, pl.segs.data(), pl.segs.size() * sizeof(TilesSeg), cudaMemcpyHostToDevice, st), "stack upload");
-  if (rc == TQ_OK)
-    rc = tq_cuda_status((int)cudaMemcpyAsync(base + off_cta, pl.cta_seg.data(), pl.cta_seg.size() * 4, cudaMemcpyHostToDevice, st), "stack upload");
+  StackPlan pls[3];  // kept alive until the copies have been made
+  for (int k = 0; k < 3 && rc == TQ_OK; ++k) {
+    std::vector<PlanMat> pm;
+    std::vector<uint32_t> ids;
+    uint32_t max_steps = 0;
+    for (int i = 0; i < n_mats; ++i) {
+      const bool short_rows = tiles_smem(s->table_words, 3u * (mats[i]->tiles.steps * 32u + 4u), kTilesWarps).total <= kSmemLimit;
+      if (k == 0 || (k == 1) == short_rows) {
+        pm.push_back(PlanMat{mats[i]->tiles.steps, mats[i]->tiles.row_blocks, mats[i]->rb_raw.data()});
+        ids.push_back((uint32_t)i);
+        max_steps = std::max(max_steps, mats[i]->tiles.steps);
+      }
+    }
+    tq_stack_plan& sp = s->plan[k];
+    sp.n_mats = (uint32_t)pm.size();
+    sp.xstride = max_steps * 32u + 4u;
+    if (pm.empty()) continue;
+    pls[k] = plan_stack(pm.data(), ids.data(), (int)pm.size(), s->grid);
+    uint8_t* pb = base + off_plans + (uint64_t)k * plan_bytes;
+    rc = tq_cuda_status((int)cudaMemcpyAsync(pb, pls[k].segs.data(), pls[k].segs.size() * sizeof(TilesSeg), cudaMemcpyHostToDevice, st), "stack upload");
+    if (rc == TQ_OK)
+      rc = tq_cuda_status((int)cudaMemcpyAsync(pb + segs_bytes, pls[k].cta_seg.data(), pls[k].cta_seg.size() * 4, cudaMemcpyHostToDevice, st), "stack upload");
+    sp.d_segs = pb;
+    sp.d_cta_seg = reinterpret_cast<const uint32_t*>(pb + segs_bytes);
+    sp.n_segs = (uint32_t)pls[k].segs.size();
+  }
   if (rc == TQ_OK) rc = tq_cuda_status((int)cudaStreamSynchronize(st), "stack upload");
   if (rc != TQ_OK) {
     delete s;
     return rc;
   }
   s->d_descs = reinterpret_cast<const tq_tiles_desc*>(base);
-  s->d_segs = base + off_segs;
-  s->d_cta_seg = reinterpret_cast<const uint32_t*>(base + off_cta);
-  s->n_segs = (uint32_t)pl.segs.size();
   *out = s;
   return TQ_OK;
 }
 
+namespace {
+// The launches of one pass over nb batch columns of a stack: matrices with short rows through the
+// kernel that keeps a whole row of digits in shared memory (nb <= 2 where it fits), the others --
+// or all of them in a wide pass -- through the column-panel kernel.  launch == false only counts.
+int stack_pass(const tq_stack* s, int b0, int nb, bool two, bool launch, cudaStream_t st, int* n_launches) {
+  auto params = [&](const tq_stack_plan& sp) {
+    TilesParams p{};
+    p.mats = s->d_descs;
+    p.segs = static_cast<const TilesSeg*>(sp.d_segs);
+    p.cta_seg = sp.d_cta_seg;
+    p.table = s->d_table;
+    p.table_words = s->table_words;
+    p.xstride = sp.xstride;
+    p.b0 = (uint32_t)b0;
+    return p;
+  };
+  const bool sg = s->levels_signed != 0;
+  const bool narrow = nb == 1 || (nb == 2 && two);
+  for (int k = narrow ? 1 : 0; k < (narrow ? 3 : 1); ++k) {
+    if (s->plan[k].n_mats == 0) continue;
+    ++*n_launches;
+    if (!launch) continue;
+    TilesParams p = params(s->plan[k]);
+    if (int rc = launch_pass(p, nb, two, sg, s->grid, st, /*wide=*/k != 1)) return rc;
+  }
+  return TQ_OK;
+}
+// Two batch columns per narrow pass where the digits of two vectors fit for the short-row matrices.
+bool stack_two(const tq_stack* s) {
+  return s->plan[1].n_mats != 0 && tiles_smem(s->table_words, 6u * s->plan[1].xstride, kTilesWarps).total <= kSmemLimit;
+}
+}  // namespace
+
 int tq_fused_gemv_stack(const tq_stack* s, void* cuda_stream) {
   if (!s || s->B < 1) return TQ_ERR_INVALID_ARG;
-  cudaStream_t st = (cudaStream_t)cuda_stream;
-  TilesParams p{};
-  p.mats = s->d_descs;
-  p.segs = static_cast<const TilesSeg*>(s->d_segs);
-  p.cta_seg = s->d_cta_seg;
-  p.table = s->d_table;
-  p.table_words = s->table_words;
-  p.xstride = s->xstride;
-  const bool two = tiles_smem(s->table_words, 6u * s->xstride, kTilesWarps).total <= kSmemLimit;
+  const bool two = stack_two(s);
+  int n = 0;
   for (int b0 = 0; b0 < s->B;) {
     const int nb = next_pass(s->B - b0, two);
-    p.b0 = (uint32_t)b0;
-    if (int rc = launch_pass(p, nb, two, s->levels_signed != 0, s->grid, st)) return rc;
+    if (int rc = stack_pass(s, b0, nb, two, true, (cudaStream_t)cuda_stream, &n)) return rc;
     b0 += nb;
   }
   return TQ_OK;
@@ -1390,8 +1433,8 @@ int tq_decompress_stack(const tq_stack* s, uint8_t* const* d_out_ptrs, void* cud
   if (!s || !d_out_ptrs) return TQ_ERR_INVALID_ARG;
   DecompParams p{};
   p.mats = s->d_descs;
-  p.segs = static_cast<const TilesSeg*>(s->d_segs);
-  p.cta_seg = s->d_cta_seg;
+  p.segs = static_cast<const TilesSeg*>(s->plan[0].d_segs);
+  p.cta_seg = s->plan[0].d_cta_seg;
   p.outs = d_out_ptrs;
   p.table = s->d_table;
   p.table_words = s->table_words;
@@ -1402,8 +1445,8 @@ int tq_decode_bf16_stack(const tq_stack* s, void* const* d_workspace_ptrs, void*
   if (!s || !d_workspace_ptrs) return TQ_ERR_INVALID_ARG;
   DecompParams p{};
   p.mats = s->d_descs;
-  p.segs = static_cast<const TilesSeg*>(s->d_segs);
-  p.cta_seg = s->d_cta_seg;
+  p.segs = static_cast<const TilesSeg*>(s->plan[0].d_segs);
+  p.cta_seg = s->plan[0].d_cta_seg;
   p.outs = reinterpret_cast<uint8_t* const*>(d_workspace_ptrs);
   p.table = s->d_table;
   p.table_words = s->table_words;
@@ -1413,9 +1456,13 @@ int tq_decode_bf16_stack(const tq_stack* s, void* const* d_workspace_ptrs, void*
 
 int tq_stack_launches(const tq_stack* s) {
   if (!s) return TQ_ERR_INVALID_ARG;
-  const bool two = tiles_smem(s->table_words, 6u * s->xstride, kTilesWarps).total <= kSmemLimit;
+  const bool two = stack_two(s);
   int n = 0;
-  for (int b0 = 0; b0 < s->B; ++n) b0 += next_pass(s->B - b0, two);
+  for (int b0 = 0; b0 < s->B;) {
+    const int nb = next_pass(s->B - b0, two);
+    stack_pass(s, b0, nb, two, false, nullptr, &n);
+    b0 += nb;
+  }
   return n;
 }
 

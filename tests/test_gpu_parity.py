@@ -297,6 +297,31 @@ def test_stack_matches_oracle_and_single_calls(tq, B):
             assert tq.tq_device_status(m) == 0
 
 
+@pytest.mark.parametrize("B", [1, 2, 5])
+def test_stack_with_short_and_long_rows(tq, B):
+    """Rows too long for a whole row of activation digits in shared memory (more than 8704 columns)
+    take the column-panel kernel; a stack that mixes both kinds launches one kernel for each."""
+    shapes = [(200, 1024), (40, 12288), (600, 3072), (33, 28672), (64, 8192)]
+    rng = np.random.default_rng(200 + B)
+    qs = [np.clip(np.rint(rng.standard_t(5, size=s) * 4), -127, 127).astype(np.int8) for s in shapes]
+    ss = [(rng.random(r) + 0.5).astype(np.float32) for r, _ in shapes]
+    d, streams = _oracle_pack(qs, top_k=5000)
+    dd = tq.tq_dict_upload(tq.tq_dict_from_entries(d.entries))
+    mats = [tq.tq_upload(dd, st, r, c, s, layout=tq.TQ_LAYOUT_TILES) for st, (r, c), s in zip(streams, shapes, ss)]
+    xs = [synth.activations(B, c, 400 + i).cuda() for i, (_, c) in enumerate(shapes)]
+    ys = [torch.full((B, r), float("nan"), dtype=torch.float32, device="cuda") for r, _ in shapes]
+    stack = tq.tq_stack_create(mats, xs, ys)
+    # one column: the two kinds of rows take a kernel each; two columns do not fit beside the table for
+    # 8192-column rows, so they and wider batches go through the column-panel kernel in one launch
+    assert stack.launches == (2 if B == 1 else 1)
+    tq.tq_fused_gemv_stack(stack)
+    torch.cuda.synchronize()
+    for m, q, s, x, y in zip(mats, qs, ss, xs, ys):
+        assert torch.equal(tq.tq_fused_gemv(m, x), y)
+        assert _rel_err(y.cpu().numpy().astype(np.float64), oracle.layer_forward(q, s, x.cpu().double().numpy())) <= TOL
+        assert tq.tq_device_status(m) == 0
+
+
 def test_decompress_stack_bit_exact(tq):
     """One persistent launch decompresses every matrix of a stack (ragged shapes, a table larger
     than the shared-memory limit so that some groups are stored raw); a stack may be made without
