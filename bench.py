@@ -287,31 +287,45 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
             groups = [list(range(i, min(i + 7, len(mats)))) for i in range(0, len(mats), 7)]
             n_slots = max(len(g) for g in groups)
             slot_bytes = [max(tq.tq_gemm_workspace_size(mats[g[k]]) for g in groups if k < len(g)) for k in range(n_slots)]
-            wss = [torch.empty(b, dtype=torch.uint8, device=device) for b in slot_bytes]
+            wsets = [[torch.empty(b, dtype=torch.uint8, device=device) for b in slot_bytes] for _ in range(2)]
             gstacks = [tq.tq_stack_create([mats[i] for i in g]) for g in groups]
 
-            # the products of one group do not depend on one another (as q/k/v or gate/up of a decoder
-            # layer do not): they are spread over three streams so that a product whose tiles do not fill
-            # the SMs shares them with the next; each stream has its own output buffer
+            # Weights do not depend on activations, so the decode of group g + 1 (HBM-bound) runs on a
+            # stream of its own while the products of group g (tensor-bound) run: two workspace sets
+            # alternate.  The products of one group do not depend on one another either (as q/k/v or
+            # gate/up of a decoder layer do not): they are spread over three streams so that a product
+            # whose tiles do not fill the SMs shares them with the next; each stream has its own output
+            # buffer.
             lanes = [stream, torch.cuda.Stream(device), torch.cuda.Stream(device)]
+            dec_stream = torch.cuda.Stream(device)
             Ys = [Y] + [torch.empty_like(Y) for _ in lanes[1:]]
-            ev_dec = torch.cuda.Event()
-            ev_done = [torch.cuda.Event() for _ in lanes[1:]]
+            ev_dec = [torch.cuda.Event() for _ in groups]
+            ev_used = [torch.cuda.Event() for _ in groups]   # the products of a group have read its workspaces
+            ev_lane = [torch.cuda.Event() for _ in lanes[1:]]
+            ev_start, ev_end = torch.cuda.Event(), torch.cuda.Event()
 
             def run_gemm():
-                for g, st in zip(groups, gstacks):
-                    tq.tq_decode_bf16_stack(st, wss[: len(g)], stream=stream)
-                    ev_dec.record(stream)
-                    for ln in lanes[1:]:
-                        ln.wait_event(ev_dec)
+                ev_start.record(stream)
+                dec_stream.wait_event(ev_start)
+                for gi, (g, st) in enumerate(zip(groups, gstacks)):
+                    if gi >= 2:
+                        dec_stream.wait_event(ev_used[gi - 2])
+                    tq.tq_decode_bf16_stack(st, wsets[gi % 2][: len(g)], stream=dec_stream)
+                    ev_dec[gi].record(dec_stream)
+                for gi, g in enumerate(groups):
+                    for ln in lanes:
+                        ln.wait_event(ev_dec[gi])
                     for k, i in enumerate(g):
                         m = mats[i]
                         ln = k % len(lanes)
-                        tq.tq_gemm_bf16_ws(m, Xs[m.info.cols], wss[k], Ys[ln][: M * m.info.rows].view(M, m.info.rows),
+                        tq.tq_gemm_bf16_ws(m, Xs[m.info.cols], wsets[gi % 2][k], Ys[ln][: M * m.info.rows].view(M, m.info.rows),
                                            stream=lanes[ln])
-                    for ln, ev in zip(lanes[1:], ev_done):  # the next decode overwrites the workspaces
+                    for ln, ev in zip(lanes[1:], ev_lane):
                         ev.record(ln)
                         stream.wait_event(ev)
+                    ev_used[gi].record(stream)
+                ev_end.record(dec_stream)
+                stream.wait_event(ev_end)
         else:
             def run_gemm():
                 for m in mats:
