@@ -106,8 +106,9 @@ void tq_dict_free(tq_dict* d);
  * Device side: upload, decompress, fused products.
  * ---------------------------------------------------------------------------------------- */
 
-/* Bytes of DEVICE memory a table needs (always the full 16-bit index range, 256 KB: words past
- * the last entry are zero, so a kernel may index the table with any token). */
+/* Bytes of DEVICE memory a table needs: the full 16-bit index range (256 KB: words past the last
+ * entry are zero, so a kernel may index the table with any token) and a 2 MB map from 4-byte
+ * windows to codes for the device-side encoder. */
 int tq_dict_upload_size(const tq_dict* d, uint64_t* device_bytes);
 
 /* Copy the table into the caller's DEVICE buffer d_buf (256-byte aligned, d_buf_bytes long) and
@@ -166,6 +167,20 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
 int tq_tiles_image_host(const tq_dict* d, const uint16_t* stream, uint64_t stream_len, uint32_t rows,
                         uint32_t cols, const float* row_scale, const float* row_zero, uint8_t* out,
                         uint64_t out_cap, uint64_t* out_bytes, uint64_t* offsets, uint32_t* dims);
+
+/* tq_upload for 8-bit levels that are already on the device (for instance the output of
+ * tq_quantize_rows_device): Listing 3's decision for every aligned group (in the table: its code;
+ * else the marker and its 4 bytes) is taken on the GPU and written straight into the
+ * TQ_LAYOUT_TILES image, which is byte for byte the image tq_upload builds from the host stream.
+ * d_levels: DEVICE, rows x cols bytes, row-major, 16-byte aligned; d_row_scale / d_row_zero: DEVICE
+ * [rows] (zero may be NULL).  d_buf: DEVICE, 256-byte aligned, tq_upload_device_size bytes (sized
+ * for the worst case of no group in the table; tq_dmat_info.device_bytes reports what the image
+ * uses, the rest may be released by a caller who can shrink its buffer).  Requires cols % 4 == 0.
+ * The dictionary must have been uploaded with tq_dict_upload.  Synchronises cuda_stream. */
+int tq_upload_device_size(uint32_t rows, uint32_t cols, uint64_t* device_bytes);
+int tq_upload_device(const tq_ddict* dict, const uint8_t* d_levels, uint32_t rows, uint32_t cols,
+                     const float* d_row_scale, const float* d_row_zero, int levels_signed, void* d_buf,
+                     uint64_t d_buf_bytes, void* cuda_stream, tq_dmat** out);
 
 typedef struct tq_dmat_info {
   uint32_t rows, cols, K;

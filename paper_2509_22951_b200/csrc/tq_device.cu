@@ -557,7 +557,7 @@ int tq_dict_upload_size(const tq_dict* d, uint64_t* device_bytes) {
   if (!d || !device_bytes) return TQ_ERR_INVALID_ARG;
   // always the full 16-bit index range, zero past the last entry: any token is a safe index
   (void)d;
-  *device_bytes = 65536ull * 4 + 256;
+  *device_bytes = 65536ull * 4 + 256 + (uint64_t)kMapSlots * sizeof(tq_map_slot);  // table, then the window -> code map
   return TQ_OK;
 }
 
@@ -573,11 +573,17 @@ int tq_dict_upload(const tq_dict* d, void* d_buf, uint64_t d_buf_bytes, void* cu
                                          cudaMemcpyHostToDevice, st), "table upload"))
       return rc;
   }
+  std::vector<tq_map_slot> map(kMapSlots);
+  for (uint32_t i = 0; i < kMapSlots; ++i) map[i] = tq_map_slot{d->map_key[i], d->map_code[i]};
+  uint8_t* d_map = static_cast<uint8_t*>(d_buf) + 65536ull * 4 + 256;
+  if (int rc = cuda_ok(cudaMemcpyAsync(d_map, map.data(), map.size() * sizeof(tq_map_slot), cudaMemcpyHostToDevice, st), "table upload"))
+    return rc;
   if (int rc = cuda_ok(cudaStreamSynchronize(st), "table upload")) return rc;
   tq_ddict* dd = new (std::nothrow) tq_ddict();
   if (!dd) return TQ_ERR_NOMEM;
   dd->K = d->K;
   dd->d_table = static_cast<const uint32_t*>(d_buf);
+  dd->d_map = reinterpret_cast<const tq_map_slot*>(d_map);
   try {
     dd->h_table.assign((size_t)d->K + 1, 0u);
   } catch (const std::bad_alloc&) {
@@ -693,6 +699,81 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
   m->info.stream_bytes = 2 * (n_hits + 5 * n_miss);
   if (layout != TQ_LAYOUT_TILES) m->info.n_raw_words = n_miss;
   m->info.device_bytes = need;
+  *out = m;
+  return TQ_OK;
+}
+
+int tq_upload_device_size(uint32_t rows, uint32_t cols, uint64_t* device_bytes) {
+  if (!device_bytes || rows == 0 || cols == 0) return TQ_ERR_INVALID_ARG;
+  if (cols % 4 != 0 || cols > TQ_TILES_MAX_COLS) return TQ_ERR_UNSUPPORTED_SHAPE;
+  const tq_tiles_geometry geo = tq_tiles_layout(rows, cols);
+  if (geo.n_tiles >= (1ull << 31) || (uint64_t)rows * (cols / 4) >= (1ull << 32) - 65536) return TQ_ERR_UNSUPPORTED_SHAPE;
+  *device_bytes = geo.total((uint64_t)rows * (cols / 4));  // every group raw
+  return TQ_OK;
+}
+
+int tq_upload_device(const tq_ddict* dict, const uint8_t* d_levels, uint32_t rows, uint32_t cols,
+                     const float* d_row_scale, const float* d_row_zero, int levels_signed, void* d_buf,
+                     uint64_t d_buf_bytes, void* cuda_stream, tq_dmat** out) {
+  if (!dict || !d_levels || !d_row_scale || !d_buf || !out || ((uintptr_t)d_buf & 255) || ((uintptr_t)d_levels & 15))
+    return TQ_ERR_INVALID_ARG;
+  uint64_t need = 0;
+  if (int rc = tq_upload_device_size(rows, cols, &need)) return rc;
+  if (d_buf_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  uint8_t* base = static_cast<uint8_t*>(d_buf);
+  if (int rc = tq_tiles_build_device(dict, d_levels, rows, cols, d_row_scale, d_row_zero, base, cuda_stream)) return rc;
+  const tq_tiles_geometry geo = tq_tiles_layout(rows, cols);
+  tq_dmat* m = new (std::nothrow) tq_dmat();
+  if (!m) return TQ_ERR_NOMEM;
+  std::vector<uint32_t> tile_raw;
+  unsigned long long counters[2] = {0, 0};
+  int rc = TQ_OK;
+  try {
+    tile_raw.resize(geo.n_tiles + 1);
+  } catch (const std::bad_alloc&) {
+    rc = TQ_ERR_NOMEM;
+  }
+  if (rc == TQ_OK)
+    rc = cuda_ok(cudaMemcpyAsync(tile_raw.data(), base + geo.off_tile_raw, tile_raw.size() * 4, cudaMemcpyDeviceToHost, st), "device upload");
+  if (rc == TQ_OK) rc = cuda_ok(cudaMemcpyAsync(counters, base + 64, sizeof(counters), cudaMemcpyDeviceToHost, st), "device upload");
+  if (rc == TQ_OK) rc = cuda_ok(cudaStreamSynchronize(st), "device upload");
+  if (rc != TQ_OK) {
+    delete m;
+    return rc;
+  }
+  const uint64_t n_raw = tile_raw[geo.n_tiles];
+  m->rb_raw.resize((size_t)geo.row_blocks + 1);
+  for (uint32_t rb = 0; rb <= geo.row_blocks; ++rb) m->rb_raw[rb] = tile_raw[(uint64_t)rb * geo.steps];
+  m->dict = dict;
+  m->has_zero = d_row_zero != nullptr;
+  m->d_status = reinterpret_cast<uint32_t*>(base + geo.off_status);
+  m->d_scale = reinterpret_cast<const float*>(base + geo.off_scale);
+  m->d_zero = reinterpret_cast<const float*>(base + geo.off_zero);
+  tq_tiles_desc& t = m->tiles;
+  t.tokens = reinterpret_cast<const uint4*>(base + geo.off_tokens);
+  t.raw = reinterpret_cast<const uint32_t*>(base + geo.off_raw);
+  t.tile_raw = reinterpret_cast<const uint32_t*>(base + geo.off_tile_raw);
+  t.scale = m->d_scale;
+  t.zero = m->d_zero;
+  t.status = m->d_status;
+  t.rows = rows;
+  t.cols = cols;
+  t.steps = geo.steps;
+  t.row_blocks = geo.row_blocks;
+  t.has_zero = d_row_zero != nullptr;
+  t.table_words = TQ_TILES_TABLE_WORDS;
+  m->info.rows = rows;
+  m->info.cols = cols;
+  m->info.K = dict->K;
+  m->info.layout = TQ_LAYOUT_TILES;
+  m->info.levels_signed = levels_signed != 0;
+  m->info.n_hits = counters[0];
+  m->info.n_miss = counters[1];
+  m->info.stream_bytes = 2 * (counters[0] + 5 * counters[1]);
+  m->info.n_raw_words = n_raw;
+  m->info.payload_bytes = geo.n_tiles * 1024 + n_raw * 4 + (geo.n_tiles + 1) * 4 + (uint64_t)rows * (4 + (d_row_zero ? 4 : 0));
+  m->info.device_bytes = geo.total(n_raw);
   *out = m;
   return TQ_OK;
 }

@@ -772,14 +772,10 @@ int tq_build_tiles_image(const uint16_t* stream, uint64_t stream_len, uint32_t r
     tile_raw_v[i + 1] = (uint32_t)n_raw;
   }
 
-  const uint64_t off_status = 0;
-  const uint64_t off_scale = 256;
-  const uint64_t off_zero = align_up(off_scale + rows_pad * 4, 256);
-  const uint64_t off_tile_raw = align_up(off_zero + rows_pad * 4, 256);
-  const uint64_t off_tokens = align_up(off_tile_raw + (n_tiles + 1 + 8) * 4, 1024);
-  // 8 KB of token padding and 16 KB of raw padding: prefetches past the last tile stay inside the buffer
-  const uint64_t off_raw = align_up(off_tokens + n_tiles * 1024 + 8192, 1024);
-  const uint64_t total = align_up(off_raw + n_raw * 4 + 16384, 256);
+  const tq_tiles_geometry geo = tq_tiles_layout(rows, cols);
+  const uint64_t off_status = geo.off_status, off_scale = geo.off_scale, off_zero = geo.off_zero;
+  const uint64_t off_tile_raw = geo.off_tile_raw, off_tokens = geo.off_tokens, off_raw = geo.off_raw;
+  const uint64_t total = geo.total(n_raw);
   if (device_bytes) *device_bytes = total;
   if (!img) return TQ_OK;
   if (!row_scale || !table) return TQ_ERR_INVALID_ARG;

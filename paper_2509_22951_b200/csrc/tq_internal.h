@@ -20,8 +20,17 @@ struct tq_dict {
   uint64_t n_windows = 0, n_distinct = 0;
 };
 
+// Slot of the device-side lookup from a 4-byte window to its code (open addressing, 2^18 slots,
+// slot = (key * 0x9E3779B1) >> 14, linear probing, code 0 = empty): the host table's own map.
+struct tq_map_slot {
+  uint32_t key;
+  uint32_t code;
+};
+constexpr uint32_t kMapSlots = 1u << 18;
+
 struct tq_ddict {
   uint32_t K = 0;
+  const tq_map_slot* d_map = nullptr;  // DEVICE: kMapSlots slots
   // DEVICE: K + 1 words indexed by code; word 0 is zero (token 0 = padding), word c holds entry
   // c - 1 with byte i of the window in bits 8i..8i+7
   const uint32_t* d_table = nullptr;
@@ -88,6 +97,31 @@ struct tq_planes_image {
   uint64_t n_hits = 0, n_miss = 0;
 };
 
+// Where the parts of a TQ_LAYOUT_TILES image lie (byte offsets from its 256-byte aligned start).
+// One definition for the host builder and the device builder, whose images must be identical.
+struct tq_tiles_geometry {
+  uint32_t steps, row_blocks;
+  uint64_t n_tiles, rows_pad;
+  uint64_t off_status, off_scale, off_zero, off_tile_raw, off_tokens, off_raw;
+  uint64_t total(uint64_t n_raw) const { return (off_raw + n_raw * 4 + 16384 + 255) / 256 * 256; }
+};
+inline tq_tiles_geometry tq_tiles_layout(uint32_t rows, uint32_t cols) {
+  auto up = [](uint64_t v, uint64_t a) { return (v + a - 1) / a * a; };
+  tq_tiles_geometry g{};
+  g.steps = (cols / 4 + 31u) / 32u;
+  g.row_blocks = (rows + 15u) / 16u;
+  g.n_tiles = (uint64_t)g.steps * g.row_blocks;
+  g.rows_pad = (uint64_t)g.row_blocks * 16;
+  g.off_status = 0;  // status word; bytes 64.. of this 256-byte header are scratch counters of the device builder
+  g.off_scale = 256;
+  g.off_zero = up(g.off_scale + g.rows_pad * 4, 256);
+  g.off_tile_raw = up(g.off_zero + g.rows_pad * 4, 256);
+  g.off_tokens = up(g.off_tile_raw + (g.n_tiles + 1 + 8) * 4, 1024);  // 8 entries read ahead by the kernels
+  // 8 KB of token padding and 16 KB of raw padding: prefetches past the last tile stay inside the buffer
+  g.off_raw = up(g.off_tokens + g.n_tiles * 1024 + 8192, 1024);
+  return g;
+}
+
 struct tq_tiles_image {
   std::vector<uint8_t> blob;
   uint64_t off_status = 0, off_scale = 0, off_zero = 0, off_tile_raw = 0, off_tokens = 0, off_raw = 0;
@@ -146,3 +180,7 @@ struct tq_stack {
 // Phase 2 of the workspace GEMM (tq_gemm_ws.cu), declared here for tq_fused_gemm_ws.
 extern "C" int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, const void* d_workspace,
                                void* cuda_stream);
+
+// Device-side builder of the TILES image (tq_encode.cu).
+int tq_tiles_build_device(const tq_ddict* dict, const uint8_t* d_levels, uint32_t rows, uint32_t cols,
+                          const float* d_row_scale, const float* d_row_zero, uint8_t* d_image, void* cuda_stream);

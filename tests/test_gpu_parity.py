@@ -267,6 +267,38 @@ def test_fused_gemm_ws_agrees_with_fused_gemv(tq):
     assert float((a - b).abs().max() / b.abs().max()) < 1e-5
 
 
+# ------------------------------------------------------------------ device-side encoder
+@pytest.mark.parametrize("rows,cols,spread,top_k", [(37, 516, 3, 300), (300, 3072, 6, 65535), (17, 8192, 4, 65535), (5, 4, 2, 10),
+                                                    (64, 2048, 20, 65535), (48, 1280, 3, 0)])
+def test_upload_device_builds_the_same_image_as_the_host(tq, rows, cols, spread, top_k):
+    """tq_upload_device (levels on the GPU -> TILES image on the GPU) against tq_tiles_image_host
+    fed with the oracle's stream: tokens, tile index, raw words, scales and zero points byte for
+    byte; then the same y from both matrices."""
+    rng = np.random.default_rng(rows + cols)
+    q = np.clip(np.rint(rng.standard_t(5, size=(rows, cols)) * spread), -127, 127).astype(np.int8)
+    s = (rng.random(rows) + 0.5).astype(np.float32)
+    z = rng.integers(0, 5, rows).astype(np.float32)
+    d, (stream,) = _oracle_pack([q], top_k=top_k)
+    hd = tq.tq_dict_from_entries(d.entries)
+    dd = tq.tq_dict_upload(hd)
+    img, offs, steps, row_blocks = tq.tq_tiles_image_host(hd, stream, rows, cols, s, z)
+    md = tq.tq_upload_device(dd, torch.from_numpy(q).cuda(), torch.from_numpy(s).cuda(), torch.from_numpy(z).cuda())
+    got = md.buf.cpu().numpy()
+    n_tiles = steps * row_blocks
+    n_raw = int(img[offs["tile_raw"]:].view(np.uint32)[n_tiles])
+    assert md.info.n_raw_words == n_raw and md.info.device_bytes == img.size
+    assert md.info.n_hits + md.info.n_miss == rows * cols // 4 and md.info.stream_bytes == stream.nbytes
+    for name, length in (("scale", 4 * row_blocks * 16), ("zero", 4 * row_blocks * 16), ("tile_raw", 4 * (n_tiles + 9)),
+                         ("tokens", 1024 * n_tiles), ("raw", 4 * n_raw)):
+        a, b = offs[name], offs[name] + length
+        assert np.array_equal(got[a:b], img[a:b]), name
+    mh = tq.tq_upload(dd, stream, rows, cols, s, z, layout=tq.TQ_LAYOUT_TILES)
+    x = synth.activations(3, cols, 77).cuda()
+    assert torch.equal(tq.tq_fused_gemv(md, x), tq.tq_fused_gemv(mh, x))
+    assert np.array_equal(tq.tq_decompress(md).cpu().numpy(), q.view(np.uint8))
+    assert tq.tq_device_status(md) == 0
+
+
 # ------------------------------------------------------------------ stack: one persistent launch
 @pytest.mark.parametrize("B", [1, 2, 3, 8, 11])
 def test_stack_matches_oracle_and_single_calls(tq, B):
