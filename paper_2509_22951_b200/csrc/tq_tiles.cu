@@ -535,8 +535,14 @@ template <int W, int NB, bool SIGNED>
 __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams p) {
   extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
   TilesCta<W, NB, SIGNED> cta;
+  // launched with programmatic stream serialisation: the next kernel of the stream may start its own
+  // set-up while this one runs, and this one has come this far (barriers, table copy under way)
+  // while its predecessor was still running.  Nothing above reads or writes what a predecessor
+  // produces (the table and the weights are constant); the activations are first read below.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   cta.setup(tiles_smem_raw, tiles_smem(p.table_words, 3u * NB * p.xstride, W), W, p.table, p.table_words);
   cta.xstride = p.xstride;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (p.mats == nullptr) {
     const uint32_t nrb = p.one.row_blocks;
@@ -844,8 +850,10 @@ template <int W, int NB, bool SIGNED>
 __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_panel_kernel(const TilesParams p) {
   extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
   PanelCta<W, NB, SIGNED> cta;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // see gemv_tiles_kernel
   cta.setup(tiles_smem_raw, tiles_smem(p.table_words, 2u * PanelCta<W, NB, SIGNED>::kBufWords, W), W, p.table, p.table_words);
   cta.nb_valid = p.nb_valid;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (p.mats == nullptr) {
     const uint32_t nrb = p.one.row_blocks;
@@ -1100,6 +1108,22 @@ int launch_decomp(const DecompParams& p, uint32_t grid, cudaStream_t st) {
   return tq_cuda_status((int)cudaGetLastError(), "decompress(tiles) launch");
 }
 
+// Launch with programmatic stream serialisation (see gemv_tiles_kernel).
+template <class Kern>
+int launch_pdl(Kern kern, uint32_t grid, uint32_t threads, size_t smem, cudaStream_t st, const TilesParams& p) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return tq_cuda_status((int)cudaLaunchKernelEx(&cfg, kern, p), "gemv(tiles) launch");
+}
+
 template <int NB, bool SIGNED>
 int launch_tiles(const TilesParams& p, uint32_t grid, size_t smem, cudaStream_t st) {
   auto kern = gemv_tiles_kernel<kTilesWarps, NB, SIGNED>;
@@ -1110,8 +1134,7 @@ int launch_tiles(const TilesParams& p, uint32_t grid, size_t smem, cudaStream_t 
       return rc;
     configured = smem;
   }
-  kern<<<grid, kTilesWarps * 32, smem, st>>>(p);
-  return tq_cuda_status((int)cudaGetLastError(), "gemv(tiles) launch");
+  return launch_pdl(kern, grid, kTilesWarps * 32, smem, st, p);
 }
 
 template <int NB, bool SIGNED>
@@ -1126,8 +1149,7 @@ int launch_panel(const TilesParams& p, uint32_t grid, cudaStream_t st) {
       return rc;
     configured = smem;
   }
-  kern<<<grid, kTilesWarps * 32, smem, st>>>(p);
-  return tq_cuda_status((int)cudaGetLastError(), "gemv(tiles, wide) launch");
+  return launch_pdl(kern, grid, kTilesWarps * 32, smem, st, p);
 }
 
 // One pass over nb batch columns (1..8) with the kernel that fits: p.one / p.mats describe the work.
