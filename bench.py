@@ -119,6 +119,8 @@ def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout
     if threads:
         tq.tq_set_num_threads(threads)
     q_host, scales, zeros = [], [], []
+    q_dev, s_dev = [], []  # levels and scales kept on the device for the device-side encoder (tiles layout)
+    on_device = layout == 2 and quantizer == "rows"
     for i, (name, rows, cols) in enumerate(shapes):
         w = synth.weight(rows, cols, synth.matrix_seed(i), device=device)
         if quantizer == "paper":
@@ -131,6 +133,9 @@ def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout
             q_host.append(q.cpu().numpy())
             scales.append(s.cpu().numpy())
             zeros.append(None)
+            if on_device:
+                q_dev.append(q)
+                s_dev.append(s)
         del w, q, s
     t1 = time.time()
     hd = tq.tq_build_dictionary(q_host) if table_entries is None else tq.tq_dict_from_entries(table_entries)
@@ -138,6 +143,10 @@ def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout
     dd = tq.tq_dict_upload(hd, device=device)
     mats = []
     for i, (name, rows, cols) in enumerate(shapes):
+        if on_device:  # Listing 3 and the tiling on the GPU, no host stream
+            mats.append(tq.tq_upload_device(dd, q_dev[i], s_dev[i]))
+            q_dev[i] = s_dev[i] = None
+            continue
         stream, h, m = tq.tq_encode(hd, q_host[i])
         mats.append(tq.tq_upload(dd, stream, rows, cols, scales[i], zeros[i], levels_signed=(quantizer != "paper"),
                                  layout=layout))
