@@ -138,7 +138,12 @@ def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout
                 s_dev.append(s)
         del w, q, s
     t1 = time.time()
-    hd = tq.tq_build_dictionary(q_host) if table_entries is None else tq.tq_dict_from_entries(table_entries)
+    if table_entries is not None:
+        hd = tq.tq_dict_from_entries(table_entries)
+    elif on_device:  # windows counted on the GPU, candidates ranked on the host: the same table
+        hd = tq.tq_build_dictionary_device([q.view(-1) for q in q_dev])
+    else:
+        hd = tq.tq_build_dictionary(q_host)
     t2 = time.time()
     dd = tq.tq_dict_upload(hd, device=device)
     mats = []

@@ -83,6 +83,20 @@ int tq_quantize_rows_device(const float* d_w, uint32_t rows, uint32_t cols, int8
 int tq_build_dictionary(const uint8_t* const* mats, const uint64_t* n_elems, int n_mats,
                         uint32_t top_k, tq_dict** out);
 
+/* tq_build_dictionary for matrices that are on the DEVICE (d_mats: HOST array of n_mats DEVICE
+ * pointers, 4-byte aligned): the windows are counted on the GPU (keys, radix sort and run lengths
+ * per matrix, a hash table over all matrices) and only the candidates for the table (count at
+ * least that of rank top_k, every tie included) come back to the host, where they are ranked by
+ * the same rule -- the result is the table tq_build_dictionary builds.  d_workspace: DEVICE,
+ * 256-byte aligned, tq_build_dictionary_device_size bytes (about 28 bytes per byte of the largest
+ * matrix plus up to 2.6 GB).  TQ_ERR_BUFFER_TOO_SMALL if the data has more distinct windows than
+ * the hash table holds (2^28 at most), TQ_ERR_UNSUPPORTED_SHAPE if more than 2^24 windows tie at
+ * the cut: use tq_build_dictionary then.  Synchronises cuda_stream. */
+int tq_build_dictionary_device_size(const uint64_t* n_elems, int n_mats, uint64_t* workspace_bytes);
+int tq_build_dictionary_device(const uint8_t* const* d_mats, const uint64_t* n_elems, int n_mats,
+                               uint32_t top_k, void* d_workspace, uint64_t workspace_bytes,
+                               void* cuda_stream, tq_dict** out);
+
 /* A table from an explicit entry list (K x 4 bytes, rank order, HOST). */
 int tq_dict_from_entries(const uint8_t* entries, uint32_t K, tq_dict** out);
 

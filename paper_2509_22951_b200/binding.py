@@ -33,7 +33,7 @@ TQ_STATUS_WAIT_EXPIRED = 4
 
 EXPORTS = [
     "tq_strerror", "tq_last_cuda_error", "tq_set_num_threads", "tq_quantize_tensor", "tq_quantize_rows",
-    "tq_quantize_rows_device", "tq_build_dictionary", "tq_dict_from_entries", "tq_dict_entries",
+    "tq_quantize_rows_device", "tq_build_dictionary", "tq_build_dictionary_device_size", "tq_build_dictionary_device", "tq_dict_from_entries", "tq_dict_entries",
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_upload_device_size", "tq_upload_device", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
     "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_gemm_workspace_size",
@@ -70,6 +70,8 @@ def _load() -> C.CDLL:
         "tq_quantize_rows": (C.c_int, [f32p, C.c_uint32, C.c_uint32, C.POINTER(C.c_int8), f32p]),
         "tq_quantize_rows_device": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, vp, vp]),
         "tq_build_dictionary": (C.c_int, [C.POINTER(u8p), u64p, C.c_int, C.c_uint32, C.POINTER(vp)]),
+        "tq_build_dictionary_device_size": (C.c_int, [u64p, C.c_int, u64p]),
+        "tq_build_dictionary_device": (C.c_int, [C.POINTER(vp), u64p, C.c_int, C.c_uint32, vp, C.c_uint64, vp, C.POINTER(vp)]),
         "tq_dict_from_entries": (C.c_int, [u8p, C.c_uint32, C.POINTER(vp)]),
         "tq_dict_entries": (C.c_int, [vp, u32p, C.POINTER(u8p), C.POINTER(u64p)]),
         "tq_encode": (C.c_int, [vp, u8p, C.c_uint64, u16p, C.c_uint64, u64p, u64p, u64p]),
@@ -203,6 +205,24 @@ def tq_build_dictionary(mats, top_k: int = 2 ** 16 - 1) -> Dict:
     lens = (C.c_uint64 * max(n, 1))(*[a.size for a in arrs])
     out = C.c_void_p()
     _check(_lib.tq_build_dictionary(ptrs, lens, n, top_k, C.byref(out)), "tq_build_dictionary")
+    return Dict(out.value)
+
+
+def tq_build_dictionary_device(mats, top_k: int = 2 ** 16 - 1, stream=None) -> Dict:
+    """mats: CUDA 1-byte tensors (levels).  Counts the windows on the GPU; same table as tq_build_dictionary."""
+    n = len(mats)
+    assert n >= 1
+    for m in mats:
+        assert m.is_cuda and m.is_contiguous() and m.element_size() == 1
+    lens = (C.c_uint64 * n)(*[m.numel() for m in mats])
+    need = C.c_uint64()
+    _check(_lib.tq_build_dictionary_device_size(lens, n, C.byref(need)), "tq_build_dictionary_device_size")
+    ws = torch.empty(need.value, dtype=torch.uint8, device=mats[0].device)
+    ptrs = (C.c_void_p * n)(*[m.data_ptr() for m in mats])
+    out = C.c_void_p()
+    with torch.cuda.device(ws.device):
+        _check(_lib.tq_build_dictionary_device(ptrs, lens, n, top_k, ws.data_ptr(), ws.numel(), _stream_ptr(stream),
+                                               C.byref(out)), "tq_build_dictionary_device")
     return Dict(out.value)
 
 

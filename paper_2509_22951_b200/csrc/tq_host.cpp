@@ -129,6 +129,33 @@ int tq_num_threads() {
   return n;
 }
 
+// A table from windows already ranked (keys little endian: byte i of the window in bits 8i..8i+7).
+int tq_dict_from_ranked(const uint32_t* keys, const uint64_t* counts, uint32_t K, uint64_t n_windows,
+                        uint64_t n_distinct, tq_dict** out) {
+  if (!out || (K && (!keys || !counts)) || K > TQ_MAX_ENTRIES) return TQ_ERR_INVALID_ARG;
+  tq_dict* d = new (std::nothrow) tq_dict();
+  if (!d) return TQ_ERR_NOMEM;
+  try {
+    d->K = K;
+    d->n_windows = n_windows;
+    d->n_distinct = n_distinct;
+    d->entries.resize(4 * (size_t)K);
+    d->counts.assign(counts, counts + K);
+    for (uint32_t r = 0; r < K; ++r) {
+      d->entries[4 * (size_t)r + 0] = (uint8_t)keys[r];
+      d->entries[4 * (size_t)r + 1] = (uint8_t)(keys[r] >> 8);
+      d->entries[4 * (size_t)r + 2] = (uint8_t)(keys[r] >> 16);
+      d->entries[4 * (size_t)r + 3] = (uint8_t)(keys[r] >> 24);
+    }
+    finish_dict(d);
+  } catch (const std::bad_alloc&) {
+    delete d;
+    return TQ_ERR_NOMEM;
+  }
+  *out = d;
+  return TQ_OK;
+}
+
 extern "C" {
 
 const char* tq_strerror(int s) {

@@ -184,3 +184,7 @@ extern "C" int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, fl
 // Device-side builder of the TILES image (tq_encode.cu).
 int tq_tiles_build_device(const tq_ddict* dict, const uint8_t* d_levels, uint32_t rows, uint32_t cols,
                           const float* d_row_scale, const float* d_row_zero, uint8_t* d_image, void* cuda_stream);
+
+// A host table from windows that are already ranked (tq_host.cpp; used by the device-side builder).
+int tq_dict_from_ranked(const uint32_t* keys, const uint64_t* counts, uint32_t K, uint64_t n_windows,
+                        uint64_t n_distinct, tq_dict** out);

@@ -267,6 +267,39 @@ def test_fused_gemm_ws_agrees_with_fused_gemv(tq):
     assert float((a - b).abs().max() / b.abs().max()) < 1e-5
 
 
+# ------------------------------------------------------------------ device-side table build
+@pytest.mark.parametrize("case", ["ties", "several", "minus_one", "odd_lengths", "top_k_small", "large"])
+def test_build_dictionary_device_matches_oracle(tq, case):
+    """Listing 2 with the counting on the GPU: entries (rank order: count descending, then first
+    occurrence) and counts must equal the oracle's and the host builder's, ties included."""
+    rng = np.random.default_rng(sum(map(ord, case)))
+    top_k = 65535
+    if case == "ties":  # few distinct values: many windows share a count
+        mats = [rng.integers(-1, 2, size=(40, 64)).astype(np.int8)]
+    elif case == "several":  # windows must not span two matrices
+        mats = [rng.integers(-3, 4, size=s).astype(np.int8) for s in [(16, 32), (7, 12), (64, 128)]]
+    elif case == "minus_one":  # the window 0xFFFFFFFF (four levels of -1) is an ordinary window
+        a = rng.integers(-2, 1, size=(32, 256)).astype(np.int8)
+        a[:, 64:192] = -1
+        mats = [a]
+    elif case == "odd_lengths":  # lengths that are no multiple of 4, and matrices too short for one window
+        mats = [rng.integers(-2, 3, size=n).astype(np.int8) for n in (1001, 3, 4, 4099, 2)]
+    elif case == "top_k_small":
+        mats = [rng.integers(-4, 5, size=(128, 256)).astype(np.int8)]
+        top_k = 37
+    else:  # more distinct windows than table entries, realistic levels
+        mats = [np.clip(np.rint(rng.standard_t(5, size=(1024, 1024)) * 6), -127, 127).astype(np.int8),
+                np.clip(np.rint(rng.standard_t(5, size=(512, 2048)) * 9), -127, 127).astype(np.int8)]
+    od = oracle.Dictionary.build(mats, top_k=top_k)
+    hd = tq.tq_build_dictionary(mats, top_k=top_k)
+    dev = [torch.from_numpy(np.ascontiguousarray(m).reshape(-1).view(np.uint8).copy()).cuda() for m in mats]
+    # 4-byte alignment of every matrix is the call's requirement; torch allocations satisfy it
+    gd = tq.tq_build_dictionary_device(dev, top_k=top_k)
+    assert gd.K == od.K == hd.K
+    assert np.array_equal(gd.entries, od.entries) and np.array_equal(gd.entries, hd.entries)
+    assert np.array_equal(gd.counts, hd.counts)
+
+
 # ------------------------------------------------------------------ device-side encoder
 @pytest.mark.parametrize("rows,cols,spread,top_k", [(37, 516, 3, 300), (300, 3072, 6, 65535), (17, 8192, 4, 65535), (5, 4, 2, 10),
                                                     (64, 2048, 20, 65535), (48, 1280, 3, 0)])
@@ -454,6 +487,8 @@ def test_full_3b_stack_as_benchmarked_on_sampled_rows(tq):
         err = np.max(np.abs(y - yref), axis=1) / np.max(np.abs(yref), axis=1)
         assert float(err.max()) <= TOL, (name, err)
         assert tq.tq_device_status(mats[i]) == 0
+    # the table was built with the counting on the GPU: it must be the host builder's table
+    assert np.array_equal(hd.entries, tq.tq_build_dictionary(q_host).entries)
     # decoded levels of two matrices, whole, against the levels that were encoded
     for i in (6, 196):
         got = tq.tq_decompress(mats[i])
