@@ -30,15 +30,17 @@
 #include <vector>
 
 #include "tq_internal.h"
+#include "tq_sm100.cuh"
 
 namespace {
+
+using namespace tq_sm100;
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kRingWords = TQ_TILES_RING_WORDS;     // 4 KB per warp
 constexpr int kChunkWords = 256;                    // one bulk copy: 1 KB of raw words
 constexpr int kSlots = kRingWords / kChunkWords;    // chunks per ring
 constexpr int kL2Ahead = 8;                         // token tiles prefetched into L2 ahead of their use (<= 8: padding)
-constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr uint32_t kNoBlock = 0xFFFFFFFFu;
 constexpr uint32_t kMissBase = 0x10000u - TQ_TILES_RING_WORDS;  // first miss token
 static_assert(kSlots == 4 && (kRingWords & (kRingWords - 1)) == 0, "ring geometry");
@@ -75,8 +77,6 @@ struct TilesParams {
   uint32_t nb_valid;          // wide passes: vectors present (<= the kernel's NB)
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
 __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
   uint4 v;
   asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -90,37 +90,11 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
   return v;
 }
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-
 // The table into shared memory with bulk copies (one thread issues them; nothing waits until the
 // first lookup, so the activation set-up and the first loads of the streams overlap the copy).
 constexpr uint32_t kTableBarOffset = 400u;  // inside the misc area of the shared-memory plan
@@ -919,12 +893,6 @@ decompress_tiles_kernel(const tq_tiles_desc d, const uint32_t* __restrict__ tabl
   if (bad) atomicOr(d.status, TQ_STATUS_BAD_CODE);
 }
 
-int sm_count_tiles() {
-  int dev = 0, n = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  return n;
-}
 
 constexpr int kTilesWarps = 16;
 constexpr uint32_t kSmemLimit = 232448u;  // 227 KB per CTA
@@ -1192,7 +1160,7 @@ int tq_tiles_gemv(const tq_dmat* m, const void* x, int B, float* y, void* cuda_s
   p.table_words = m->tiles.table_words;
   p.xstride = m->tiles.steps * 32u + 4u;
   const bool narrow_two = tq_tiles_max_nb(m) >= 2;
-  const uint32_t grid = std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count_tiles());
+  const uint32_t grid = std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count());
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const bool sg = m->info.levels_signed != 0;
   for (int b0 = 0; b0 < B;) {
@@ -1208,15 +1176,15 @@ int tq_tiles_gemv(const tq_dmat* m, const void* x, int B, float* y, void* cuda_s
 int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
   const uint32_t n_tiles = m->tiles.steps * m->tiles.row_blocks;
   // loading the table into every SM's shared memory pays off from a few thousand tiles per SM on
-  if ((uint64_t)n_tiles >= 64ull * (uint64_t)sm_count_tiles()) {
+  if ((uint64_t)n_tiles >= 64ull * (uint64_t)sm_count()) {
     DecompParams p{};
     p.one = m->tiles;
     p.out_one = d_codes;
     p.table = m->dict->d_table;
     p.table_words = m->tiles.table_words;
-    return launch_decomp<false>(p, std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count_tiles()), (cudaStream_t)cuda_stream);
+    return launch_decomp<false>(p, std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count()), (cudaStream_t)cuda_stream);
   }
-  const uint32_t grid = std::min<uint32_t>((n_tiles + 7u) / 8u, (uint32_t)sm_count_tiles() * 8u);
+  const uint32_t grid = std::min<uint32_t>((n_tiles + 7u) / 8u, (uint32_t)sm_count() * 8u);
   decompress_tiles_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(m->tiles, m->dict->d_table,
                                                                        reinterpret_cast<uint32_t*>(d_codes));
   return tq_cuda_status((int)cudaGetLastError(), "decompress(tiles) launch");
@@ -1230,7 +1198,7 @@ int tq_tiles_decode_bf16(const tq_dmat* m, void* d_out, void* cuda_stream) {
   p.table = m->dict->d_table;
   p.table_words = m->tiles.table_words;
   p.levels_signed = m->info.levels_signed != 0;
-  return launch_decomp<true>(p, std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count_tiles()), (cudaStream_t)cuda_stream);
+  return launch_decomp<true>(p, std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count()), (cudaStream_t)cuda_stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1317,7 +1285,7 @@ int tq_stack_plan_host(int n_mats, const uint32_t* steps, const uint32_t* row_bl
 
 int tq_stack_size(int n_mats, uint64_t* device_bytes) {
   if (n_mats < 1 || !device_bytes) return TQ_ERR_INVALID_ARG;
-  const uint64_t grid = (uint64_t)sm_count_tiles();
+  const uint64_t grid = (uint64_t)sm_count();
   *device_bytes = align256((uint64_t)n_mats * sizeof(tq_tiles_desc)) +
                   3 * (align256(((uint64_t)n_mats + grid) * sizeof(TilesSeg)) + align256((grid + 1) * 4));
   return TQ_OK;
@@ -1344,7 +1312,7 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   s->n = n_mats;
   s->B = bound ? B : 0;
   s->levels_signed = mats[0]->info.levels_signed;
-  s->grid = (uint32_t)sm_count_tiles();
+  s->grid = (uint32_t)sm_count();
   s->table_words = mats[0]->tiles.table_words;
   s->d_table = mats[0]->dict->d_table;
 
