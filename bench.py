@@ -107,6 +107,11 @@ class ClockSampler:
 # summarised under profiles/ (None: not captured for that launch shape, or kernel changed since).
 # tiles_stack: 213.2 MB read + 4.2 MB written for 207.7 MB of algorithmic bytes on a 14-matrix stack (2 decoder
 # layers), i.e. 1.047 x; traffic grows with the bytes streamed, so the 3B launch (3.333 GB) is scaled by that ratio.
+# the arithmetic each layout's product kernel computes in
+DTYPE = {"tiles": "s8 x s8 -> s32 (int8 levels x three base-256 digits of block-fixed-point bf16 activations, "
+                  "exact integer tensor-core sums, fp64 epilogue)",
+         "planes": "int8 weights x bf16 activations, fp32 accumulate",
+         "stream": "int8 weights x bf16 activations, fp32 accumulate"}
 TRAFFIC_RATIO = {"tiles_stack": 1.047}
 TRAFFIC = {}
 
@@ -583,7 +588,7 @@ def main():
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "int8 weights x bf16 activations, fp32 accumulate",
+        "scaling": "weak", "vs_baseline": None, "dtype": DTYPE[args.layout],
         "data": "synthetic",
         "config": {"workload": workload, "n_weights": n_weights, "hit_rate": hits / (hits + miss),
                    "hit_rate_device_layout": hit_rate_device, "K": stats["K"],
