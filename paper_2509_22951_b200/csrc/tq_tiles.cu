@@ -895,6 +895,7 @@ decompress_tiles_kernel(const tq_tiles_desc d, const uint32_t* __restrict__ tabl
 
 
 constexpr int kTilesWarps = 16;
+constexpr int kDecompWarps = 16;
 constexpr uint32_t kSmemLimit = 232448u;  // 227 KB per CTA
 
 // ---------------------------------------------------------------------------------------------
@@ -928,6 +929,8 @@ struct DecompCta : CtaBase {
     const uint32_t S = d.steps, gpr = d.cols >> 2;
     const uint32_t g = lane >> 2, t = lane & 3u;
     const bool vec_ok = (gpr & 3u) == 0u;  // every row starts on a 16-byte boundary
+    // ... on a 32-byte one (bf16 rows have a pitch of whole tiles)
+    const bool wide_ok = (BF16 || (gpr & 7u) == 0u) && (reinterpret_cast<uintptr_t>(out) & 31u) == 0u;
     const uint32_t xor_mask = levels_signed ? 0x80808080u : 0u;          // int8 bit pattern -> biased byte
     const float magic = levels_signed ? 8388736.0f : 8388608.0f;         // 2^23 (+ 128): as_float(0x4B000000 | byte) - magic = level
 
@@ -975,10 +978,10 @@ struct DecompCta : CtaBase {
           const float off = magic + (d.has_zero ? __ldg(d.zero + r) : 0.f);
           uint32_t* o = out + ((size_t)r * (S * 32u) + g0) * 2u;  // 2 words of bf16 per group
 #pragma unroll
-          for (int i = 0; i < 8; i += 2) {
-            uint32_t pk[4];
+          for (int i = 0; i < 8; i += 4) {
+            uint32_t pk[8];
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
+            for (int e = 0; e < 4; ++e) {
               const uint32_t v = w[8 * h + i + e] ^ xor_mask;
               const float f0 = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7540)) - off;
               const float f1 = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7541)) - off;
@@ -988,8 +991,17 @@ struct DecompCta : CtaBase {
               pk[2 * e] = *reinterpret_cast<const uint32_t*>(&lo);
               pk[2 * e + 1] = *reinterpret_cast<const uint32_t*>(&hi);
             }
-            asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(o + 2 * i), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3])
-                         : "memory");
+            if (wide_ok) {  // one whole 32-byte sector per store
+              asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(o + 2 * i), "r"(pk[0]), "r"(pk[1]),
+                           "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7])
+                           : "memory");
+            } else {
+              asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(o + 2 * i), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3])
+                           : "memory");
+              asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(o + 2 * i + 4), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]),
+                           "r"(pk[7])
+                           : "memory");
+            }
           }
         }
       }
@@ -998,7 +1010,12 @@ struct DecompCta : CtaBase {
         const uint32_t r = rb * 16u + g + 8u * h;
         if (r < d.rows && g0 < gpr) {
           uint32_t* o = out + (size_t)r * gpr + g0;
-          if (vec_ok && g0 + 8u <= gpr) {
+          if (wide_ok && g0 + 8u <= gpr) {  // one whole 32-byte sector per lane
+            asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(o), "r"(w[8 * h]), "r"(w[8 * h + 1]),
+                         "r"(w[8 * h + 2]), "r"(w[8 * h + 3]), "r"(w[8 * h + 4]), "r"(w[8 * h + 5]), "r"(w[8 * h + 6]),
+                         "r"(w[8 * h + 7])
+                         : "memory");
+          } else if (vec_ok && g0 + 8u <= gpr) {
             asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(o), "r"(w[8 * h]), "r"(w[8 * h + 1]),
                          "r"(w[8 * h + 2]), "r"(w[8 * h + 3])
                          : "memory");
@@ -1063,8 +1080,8 @@ __global__ void __launch_bounds__(W * 32, 1) decompress_tiles_smem_kernel(const 
 
 template <bool BF16>
 int launch_decomp(const DecompParams& p, uint32_t grid, cudaStream_t st) {
-  auto kern = decompress_tiles_smem_kernel<kTilesWarps, BF16>;
-  const size_t smem = tiles_smem(p.table_words, 0u, kTilesWarps).total;
+  auto kern = decompress_tiles_smem_kernel<kDecompWarps, BF16>;
+  const size_t smem = tiles_smem(p.table_words, 0u, kDecompWarps).total;
   static bool configured = false;
   if (!configured) {
     if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
@@ -1072,7 +1089,7 @@ int launch_decomp(const DecompParams& p, uint32_t grid, cudaStream_t st) {
       return rc;
     configured = true;
   }
-  kern<<<grid, kTilesWarps * 32, smem, st>>>(p);
+  kern<<<grid, kDecompWarps * 32, smem, st>>>(p);
   return tq_cuda_status((int)cudaGetLastError(), "decompress(tiles) launch");
 }
 
