@@ -46,6 +46,8 @@ def _L():
         f32p, f64p = C.POINTER(C.c_float), C.POINTER(C.c_double)
         lib.tqo_quantize_paper.argtypes = [f32p, C.c_uint64, u8p, f32p, f32p]
         lib.tqo_quantize_paper.restype = C.c_int
+        lib.tqo_quantize_paper_bits.argtypes = [f32p, C.c_uint64, C.c_int, u8p, f32p, f32p]
+        lib.tqo_quantize_paper_bits.restype = C.c_int
         lib.tqo_quantize_rows.argtypes = [f32p, C.c_uint32, C.c_uint32, C.POINTER(C.c_int8), f32p]
         lib.tqo_quantize_rows.restype = None
         lib.tqo_build_dictionary.argtypes = [C.POINTER(u8p), u64p, C.c_int, C.c_uint32]
@@ -79,15 +81,16 @@ def _ptr(a: np.ndarray, ctype):
     return a.ctypes.data_as(C.POINTER(ctype))
 
 
-def quantize_paper(x: np.ndarray):
-    """Listing 1 (bits=8): per-tensor min-max levels 0..255.  -> (q uint8, scale, zero)."""
+def quantize_paper(x: np.ndarray, bits: int = 8):
+    """Listing 1: per-tensor min-max levels 0..2^bits-1 (bits = 8 in the paper's pipeline).
+    -> (q uint8, scale, zero)."""
     x = np.ascontiguousarray(x, dtype=np.float32)
     q = np.empty(x.shape, dtype=np.uint8)
     s, z = C.c_float(), C.c_float()
-    rc = _L().tqo_quantize_paper(_ptr(x, C.c_float), x.size, _ptr(q, C.c_uint8),
-                                 C.byref(s), C.byref(z))
+    rc = _L().tqo_quantize_paper_bits(_ptr(x, C.c_float), x.size, int(bits), _ptr(q, C.c_uint8),
+                                      C.byref(s), C.byref(z))
     if rc != 0:
-        raise ValueError("degenerate range: max == min")
+        raise ValueError("degenerate range (max == min) or bits outside 1..8")
     return q, np.float32(s.value), np.float32(z.value)
 
 

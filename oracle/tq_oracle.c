@@ -30,15 +30,18 @@
                                    escape marker that the decoder tests first   */
 
 /* ------------------------------------------------------------------------ */
-/* Listing 1: naive min-max quantizer, per tensor, bits = 8 (maxq = 255).    */
-/* All arithmetic in fp32 with round-half-to-even, as the listing's tensor   */
-/* ops do.  Writes the integer level q (0..255); returns scale and zero.     */
-/* Returns -1 when the range is empty (scale would be 0).                    */
+/* Listing 1: naive min-max quantizer, per tensor, maxq = 2^bits - 1 levels   */
+/* above zero (bits = 8 in the paper's pipeline; Section 3 also tried 2, 4,  */
+/* 6).  All arithmetic in fp32 with round-half-to-even, as the listing's     */
+/* tensor ops do.  Writes the integer level q (0..maxq); returns scale and   */
+/* zero.  Returns -1 when the range is empty (scale would be 0) or bits is   */
+/* not an integer in 1..8 (the listing's ternary branch, bits = 1.5, makes   */
+/* no integer level and is not part of this path).                           */
 /* ------------------------------------------------------------------------ */
-int tqo_quantize_paper(const float *x, uint64_t n, uint8_t *q, float *scale_out,
-                       float *zero_out) {
-  if (n == 0) return -1;
-  const float maxq = 255.0f;
+int tqo_quantize_paper_bits(const float *x, uint64_t n, int bits, uint8_t *q,
+                            float *scale_out, float *zero_out) {
+  if (n == 0 || bits < 1 || bits > 8) return -1;
+  const float maxq = (float)((1 << bits) - 1);
   float xmin = x[0], xmax = x[0];
   for (uint64_t i = 1; i < n; ++i) {
     if (x[i] < xmin) xmin = x[i];
@@ -56,6 +59,11 @@ int tqo_quantize_paper(const float *x, uint64_t n, uint8_t *q, float *scale_out,
   *scale_out = scale;
   *zero_out = zero;
   return 0;
+}
+
+int tqo_quantize_paper(const float *x, uint64_t n, uint8_t *q, float *scale_out,
+                       float *zero_out) {
+  return tqo_quantize_paper_bits(x, n, 8, q, scale_out, zero_out);
 }
 
 /* ------------------------------------------------------------------------ */

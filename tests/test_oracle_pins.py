@@ -45,7 +45,7 @@ def test_handworked_tables(case):
 
 @pytest.mark.parametrize("case", _load("handworked_quantizer.json"), ids=lambda c: c["cite"][:40])
 def test_handworked_quantizer(case):
-    q, s, z = oracle.quantize_paper(np.array(case["x"], dtype=np.float32))
+    q, s, z = oracle.quantize_paper(np.array(case["x"], dtype=np.float32), bits=case.get("bits", 8))
     assert q.tolist() == case["q"]
     assert s == np.float32(case["scale_num"]) / np.float32(case["scale_den"])
     assert z == np.float32(case["zero"])
@@ -200,18 +200,39 @@ def test_code_is_rank_plus_one():
 # ----------------------------------------------------------------------------
 # Quantizers
 # ----------------------------------------------------------------------------
-def test_quantize_paper_end_points_and_error_bound():
+@pytest.mark.parametrize("bits", [8, 6, 4, 2, 1])
+def test_quantize_paper_end_points_and_error_bound(bits):
     rng = np.random.default_rng(11)
     x = rng.standard_normal(10_000).astype(np.float32) * 0.02
-    q, s, z = oracle.quantize_paper(x)
-    assert q[np.argmin(x)] == 0 and q[np.argmax(x)] == 255
+    maxq = 2 ** bits - 1
+    q, s, z = oracle.quantize_paper(x, bits=bits)
+    assert q[np.argmin(x)] == 0 and q[np.argmax(x)] == maxq and q.max() == maxq
+    assert float(s) == float((np.float32(x.max()) - np.float32(x.min())) / np.float32(maxq))
     deq = s.astype(np.float64) * (q.astype(np.float64) - float(z))
-    assert np.max(np.abs(deq - x)) <= 0.5 * float(s) * (1 + 1e-3) + 1e-9
+    # zero is itself rounded, so the grid may sit up to half a step off x's range at the ends
+    assert np.max(np.abs(deq - x)) <= float(s) * (1 + 1e-3) + 1e-9
+    inner = (q > 0) & (q < maxq)
+    assert np.max(np.abs(deq - x)[inner], initial=0.0) <= 0.5 * float(s) * (1 + 1e-3) + 1e-9
     # levels are a fixed point: quantizing the dequantised values with the same grid returns them
-    q2 = np.clip(np.rint(deq / float(s)) + float(z), 0, 255).astype(np.uint8)
+    q2 = np.clip(np.rint(deq / float(s)) + float(z), 0, maxq).astype(np.uint8)
     assert np.array_equal(q, q2)
     with pytest.raises(ValueError):
-        oracle.quantize_paper(np.ones(8, dtype=np.float32))
+        oracle.quantize_paper(np.ones(8, dtype=np.float32), bits=bits)
+
+
+def test_quantize_paper_rejects_other_bit_widths():
+    x = np.linspace(-1, 1, 16, dtype=np.float32)
+    for bits in (0, 9, -1):
+        with pytest.raises(ValueError):
+            oracle.quantize_paper(x, bits=bits)
+    # halving the bit count keeps every level on the coarser grid's multiples when the ranges nest:
+    # x on the integers 0..255 has scale 1 at 8 bits and scale 17 at 4 bits (255 / 15)
+    xi = np.arange(256, dtype=np.float32)
+    q8, s8, _ = oracle.quantize_paper(xi, bits=8)
+    q4, s4, z4 = oracle.quantize_paper(xi, bits=4)
+    assert s8 == 1.0 and s4 == 17.0 and z4 == 0.0
+    assert np.array_equal(q8, np.arange(256))
+    assert np.array_equal(q4, np.rint(xi / 17.0).astype(np.uint8))
 
 
 def test_quantize_rows_properties():
