@@ -116,7 +116,7 @@ DTYPE = {"tiles": "s8 x s8 -> s32 (int8 levels x three base-256 digits of block-
          "stream": "int8 weights x bf16 activations, fp32 accumulate"}
 
 
-def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout=1, quantizer="rows"):
+def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout=1, quantizer="rows", bits=8):
     """Generate, quantize, build the table and encode (host), upload.  quantizer "rows": per-row
     symmetric int8 on the GPU (the workload definition); "paper": Listing 1, one scale and zero point
     per tensor, unsigned levels (host).  Returns (matrices, xs, ys, table, ...)."""
@@ -129,7 +129,7 @@ def build_model(tq, shapes, batch, device, threads=0, table_entries=None, layout
     for i, (name, rows, cols) in enumerate(shapes):
         w = synth.weight(rows, cols, synth.matrix_seed(i), device=device)
         if quantizer == "paper":
-            q, s, z = tq.tq_quantize_tensor(w.cpu().numpy())
+            q, s, z = tq.tq_quantize_tensor_bits(w.cpu().numpy(), bits)
             q_host.append(q.reshape(rows, cols))
             scales.append(np.full(rows, s, dtype=np.float32))
             zeros.append(np.full(rows, z, dtype=np.float32))
@@ -382,6 +382,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="tq", choices=["tq", "reference"])
     ap.add_argument("--model", default="3b", choices=["1b", "3b", "11b"])
+    ap.add_argument("--bits", type=int, default=8, help="bit count of the per-tensor quantizer (--quantizer paper)")
     ap.add_argument("--quantizer", default="rows", choices=["rows", "paper"],
                     help="rows: per-row symmetric int8 (the workload definition); paper: Listing 1, per tensor, unsigned levels "
                          "with a zero point (a regime where nearly every group is in the table); single GPU, no CPU baseline")
@@ -404,7 +405,7 @@ def main():
     shapes = synth.llama32_linear_shapes(args.model, args.layers, lm_head=not args.no_lm_head)
     workload = f"llama3.2-{args.model} linear stack ({len(shapes)} matrices), batch {args.batch}"
     if args.quantizer == "paper":
-        workload += ", per-tensor quantizer of Listing 1"
+        workload += ", per-tensor quantizer of Listing 1" + ("" if args.bits == 8 else " at %d bits" % args.bits)
         assert int(os.environ.get("WORLD_SIZE", "1")) == 1 and not args.per_layer
     if args.shapes:
         shapes = [(f"m{i}", int(t.split("x")[0]), int(t.split("x")[1])) for i, t in enumerate(args.shapes.split(","))]
@@ -447,7 +448,7 @@ def main():
         dist.broadcast(ent, 0)
         table_entries = ent.cpu().numpy()
 
-    mats, xs, ys, hd, q_host, scales, stats, x_arena, y_arena, dd = build_model(tq, shapes, args.batch, device, threads, table_entries, layout={"stream": 0, "planes": 1, "tiles": 2}[args.layout], quantizer=args.quantizer)
+    mats, xs, ys, hd, q_host, scales, stats, x_arena, y_arena, dd = build_model(tq, shapes, args.batch, device, threads, table_entries, layout={"stream": 0, "planes": 1, "tiles": 2}[args.layout], quantizer=args.quantizer, bits=args.bits)
     infos = [m.info for m in mats]
     hits = sum(i.n_hits for i in infos)
     miss = sum(i.n_miss for i in infos)

@@ -64,6 +64,12 @@ int tq_set_num_threads(int n);
  * x, q: HOST, n elements.  Fails with TQ_ERR_INVALID_ARG when max == min. */
 int tq_quantize_tensor(const float* x, uint64_t n, uint8_t* q, float* scale, float* zero);
 
+/* The same quantizer at another bit count (Listing 1's configure step: maxq = 2^bits - 1; Section 3
+ * reports 2, 4, 6 and 8 bits): levels 0..maxq, still one byte per level, so every later step of the
+ * path (table, tokens, decode, products) takes them unchanged.  bits: integer 1..8, anything else
+ * (the listing's ternary setting included, which makes no integer level) is TQ_ERR_INVALID_ARG. */
+int tq_quantize_tensor_bits(const float* x, uint64_t n, int bits, uint8_t* q, float* scale, float* zero);
+
 /* Per-output-row symmetric int8 quantizer used by the benchmark workloads (not in the paper;
  * it produces the same kind of 8-bit level Listing 1 does, W ~ scale_r * q):
  * scale_r = max_c |w[r][c]| / 127 (1 for an all-zero row), q = clamp(round(w/scale_r), -127, 127).

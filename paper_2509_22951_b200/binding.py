@@ -32,7 +32,7 @@ TQ_STATUS_BAD_ROW = 2
 TQ_STATUS_WAIT_EXPIRED = 4
 
 EXPORTS = [
-    "tq_strerror", "tq_last_cuda_error", "tq_set_num_threads", "tq_quantize_tensor", "tq_quantize_rows",
+    "tq_strerror", "tq_last_cuda_error", "tq_set_num_threads", "tq_quantize_tensor", "tq_quantize_tensor_bits", "tq_quantize_rows",
     "tq_quantize_rows_device", "tq_build_dictionary", "tq_build_dictionary_device_size", "tq_build_dictionary_device", "tq_dict_from_entries", "tq_dict_entries",
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_upload_device_size", "tq_upload_device", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
@@ -67,6 +67,7 @@ def _load() -> C.CDLL:
         "tq_last_cuda_error": (C.c_char_p, []),
         "tq_set_num_threads": (C.c_int, [C.c_int]),
         "tq_quantize_tensor": (C.c_int, [f32p, C.c_uint64, u8p, f32p, f32p]),
+        "tq_quantize_tensor_bits": (C.c_int, [f32p, C.c_uint64, C.c_int, u8p, f32p, f32p]),
         "tq_quantize_rows": (C.c_int, [f32p, C.c_uint32, C.c_uint32, C.POINTER(C.c_int8), f32p]),
         "tq_quantize_rows_device": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, vp, vp]),
         "tq_build_dictionary": (C.c_int, [C.POINTER(u8p), u64p, C.c_int, C.c_uint32, C.POINTER(vp)]),
@@ -144,6 +145,15 @@ def tq_quantize_tensor(x: np.ndarray):
     s, z = C.c_float(), C.c_float()
     _check(_lib.tq_quantize_tensor(_np_ptr(x, C.c_float), x.size, _np_ptr(q, C.c_uint8), C.byref(s), C.byref(z)),
            "tq_quantize_tensor")
+    return q, np.float32(s.value), np.float32(z.value)
+
+
+def tq_quantize_tensor_bits(x: np.ndarray, bits: int):
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    q = np.empty(x.shape, dtype=np.uint8)
+    s, z = C.c_float(), C.c_float()
+    _check(_lib.tq_quantize_tensor_bits(_np_ptr(x, C.c_float), x.size, int(bits), _np_ptr(q, C.c_uint8), C.byref(s),
+                                        C.byref(z)), "tq_quantize_tensor_bits")
     return q, np.float32(s.value), np.float32(z.value)
 
 

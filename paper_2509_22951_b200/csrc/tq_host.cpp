@@ -177,14 +177,15 @@ int tq_set_num_threads(int n) {
   return tq_num_threads();
 }
 
-int tq_quantize_tensor(const float* x, uint64_t n, uint8_t* q, float* scale, float* zero) {
-  if (!x || !q || !scale || !zero || n == 0) return TQ_ERR_INVALID_ARG;
+int tq_quantize_tensor_bits(const float* x, uint64_t n, int bits, uint8_t* q, float* scale, float* zero) {
+  if (!x || !q || !scale || !zero || n == 0 || bits < 1 || bits > 8) return TQ_ERR_INVALID_ARG;
+  const float maxq = (float)((1 << bits) - 1);
   float lo = x[0], hi = x[0];
   for (uint64_t i = 1; i < n; ++i) {
     lo = std::min(lo, x[i]);
     hi = std::max(hi, x[i]);
   }
-  const float s = (hi - lo) / 255.0f;
+  const float s = (hi - lo) / maxq;
   if (!(s > 0.0f)) return TQ_ERR_INVALID_ARG;
   const float z = std::nearbyintf(-lo / s);
   const int nt = (int)std::min<uint64_t>(tq_num_threads(), n / 65536 + 1);
@@ -192,13 +193,17 @@ int tq_quantize_tensor(const float* x, uint64_t n, uint8_t* q, float* scale, flo
     uint64_t a = n * t / nt, b = n * (t + 1) / nt;
     for (uint64_t i = a; i < b; ++i) {
       float v = std::nearbyintf(x[i] / s) + z;
-      v = v < 0.0f ? 0.0f : (v > 255.0f ? 255.0f : v);
+      v = v < 0.0f ? 0.0f : (v > maxq ? maxq : v);
       q[i] = (uint8_t)v;
     }
   });
   *scale = s;
   *zero = z;
   return TQ_OK;
+}
+
+int tq_quantize_tensor(const float* x, uint64_t n, uint8_t* q, float* scale, float* zero) {
+  return tq_quantize_tensor_bits(x, n, 8, q, scale, zero);
 }
 
 int tq_quantize_rows(const float* w, uint32_t rows, uint32_t cols, int8_t* q, float* scale) {

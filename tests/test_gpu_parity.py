@@ -119,6 +119,19 @@ def test_unsigned_levels_with_zero_point(tq, layout):
     _check_layer(tq, qu, s, d, stream, batches=(1, 4), zero=z, layout=layout)
 
 
+@pytest.mark.parametrize("bits", [6, 4, 2])
+def test_lower_bit_grids_of_the_per_tensor_quantizer(tq, layout, bits):
+    # Listing 1 at fewer bits: levels 0..2^bits-1 in one byte each; table, tokens, decode and products unchanged
+    w = synth.weight(144, 1536, synth.matrix_seed(20 + bits)).numpy()
+    qu, sc, zp = oracle.quantize_paper(w, bits=bits)
+    qu = qu.reshape(144, 1536)
+    assert int(qu.max()) == 2 ** bits - 1
+    s = np.full(144, sc, dtype=np.float32)
+    z = np.full(144, zp, dtype=np.float32)
+    d, (stream,) = _oracle_pack([qu])
+    _check_layer(tq, qu, s, d, stream, batches=(1, 3, 8), zero=z, layout=layout)
+
+
 def test_batch_up_to_32(tq, layout):
     rng = np.random.default_rng(8)
     q = np.clip(np.rint(rng.standard_t(5, size=(130, 3072)) * 6), -127, 127).astype(np.int8)

@@ -40,6 +40,17 @@ def test_quantize_tensor_matches_oracle_bit_exact():
         tq.tq_quantize_tensor(np.zeros(16, dtype=np.float32))
 
 
+@pytest.mark.parametrize("bits", [1, 2, 4, 6, 8])
+def test_quantize_tensor_bits_matches_oracle_bit_exact(bits):
+    x = synth.weight(48, 320, synth.matrix_seed(5)).numpy()
+    q, s, z = tq.tq_quantize_tensor_bits(x, bits)
+    qo, so, zo = oracle.quantize_paper(x, bits=bits)
+    assert np.array_equal(q, qo) and s == so and z == zo and q.max() == 2 ** bits - 1
+    for bad in (0, 9):
+        with pytest.raises(tq.TqError):
+            tq.tq_quantize_tensor_bits(x, bad)
+
+
 def _check_same(mats, top_k):
     d = tq.tq_build_dictionary(mats, top_k)
     o = oracle.Dictionary.build(mats, top_k)
