@@ -594,23 +594,23 @@ struct PanelCta : CtaBase {
   __device__ __forceinline__ XInfo8* xinfo() { return reinterpret_cast<XInfo8*>(smem + L.misc + 128); }
   __device__ __forceinline__ long long* sums() { return reinterpret_cast<long long*>(smem + L.misc + 256); }
 
-  // digits of one activation group (4 columns) -> three words
-  static __device__ __forceinline__ void digits(uint2 v, float scale, bool finite, uint32_t& w0, uint32_t& w1,
-                                                uint32_t& w2, long long* sum) {
+  // digits of one activation group (4 columns) -> three words.  X = d0 + 256 d1 + 65536 d2 with
+  // balanced digits: d0 is the low byte of X, d1 byte 1 of X + 128, d2 byte 2 of X + 128 + 32768.
+  static __device__ __forceinline__ void digits(uint2 v, float scale, uint32_t& w0, uint32_t& w1, uint32_t& w2,
+                                                long long* sum) {
     const uint32_t h[4] = {v.x << 16, v.x & 0xFFFF0000u, v.y << 16, v.y & 0xFFFF0000u};
-    w0 = w1 = w2 = 0;
+    uint32_t X[4], Y[4], Z[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      int X = finite ? __float2int_rn(__uint_as_float(h[i]) * scale) : 0;
-      if (sum) *sum += X;
-      const int d0 = (int)(signed char)(X & 0xFF);
-      X = (X - d0) >> 8;
-      const int d1 = (int)(signed char)(X & 0xFF);
-      const int d2 = (X - d1) >> 8;
-      w0 |= (uint32_t)(d0 & 0xFF) << (8 * i);
-      w1 |= (uint32_t)(d1 & 0xFF) << (8 * i);
-      w2 |= (uint32_t)(d2 & 0xFF) << (8 * i);
+      const int xi = __float2int_rn(__uint_as_float(h[i]) * scale);
+      if (sum) *sum += xi;
+      X[i] = (uint32_t)xi;
+      Y[i] = X[i] + 128u;
+      Z[i] = X[i] + 32896u;
     }
+    w0 = __byte_perm(__byte_perm(X[0], X[1], 0x0040), __byte_perm(X[2], X[3], 0x0040), 0x5410);
+    w1 = __byte_perm(__byte_perm(Y[0], Y[1], 0x0051), __byte_perm(Y[2], Y[3], 0x0051), 0x5410);
+    w2 = __byte_perm(__byte_perm(Z[0], Z[1], 0x0062), __byte_perm(Z[2], Z[3], 0x0062), 0x5410);
   }
 
   // Per-vector scales (and, with zero points, the sum of each vector's fixed-point values).
@@ -651,7 +651,7 @@ struct PanelCta : CtaBase {
         long long sum = 0;
         for (uint32_t g = tid; g < G; g += kThreads) {
           uint32_t w0, w1, w2;
-          digits(__ldg(xg + (size_t)b * G + g), sc, true, w0, w1, w2, &sum);
+          digits(__ldg(xg + (size_t)b * G + g), sc, w0, w1, w2, &sum);
         }
 #pragma unroll
         for (int sft = 16; sft > 0; sft >>= 1) sum += __shfl_xor_sync(kFull, sum, sft);
@@ -686,7 +686,7 @@ struct PanelCta : CtaBase {
       const uint32_t gl = idx % kGroups, b = idx / kGroups;
       if (idx < kGroups * NB) {
         uint32_t w0, w1, w2;
-        digits(v[it], b < nb_valid ? in_scale()[b] : 0.f, true, w0, w1, w2, nullptr);
+        digits(v[it], b < nb_valid ? in_scale()[b] : 0.f, w0, w1, w2, nullptr);
         xs[(3 * b + 0) * kPanelStride + gl] = w0;
         xs[(3 * b + 1) * kPanelStride + gl] = w1;
         xs[(3 * b + 2) * kPanelStride + gl] = w2;
