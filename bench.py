@@ -436,9 +436,12 @@ def main():
             q0 = []
             for i, (name, rows, cols) in enumerate(shapes):
                 w = synth.weight(rows, cols, synth.matrix_seed(i), device=device)
-                q0.append(tq.tq_quantize_rows_device(w)[0].cpu().numpy())
-            ent = torch.from_numpy(tq.tq_build_dictionary(q0).entries).to(device)
+                q0.append(tq.tq_quantize_rows_device(w)[0])
+                del w
+            # windows counted on the GPU, candidates ranked on the host: the same table as tq_build_dictionary
+            ent = torch.from_numpy(np.ascontiguousarray(tq.tq_build_dictionary_device([q.view(-1) for q in q0]).entries)).to(device)
             del q0
+            torch.cuda.empty_cache()
             meta = torch.tensor([ent.shape[0]], device=device)
         else:
             meta = torch.zeros(1, dtype=torch.int64, device=device)
