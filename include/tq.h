@@ -312,6 +312,26 @@ int tq_decompress_stack(const tq_stack* s, uint8_t* const* d_out_ptrs, void* cud
  * d_workspace_ptrs: DEVICE array of n_mats DEVICE pointers (256-byte aligned, tq_gemm_workspace_size
  * bytes each). */
 int tq_decode_bf16_stack(const tq_stack* s, void* const* d_workspace_ptrs, void* cuda_stream);
+
+/* Phase 2 of tq_fused_gemm_ws for several matrices and one token count in ONE persistent launch: the
+ * output tiles of all products form one sequence (longest rows first) that the CTAs share, so no SM
+ * idles at the end of a small matrix.  Y_i[M][rows_i] = scale_i * (W_i as bf16 in d_workspaces[i]) x
+ * X_i[M][cols_i]; the workspaces are the ones tq_decode_bf16 / tq_decode_bf16_stack fill.
+ * tq_gemm_plan_create binds the operands (HOST arrays of n_mats DEVICE pointers; alignment as for
+ * tq_gemm_bf16_ws), writes the tensor maps and the tile index into d_buf (DEVICE, 256-byte aligned,
+ * tq_gemm_plan_size bytes, caller-owned, must outlive the plan) on cuda_stream and synchronises it
+ * once; tq_gemm_plan_run launches without synchronising and may be called any number of times while
+ * the bound buffers are alive.  Matrices must be TQ_LAYOUT_TILES with cols a multiple of 8
+ * (TQ_ERR_UNSUPPORTED_SHAPE otherwise).  tq_gemm_plan_status synchronises cuda_stream and returns the
+ * plan's own sticky status word (TQ_STATUS_WAIT_EXPIRED if a bounded wait inside the kernel ran out). */
+typedef struct tq_gemm_plan tq_gemm_plan;
+int tq_gemm_plan_size(int n_mats, uint64_t* device_bytes);
+int tq_gemm_plan_create(const tq_dmat* const* mats, const void* const* d_X_bf16, float* const* d_Y,
+                        const void* const* d_workspaces, int n_mats, int M, void* d_buf,
+                        uint64_t d_buf_bytes, void* cuda_stream, tq_gemm_plan** out);
+int tq_gemm_plan_run(const tq_gemm_plan* plan, void* cuda_stream);
+int tq_gemm_plan_status(const tq_gemm_plan* plan, void* cuda_stream, uint32_t* status);
+void tq_gemm_plan_free(tq_gemm_plan* plan); /* host handle only */
 void tq_stack_free(tq_stack* s);
 
 /* Read and clear the matrix's device status word (TQ_STATUS_* bits); synchronises cuda_stream. */

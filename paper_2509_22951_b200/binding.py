@@ -37,7 +37,8 @@ EXPORTS = [
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
     "tq_upload_size", "tq_upload", "tq_upload_device_size", "tq_upload_device", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
     "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_gemm_workspace_size",
-    "tq_fused_gemm_ws", "tq_decode_bf16", "tq_gemm_bf16_ws", "tq_decode_bf16_stack", "tq_stack_size", "tq_stack_plan_host", "tq_stack_create",
+    "tq_fused_gemm_ws", "tq_decode_bf16", "tq_gemm_bf16_ws", "tq_decode_bf16_stack", "tq_gemm_plan_size", "tq_gemm_plan_create", "tq_gemm_plan_run",
+    "tq_gemm_plan_status", "tq_gemm_plan_free", "tq_stack_size", "tq_stack_plan_host", "tq_stack_create",
     "tq_fused_gemv_stack", "tq_fused_gemv_stack_host", "tq_stack_launches", "tq_decompress_stack", "tq_stack_free", "tq_device_status", "tq_dmat_free",
 ]
 
@@ -98,6 +99,12 @@ def _load() -> C.CDLL:
         "tq_decode_bf16": (C.c_int, [vp, vp, C.c_uint64, vp]),
         "tq_gemm_bf16_ws": (C.c_int, [vp, vp, C.c_int, vp, vp, vp]),
         "tq_decode_bf16_stack": (C.c_int, [vp, vp, vp]),
+        "tq_gemm_plan_size": (C.c_int, [C.c_int, u64p]),
+        "tq_gemm_plan_create": (C.c_int, [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int, C.c_int, vp,
+                                          C.c_uint64, vp, C.POINTER(vp)]),
+        "tq_gemm_plan_run": (C.c_int, [vp, vp]),
+        "tq_gemm_plan_status": (C.c_int, [vp, vp, u32p]),
+        "tq_gemm_plan_free": (None, [vp]),
         "tq_stack_size": (C.c_int, [C.c_int, u64p]),
         "tq_stack_plan_host": (C.c_int, [C.c_int, u32p, u32p, C.POINTER(u32p), C.c_uint32, u32p, C.c_uint32, u32p, u32p]),
         "tq_stack_create": (C.c_int, [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int, C.c_int, vp, C.c_uint64, vp,
@@ -555,6 +562,56 @@ def tq_decode_bf16_stack(s: Stack, workspaces, stream=None) -> None:
     ptrs = torch.tensor([w.data_ptr() for w in workspaces], dtype=torch.int64).to(s.buf.device)
     _check(_lib.tq_decode_bf16_stack(s._h, ptrs.data_ptr(), _stream_ptr(stream)), "tq_decode_bf16_stack")
     s._ws_ptrs = ptrs  # keep the pointer array alive until the stream has used it
+
+
+class GemmPlan:
+    """Several workspace GEMMs of one token count bound for one persistent launch.  Keeps the
+    matrices, operands, workspaces and its own device buffer alive."""
+
+    def __init__(self, handle: int, buf: torch.Tensor, mats, Xs, Ys, workspaces, M: int):
+        self._h = C.c_void_p(handle)
+        self.buf, self.mats, self.Xs, self.Ys, self.workspaces, self.M = buf, list(mats), list(Xs), list(Ys), list(workspaces), M
+
+    def __del__(self):
+        if getattr(self, "_h", None) and _lib is not None:
+            _lib.tq_gemm_plan_free(self._h)
+            self._h = None
+
+
+def tq_gemm_plan_create(mats, Xs, workspaces, Ys=None, stream=None) -> GemmPlan:
+    """Xs[i]: CUDA bf16 [M][cols_i]; workspaces[i]: filled (now or later, before the run) by tq_decode_bf16(_stack);
+    Ys[i]: CUDA fp32 [M][rows_i] (made here when None)."""
+    n = len(mats)
+    assert n >= 1 and len(Xs) == n and len(workspaces) == n
+    M = Xs[0].view(-1, mats[0].info.cols).shape[0]
+    dev = Xs[0].device
+    if Ys is None:
+        Ys = [torch.empty((M, m.info.rows), dtype=torch.float32, device=dev) for m in mats]
+    for m, X, Y, w in zip(mats, Xs, Ys, workspaces):
+        assert X.is_cuda and X.dtype == torch.bfloat16 and X.is_contiguous() and X.numel() == M * m.info.cols
+        assert Y.is_cuda and Y.dtype == torch.float32 and Y.is_contiguous() and Y.numel() == M * m.info.rows
+        assert w.is_cuda and w.numel() * w.element_size() >= tq_gemm_workspace_size(m)
+    need = C.c_uint64()
+    _check(_lib.tq_gemm_plan_size(n, C.byref(need)), "tq_gemm_plan_size")
+    buf = torch.empty(need.value + 256, dtype=torch.uint8, device=dev)
+    off = (-buf.data_ptr()) % 256
+    arr = lambda ts: (C.c_void_p * n)(*[t.data_ptr() for t in ts])  # noqa: E731
+    out = C.c_void_p()
+    with torch.cuda.device(dev):
+        _check(_lib.tq_gemm_plan_create((C.c_void_p * n)(*[m._h for m in mats]), arr(Xs), arr(Ys), arr(workspaces), n, M,
+                                        buf.data_ptr() + off, need.value, _stream_ptr(stream), C.byref(out)),
+               "tq_gemm_plan_create")
+    return GemmPlan(out.value, buf, mats, Xs, Ys, workspaces, M)
+
+
+def tq_gemm_plan_run(p: GemmPlan, stream=None) -> None:
+    _check(_lib.tq_gemm_plan_run(p._h, _stream_ptr(stream)), "tq_gemm_plan_run")
+
+
+def tq_gemm_plan_status(p: GemmPlan, stream=None) -> int:
+    st = C.c_uint32()
+    _check(_lib.tq_gemm_plan_status(p._h, _stream_ptr(stream), C.byref(st)), "tq_gemm_plan_status")
+    return st.value
 
 
 def tq_fused_gemv_stack(s: Stack, stream=None) -> None:

@@ -16,6 +16,8 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <new>
+#include <vector>
 
 #include "tq_internal.h"
 #include "tq_sm100.cuh"
@@ -44,9 +46,88 @@ struct GemmWsParams {
   uint32_t row_tiles, token_tiles;
 };
 
-template <int BN>
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, const GemmWsParams p) {
+// What one output tile needs: the two tensor maps, where it sits, how many 64-column stages it
+// takes, and where its results go.
+struct TileInfo {
+  const CUtensorMap* map_w;
+  const CUtensorMap* map_x;
+  const float* scale;
+  float* Y;
+  uint32_t rows, n_k, r0, n0;
+};
+
+// One matrix: tensor maps in the kernel's parameter space.
+struct SingleSrc {
+  const CUtensorMap* map_w;
+  const CUtensorMap* map_x;
+  GemmWsParams p;
+  __device__ __forceinline__ uint32_t total() const { return p.row_tiles * p.token_tiles; }
+  __device__ __forceinline__ uint32_t M() const { return p.M; }
+  __device__ __forceinline__ uint32_t* status() const { return p.status; }
+  // `cursor` (unused here) and `fresh` (the maps were not used by this thread before) serve GroupSrc
+  template <int BN>
+  __device__ __forceinline__ TileInfo locate(uint32_t tile, uint32_t& cursor, bool& fresh) const {
+    (void)cursor;
+    fresh = false;
+    TileInfo t;
+    t.map_w = map_w;
+    t.map_x = map_x;
+    t.scale = p.scale;
+    t.Y = p.Y;
+    t.rows = p.rows;
+    t.n_k = (p.cols + BK - 1) / BK;
+    t.r0 = (tile / p.token_tiles) * BM;
+    t.n0 = (tile % p.token_tiles) * BN;
+    return t;
+  }
+};
+
+// Several matrices, one token count: the tiles of all of them in one sequence.  Everything lives in
+// DEVICE memory, the tensor maps included (2 per matrix: weights, activations; 128 bytes each).
+struct GroupEntry {
+  const float* scale;
+  float* Y;
+  uint32_t rows, cols;
+};
+struct GroupSrc {
+  const CUtensorMap* maps;
+  const GroupEntry* groups;
+  const uint32_t* tile_begin;  // n_groups + 1
+  uint32_t* status_word;
+  uint32_t n_groups, token_tiles, n_tokens, n_tiles;
+  __device__ __forceinline__ uint32_t total() const { return n_tiles; }
+  __device__ __forceinline__ uint32_t M() const { return n_tokens; }
+  __device__ __forceinline__ uint32_t* status() const { return status_word; }
+  // Tiles come in ascending order, so the group index only moves forward from `cursor`.
+  template <int BN>
+  __device__ __forceinline__ TileInfo locate(uint32_t tile, uint32_t& cursor, bool& fresh) const {
+    uint32_t g = cursor == 0xFFFFFFFFu ? 0u : cursor;
+    while (g + 1 < n_groups && tile >= __ldg(tile_begin + g + 1)) ++g;
+    fresh = g != cursor;
+    cursor = g;
+    const uint32_t local = tile - __ldg(tile_begin + g);
+    const GroupEntry e = groups[g];
+    TileInfo t;
+    t.map_w = maps + 2 * g;
+    t.map_x = maps + 2 * g + 1;
+    t.scale = e.scale;
+    t.Y = e.Y;
+    t.rows = e.rows;
+    t.n_k = (e.cols + BK - 1) / BK;
+    t.r0 = (local / token_tiles) * BM;
+    t.n0 = (local % token_tiles) * BN;
+    return t;
+  }
+};
+
+// A tensor map read from global memory: the copy unit reads it through its own path, so the thread
+// that is about to use it orders that read after the writes that made the map.
+__device__ __forceinline__ void tensormap_acquire(const CUtensorMap* map) {
+  asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(map) : "memory");
+}
+
+template <int BN, class Src>
+__device__ __forceinline__ void gemm_ws_body(const Src& src) {
   constexpr uint32_t STAGE_BYTES = Geo<BN>::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // operand tiles need 1024-byte alignment
@@ -60,8 +141,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
-  const uint32_t n_tiles = p.row_tiles * p.token_tiles;
-  const uint32_t n_k = (p.cols + BK - 1) / BK;
+  const uint32_t n_tiles = src.total();
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < kStages; ++s) {
@@ -89,16 +169,22 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     if (lane == 0) {
       bool alive = true;
       uint32_t it = 0;
+      uint32_t cursor = 0xFFFFFFFFu;
       for (uint32_t tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
-        const int r0 = (int)((tile / p.token_tiles) * BM), n0 = (int)((tile % p.token_tiles) * BN);
-        for (uint32_t ks = 0; ks < n_k && alive; ++ks, ++it) {
+        bool fresh;
+        const TileInfo t = src.template locate<BN>(tile, cursor, fresh);
+        if (fresh) {
+          tensormap_acquire(t.map_w);
+          tensormap_acquire(t.map_x);
+        }
+        for (uint32_t ks = 0; ks < t.n_k && alive; ++ks, ++it) {
           const uint32_t s = it % kStages;
           alive = mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag);
           if (!alive) break;
           const uint32_t a_tile = base + s * STAGE_BYTES;
           mbar_expect_tx(full_bar(s), STAGE_BYTES);
-          tma_load_2d(a_tile, &tmap_w, (int)(ks * BK), r0, full_bar(s));
-          tma_load_2d(a_tile + A_BYTES, &tmap_x, (int)(ks * BK), n0, full_bar(s));
+          tma_load_2d(a_tile, t.map_w, (int)(ks * BK), (int)t.r0, full_bar(s));
+          tma_load_2d(a_tile + A_BYTES, t.map_x, (int)(ks * BK), (int)t.n0, full_bar(s));
         }
       }
       if (!alive) {  // let the copies already in flight land before the CTA's shared memory is released
@@ -110,8 +196,10 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc(BM, BN);
       bool alive = true;
-      uint32_t it = 0, local = 0;
+      uint32_t it = 0, local = 0, cursor = 0xFFFFFFFFu;
       for (uint32_t tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++local) {
+        bool fresh;
+        const uint32_t n_k = src.template locate<BN>(tile, cursor, fresh).n_k;
         const uint32_t buf = local & 1u, use = local >> 1;
         alive = mbar_wait(acc_empty(buf), (use & 1u) ^ 1u, abort_flag);  // the epilogue has drained this accumulator
         if (!alive) break;
@@ -135,15 +223,18 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     // ------------------------------------------------------------------ epilogue: TMEM -> scale -> Y
     const uint32_t quarter = warp & 3u;  // the TMEM lanes this warp may read: 32 * (warp % 4) ..
     bool alive = true;
-    uint32_t local = 0;
+    uint32_t local = 0, cursor = 0xFFFFFFFFu;
+    const uint32_t n_tokens = src.M();
     for (uint32_t tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++local) {
       const uint32_t buf = local & 1u, use = local >> 1;
-      const uint32_t r0 = (tile / p.token_tiles) * BM, n0 = (tile % p.token_tiles) * BN;
+      bool fresh;
+      const TileInfo t = src.template locate<BN>(tile, cursor, fresh);
+      const uint32_t n0 = t.n0;
       alive = mbar_wait(acc_full(buf), use & 1u, abort_flag);
       if (!alive) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t row = r0 + quarter * 32u + lane;
-      const float sc = row < p.rows ? __ldg(p.scale + row) : 0.f;
+      const uint32_t row = t.r0 + quarter * 32u + lane;
+      const float sc = row < t.rows ? __ldg(t.scale + row) : 0.f;
 #pragma unroll 1
       for (uint32_t c = 0; c < BN; c += 32) {
         uint32_t v[32];
@@ -157,11 +248,11 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
               "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
             : "r"(taddr));
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (row < p.rows) {
+        if (row < t.rows) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const uint32_t token = n0 + c + j;
-            if (token < p.M) p.Y[(size_t)token * p.rows + row] = sc * __uint_as_float(v[j]);
+            if (token < n_tokens) t.Y[(size_t)token * t.rows + row] = sc * __uint_as_float(v[j]);
           }
         }
       }
@@ -177,7 +268,18 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(2 * BN) : "memory");
   }
-  if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, TQ_STATUS_WAIT_EXPIRED);
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(src.status(), TQ_STATUS_WAIT_EXPIRED);
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, const GemmWsParams p) {
+  gemm_ws_body<BN>(SingleSrc{&tmap_w, &tmap_x, p});
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1) gemm_ws_group_kernel(const GroupSrc src) {
+  gemm_ws_body<BN>(src);
 }
 
 }  // namespace
@@ -207,26 +309,69 @@ int tq_fused_gemm_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, 
   return tq_gemm_bf16_ws(m, d_X_bf16, M, d_Y, d_workspace, cuda_stream);
 }
 
+}  // extern "C"
+
+namespace {
+
+// Tensor maps of one product: the weights as bf16 in a workspace (rows padded to whole tiles, pitch of
+// whole tiles), the activations [M][cols]; boxes of 64 columns x 128 rows / bn tokens, 128-byte swizzle.
+int encode_maps(const tq_dmat* m, const void* d_workspace, const void* d_X_bf16, uint32_t M, uint32_t bn, CUtensorMap* map_w,
+                CUtensorMap* map_x) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return tq_cuda_status((int)cudaErrorUnknown, "gemm: cuTensorMapEncodeTiled not available");
+  const uint32_t rows_pad = m->tiles.row_blocks * 16u, pitch = m->tiles.steps * 128u;
+  const cuuint32_t estr[2] = {1, 1};
+  {
+    const cuuint64_t gdim[2] = {m->info.cols, rows_pad};
+    const cuuint64_t gstride[1] = {(cuuint64_t)pitch * 2};
+    const cuuint32_t box[2] = {BK, BM};
+    if (enc(map_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d_workspace), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return tq_cuda_status((int)cudaErrorInvalidValue, "gemm: tensor map of the weights");
+  }
+  {
+    const cuuint64_t gdim[2] = {m->info.cols, (cuuint64_t)M};
+    const cuuint64_t gstride[1] = {(cuuint64_t)m->info.cols * 2};
+    const cuuint32_t box[2] = {BK, bn};
+    if (enc(map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d_X_bf16), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return tq_cuda_status((int)cudaErrorInvalidValue, "gemm: tensor map of the activations");
+  }
+  return TQ_OK;
+}
+
+int configure_gemm_kernels() {
+  static bool configured = false;
+  if (configured) return TQ_OK;
+  const void* kerns[4] = {(const void*)gemm_ws_kernel<256>, (const void*)gemm_ws_kernel<128>, (const void*)gemm_ws_group_kernel<256>,
+                          (const void*)gemm_ws_group_kernel<128>};
+  const int smem[4] = {(int)Geo<256>::SMEM_BYTES, (int)Geo<128>::SMEM_BYTES, (int)Geo<256>::SMEM_BYTES, (int)Geo<128>::SMEM_BYTES};
+  for (int i = 0; i < 4; ++i)
+    if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(kerns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, smem[i]),
+                                "gemm: raising the dynamic shared memory limit"))
+      return rc;
+  configured = true;
+  return TQ_OK;
+}
+
+inline uint64_t align256(uint64_t v) { return (v + 255) / 256 * 256; }
+
+}  // namespace
+
+struct tq_gemm_plan {
+  GroupSrc src{};
+  uint32_t bn = 256, grid = 0;
+};
+
+extern "C" {
+
 int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, const void* d_workspace,
                     void* cuda_stream) {
   if (!m || !d_X_bf16 || !d_Y || !d_workspace || M < 1 || ((uintptr_t)d_X_bf16 & 15) || ((uintptr_t)d_workspace & 255))
     return TQ_ERR_INVALID_ARG;
   if (m->info.layout != TQ_LAYOUT_TILES) return TQ_ERR_UNSUPPORTED_SHAPE;
   if ((m->info.cols * 2u) % 16u != 0) return TQ_ERR_UNSUPPORTED_SHAPE;  // TMA row pitch must be a multiple of 16 bytes
-  EncodeTiledFn enc = encode_fn();
-  if (!enc) return tq_cuda_status((int)cudaErrorUnknown, "gemm: cuTensorMapEncodeTiled not available");
-
-  const uint32_t rows_pad = m->tiles.row_blocks * 16u, pitch = m->tiles.steps * 128u;
-  CUtensorMap tmap_w;
-  const cuuint32_t estr[2] = {1, 1};
-  {
-    const cuuint64_t gdim[2] = {m->info.cols, rows_pad};
-    const cuuint64_t gstride[1] = {(cuuint64_t)pitch * 2};
-    const cuuint32_t box[2] = {BK, BM};
-    if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d_workspace), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return tq_cuda_status((int)cudaErrorInvalidValue, "gemm: tensor map of the weights");
-  }
   GemmWsParams p;
   p.scale = m->d_scale;
   p.Y = d_Y;
@@ -246,32 +391,106 @@ int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, c
   const bool narrow = (uint32_t)M <= 128u && fill(128) >= fill(256);
   const uint32_t bn = narrow ? 128u : 256u;
   p.token_tiles = ((uint32_t)M + bn - 1) / bn;
-  CUtensorMap tmap_x;
-  {
-    const cuuint64_t gdim[2] = {m->info.cols, (cuuint64_t)M};
-    const cuuint64_t gstride[1] = {(cuuint64_t)m->info.cols * 2};
-    const cuuint32_t box[2] = {BK, bn};
-    if (enc(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d_X_bf16), gdim, gstride, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return tq_cuda_status((int)cudaErrorInvalidValue, "gemm: tensor map of the activations");
-  }
+  CUtensorMap tmap_w, tmap_x;
+  if (int rc = encode_maps(m, d_workspace, d_X_bf16, (uint32_t)M, bn, &tmap_w, &tmap_x)) return rc;
   const uint32_t grid = std::min<uint32_t>(p.row_tiles * p.token_tiles, sms);
-  static bool configured = false;
-  if (!configured) {
-    int rc = tq_cuda_status((int)cudaFuncSetAttribute(gemm_ws_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                      (int)Geo<256>::SMEM_BYTES), "gemm: raising the dynamic shared memory limit");
-    if (rc == TQ_OK)
-      rc = tq_cuda_status((int)cudaFuncSetAttribute(gemm_ws_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                    (int)Geo<128>::SMEM_BYTES), "gemm: raising the dynamic shared memory limit");
-    if (rc != TQ_OK) return rc;
-    configured = true;
-  }
+  if (int rc = configure_gemm_kernels()) return rc;
   if (narrow)
     gemm_ws_kernel<128><<<grid, kThreads, Geo<128>::SMEM_BYTES, (cudaStream_t)cuda_stream>>>(tmap_w, tmap_x, p);
   else
     gemm_ws_kernel<256><<<grid, kThreads, Geo<256>::SMEM_BYTES, (cudaStream_t)cuda_stream>>>(tmap_w, tmap_x, p);
   return tq_cuda_status((int)cudaGetLastError(), "gemm launch");
 }
+
+int tq_gemm_plan_size(int n_mats, uint64_t* device_bytes) {
+  if (n_mats < 1 || !device_bytes) return TQ_ERR_INVALID_ARG;
+  *device_bytes = align256((uint64_t)n_mats * 2 * sizeof(CUtensorMap)) + align256((uint64_t)n_mats * sizeof(GroupEntry)) +
+                  align256(((uint64_t)n_mats + 1) * 4) + 256 /* status word */;
+  return TQ_OK;
+}
+
+int tq_gemm_plan_create(const tq_dmat* const* mats, const void* const* d_X_bf16, float* const* d_Y,
+                        const void* const* d_workspaces, int n_mats, int M, void* d_buf, uint64_t d_buf_bytes,
+                        void* cuda_stream, tq_gemm_plan** out) {
+  if (!mats || !d_X_bf16 || !d_Y || !d_workspaces || n_mats < 1 || M < 1 || !d_buf || ((uintptr_t)d_buf & 255) || !out)
+    return TQ_ERR_INVALID_ARG;
+  uint64_t need = 0;
+  tq_gemm_plan_size(n_mats, &need);
+  if (d_buf_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
+  for (int i = 0; i < n_mats; ++i) {
+    if (!mats[i] || !d_X_bf16[i] || !d_Y[i] || !d_workspaces[i] || ((uintptr_t)d_X_bf16[i] & 15) || ((uintptr_t)d_workspaces[i] & 255))
+      return TQ_ERR_INVALID_ARG;
+    if (mats[i]->info.layout != TQ_LAYOUT_TILES || (mats[i]->info.cols * 2u) % 16u != 0) return TQ_ERR_UNSUPPORTED_SHAPE;
+  }
+  const uint32_t bn = (uint32_t)M <= 128u ? 128u : 256u;
+  const uint32_t token_tiles = ((uint32_t)M + bn - 1) / bn;
+  // longest rows first: the tiles that take longest start first, so the last, partly filled round of
+  // tiles is made of short ones
+  std::vector<int> order((size_t)n_mats);
+  for (int i = 0; i < n_mats; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return mats[a]->info.cols > mats[b]->info.cols; });
+  std::vector<CUtensorMap> maps((size_t)n_mats * 2);
+  std::vector<GroupEntry> groups((size_t)n_mats);
+  std::vector<uint32_t> tile_begin((size_t)n_mats + 1);
+  uint64_t tiles = 0;
+  for (int k = 0; k < n_mats; ++k) {
+    const tq_dmat* m = mats[order[k]];
+    if (int rc = encode_maps(m, d_workspaces[order[k]], d_X_bf16[order[k]], (uint32_t)M, bn, &maps[2 * k], &maps[2 * k + 1])) return rc;
+    groups[k] = GroupEntry{m->d_scale, d_Y[order[k]], m->info.rows, m->info.cols};
+    tile_begin[k] = (uint32_t)tiles;
+    tiles += (uint64_t)((m->info.rows + BM - 1) / BM) * token_tiles;
+    if (tiles > 0x7FFFFFFFull) return TQ_ERR_UNSUPPORTED_SHAPE;
+  }
+  tile_begin[n_mats] = (uint32_t)tiles;
+  if (int rc = configure_gemm_kernels()) return rc;
+  tq_gemm_plan* pl = new (std::nothrow) tq_gemm_plan();
+  if (!pl) return TQ_ERR_NOMEM;
+  uint8_t* base = static_cast<uint8_t*>(d_buf);
+  const uint64_t off_groups = align256(maps.size() * sizeof(CUtensorMap));
+  const uint64_t off_begin = off_groups + align256(groups.size() * sizeof(GroupEntry));
+  const uint64_t off_status = off_begin + align256(tile_begin.size() * 4);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int rc = tq_cuda_status((int)cudaMemcpyAsync(base, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, st), "gemm plan upload");
+  if (rc == TQ_OK)
+    rc = tq_cuda_status((int)cudaMemcpyAsync(base + off_groups, groups.data(), groups.size() * sizeof(GroupEntry), cudaMemcpyHostToDevice, st), "gemm plan upload");
+  if (rc == TQ_OK)
+    rc = tq_cuda_status((int)cudaMemcpyAsync(base + off_begin, tile_begin.data(), tile_begin.size() * 4, cudaMemcpyHostToDevice, st), "gemm plan upload");
+  if (rc == TQ_OK) rc = tq_cuda_status((int)cudaMemsetAsync(base + off_status, 0, 256, st), "gemm plan upload");
+  if (rc == TQ_OK) rc = tq_cuda_status((int)cudaStreamSynchronize(st), "gemm plan upload");  // the host vectors go away
+  if (rc != TQ_OK) {
+    delete pl;
+    return rc;
+  }
+  pl->src.maps = reinterpret_cast<const CUtensorMap*>(base);
+  pl->src.groups = reinterpret_cast<const GroupEntry*>(base + off_groups);
+  pl->src.tile_begin = reinterpret_cast<const uint32_t*>(base + off_begin);
+  pl->src.status_word = reinterpret_cast<uint32_t*>(base + off_status);
+  pl->src.n_groups = (uint32_t)n_mats;
+  pl->src.token_tiles = token_tiles;
+  pl->src.n_tokens = (uint32_t)M;
+  pl->src.n_tiles = (uint32_t)tiles;
+  pl->bn = bn;
+  pl->grid = std::min<uint32_t>((uint32_t)tiles, (uint32_t)sm_count());
+  *out = pl;
+  return TQ_OK;
+}
+
+int tq_gemm_plan_run(const tq_gemm_plan* pl, void* cuda_stream) {
+  if (!pl) return TQ_ERR_INVALID_ARG;
+  if (pl->bn == 128u)
+    gemm_ws_group_kernel<128><<<pl->grid, kThreads, Geo<128>::SMEM_BYTES, (cudaStream_t)cuda_stream>>>(pl->src);
+  else
+    gemm_ws_group_kernel<256><<<pl->grid, kThreads, Geo<256>::SMEM_BYTES, (cudaStream_t)cuda_stream>>>(pl->src);
+  return tq_cuda_status((int)cudaGetLastError(), "gemm plan launch");
+}
+
+int tq_gemm_plan_status(const tq_gemm_plan* pl, void* cuda_stream, uint32_t* status) {
+  if (!pl || !status) return TQ_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (int rc = tq_cuda_status((int)cudaMemcpyAsync(status, pl->src.status_word, 4, cudaMemcpyDeviceToHost, st), "gemm plan status")) return rc;
+  return tq_cuda_status((int)cudaStreamSynchronize(st), "gemm plan status");
+}
+
+void tq_gemm_plan_free(tq_gemm_plan* pl) { delete pl; }
 
 }  // extern "C"

@@ -280,6 +280,40 @@ def test_fused_gemm_ws_agrees_with_fused_gemv(tq):
     assert float((a - b).abs().max() / b.abs().max()) < 1e-5
 
 
+@pytest.mark.parametrize("M", [5, 130, 600])
+def test_gemm_plan_matches_oracle(tq, M):
+    """Several workspace GEMMs in one persistent launch: matrices of different row and column counts
+    (ragged in both), one table, tiles of all products in one sequence; run twice on the same plan."""
+    shapes = [(200, 512), (128, 1032), (17, 8), (384, 3072), (130, 264)]
+    rng = np.random.default_rng(900 + M)
+    qs = [np.clip(np.rint(rng.standard_t(5, size=sh) * 6), -127, 127).astype(np.int8) for sh in shapes]
+    ss = [(rng.random(sh[0]) + 0.5).astype(np.float32) for sh in shapes]
+    d, streams = _oracle_pack(qs, top_k=3000)
+    hd = tq.tq_dict_from_entries(d.entries)
+    dd = tq.tq_dict_upload(hd)
+    mats = [tq.tq_upload(dd, st, sh[0], sh[1], sc, None, levels_signed=True, layout=2) for st, sh, sc in zip(streams, shapes, ss)]
+    wss = [torch.full((tq.tq_gemm_workspace_size(m),), 0x7F, dtype=torch.uint8, device="cuda") for m in mats]
+    Xs = [synth.activations(M, sh[1], 50 + i) for i, sh in enumerate(shapes)]
+    Xd = [x.cuda() for x in Xs]
+    plan = tq.tq_gemm_plan_create(mats, Xd, wss)
+    stack = tq.tq_stack_create(mats)
+    tq.tq_decode_bf16_stack(stack, wss)
+    for _ in range(2):
+        for y in plan.Ys:
+            y.fill_(float("nan"))
+        tq.tq_gemm_plan_run(plan)
+    assert tq.tq_gemm_plan_status(plan) == 0
+    for q, sc, x, y, m in zip(qs, ss, Xs, plan.Ys, mats):
+        Y = y.cpu().numpy().astype(np.float64)
+        sample = np.arange(M) if M <= 300 else np.sort(rng.choice(M, 64, replace=False))
+        Yref = oracle.layer_forward(q, sc, x[sample].double().numpy())
+        assert Y.shape == (M, q.shape[0]) and np.isfinite(Y).all()
+        assert _rel_err(Y[sample], Yref) <= TOL
+        # and bit for bit what the single-matrix call gives
+        Y1 = tq.tq_gemm_bf16_ws(m, x.cuda(), wss[mats.index(m)])
+        assert torch.equal(Y1, y)
+
+
 # ------------------------------------------------------------------ device-side table build
 @pytest.mark.parametrize("case", ["ties", "several", "minus_one", "odd_lengths", "top_k_small", "large"])
 def test_build_dictionary_device_matches_oracle(tq, case):
