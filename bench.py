@@ -302,25 +302,26 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
         Y = torch.empty(M * max_rows, dtype=torch.float32, device=device)
         Xs = {c: synth.activations(M, c, 99, device=device) for c in sorted({i.cols for i in infos})}
         if args.layout == "tiles":
-            # phase 1 for a whole decoder layer (7 matrices) in one launch, then one tensor-core product per matrix
-            groups = [list(range(i, min(i + 7, len(mats)))) for i in range(0, len(mats), 7)]
+            # phase 1 for a group of decoder layers (7 matrices each) in one launch, then all their tensor-core
+            # products in one persistent launch (tq_gemm_plan: the tiles of all products in one sequence)
+            per_group = 7 * max(1, args.prefill_layers_per_launch)
+            groups = [list(range(i, min(i + per_group, len(mats)))) for i in range(0, len(mats), per_group)]
             n_slots = max(len(g) for g in groups)
             slot_bytes = [max(tq.tq_gemm_workspace_size(mats[g[k]]) for g in groups if k < len(g)) for k in range(n_slots)]
+            slot_rows = [max(mats[g[k]].info.rows for g in groups if k < len(g)) for k in range(n_slots)]
             wsets = [[torch.empty(b, dtype=torch.uint8, device=device) for b in slot_bytes] for _ in range(2)]
+            Yslots = [torch.empty(M * r, dtype=torch.float32, device=device) for r in slot_rows]  # reused by every group
+            del Y
             gstacks = [tq.tq_stack_create([mats[i] for i in g]) for g in groups]
+            plans = [tq.tq_gemm_plan_create([mats[i] for i in g], [Xs[mats[i].info.cols] for i in g], wsets[gi % 2][: len(g)],
+                                            [Yslots[k][: M * mats[i].info.rows].view(M, mats[i].info.rows) for k, i in enumerate(g)])
+                     for gi, g in enumerate(groups)]
 
-            # Weights do not depend on activations, so the decode of group g + 1 (HBM-bound) runs on a
-            # stream of its own while the products of group g (tensor-bound) run: two workspace sets
-            # alternate.  The products of one group do not depend on one another either (as q/k/v or
-            # gate/up of a decoder layer do not): they are spread over three streams so that a product
-            # whose tiles do not fill the SMs shares them with the next; each stream has its own output
-            # buffer.
-            lanes = [stream, torch.cuda.Stream(device), torch.cuda.Stream(device)]
+            # Weights do not depend on activations, so the decode of group g + 1 runs on a stream of its
+            # own, ahead of the products of group g: two workspace sets alternate.
             dec_stream = torch.cuda.Stream(device)
-            Ys = [Y] + [torch.empty_like(Y) for _ in lanes[1:]]
             ev_dec = [torch.cuda.Event() for _ in groups]
             ev_used = [torch.cuda.Event() for _ in groups]   # the products of a group have read its workspaces
-            ev_lane = [torch.cuda.Event() for _ in lanes[1:]]
             ev_start, ev_end = torch.cuda.Event(), torch.cuda.Event()
 
             def run_gemm():
@@ -331,17 +332,8 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
                         dec_stream.wait_event(ev_used[gi - 2])
                     tq.tq_decode_bf16_stack(st, wsets[gi % 2][: len(g)], stream=dec_stream)
                     ev_dec[gi].record(dec_stream)
-                for gi, g in enumerate(groups):
-                    for ln in lanes:
-                        ln.wait_event(ev_dec[gi])
-                    for k, i in enumerate(g):
-                        m = mats[i]
-                        ln = k % len(lanes)
-                        tq.tq_gemm_bf16_ws(m, Xs[m.info.cols], wsets[gi % 2][k], Ys[ln][: M * m.info.rows].view(M, m.info.rows),
-                                           stream=lanes[ln])
-                    for ln, ev in zip(lanes[1:], ev_lane):
-                        ev.record(ln)
-                        stream.wait_event(ev)
+                    stream.wait_event(ev_dec[gi])
+                    tq.tq_gemm_plan_run(plans[gi], stream=stream)
                     ev_used[gi].record(stream)
                 ev_end.record(dec_stream)
                 stream.wait_event(ev_end)
@@ -355,12 +347,15 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
         pk = float(peaks.get("bf16_tflops_sustained", 1400.0))
         out["prefill"] = {"tokens": M, "ms": ms,
-                          "call": "tq_decode_bf16_stack per 7 matrices (one decoder layer) + tq_gemm_bf16_ws per matrix (TMA-fed tcgen05 GEMM)" if args.layout == "tiles"
+                          "call": ("tq_decode_bf16_stack + tq_gemm_plan_run (TMA-fed tcgen05 GEMM over all products of the group) per %d decoder layer(s)" % max(1, args.prefill_layers_per_launch)) if args.layout == "tiles"
                           else "tq_fused_gemm (decode inside the GEMM)", "TFLOP_per_s": flops / (ms * 1e-3) / 1e12,
                           "frac_of_measured_bf16_sustained": flops / (ms * 1e-3) / 1e12 / pk, "peak_TFLOP_per_s": pk}
         status = 0
         for m in mats:
             status |= tq.tq_device_status(m)
+        if args.layout == "tiles":
+            for pl in plans:
+                status |= tq.tq_gemm_plan_status(pl)
         assert status == 0, f"device status {status}"
     return out
 
@@ -397,6 +392,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the tq_decompress / tq_fused_gemm timings")
     ap.add_argument("--prefill-tokens", type=int, default=2048)
+    ap.add_argument("--prefill-layers-per-launch", type=int, default=14, help="decoder layers per decode + GEMM launch pair of the prefill leg")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
