@@ -107,6 +107,7 @@ class ClockSampler:
 # summarised under profiles/ (None: not captured for that launch shape, or kernel changed since).
 # tiles_stack: 213.1 MB read + 3.7 MB written for 207.7 MB of algorithmic bytes on a 14-matrix stack (2 decoder
 # layers), i.e. 1.044 x; traffic grows with the bytes streamed, so the 3B launch (3.333 GB) is scaled by that ratio.
+L2_BYTES = 126 << 20
 TRAFFIC_RATIO = {"tiles_stack": 1.044}
 TRAFFIC = {}
 # the arithmetic each layout's product kernel computes in
@@ -505,6 +506,20 @@ def main():
             run_step()
         ev1.record(stream)
         stream.synchronize()
+        ms_flushed = None
+        if payload_bytes < 2 * L2_BYTES:
+            # a workload that fits L2 would be read from L2 from the second step on: write a buffer larger
+            # than L2 between steps and time every step on its own
+            flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+            pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+            for a, b in pairs:
+                flush.zero_()
+                a.record(stream)
+                run_step()
+                b.record(stream)
+            stream.synchronize()
+            ms_flushed = sum(a.elapsed_time(b) for a, b in pairs)
+            del flush
         torch.cuda.synchronize()
         t_end = time.time()
         barrier()
@@ -517,7 +532,8 @@ def main():
             t_end = time.time()
         clocks = sampler.stop(t_start, t_end)
         clocks["sampled_over"] = "timed region" if not extended else "timed region plus identical untimed steps"
-        ms_total = ev0.elapsed_time(ev1)
+        ms_unflushed = ev0.elapsed_time(ev1) / args.steps
+        ms_total = ev0.elapsed_time(ev1) if ms_flushed is None else ms_flushed
 
         status = 0
         for m in mats:
@@ -598,7 +614,10 @@ def main():
                               "tiles": "1 KB token tiles of 16 rows x 32 groups in integer-MMA operand order + one raw-word stream; "
                                        "table limited to the %d words shared memory holds" % tq.TQ_TILES_TABLE_WORDS}[args.layout],
                    "cuda_graph": graph is not None,
-                   "l2": "inputs larger than L2: each step streams %.2f GB" % (payload_bytes / 1e9),
+                   "l2": ("inputs larger than L2: each step streams %.2f GB" % (payload_bytes / 1e9) if ms_flushed is None else
+                          "L2 flushed between steps (a %d MB buffer written), every step timed on its own; back to back without "
+                          "the flush a step takes %.5f ms (%.1f MB served from L2)"
+                          % (2 * L2_BYTES >> 20, ms_unflushed, payload_bytes / 1e6)),
                    "multi_gpu": "independent replicas, no data-path collective" if world > 1 else "single GPU"},
         "us_per_token": ms_step * 1e3 / args.batch,
         "bytes_per_step": {"algorithmic": alg_bytes, "paper_stream": stream_bytes, "device_payload": payload_bytes,
