@@ -393,15 +393,16 @@ struct TilesCta : CtaBase {
       rd = rd_next;
       return true;
     };
-    auto refill = [&]() {
+    auto refill = [&](bool prefetch) {
       // every lane has issued its reads of the chunks below rd; the warp barrier orders them before
       // the copies that overwrite those chunks
       __syncwarp();
       const uint32_t lim = min(stop_pos, (rd & ~(uint32_t)(kChunkWords - 1)) + kRingWords);
       for (; i_pos < lim; i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
-      // the token tile kL2Ahead tiles further on: brought into L2 now, so that the register load two
-      // tiles ahead of its use finds it there (tok already points two tiles ahead)
-      if (lane == 0 && tok + (kL2Ahead - 2) * 64 < tok_end) bulk_prefetch_l2(tok + (kL2Ahead - 2) * 64, 1024u);
+      // the two token tiles kL2Ahead tiles further on (every other tile): brought into L2 now, so that
+      // the register loads two tiles ahead of their use find them there (tok already points two tiles
+      // ahead; a prefetch that runs past the run's end stays inside the padding of the token array)
+      if (prefetch && lane == 0 && tok + (kL2Ahead - 2) * 64 < tok_end) bulk_prefetch_l2(tok + (kL2Ahead - 2) * 64, 2048u);
     };
     auto consume = [&](const uint32_t (&wc)[16]) {
       uint4 xa, xb;
@@ -432,17 +433,17 @@ struct TilesCta : CtaBase {
 
     const uint32_t n = t1 - t0;
     bool ok = lookups(0);
-    if (ok) refill();
+    if (ok) refill(true);
     uint32_t i = 1;
     for (; ok && i + 1 < n; i += 2) {
       ok = lookups(1);
       if (!ok) break;
       consume(wbuf[0]);
-      refill();
+      refill(false);
       ok = lookups(0);
       if (!ok) break;
       consume(wbuf[1]);
-      refill();
+      refill(true);
     }
     if (ok && i < n) {
       ok = lookups(1);
