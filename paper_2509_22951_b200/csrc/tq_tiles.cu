@@ -231,9 +231,20 @@ struct CtaBase {
     const uint32_t R[8] = {q[0].x, q[0].y, q[0].z, q[0].w, q[1].x, q[1].y, q[1].z, q[1].w};
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const uint32_t lo4 = (R[i] << 2) & 0x3FFFCu, hi4 = (R[i] >> 14) & 0x3FFFCu;  // token * 4
-      w[2 * i] = lds_u32(lo4 + (lo4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
-      w[2 * i + 1] = lds_u32(hi4 + (hi4 >= 4u * kMissBase ? miss_adj4 : tbl_addr));
+      asm volatile(
+          "{\n\t.reg .pred p0, p1;\n\t.reg .u32 t0, t1, b0, b1, a0, a1;\n\t"
+          "and.b32 t0, %2, 0xFFFF;\n\t"
+          "shr.u32 t1, %2, 16;\n\t"
+          "setp.ge.u32 p0, t0, 64512;\n\t"
+          "setp.ge.u32 p1, t1, 64512;\n\t"
+          "selp.u32 b0, %4, %3, p0;\n\t"
+          "selp.u32 b1, %4, %3, p1;\n\t"
+          "mad.lo.u32 a0, t0, 4, b0;\n\t"
+          "mad.lo.u32 a1, t1, 4, b1;\n\t"
+          "ld.shared.u32 %0, [a0];\n\t"
+          "ld.shared.u32 %1, [a1];\n\t}"
+          : "=r"(w[2 * i]), "=r"(w[2 * i + 1])
+          : "r"(R[i]), "r"(tbl_addr), "r"(miss_adj4));
     }
   }
 };
