@@ -18,7 +18,7 @@
 // memory: lookups there are bank-conflict limited, not tag limited like divergent global loads.
 // Each warp walks a contiguous run of tiles.  Token tiles come through registers, two tiles
 // ahead.  Raw words come through a per-warp ring of TQ_TILES_RING_WORDS words in shared memory
-// that one lane keeps filled with 1 KB bulk copies (cp.async.bulk + mbarrier); raw word p of
+// that one lane keeps filled with 2 KB bulk copies (cp.async.bulk + mbarrier); raw word p of
 // the matrix always sits in ring slot p mod ring size, and that slot number is what a miss token
 // carries, so a lookup is: token -> (token >= 0xFC00 ? ring : table)[token] -> MMA operand.
 #include <cuda_bf16.h>
@@ -38,12 +38,12 @@ using namespace tq_sm100;
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kRingWords = TQ_TILES_RING_WORDS;     // 4 KB per warp
-constexpr int kChunkWords = 256;                    // one bulk copy: 1 KB of raw words
+constexpr int kChunkWords = 512;                    // one bulk copy: 2 KB of raw words
 constexpr int kSlots = kRingWords / kChunkWords;    // chunks per ring
 constexpr int kL2Ahead = 8;                         // token tiles prefetched into L2 ahead of their use (<= 8: padding)
 constexpr uint32_t kNoBlock = 0xFFFFFFFFu;
 constexpr uint32_t kMissBase = 0x10000u - TQ_TILES_RING_WORDS;  // first miss token
-static_assert(kSlots == 4 && (kRingWords & (kRingWords - 1)) == 0, "ring geometry");
+static_assert(kSlots == 2 && (kRingWords & (kRingWords - 1)) == 0 && kRingWords - kChunkWords >= 512, "ring geometry: a tile has up to 512 raw words");
 
 __host__ __device__ inline uint32_t align_up_u32(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 
@@ -166,10 +166,11 @@ __device__ __noinline__ void tiles_finalize(const float* __restrict__ scale, con
 
 // What every CTA of these kernels carries: the shared-memory plan, the table and this warp's raw ring.
 //
-// Raw ring: chunk c of a matrix's raw stream (words 256c .. 256c+255) always lands at ring offset
-// (c mod 4) KB, the place its tokens point to.  The barriers are used round robin in issue order,
-// which is also the order of the waits: use number n takes barrier n mod 4 and completes its phase
-// (n / 4) mod 2.
+// Raw ring: chunk c of a matrix's raw stream (words 512c .. 512c+511) always lands in half c mod 2
+// of the ring, the place its tokens point to.  A tile has at most 512 raw words, so the two chunks in
+// flight always cover the tile being looked up.  The barriers are used round robin in issue order,
+// which is also the order of the waits: use number n takes barrier n mod 2 and completes its phase
+// (n / 2) mod 2.
 struct CtaBase {
   uint8_t* smem;
   TilesSmem L;
@@ -219,7 +220,7 @@ struct CtaBase {
   }
   __device__ __forceinline__ bool wait_chunk() {
     const uint32_t bar = bar_base + (n_waited & (kSlots - 1u)) * 8u;
-    const uint32_t par = (n_waited >> 2) & 1u;
+    const uint32_t par = (n_waited / kSlots) & 1u;
     ++n_waited;
     if (__all_sync(kFull, mbar_try(bar, par))) return true;  // one answer per warp: the slow path votes too
     return tiles_wait_slow(bar, par, dead_flag());
