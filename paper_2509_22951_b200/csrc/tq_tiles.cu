@@ -84,11 +84,6 @@ __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
                : "l"(p));
   return v;
 }
-__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
-  uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
-}
 
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
@@ -913,7 +908,7 @@ constexpr uint32_t kSmemLimit = 232448u;  // 227 KB per CTA
 
 // ---------------------------------------------------------------------------------------------
 // Decompress for large inputs: the data path of the GEMV kernel (table in shared memory, raw words
-// through the ring, two-tile register pipeline) with the MMAs replaced by 32-byte stores.  A lane
+// through the ring, two-tile register pipeline, no L2 prefetch) with the MMAs replaced by 32-byte stores.  A lane
 // holds, per tile and half, the 8 words of one row = 32 consecutive bytes of the output row; the 4
 // lanes of a quad cover 128 consecutive bytes.
 // ---------------------------------------------------------------------------------------------
@@ -952,7 +947,6 @@ struct DecompCta : CtaBase {
     uint32_t w_pos = rd & ~(uint32_t)(kChunkWords - 1), i_pos = w_pos;
     for (int k = 0; k < kSlots && i_pos < stop_pos; ++k, i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
     const uint4* tok = d.tokens + (size_t)t0 * 64u + lane;
-    const uint4* tok_end = d.tokens + (size_t)t1 * 64u;
     const uint32_t* trp = d.tile_raw + t0 + 1;
     uint4 q[2][2];
     uint32_t tr[2];
@@ -1049,7 +1043,8 @@ struct DecompCta : CtaBase {
       __syncwarp();
       const uint32_t lim = min(stop_pos, (rd & ~(uint32_t)(kChunkWords - 1)) + kRingWords);
       for (; i_pos < lim; i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
-      if (lane == 0 && tok + (kL2Ahead - 2) * 64 < tok_end) bulk_prefetch_l2(tok + (kL2Ahead - 2) * 64, 1024u);
+      // no L2 prefetch of the tokens here: with as many bytes written as read it was measured to cost
+      // 5 % (prefetched lines are pushed out by the stores before their use)
     };
 
     for (uint32_t i = t0; i < t1 && ok; i += 2) {
