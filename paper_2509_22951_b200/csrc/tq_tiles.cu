@@ -729,7 +729,6 @@ struct PanelCta : CtaBase {
 
     uint32_t rd = 0, stop_pos = 0, w_pos = 0, i_pos = 0;
     const uint4* tok = d.tokens + (size_t)t0 * 64u + lane;
-    const uint4* tok_end = d.tokens + (size_t)t1 * 64u;
     const uint32_t* trp = d.tile_raw + t0 + 1;
     uint4 q[2][2] = {};
     uint32_t tr[2] = {0, 0};
@@ -773,7 +772,6 @@ struct PanelCta : CtaBase {
       __syncwarp();
       const uint32_t lim = min(stop_pos, (rd & ~(uint32_t)(kChunkWords - 1)) + kRingWords);
       for (; i_pos < lim; i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
-      if (lane == 0 && tok + (kL2Ahead - 2) * 64 < tok_end) bulk_prefetch_l2(tok + (kL2Ahead - 2) * 64, 1024u);
     };
     // MMAs of one tile (real == false: the warp has no tile in this iteration but keeps step with the others)
     auto consume = [&](const uint32_t (&wc)[16], bool real) {
