@@ -111,7 +111,7 @@ L2_BYTES = 126 << 20
 TRAFFIC_RATIO = {"tiles_stack": 1.053}
 TRAFFIC = {}
 # the arithmetic each layout's product kernel computes in
-DTYPE = {"tiles": "s8 x s8 -> s32 (int8 levels x three base-256 digits of block-fixed-point bf16 activations, "
+DTYPE = {"tiles": "s8 x s8 -> s32 (int8 levels x four base-256 digits of block-fixed-point bf16 activations, "
                   "exact integer tensor-core sums, fp64 epilogue)",
          "planes": "int8 weights x bf16 activations, fp32 accumulate",
          "stream": "int8 weights x bf16 activations, fp32 accumulate"}

@@ -155,8 +155,8 @@ void tq_ddict_free(tq_ddict* d); /* host handle only */
                               (marker + its 4 bytes), i.e. the image is the stream Listing 3 produces with
                               top_k = TQ_TILES_TABLE_WORDS - 1.  Same decoded bytes, 4 more bytes per such
                               group (tq_dmat_info.n_raw_words counts them). */
-#define TQ_TILES_TABLE_WORDS 34816u
-#define TQ_TILES_MAX_COLS 65536u /* 32-bit integer accumulators; rows of more than 8704 columns go through the
+#define TQ_TILES_TABLE_WORDS 33024u
+#define TQ_TILES_MAX_COLS 65536u /* 32-bit integer accumulators; rows of more than 8448 columns go through the
                                     column-panel kernel, whose shared memory need does not grow with the row */
 #define TQ_TILES_RING_WORDS 1024u /* a miss token of the image is 0xFC00 + (index of its raw word mod 1024) */
 
@@ -221,8 +221,20 @@ int tq_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream);
 /* Compressed linear layer for small batches (Section 2.3: weights are expanded layer by layer,
  * then used as an ordinary linear layer; here the expansion, Listing 1's scale*(q-zero) and the
  * product are one kernel and the weights never reach memory):
- *   y[b][r] = scale_r * sum_c (q[r][c] - zero_r) * x[b][c],   fp32 accumulation.
- * d_x_bf16: DEVICE [B][cols] bf16, 16-byte aligned; B in 1..32; d_y: DEVICE [B][rows] fp32. */
+ *   y[b][r] = scale_r * sum_c (q[r][c] - zero_r) * x[b][c].
+ * d_x_bf16: DEVICE [B][cols] bf16, 16-byte aligned; B in 1..32; d_y: DEVICE [B][rows] fp32.
+ *
+ * Arithmetic and its domain.  TQ_LAYOUT_STREAM / TQ_LAYOUT_PLANES: exact int8 x bf16 products,
+ * fp32 accumulation.  TQ_LAYOUT_TILES: each vector x[b] is put on a fixed-point grid 30 bits below
+ * the power of two above its largest magnitude (X = round(x * 2^(30-e)), max |x[b]| < 2^e) and the
+ * sums are exact integers, so the result does not depend on how the work is split and
+ *   |y[b][r] - exact| <= scale_r * 2^(e-31) * sum_c |q[r][c] - zero_r|   (+ one fp32 rounding of y).
+ * An element keeps every bit of its bf16 value while it is at most 2^22 times smaller than the
+ * largest element of its vector; smaller ones are rounded to the grid.  Against max_r |y[b][r]| this
+ * is far inside 2e-3 unless the row sums rest on elements more than about 2^20 times smaller than one
+ * that meets (near-)zero weights.  Subnormal and smallest-normal bf16 inputs are exact.  A vector with
+ * an Inf or NaN element yields NaN for all of its outputs (other vectors are unaffected); the status
+ * word is not touched. */
 int tq_fused_gemv(const tq_dmat* m, const void* d_x_bf16, int B, float* d_y, void* cuda_stream);
 
 /* The same call with HOST operands: copies x to the DEVICE staging buffer d_x_stage ([B][cols]
@@ -243,8 +255,9 @@ int tq_fused_gemv_host(const tq_dmat* m, const void* h_x_bf16, int B, float* h_y
  * address with that device current; make that first call outside any stream capture.  All calls
  * on a device share the one array: nothing in it has to start at zero (x is overwritten by the
  * copy, y by the kernel, before either is read), but two calls whose GPU work overlaps (different
- * streams, or different threads) race on it -- serialise them.  h_x_bf16, h_y: HOST, as for
- * tq_fused_gemv_host; asynchronous on cuda_stream. */
+ * streams, or different threads) race on it -- serialise them.  The array that is used is the
+ * current device's, so the device the matrix lives on must be current: TQ_ERR_INVALID_ARG otherwise.
+ * h_x_bf16, h_y: HOST, as for tq_fused_gemv_host; asynchronous on cuda_stream. */
 int tq_fused_gemv_host_static(const tq_dmat* m, const void* h_x_bf16, int B, float* h_y,
                               void* cuda_stream);
 
@@ -257,7 +270,9 @@ int tq_fused_gemm(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, voi
 /* The prefill-sized product for a TQ_LAYOUT_TILES matrix, in two phases on cuda_stream that share a
  * caller-provided DEVICE workspace (256-byte aligned, tq_gemm_workspace_size bytes = the matrix as
  * bf16, padded to whole tiles): the layer is decompressed once into the workspace as bf16
- * (level - zero point: exact for integer zero points), then a persistent tcgen05 GEMM reads both
+ * (level - zero point: exact when every zero point is an integer no further than 256 from any level,
+ * which holds for Listing 1's zero points of tensors that straddle 0; TQ_ERR_UNSUPPORTED_SHAPE for
+ * other zero points, here and in tq_fused_gemm), then a persistent tcgen05 GEMM reads both
  * operands by TMA and applies the row scale in fp32.  Same result definition, argument layout and
  * alignment as tq_fused_gemm; the workspace may be reused by the next call on the same stream. */
 int tq_gemm_workspace_size(const tq_dmat* m, uint64_t* bytes);
@@ -277,8 +292,7 @@ int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, c
  * then streams its share of the row blocks of all the matrices.  The products are independent of
  * one another: a caller whose layers feed each other makes one stack per group of layers that can
  * run together (q/k/v; gate/up; ...).  d_x[i]: DEVICE bf16 [B][cols_i], 16-byte aligned; d_y[i]:
- * DEVICE fp32 [B][rows_i]; B in 1..32 (one launch per two batch columns, or per column when the
- * widest matrix leaves no room for two).  mats, d_x, d_y: HOST arrays of n_mats entries.  The
+ * DEVICE fp32 [B][rows_i]; B in 1..32 (tq_stack_launches tells how many kernel launches a call makes).  mats, d_x, d_y: HOST arrays of n_mats entries.  The
  * work split and the operand addresses are written to the caller's DEVICE buffer d_buf (256-byte
  * aligned, tq_stack_size bytes), which must outlive the handle, as must the matrices.
  * TQ_ERR_UNSUPPORTED_SHAPE if the matrices do not share table, level type and layout.

@@ -25,7 +25,7 @@ TQ_ERR_NOMEM = -7
 TQ_LAYOUT_STREAM = 0
 TQ_LAYOUT_PLANES = 1
 TQ_LAYOUT_TILES = 2
-TQ_TILES_TABLE_WORDS = 34816
+TQ_TILES_TABLE_WORDS = 33024
 TQ_TILES_MAX_COLS = 65536
 TQ_STATUS_BAD_CODE = 1
 TQ_STATUS_BAD_ROW = 2

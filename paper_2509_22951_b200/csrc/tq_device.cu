@@ -14,7 +14,9 @@
 
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <mutex>
+#include <utility>
 #include <new>
 
 #include "tq_internal.h"
@@ -484,12 +486,9 @@ template <int NB>
 int launch_gemv(const tq_dmat* m, const __nv_bfloat16* x, float* y, cudaStream_t st) {
   const uint32_t rows = m->info.rows, cols = m->info.cols;
   const size_t smem = (size_t)NB * cols * sizeof(float);
-  static size_t configured = 0;
-  if (smem + 20 * 1024 > 48 * 1024 && smem > configured) {  // static shared memory counts too
-    if (int rc = cuda_ok(cudaFuncSetAttribute(gemv_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
-                         "gemv: raising the dynamic shared memory limit"))
+  if (smem + 20 * 1024 > 48 * 1024) {  // static shared memory counts too
+    if (int rc = tq_ensure_dynamic_smem((const void*)gemv_kernel<NB>, smem, "gemv: raising the dynamic shared memory limit"))
       return rc;
-    configured = smem;
   }
   int per_sm = 0;
   if (int rc = cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gemv_kernel<NB>, kThreads, smem),
@@ -513,12 +512,9 @@ int launch_gemv_planes(const tq_dmat* m, const __nv_bfloat16* x, float* y, cudaS
   const uint32_t rows = m->info.rows, cols = m->info.cols;
   const size_t slots = ((size_t)(m->gpr_pad + 255u) >> 8) << 8;
   const size_t smem = (size_t)NB * slots * sizeof(float4);
-  static size_t configured = 0;
-  if (smem + 4 * 1024 > 48 * 1024 && smem > configured) {
-    if (int rc = cuda_ok(cudaFuncSetAttribute(gemv_planes_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
-                         "gemv(planes): raising the dynamic shared memory limit"))
+  if (smem + 4 * 1024 > 48 * 1024) {
+    if (int rc = tq_ensure_dynamic_smem((const void*)gemv_planes_kernel<NB>, smem, "gemv(planes): raising the dynamic shared memory limit"))
       return rc;
-    configured = smem;
   }
   int per_sm = 0;
   if (int rc = cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gemv_planes_kernel<NB>, kThreads, smem),
@@ -540,6 +536,20 @@ int launch_gemv_planes(const tq_dmat* m, const __nv_bfloat16* x, float* y, cudaS
 }  // namespace
 
 int tq_cuda_status(int cuda_error, const char* what) { return cuda_ok((cudaError_t)cuda_error, what); }
+
+int tq_ensure_dynamic_smem(const void* func, size_t bytes, const char* what) {
+  static std::mutex mu;
+  static std::map<std::pair<int, const void*>, size_t> raised;  // (device, kernel) -> limit set so far
+  int dev = 0;
+  if (int rc = cuda_ok(cudaGetDevice(&dev), what)) return rc;
+  std::lock_guard<std::mutex> lock(mu);
+  size_t& have = raised[std::make_pair(dev, func)];
+  if (bytes > have) {
+    if (int rc = cuda_ok(cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes), what)) return rc;
+    have = bytes;
+  }
+  return TQ_OK;
+}
 
 extern "C" {
 
@@ -689,6 +699,7 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
   }
   m->dict = dict;
   m->has_zero = row_zero != nullptr;
+  m->zero_bf16_exact = tq_zero_bf16_exact(row_zero, rows, levels_signed != 0);
   m->info.rows = rows;
   m->info.cols = cols;
   m->info.K = dict->K;
@@ -727,13 +738,17 @@ int tq_upload_device(const tq_ddict* dict, const uint8_t* d_levels, uint32_t row
   tq_dmat* m = new (std::nothrow) tq_dmat();
   if (!m) return TQ_ERR_NOMEM;
   std::vector<uint32_t> tile_raw;
+  std::vector<float> zeros;
   unsigned long long counters[2] = {0, 0};
   int rc = TQ_OK;
   try {
     tile_raw.resize(geo.n_tiles + 1);
+    if (d_row_zero) zeros.resize(rows);
   } catch (const std::bad_alloc&) {
     rc = TQ_ERR_NOMEM;
   }
+  if (rc == TQ_OK && d_row_zero)
+    rc = cuda_ok(cudaMemcpyAsync(zeros.data(), d_row_zero, (size_t)rows * 4, cudaMemcpyDeviceToHost, st), "device upload");
   if (rc == TQ_OK)
     rc = cuda_ok(cudaMemcpyAsync(tile_raw.data(), base + geo.off_tile_raw, tile_raw.size() * 4, cudaMemcpyDeviceToHost, st), "device upload");
   if (rc == TQ_OK) rc = cuda_ok(cudaMemcpyAsync(counters, base + 64, sizeof(counters), cudaMemcpyDeviceToHost, st), "device upload");
@@ -747,6 +762,7 @@ int tq_upload_device(const tq_ddict* dict, const uint8_t* d_levels, uint32_t row
   for (uint32_t rb = 0; rb <= geo.row_blocks; ++rb) m->rb_raw[rb] = tile_raw[(uint64_t)rb * geo.steps];
   m->dict = dict;
   m->has_zero = d_row_zero != nullptr;
+  m->zero_bf16_exact = tq_zero_bf16_exact(d_row_zero ? zeros.data() : nullptr, rows, levels_signed != 0);
   m->d_status = reinterpret_cast<uint32_t*>(base + geo.off_status);
   m->d_scale = reinterpret_cast<const float*>(base + geo.off_scale);
   m->d_zero = reinterpret_cast<const float*>(base + geo.off_zero);
@@ -879,6 +895,17 @@ int tq_fused_gemv_host_static(const tq_dmat* m, const void* h_x_bf16, int B, flo
              (unsigned long long)B * m->info.cols, (unsigned long long)kStaticXElems,
              (unsigned long long)B * m->info.rows, (unsigned long long)kStaticYElems);
     return TQ_ERR_UNSUPPORTED_SHAPE;
+  }
+  // The staging array that is looked up belongs to the current device; the kernel runs where the
+  // matrix lives.  A caller who has another device current would hand the kernel that device's address.
+  int dev = -1;
+  cudaPointerAttributes attr{};
+  if (int rc = cuda_ok(cudaGetDevice(&dev), "static staging: current device")) return rc;
+  if (int rc = cuda_ok(cudaPointerGetAttributes(&attr, m->d_status), "static staging: device of the matrix")) return rc;
+  if (attr.type != cudaMemoryTypeDevice || attr.device != dev) {
+    snprintf(g_cuda_msg, sizeof(g_cuda_msg),
+             "tq_fused_gemv_host_static: the matrix lives on device %d but device %d is current", attr.device, dev);
+    return TQ_ERR_INVALID_ARG;
   }
   unsigned char* stage = nullptr;
   if (int rc = static_stage(&stage)) return rc;

@@ -236,6 +236,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
 extern "C" int tq_fused_gemm(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, void* cuda_stream) {
   if (!m || !d_X_bf16 || !d_Y || M < 1 || ((uintptr_t)d_X_bf16 & 15)) return TQ_ERR_INVALID_ARG;
   if (m->info.layout != TQ_LAYOUT_PLANES) return TQ_ERR_UNSUPPORTED_SHAPE;  // needs the fixed-stride token plane
+  if (!m->zero_bf16_exact) return TQ_ERR_UNSUPPORTED_SHAPE;                 // level - zero point would be rounded to bf16
   if ((m->info.cols * 2u) % 16u != 0) return TQ_ERR_UNSUPPORTED_SHAPE;     // TMA row pitch must be a multiple of 16 bytes
   EncodeTiledFn enc = encode_fn();
   if (!enc) return tq_cuda_status((int)cudaErrorUnknown, "gemm: cuTensorMapEncodeTiled not available");
@@ -250,13 +251,7 @@ extern "C" int tq_fused_gemm(const tq_dmat* m, const void* d_X_bf16, int M, floa
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS) return tq_cuda_status((int)cudaErrorInvalidValue, "gemm: tensor map encode failed");
 
-  static bool configured = false;
-  if (!configured) {
-    if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES),
-                                "gemm: raising the dynamic shared memory limit"))
-      return rc;
-    configured = true;
-  }
+  if (int rc = tq_ensure_dynamic_smem((const void*)gemm_kernel, SMEM_BYTES, "gemm: raising the dynamic shared memory limit")) return rc;
   GemmParams p;
   p.codes = m->d_codes;
   p.rawbase = m->d_rawbase;

@@ -342,16 +342,11 @@ int encode_maps(const tq_dmat* m, const void* d_workspace, const void* d_X_bf16,
 }
 
 int configure_gemm_kernels() {
-  static bool configured = false;
-  if (configured) return TQ_OK;
   const void* kerns[4] = {(const void*)gemm_ws_kernel<256>, (const void*)gemm_ws_kernel<128>, (const void*)gemm_ws_group_kernel<256>,
                           (const void*)gemm_ws_group_kernel<128>};
   const int smem[4] = {(int)Geo<256>::SMEM_BYTES, (int)Geo<128>::SMEM_BYTES, (int)Geo<256>::SMEM_BYTES, (int)Geo<128>::SMEM_BYTES};
   for (int i = 0; i < 4; ++i)
-    if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(kerns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, smem[i]),
-                                "gemm: raising the dynamic shared memory limit"))
-      return rc;
-  configured = true;
+    if (int rc = tq_ensure_dynamic_smem(kerns[i], (size_t)smem[i], "gemm: raising the dynamic shared memory limit")) return rc;
   return TQ_OK;
 }
 

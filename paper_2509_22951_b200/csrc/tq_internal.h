@@ -71,6 +71,9 @@ struct tq_dmat {
   const uint16_t* d_tokens = nullptr;  // DEVICE: token area, 256-byte aligned (STREAM layout)
   uint64_t token_chunks = 0;           // token area length in 16-byte units
   int has_zero = 0;
+  // every level - zero point is an integer of magnitude <= 256, i.e. exact as bf16 (what the workspace
+  // GEMM stores); false for zero points that are fractional or far outside the level range
+  bool zero_bf16_exact = true;
   // PLANES layout
   const uint32_t* d_rawbase = nullptr; // DEVICE: rows + 1, index of each row's first raw word
   const uint16_t* d_rawidx = nullptr;  // DEVICE: rows x nidx_pad, markers before group 32*c of the row
@@ -133,8 +136,25 @@ struct tq_tiles_image {
 
 int tq_num_threads();
 
+// True if level - zero is an integer of magnitude <= 256 for every level of the given kind and every
+// zero point of the list (zero == nullptr: no zero points).
+inline bool tq_zero_bf16_exact(const float* zero, uint32_t rows, bool levels_signed) {
+  if (!zero) return true;
+  const float lo = levels_signed ? -128.f : 0.f, hi = levels_signed ? 127.f : 255.f;
+  for (uint32_t r = 0; r < rows; ++r) {
+    const float z = zero[r];
+    if (!(z == (float)(int)z) || hi - z > 256.f || z - lo > 256.f) return false;
+  }
+  return true;
+}
+
 // Maps a cudaError_t (passed as int) to TQ_OK / TQ_ERR_CUDA and records its text for tq_last_cuda_error.
 int tq_cuda_status(int cuda_error, const char* what);
+
+// Raises a kernel's limit of dynamic shared memory to `bytes` on the current device, once per device
+// and kernel (the attribute belongs to the device the call is made on); safe to call from several
+// host threads.  func: the kernel's host-side address.
+int tq_ensure_dynamic_smem(const void* func, size_t bytes, const char* what);
 
 // Validates the stream and computes the layout size; if img != nullptr also builds the image.
 // K == 0xFFFFFFFF skips the code-range check (size query without a table).
@@ -169,6 +189,7 @@ struct tq_stack_plan {
 struct tq_stack {
   int n = 0, B = 0;
   int levels_signed = 0;
+  bool zero_bf16_exact = true;  // of every matrix
   uint32_t grid = 0, table_words = 0;
   const uint32_t* d_table = nullptr;
   const tq_tiles_desc* d_descs = nullptr;  // DEVICE

@@ -6,13 +6,15 @@
 // of 8-bit values, 32-bit accumulators).  A warp that owns 16 rows therefore feeds every word it
 // looks up to the tensor core as is: no unpacking, no int->float conversion, no FMA chain.  The
 // activations take the B operand.  A bf16 activation vector is turned, once per CTA, into a
-// block-fixed-point integer X[c] = round(x[c] * 2^(22-e)) (2^e > max |x|, so |X| <= 2^22) and
-// split into three balanced base-256 digits X = d0 + 256 d1 + 65536 d2, each a signed byte; the
-// three digit vectors are three of the eight B columns.  All sums are exact integers, so
-//   y[r] = scale_r * ( 2^(e-22) * (D0 + 256 D1 + 65536 D2) - zero_r * 2^(e-22) * sum_c X[c] )
-// differs from the exact product only by the rounding of x to 22 bits below its largest element
-// (bf16 carries 8), far inside the fp32-accumulation tolerance, and is independent of how the
-// columns are split among warps.  Two batch columns fit one MMA (6 of 8 B columns).
+// block-fixed-point integer X[c] = round(x[c] * 2^(30-e)) (2^e > max |x|, so |X| <= 2^30) and
+// split into four balanced base-256 digits X = d0 + 2^8 d1 + 2^16 d2 + 2^24 d3, each a signed
+// byte; the four digit vectors are four of the eight B columns.  All sums are exact integers, so
+//   y[r] = scale_r * ( 2^(e-30) * (D0 + 2^8 D1 + 2^16 D2 + 2^24 D3) - zero_r * 2^(e-30) * sum_c X[c] )
+// differs from the exact product only by the rounding of x to a grid 30 bits below the power of
+// two above its largest element: |error of the sum for row r| <= 2^(e-31) * sum_c |q[r][c] - zero_r|.
+// An element keeps all 8 significant bits of its bf16 value while it is no more than 2^22 times
+// smaller than the largest one.  The result does not depend on how the columns are split among
+// warps.  Two batch columns fill one MMA (8 of 8 B columns).
 //
 // Data movement.  One persistent CTA per SM keeps the table (TQ_TILES_TABLE_WORDS words) in shared
 // memory: lookups there are bank-conflict limited, not tag limited like divergent global loads.
@@ -42,6 +44,8 @@ constexpr int kChunkWords = 512;                    // one bulk copy: 2 KB of ra
 constexpr int kSlots = kRingWords / kChunkWords;    // chunks per ring
 constexpr int kL2Ahead = 8;                         // token tiles prefetched into L2 ahead of their use (<= 8: padding)
 constexpr uint32_t kNoBlock = 0xFFFFFFFFu;
+constexpr int kDigits = 4;    // signed base-256 digits of a fixed-point activation
+constexpr int kFixBits = 30;  // |X| <= 2^kFixBits
 constexpr uint32_t kMissBase = 0x10000u - TQ_TILES_RING_WORDS;  // first miss token
 static_assert(kSlots == 2 && (kRingWords & (kRingWords - 1)) == 0 && kRingWords - kChunkWords >= 512, "ring geometry: a tile has up to 512 raw words");
 
@@ -100,6 +104,56 @@ __device__ __forceinline__ void table_load_async(uint32_t tbl_addr, uint32_t bar
     bulk_g2s(tbl_addr + off, reinterpret_cast<const uint8_t*>(table) + off, min(8192u, bytes - off), bar);
 }
 
+// ---- activations as block fixed point ------------------------------------------------------
+// A vector whose largest magnitude has the bf16 bit pattern `amax_bits` (sign cleared) satisfies
+// max |x| < 2^e with e = exponent field - 126, and is put on the grid X = round(x * 2^(kFixBits - e)).
+// The power of two spans [2^-98, 2^156], so it is applied as two float factors; both products are
+// exact wherever the result matters (a power of two times a bf16 value).
+struct FixScale {
+  float s1, s2;  // X = round(x * s1 * s2)
+  int e;
+  bool finite;   // false: the vector holds an Inf or a NaN
+};
+__device__ __forceinline__ FixScale fix_scale(uint32_t amax_bits) {
+  FixScale f;
+  f.finite = amax_bits < 0x7F80u;
+  f.e = (int)(min(amax_bits, 0x7F7Fu) >> 7) - 126;  // in [-126, 128]
+  const int k = kFixBits - f.e, k1 = k / 2, k2 = k - k1;
+  f.s1 = __uint_as_float((uint32_t)(127 + k1) << 23);
+  f.s2 = __uint_as_float((uint32_t)(127 + k2) << 23);
+  return f;
+}
+// 2^(e - kFixBits) as a double, built from its exponent field; NaN for a non-finite vector.
+__device__ __forceinline__ double fix_out_scale(const FixScale& f) {
+  return f.finite ? __longlong_as_double((long long)(1023 + f.e - kFixBits) << 52)
+                  : __longlong_as_double(0x7FF8000000000000ll);
+}
+// Largest magnitude of four bf16 values (bit patterns, monotonic; Inf and NaN sort last).
+__device__ __forceinline__ uint32_t amax4(uint2 v, uint32_t m) {
+  const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu;
+  return max(max(m, a0 & 0xFFFFu), max(a0 >> 16, max(a1 & 0xFFFFu, a1 >> 16)));
+}
+// Digits of one activation group (4 columns) -> four words, word k holding digit k of the four
+// values.  X = d0 + 2^8 d1 + 2^16 d2 + 2^24 d3 with balanced digits (signed bytes): d0 is the low
+// byte of X, d1 byte 1 of X + 2^7, d2 byte 2 of X + 2^7 + 2^15, d3 byte 3 of X + 2^7 + 2^15 + 2^23.
+__device__ __forceinline__ void fix_digits(uint2 v, float s1, float s2, uint32_t (&w)[kDigits], long long* sum) {
+  const uint32_t h[4] = {v.x << 16, v.x & 0xFFFF0000u, v.y << 16, v.y & 0xFFFF0000u};
+  uint32_t X[4], Y[4], Z[4], U[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int xi = __float2int_rn(__uint_as_float(h[i]) * s1 * s2);
+    if (sum) *sum += xi;
+    X[i] = (uint32_t)xi;
+    Y[i] = X[i] + 128u;
+    Z[i] = X[i] + 32896u;
+    U[i] = X[i] + 8421504u;
+  }
+  w[0] = __byte_perm(__byte_perm(X[0], X[1], 0x0040), __byte_perm(X[2], X[3], 0x0040), 0x5410);
+  w[1] = __byte_perm(__byte_perm(Y[0], Y[1], 0x0051), __byte_perm(Y[2], Y[3], 0x0051), 0x5410);
+  w[2] = __byte_perm(__byte_perm(Z[0], Z[1], 0x0062), __byte_perm(Z[2], Z[3], 0x0062), 0x5410);
+  w[3] = __byte_perm(__byte_perm(U[0], U[1], 0x0073), __byte_perm(U[2], U[3], 0x0073), 0x5410);
+}
+
 template <bool SIGNED>
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
@@ -133,7 +187,7 @@ __device__ __noinline__ bool tiles_wait_slow(uint32_t bar, uint32_t par, volatil
 }
 
 // Turns the 16 x 8 accumulator tile (MMA fragment layout: lane 4g+t holds rows g, g+8 and columns
-// 2t, 2t+1) of row block rb into y.  Lane L gathers the three digit sums of row L & 15, batch
+// 2t, 2t+1) of row block rb into y.  Lane L gathers the four digit sums of row L & 15, batch
 // column L >> 4 with shuffles.
 template <int NB>
 __device__ __noinline__ void tiles_finalize(const float* __restrict__ scale, const float* __restrict__ zero,
@@ -143,8 +197,8 @@ __device__ __noinline__ void tiles_finalize(const float* __restrict__ scale, con
   const uint32_t row = lane & 15u, b = lane >> 4;
   long long Y = 0;
 #pragma unroll
-  for (int k = 0; k < 3; ++k) {
-    const uint32_t col = min(3u * b + k, 7u);
+  for (int k = 0; k < kDigits; ++k) {
+    const uint32_t col = min((uint32_t)kDigits * b + k, 7u);
     const uint32_t src = (row & 7u) * 4u + (col >> 1);
     const int v0 = __shfl_sync(kFull, c0, src), v1 = __shfl_sync(kFull, c1, src);
     const int v2 = __shfl_sync(kFull, c2, src), v3 = __shfl_sync(kFull, c3, src);
@@ -248,7 +302,7 @@ struct CtaBase {
 template <int W, int NB, bool SIGNED>
 struct TilesCta : CtaBase {
   static constexpr int kThreads = W * 32;
-  static constexpr int NCOL = 3 * NB;
+  static constexpr int NCOL = kDigits * NB;
 
   uint32_t xstride;
   bool dead = false;
@@ -269,15 +323,11 @@ struct TilesCta : CtaBase {
     if (tid < 2) misc_u32()[1 + tid] = 0u;
     if (tid < 2 * NB) sum_scratch()[tid] = 0;
     __syncthreads();
-    // largest magnitude, on the bf16 bit patterns (monotonic; Inf and NaN sort last)
+    // largest magnitude per vector
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
       uint32_t m = 0;
-      for (uint32_t g = tid; g < G; g += kThreads) {
-        const uint2 v = __ldg(xg + (size_t)b * G + g);
-        const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu;
-        m = max(max(m, a0 & 0xFFFFu), max(a0 >> 16, max(a1 & 0xFFFFu, a1 >> 16)));
-      }
+      for (uint32_t g = tid; g < G; g += kThreads) m = amax4(__ldg(xg + (size_t)b * G + g), m);
 #pragma unroll
       for (int s = 16; s > 0; s >>= 1) m = max(m, __shfl_xor_sync(kFull, m, s));
       if (lane == 0) atomicMax(&misc_u32()[1 + b], m);
@@ -285,42 +335,21 @@ struct TilesCta : CtaBase {
     __syncthreads();
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-      const uint32_t mb = misc_u32()[1 + b];
-      const bool finite = mb < 0x7F80u;
-      int e = (int)(mb >> 7) - 126;  // max |x| < 2^e
-      e = max(e, -100);
-      const float in_scale = __uint_as_float((uint32_t)(127 + 22 - e) << 23);  // 2^(22-e), e in [-100, 128]
+      const FixScale f = fix_scale(misc_u32()[1 + b]);
+      const float s1 = f.finite ? f.s1 : 0.f;  // a non-finite vector: all digits zero, NaN output scale
       long long sum = 0;
       for (uint32_t g = tid; g < G; g += kThreads) {
-        const uint2 v = __ldg(xg + (size_t)b * G + g);
-        const uint32_t h[4] = {v.x << 16, v.x & 0xFFFF0000u, v.y << 16, v.y & 0xFFFF0000u};
-        uint32_t w0 = 0, w1 = 0, w2 = 0;
+        uint32_t w[kDigits];
+        fix_digits(__ldg(xg + (size_t)b * G + g), s1, f.s2, w, &sum);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          int X = finite ? __float2int_rn(__uint_as_float(h[i]) * in_scale) : 0;
-          sum += X;
-          const int d0 = (int)(signed char)(X & 0xFF);
-          X = (X - d0) >> 8;
-          const int d1 = (int)(signed char)(X & 0xFF);
-          const int d2 = (X - d1) >> 8;
-          w0 |= (uint32_t)(d0 & 0xFF) << (8 * i);
-          w1 |= (uint32_t)(d1 & 0xFF) << (8 * i);
-          w2 |= (uint32_t)(d2 & 0xFF) << (8 * i);
-        }
-        xs[(3 * b + 0) * xstride + g] = w0;
-        xs[(3 * b + 1) * xstride + g] = w1;
-        xs[(3 * b + 2) * xstride + g] = w2;
+        for (int k = 0; k < kDigits; ++k) xs[(kDigits * b + k) * xstride + g] = w[k];
       }
       if (d.has_zero) {
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) sum += __shfl_xor_sync(kFull, sum, s);
         if (lane == 0) atomicAdd(reinterpret_cast<unsigned long long*>(&sum_scratch()[b]), (unsigned long long)sum);
       }
-      if (tid == 0) {
-        // 2^(e-22) as a double, built from its exponent field
-        const double os = __longlong_as_double((long long)(1023 + e - 22) << 52);
-        xinfo()->out_scale[b] = finite ? os : __longlong_as_double(0x7FF8000000000000ll);
-      }
+      if (tid == 0) xinfo()->out_scale[b] = fix_out_scale(f);
     }
     __syncthreads();
     if (tid < NB) xinfo()->sum_x[tid] = xinfo()->out_scale[tid] * (double)sum_scratch()[tid];
@@ -522,7 +551,7 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
   // while its predecessor was still running.  Nothing above reads or writes what a predecessor
   // produces (the table and the weights are constant); the activations are first read below.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  cta.setup(tiles_smem_raw, tiles_smem(p.table_words, 3u * NB * p.xstride, W), W, p.table, p.table_words);
+  cta.setup(tiles_smem_raw, tiles_smem(p.table_words, (uint32_t)kDigits * NB * p.xstride, W), W, p.table, p.table_words);
   cta.xstride = p.xstride;
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -568,9 +597,9 @@ __device__ __noinline__ void panel_finalize(const float* __restrict__ scale, con
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t row = lane & 15u, half = lane >> 4;
   const uint32_t r = rb * 16u + row;
-  int dsum[3 * NB];
+  int dsum[kDigits * NB];
 #pragma unroll
-  for (int col = 0; col < 3 * NB; ++col) {
+  for (int col = 0; col < kDigits * NB; ++col) {
     const int nt = col >> 3, w = col & 7;
     const uint32_t src = (row & 7u) * 4u + (uint32_t)(w >> 1);
     const int lo = __shfl_sync(kFull, c[nt][w & 1], src), hi = __shfl_sync(kFull, c[nt][2 + (w & 1)], src);
@@ -579,7 +608,9 @@ __device__ __noinline__ void panel_finalize(const float* __restrict__ scale, con
 #pragma unroll
   for (int b = 0; b < NB; ++b) {
     if ((uint32_t)(b & 1) == half && (uint32_t)b < nb_valid && r < rows) {
-      const long long Y = (long long)dsum[3 * b] + 256ll * dsum[3 * b + 1] + 65536ll * dsum[3 * b + 2];
+      long long Y = 0;
+#pragma unroll
+      for (int k = 0; k < kDigits; ++k) Y += (long long)dsum[kDigits * b + k] << (8 * k);
       double v = (double)Y * xi->out_scale[b];
       if (has_zero) v -= (double)zero[r] * xi->sum_x[b];
       y[(size_t)b * rows + r] = (float)((double)scale[r] * v);
@@ -590,36 +621,17 @@ __device__ __noinline__ void panel_finalize(const float* __restrict__ scale, con
 template <int W, int NB, bool SIGNED>
 struct PanelCta : CtaBase {
   static constexpr int kThreads = W * 32;
-  static constexpr int NCOL = 3 * NB;
+  static constexpr int NCOL = kDigits * NB;
   static constexpr int NT = (NCOL + 7) / 8;
   static constexpr int kBufWords = 8 * NT * kPanelStride;  // one panel buffer: whole MMA tiles of columns
 
   uint32_t nb_valid;
 
-  // misc: [0] dead flag, +16 amax bits[8], +64 in_scale[8], +128 XInfo8, +256 sums[8]
+  // misc: [0] dead flag, +16 amax bits[8], +64 in_scale[8][2], +128 XInfo8, +256 sums[8]
   __device__ __forceinline__ uint32_t* amax_bits() { return reinterpret_cast<uint32_t*>(smem + L.misc + 16); }
-  __device__ __forceinline__ float* in_scale() { return reinterpret_cast<float*>(smem + L.misc + 64); }
+  __device__ __forceinline__ float2* in_scale() { return reinterpret_cast<float2*>(smem + L.misc + 64); }
   __device__ __forceinline__ XInfo8* xinfo() { return reinterpret_cast<XInfo8*>(smem + L.misc + 128); }
   __device__ __forceinline__ long long* sums() { return reinterpret_cast<long long*>(smem + L.misc + 256); }
-
-  // digits of one activation group (4 columns) -> three words.  X = d0 + 256 d1 + 65536 d2 with
-  // balanced digits: d0 is the low byte of X, d1 byte 1 of X + 128, d2 byte 2 of X + 128 + 32768.
-  static __device__ __forceinline__ void digits(uint2 v, float scale, uint32_t& w0, uint32_t& w1, uint32_t& w2,
-                                                long long* sum) {
-    const uint32_t h[4] = {v.x << 16, v.x & 0xFFFF0000u, v.y << 16, v.y & 0xFFFF0000u};
-    uint32_t X[4], Y[4], Z[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int xi = __float2int_rn(__uint_as_float(h[i]) * scale);
-      if (sum) *sum += xi;
-      X[i] = (uint32_t)xi;
-      Y[i] = X[i] + 128u;
-      Z[i] = X[i] + 32896u;
-    }
-    w0 = __byte_perm(__byte_perm(X[0], X[1], 0x0040), __byte_perm(X[2], X[3], 0x0040), 0x5410);
-    w1 = __byte_perm(__byte_perm(Y[0], Y[1], 0x0051), __byte_perm(Y[2], Y[3], 0x0051), 0x5410);
-    w2 = __byte_perm(__byte_perm(Z[0], Z[1], 0x0062), __byte_perm(Z[2], Z[3], 0x0062), 0x5410);
-  }
 
   // Per-vector scales (and, with zero points, the sum of each vector's fixed-point values).
   __device__ void prepare_scales(const tq_tiles_desc& d) {
@@ -633,33 +645,26 @@ struct PanelCta : CtaBase {
     __syncthreads();
     for (uint32_t b = 0; b < nb_valid; ++b) {
       uint32_t m = 0;
-      for (uint32_t g = tid; g < G; g += kThreads) {
-        const uint2 v = __ldg(xg + (size_t)b * G + g);
-        const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu;
-        m = max(max(m, a0 & 0xFFFFu), max(a0 >> 16, max(a1 & 0xFFFFu, a1 >> 16)));
-      }
+      for (uint32_t g = tid; g < G; g += kThreads) m = amax4(__ldg(xg + (size_t)b * G + g), m);
 #pragma unroll
       for (int sft = 16; sft > 0; sft >>= 1) m = max(m, __shfl_xor_sync(kFull, m, sft));
       if (lane == 0) atomicMax(&amax_bits()[b], m);
     }
     __syncthreads();
     if (tid < 8) {
-      const uint32_t mb = amax_bits()[tid];
-      const bool finite = mb < 0x7F80u;
-      const int e = max((int)(mb >> 7) - 126, -100);
+      const FixScale f = fix_scale(amax_bits()[tid]);
       // a non-finite vector: scale 0 (all digits zero) and a NaN output scale
-      in_scale()[tid] = finite ? __uint_as_float((uint32_t)(127 + 22 - e) << 23) : 0.f;
-      xinfo()->out_scale[tid] = finite ? __longlong_as_double((long long)(1023 + e - 22) << 52)
-                                       : __longlong_as_double(0x7FF8000000000000ll);
+      in_scale()[tid] = make_float2(f.finite ? f.s1 : 0.f, f.s2);
+      xinfo()->out_scale[tid] = fix_out_scale(f);
     }
     __syncthreads();
     if (d.has_zero) {
       for (uint32_t b = 0; b < nb_valid; ++b) {
-        const float sc = in_scale()[b];
+        const float2 sc = in_scale()[b];
         long long sum = 0;
         for (uint32_t g = tid; g < G; g += kThreads) {
-          uint32_t w0, w1, w2;
-          digits(__ldg(xg + (size_t)b * G + g), sc, w0, w1, w2, &sum);
+          uint32_t w[kDigits];
+          fix_digits(__ldg(xg + (size_t)b * G + g), sc.x, sc.y, w, &sum);
         }
 #pragma unroll
         for (int sft = 16; sft > 0; sft >>= 1) sum += __shfl_xor_sync(kFull, sum, sft);
@@ -693,11 +698,11 @@ struct PanelCta : CtaBase {
       const uint32_t idx = threadIdx.x + (uint32_t)it * kThreads;
       const uint32_t gl = idx % kGroups, b = idx / kGroups;
       if (idx < kGroups * NB) {
-        uint32_t w0, w1, w2;
-        digits(v[it], b < nb_valid ? in_scale()[b] : 0.f, w0, w1, w2, nullptr);
-        xs[(3 * b + 0) * kPanelStride + gl] = w0;
-        xs[(3 * b + 1) * kPanelStride + gl] = w1;
-        xs[(3 * b + 2) * kPanelStride + gl] = w2;
+        uint32_t w[kDigits];
+        const float2 sc = b < nb_valid ? in_scale()[b] : make_float2(0.f, 0.f);
+        fix_digits(v[it], sc.x, sc.y, w, nullptr);
+#pragma unroll
+        for (int k = 0; k < kDigits; ++k) xs[(kDigits * b + k) * kPanelStride + gl] = w[k];
       }
     }
   }
@@ -1088,13 +1093,7 @@ template <bool BF16>
 int launch_decomp(const DecompParams& p, uint32_t grid, cudaStream_t st) {
   auto kern = decompress_tiles_smem_kernel<kDecompWarps, BF16>;
   const size_t smem = tiles_smem(p.table_words, 0u, kDecompWarps).total;
-  static bool configured = false;
-  if (!configured) {
-    if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
-                                "decompress(tiles): raising the dynamic shared memory limit"))
-      return rc;
-    configured = true;
-  }
+  if (int rc = tq_ensure_dynamic_smem((const void*)kern, smem, "decompress(tiles): raising the dynamic shared memory limit")) return rc;
   kern<<<grid, kDecompWarps * 32, smem, st>>>(p);
   return tq_cuda_status((int)cudaGetLastError(), "decompress(tiles) launch");
 }
@@ -1118,13 +1117,7 @@ int launch_pdl(Kern kern, uint32_t grid, uint32_t threads, size_t smem, cudaStre
 template <int NB, bool SIGNED>
 int launch_tiles(const TilesParams& p, uint32_t grid, size_t smem, cudaStream_t st) {
   auto kern = gemv_tiles_kernel<kTilesWarps, NB, SIGNED>;
-  static size_t configured = 0;
-  if (smem > configured) {
-    if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
-                                "gemv(tiles): raising the dynamic shared memory limit"))
-      return rc;
-    configured = smem;
-  }
+  if (int rc = tq_ensure_dynamic_smem((const void*)kern, smem, "gemv(tiles): raising the dynamic shared memory limit")) return rc;
   return launch_pdl(kern, grid, kTilesWarps * 32, smem, st, p);
 }
 
@@ -1133,21 +1126,15 @@ int launch_panel(const TilesParams& p, uint32_t grid, cudaStream_t st) {
   auto kern = gemv_tiles_panel_kernel<kTilesWarps, NB, SIGNED>;
   const size_t smem = tiles_smem(p.table_words, 2u * PanelCta<kTilesWarps, NB, SIGNED>::kBufWords, kTilesWarps).total;
   if (smem > kSmemLimit) return TQ_ERR_UNSUPPORTED_SHAPE;
-  static size_t configured = 0;
-  if (smem > configured) {
-    if (int rc = tq_cuda_status((int)cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
-                                "gemv(tiles, wide): raising the dynamic shared memory limit"))
-      return rc;
-    configured = smem;
-  }
+  if (int rc = tq_ensure_dynamic_smem((const void*)kern, smem, "gemv(tiles, wide): raising the dynamic shared memory limit")) return rc;
   return launch_pdl(kern, grid, kTilesWarps * 32, smem, st, p);
 }
 
 // One pass over nb batch columns (1..8) with the kernel that fits: p.one / p.mats describe the work.
 int launch_pass(TilesParams& p, int nb, bool narrow_two, bool sg, uint32_t grid, cudaStream_t st, bool wide = false) {
   // the narrow kernel keeps the digits of a whole row in shared memory; rows too long for that
-  // (more than 8704 columns) take the wide kernel, which works in column panels, for any batch
-  const TilesSmem L = tiles_smem(p.table_words, 3u * std::min(nb, 2) * p.xstride, kTilesWarps);
+  // (more than 8448 columns) take the wide kernel, which works in column panels, for any batch
+  const TilesSmem L = tiles_smem(p.table_words, (uint32_t)kDigits * std::min(nb, 2) * p.xstride, kTilesWarps);
   if (!wide && nb <= 2 && (nb == 1 || narrow_two) && L.total <= kSmemLimit) {
     if (nb == 1) return sg ? launch_tiles<1, true>(p, grid, L.total, st) : launch_tiles<1, false>(p, grid, L.total, st);
     return sg ? launch_tiles<2, true>(p, grid, L.total, st) : launch_tiles<2, false>(p, grid, L.total, st);
@@ -1171,7 +1158,7 @@ int next_pass(int left, bool narrow_two) {
 int tq_tiles_max_nb(const tq_dmat* m) {
   const uint32_t xstride = m->tiles.steps * 32u + 4u;
   for (int nb = 2; nb >= 1; --nb)
-    if (tiles_smem(m->tiles.table_words, 3u * nb * xstride, kTilesWarps).total <= kSmemLimit) return nb;
+    if (tiles_smem(m->tiles.table_words, (uint32_t)kDigits * nb * xstride, kTilesWarps).total <= kSmemLimit) return nb;
   return 0;
 }
 
@@ -1215,6 +1202,7 @@ int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
 
 // The matrix as bf16 (level - zero point) in whole tiles: row_blocks * 16 rows of steps * 128 columns.
 int tq_tiles_decode_bf16(const tq_dmat* m, void* d_out, void* cuda_stream) {
+  if (!m->zero_bf16_exact) return TQ_ERR_UNSUPPORTED_SHAPE;  // level - zero point would be rounded
   DecompParams p{};
   p.one = m->tiles;
   p.out_one = static_cast<uint8_t*>(d_out);
@@ -1335,6 +1323,7 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   s->n = n_mats;
   s->B = bound ? B : 0;
   s->levels_signed = mats[0]->info.levels_signed;
+  for (int i = 0; i < n_mats; ++i) s->zero_bf16_exact = s->zero_bf16_exact && mats[i]->zero_bf16_exact;
   s->grid = (uint32_t)sm_count();
   s->table_words = mats[0]->tiles.table_words;
   s->d_table = mats[0]->dict->d_table;
@@ -1357,7 +1346,7 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
     std::vector<uint32_t> ids;
     uint32_t max_steps = 0;
     for (int i = 0; i < n_mats; ++i) {
-      const bool short_rows = tiles_smem(s->table_words, 3u * (mats[i]->tiles.steps * 32u + 4u), kTilesWarps).total <= kSmemLimit;
+      const bool short_rows = tiles_smem(s->table_words, (uint32_t)kDigits * (mats[i]->tiles.steps * 32u + 4u), kTilesWarps).total <= kSmemLimit;
       if (k == 0 || (k == 1) == short_rows) {
         pm.push_back(PlanMat{mats[i]->tiles.steps, mats[i]->tiles.row_blocks, mats[i]->rb_raw.data()});
         ids.push_back((uint32_t)i);
@@ -1416,7 +1405,7 @@ int stack_pass(const tq_stack* s, int b0, int nb, bool two, bool launch, cudaStr
 }
 // Two batch columns per narrow pass where the digits of two vectors fit for the short-row matrices.
 bool stack_two(const tq_stack* s) {
-  return s->plan[1].n_mats != 0 && tiles_smem(s->table_words, 6u * s->plan[1].xstride, kTilesWarps).total <= kSmemLimit;
+  return s->plan[1].n_mats != 0 && tiles_smem(s->table_words, 2u * kDigits * s->plan[1].xstride, kTilesWarps).total <= kSmemLimit;
 }
 }  // namespace
 
@@ -1456,6 +1445,7 @@ int tq_decompress_stack(const tq_stack* s, uint8_t* const* d_out_ptrs, void* cud
 
 int tq_decode_bf16_stack(const tq_stack* s, void* const* d_workspace_ptrs, void* cuda_stream) {
   if (!s || !d_workspace_ptrs) return TQ_ERR_INVALID_ARG;
+  if (!s->zero_bf16_exact) return TQ_ERR_UNSUPPORTED_SHAPE;  // level - zero point would be rounded
   DecompParams p{};
   p.mats = s->d_descs;
   p.segs = static_cast<const TilesSeg*>(s->plan[0].d_segs);

@@ -1,6 +1,6 @@
 """CUDA path against the oracle, through the C ABI.  Decoded bytes must be bit-exact; layer
-outputs must satisfy max_r |y - y_ref| <= 2e-3 * max_r |y_ref| per batch column (fp32
-accumulation of exact int8 x bf16 products against an fp64 reference)."""
+outputs must satisfy max_r |y - y_ref| <= 2e-3 * max_r |y_ref| per batch column (the contract),
+and the fused GEMV calls are held to the 1e-5 they deliver on N(0, 1) activations."""
 import numpy as np
 import pytest
 import torch
@@ -9,7 +9,10 @@ from inputs import synth
 from oracle import oracle
 
 pytestmark = pytest.mark.gpu
-TOL = 2e-3
+TOL = 2e-3    # the contract: max_r |y - y_ref| <= TOL * max_r |y_ref| per vector
+TIGHT = 1e-5  # what the GEMV kernels deliver on N(0, 1) activations (exact products; integer sums in the
+              # tiles layout, fp32 sums in the others): a defect a hundred times smaller than TOL fails
+GEMM_TIGHT = 5e-5  # the tensor-core products: exact bf16 operands, fp32 accumulation over up to 8192 columns
 
 
 @pytest.fixture(scope="module")
@@ -57,7 +60,7 @@ def _check_layer(tq, q, scale, odict, stream, batches=(1,), zero=None, seed=1, l
         y = tq.tq_fused_gemv(m, x.cuda()).cpu().numpy().astype(np.float64)
         yref = oracle.layer_forward(q, scale, x.double().numpy(), zero=zero)
         assert y.shape == yref.shape
-        assert _rel_err(y, yref) <= TOL
+        assert _rel_err(y, yref) <= TIGHT
     assert tq.tq_device_status(m) == 0
     return m
 
@@ -181,7 +184,7 @@ def test_host_library_pipeline_matches_oracle_pipeline(tq, layout):
             y = tq.tq_fused_gemv(m, x.cuda()).cpu().numpy().astype(np.float64)
             yref = oracle.layer_forward(qo, so, x.double().numpy())
             err = np.max(np.abs(y[:, sample] - yref), axis=1) / np.max(np.abs(yref), axis=1)
-            assert float(err.max()) <= TOL
+            assert float(err.max()) <= TIGHT
         assert tq.tq_device_status(m) == 0
 
 
@@ -199,7 +202,7 @@ def test_fused_gemm_matches_oracle(tq, rows, cols, M):
     sample = np.arange(M) if M <= 300 else np.sort(rng.choice(M, 64, replace=False))
     Yref = oracle.layer_forward(q, s, X[sample].double().numpy())
     assert Y.shape == (M, rows)
-    assert _rel_err(Y[sample], Yref) <= TOL
+    assert _rel_err(Y[sample], Yref) <= GEMM_TIGHT
 
 
 def test_fused_gemm_unsigned_levels_with_zero_point(tq):
@@ -213,7 +216,7 @@ def test_fused_gemm_unsigned_levels_with_zero_point(tq):
     X = synth.activations(64, 512, 9)
     Y = tq.tq_fused_gemm(m, X.cuda()).cpu().numpy().astype(np.float64)
     Yref = oracle.layer_forward(qu, s, X.double().numpy(), zero=z)
-    assert _rel_err(Y, Yref) <= TOL
+    assert _rel_err(Y, Yref) <= GEMM_TIGHT
     assert tq.tq_device_status(m) == 0
 
 
@@ -248,7 +251,7 @@ def test_fused_gemm_ws_matches_oracle(tq, rows, cols, M):
     sample = np.arange(M) if M <= 300 else np.sort(rng.choice(M, 64, replace=False))
     Yref = oracle.layer_forward(q, s, X[sample].double().numpy())
     assert Y.shape == (M, rows)
-    assert _rel_err(Y[sample], Yref) <= TOL
+    assert _rel_err(Y[sample], Yref) <= GEMM_TIGHT
 
 
 def test_fused_gemm_ws_unsigned_levels_with_zero_point(tq):
@@ -263,7 +266,7 @@ def test_fused_gemm_ws_unsigned_levels_with_zero_point(tq):
     X = synth.activations(64, 512, 9)
     Y = tq.tq_fused_gemm_ws(m, X.cuda(), ws).cpu().numpy().astype(np.float64)
     Yref = oracle.layer_forward(qu, s, X.double().numpy(), zero=z)
-    assert _rel_err(Y, Yref) <= TOL
+    assert _rel_err(Y, Yref) <= GEMM_TIGHT
     assert tq.tq_device_status(m) == 0
 
 
@@ -308,7 +311,7 @@ def test_gemm_plan_matches_oracle(tq, M):
         sample = np.arange(M) if M <= 300 else np.sort(rng.choice(M, 64, replace=False))
         Yref = oracle.layer_forward(q, sc, x[sample].double().numpy())
         assert Y.shape == (M, q.shape[0]) and np.isfinite(Y).all()
-        assert _rel_err(Y[sample], Yref) <= TOL
+        assert _rel_err(Y[sample], Yref) <= GEMM_TIGHT
         # and bit for bit what the single-matrix call gives
         Y1 = tq.tq_gemm_bf16_ws(m, x.cuda(), wss[mats.index(m)])
         assert torch.equal(Y1, y)
@@ -405,13 +408,13 @@ def test_stack_matches_oracle_and_single_calls(tq, B):
             single = tq.tq_fused_gemv(m, x)
             assert torch.equal(single, y)
             yref = oracle.layer_forward(q, s, x.cpu().double().numpy())
-            assert _rel_err(y.cpu().numpy().astype(np.float64), yref) <= TOL
+            assert _rel_err(y.cpu().numpy().astype(np.float64), yref) <= TIGHT
             assert tq.tq_device_status(m) == 0
 
 
 @pytest.mark.parametrize("B", [1, 2, 5])
 def test_stack_with_short_and_long_rows(tq, B):
-    """Rows too long for a whole row of activation digits in shared memory (more than 8704 columns)
+    """Rows too long for a whole row of activation digits in shared memory (more than 8448 columns)
     take the column-panel kernel; a stack that mixes both kinds launches one kernel for each."""
     shapes = [(200, 1024), (40, 12288), (600, 3072), (33, 28672), (64, 8192)]
     rng = np.random.default_rng(200 + B)
@@ -430,7 +433,7 @@ def test_stack_with_short_and_long_rows(tq, B):
     torch.cuda.synchronize()
     for m, q, s, x, y in zip(mats, qs, ss, xs, ys):
         assert torch.equal(tq.tq_fused_gemv(m, x), y)
-        assert _rel_err(y.cpu().numpy().astype(np.float64), oracle.layer_forward(q, s, x.cpu().double().numpy())) <= TOL
+        assert _rel_err(y.cpu().numpy().astype(np.float64), oracle.layer_forward(q, s, x.cpu().double().numpy())) <= TIGHT
         assert tq.tq_device_status(m) == 0
 
 
@@ -476,7 +479,7 @@ def test_decode_bf16_stack_then_gemm(tq):
     for m, q, s, w, (r, c) in zip(mats, qs, ss, wss, shapes):
         X = synth.activations(M, c, 17)
         Y = tq.tq_gemm_bf16_ws(m, X.cuda(), w).cpu().numpy().astype(np.float64)
-        assert _rel_err(Y, oracle.layer_forward(q, s, X.double().numpy())) <= TOL
+        assert _rel_err(Y, oracle.layer_forward(q, s, X.double().numpy())) <= GEMM_TIGHT
         # the workspace holds the levels themselves as bf16, in whole tiles
         rows_pad, pitch = -(-r // 16) * 16, -(-c // 128) * 128
         wb = w.view(torch.bfloat16)[: rows_pad * pitch].view(rows_pad, pitch)[:r, :c].float().cpu().numpy()
@@ -503,23 +506,35 @@ def test_stack_rejects_mixed_tables_and_layouts(tq):
 
 
 # ------------------------------------------------------------------ full size, as benchmarked
-def test_full_3b_stack_as_benchmarked_on_sampled_rows(tq):
-    """The whole LLaMA-3.2-3B linear stack (197 matrices, 3.2 G weights) built by the benchmark's
-    own builder and run in the launch configuration the benchmark times (one persistent launch,
-    batch 1).  The oracle regenerates sampled rows, quantizes them itself and computes their
-    outputs one by one; decoded levels of those rows must match bit for bit."""
+@pytest.fixture(scope="module")
+def model3b(tq):
+    """The whole LLaMA-3.2-3B linear stack (197 matrices, 3.2 G weights) built by the benchmark's own
+    builder, with 32 activation vectors per matrix; smaller batches use the first vectors."""
     import bench
 
     shapes = synth.llama32_linear_shapes("3b")
     device = torch.device("cuda", 0)
     mats, xs, ys, hd, q_host, scales, stats, x_arena, y_arena, dd = bench.build_model(
-        tq, shapes, 1, device, 0, None, layout=tq.TQ_LAYOUT_TILES)
+        tq, shapes, 32, device, 0, None, layout=tq.TQ_LAYOUT_TILES)
+    yield {"shapes": shapes, "device": device, "mats": mats, "xs": xs, "ys": ys, "hd": hd, "q_host": q_host,
+           "scales": scales, "y_arena": y_arena}
+    del mats, xs, ys, x_arena, y_arena
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("B", [1, 8, 32])
+def test_full_3b_stack_as_benchmarked_on_sampled_rows(tq, model3b, B):
+    """The launch configuration the benchmark times (one tq_fused_gemv_stack call over all 197
+    matrices) at 1, 8 and 32 vectors.  The oracle regenerates sampled rows, quantizes them itself and
+    computes their outputs one by one; decoded levels of those rows must match bit for bit."""
+    shapes, device, mats, q_host, scales = (model3b[k] for k in ("shapes", "device", "mats", "q_host", "scales"))
+    xs = [x[:B] for x in model3b["xs"]]
+    ys = [torch.full((B, r), float("nan"), dtype=torch.float32, device=device) for _, r, _ in shapes]
     stack = tq.tq_stack_create(mats, xs, ys)
-    y_arena.fill_(float("nan"))
     tq.tq_fused_gemv_stack(stack)
     torch.cuda.synchronize()
-    assert not torch.isnan(y_arena).any()
-    rng = np.random.default_rng(2025)
+    assert not any(bool(torch.isnan(y).any()) for y in ys)
+    rng = np.random.default_rng(2025 + B)
     picks = [0, 1, 2, 3, 4, 5, 6, 97, 100, 103, 190, 195, 196]  # every kind of layer, first/middle/last, lm_head
     for i in picks:
         name, rows, cols = shapes[i]
@@ -528,16 +543,54 @@ def test_full_3b_stack_as_benchmarked_on_sampled_rows(tq):
         w = synth.weight(rows, cols, synth.matrix_seed(i), device=device)[torch.from_numpy(sample).to(device)].cpu().numpy()
         qo, so = oracle.quantize_rows(w)
         assert np.array_equal(qo, q_host[i][sample]) and np.array_equal(so, scales[i][sample])
-        x = xs[i].cpu().double().numpy()
-        yref = oracle.layer_forward(qo, so, x)
+        yref = oracle.layer_forward(qo, so, xs[i].cpu().double().numpy())
         y = ys[i][:, torch.from_numpy(sample).to(device)].cpu().numpy().astype(np.float64)
         err = np.max(np.abs(y - yref), axis=1) / np.max(np.abs(yref), axis=1)
-        assert float(err.max()) <= TOL, (name, err)
+        assert float(err.max()) <= TIGHT, (name, err)
         assert tq.tq_device_status(mats[i]) == 0
-    # the table was built with the counting on the GPU: it must be the host builder's table
+
+
+def test_full_3b_table_and_decompress_stack(tq, model3b):
+    """The table was built with the counting on the GPU: it must be the host builder's table.  Then
+    tq_decompress_stack of the whole set (3.2 GB of levels, one persistent launch), every matrix
+    compared with the levels that were encoded."""
+    mats, q_host, hd, device = (model3b[k] for k in ("mats", "q_host", "hd", "device"))
     assert np.array_equal(hd.entries, tq.tq_build_dictionary(q_host).entries)
-    # decoded levels of two matrices, whole, against the levels that were encoded
+    outs = [torch.full((m.info.rows * m.info.cols,), 0x55, dtype=torch.uint8, device=device) for m in mats]
+    tq.tq_decompress_stack(tq.tq_stack_create(mats), outs)
+    torch.cuda.synchronize()
+    for o, q, m in zip(outs, q_host, mats):
+        assert torch.equal(o.view(torch.int8), torch.from_numpy(q).to(device).view(-1))
+        assert tq.tq_device_status(m) == 0
+    # and the single-matrix call on one decoder matrix and on the output head
     for i in (6, 196):
         got = tq.tq_decompress(mats[i])
         assert np.array_equal(got.cpu().numpy().view(np.int8), q_host[i])
         del got
+
+
+def test_full_3b_prefill_group_at_2048_tokens(tq, model3b):
+    """The prefill leg as the benchmark launches it: 14 decoder layers (98 matrices) decoded to bf16 by
+    one launch, then all their products at M = 2048 tokens by one tq_gemm_plan_run launch; sampled
+    (token, row) outputs against the oracle."""
+    shapes, device, mats, q_host, scales = (model3b[k] for k in ("shapes", "device", "mats", "q_host", "scales"))
+    M, group = 2048, list(range(98))
+    gm = [mats[i] for i in group]
+    Xs = {c: synth.activations(M, c, 99, device=device) for c in sorted({m.info.cols for m in gm})}
+    wss = [torch.empty(tq.tq_gemm_workspace_size(m), dtype=torch.uint8, device=device) for m in gm]
+    plan = tq.tq_gemm_plan_create(gm, [Xs[m.info.cols] for m in gm], wss)
+    tq.tq_decode_bf16_stack(tq.tq_stack_create(gm), wss)
+    tq.tq_gemm_plan_run(plan)
+    torch.cuda.synchronize()
+    assert tq.tq_gemm_plan_status(plan) == 0
+    rng = np.random.default_rng(77)
+    for k in (0, 1, 3, 5, 6, 49, 52, 91, 97):
+        i = group[k]
+        name, rows, cols = shapes[i]
+        rsel = np.sort(rng.choice(rows, 16, replace=False))
+        tsel = np.sort(rng.choice(M, 12, replace=False))
+        tsel[0], tsel[-1] = 0, M - 1
+        yref = oracle.layer_forward(q_host[i][rsel], scales[i][rsel], Xs[cols][torch.from_numpy(tsel).to(device)].cpu().double().numpy())
+        y = plan.Ys[k][torch.from_numpy(tsel).to(device)][:, torch.from_numpy(rsel).to(device)].cpu().numpy().astype(np.float64)
+        assert _rel_err(y, yref) <= GEMM_TIGHT, name
+        assert tq.tq_device_status(mats[i]) == 0
