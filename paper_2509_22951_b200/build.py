@@ -11,7 +11,7 @@ ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libtq.so"
 SOURCES = [CSRC / "tq_device.cu", CSRC / "tq_gemm.cu", CSRC / "tq_gemm_ws.cu", CSRC / "tq_tiles.cu", CSRC / "tq_encode.cu", CSRC / "tq_dict_device.cu", CSRC / "tq_host.cpp"]
-HEADERS = [CSRC / "tq_internal.h", CSRC / "tq_sm100.cuh", ROOT / "include" / "tq.h"]
+HEADERS = [CSRC / "tq_internal.h", CSRC / "tq_sm100.cuh", CSRC / "tq_tiles_common.cuh", ROOT / "include" / "tq.h"]
 
 
 def _nvcc() -> str | None:
