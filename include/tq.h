@@ -234,7 +234,11 @@ int tq_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream);
  * is far inside 2e-3 unless the row sums rest on elements more than about 2^20 times smaller than one
  * that meets (near-)zero weights.  Subnormal and smallest-normal bf16 inputs are exact.  A vector with
  * an Inf or NaN element yields NaN for all of its outputs (other vectors are unaffected); the status
- * word is not touched. */
+ * word is not touched.
+ *
+ * TQ_LAYOUT_TILES with more than two vectors (or rows too long for the one-vector kernel) stages
+ * digit planes of the activations in a scratch area inside the matrix's own device image: calls
+ * on the same matrix must not overlap on the GPU (calls on one stream never do). */
 int tq_fused_gemv(const tq_dmat* m, const void* d_x_bf16, int B, float* d_y, void* cuda_stream);
 
 /* The same call with HOST operands: copies x to the DEVICE staging buffer d_x_stage ([B][cols]
@@ -292,13 +296,19 @@ int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, c
  * then streams its share of the row blocks of all the matrices.  The products are independent of
  * one another: a caller whose layers feed each other makes one stack per group of layers that can
  * run together (q/k/v; gate/up; ...).  d_x[i]: DEVICE bf16 [B][cols_i], 16-byte aligned; d_y[i]:
- * DEVICE fp32 [B][rows_i]; B in 1..32 (tq_stack_launches tells how many kernel launches a call makes).  mats, d_x, d_y: HOST arrays of n_mats entries.  The
- * work split and the operand addresses are written to the caller's DEVICE buffer d_buf (256-byte
- * aligned, tq_stack_size bytes), which must outlive the handle, as must the matrices.
+ * DEVICE fp32 [B][rows_i]; B in 1..32.  One vector (two where the digits of two fit beside the
+ * table for every matrix) runs the kernel whose decoding warps multiply on the spot; more vectors,
+ * and matrices whose rows are too long for that kernel, run ONE pass of the tcgen05 kernel for all
+ * vectors, preceded by a small launch that turns the activations into digit planes
+ * (tq_stack_launches tells how many launches a call makes).  mats, d_x, d_y: HOST arrays of n_mats
+ * entries.  The work split, the operand addresses and the scratch of the digit planes are written
+ * to the caller's DEVICE buffer d_buf (256-byte aligned, tq_stack_size bytes for these matrices and
+ * this B; B = 0 for a stack without operands), which must outlive the handle, as must the matrices.
  * TQ_ERR_UNSUPPORTED_SHAPE if the matrices do not share table, level type and layout.
- * tq_stack_create synchronises cuda_stream; tq_fused_gemv_stack is asynchronous. */
+ * tq_stack_create synchronises cuda_stream; tq_fused_gemv_stack is asynchronous.  Calls on one
+ * stack share its scratch: they must not overlap on the GPU. */
 typedef struct tq_stack tq_stack;
-int tq_stack_size(int n_mats, uint64_t* device_bytes);
+int tq_stack_size(const tq_dmat* const* mats, int n_mats, int B, uint64_t* device_bytes);
 /* The work split tq_stack_create computes, as a host-only call (no device needed): the row blocks
  * (16 rows) of the matrices, in order, are cut into n_ctas consecutive shares of about equal cost
  * (bytes streamed plus a fixed charge per segment); a share is a list of segments (matrix, first

@@ -54,6 +54,12 @@ def _L():
         lib.tqo_build_dictionary.restype = C.c_void_p
         lib.tqo_dict_from_entries.argtypes = [u8p, C.c_uint32]
         lib.tqo_dict_from_entries.restype = C.c_void_p
+        lib.tqo_build_dictionary_seq.argtypes = [C.POINTER(u8p), u64p, C.c_int, C.c_uint32, C.c_uint32]
+        lib.tqo_build_dictionary_seq.restype = C.c_void_p
+        lib.tqo_dict_from_entries_seq.argtypes = [u8p, C.c_uint32, C.c_uint32]
+        lib.tqo_dict_from_entries_seq.restype = C.c_void_p
+        lib.tqo_dict_seq.argtypes = [C.c_void_p]
+        lib.tqo_dict_seq.restype = C.c_uint32
         lib.tqo_dict_free.argtypes = [C.c_void_p]
         lib.tqo_dict_free.restype = None
         lib.tqo_dict_size.argtypes = [C.c_void_p]
@@ -105,7 +111,8 @@ def quantize_rows(w: np.ndarray):
 
 
 class Dictionary:
-    """Listing 2's compression table: K <= 65534 four-byte entries, code = rank + 1."""
+    """Listing 2's compression table: K <= 65534 entries of `seq` bytes (Listing 2's sequence_length,
+    4 unless stated), code = rank + 1."""
 
     def __init__(self, handle):
         if not handle:
@@ -113,17 +120,19 @@ class Dictionary:
         self._h = C.c_void_p(handle)
 
     @classmethod
-    def build(cls, mats, top_k: int = 2 ** 16 - 1) -> "Dictionary":
+    def build(cls, mats, top_k: int = 2 ** 16 - 1, seq: int = 4) -> "Dictionary":
         arrs = [np.ascontiguousarray(m).view(np.uint8).reshape(-1) for m in mats]
         n = len(arrs)
         ptrs = (C.POINTER(C.c_uint8) * n)(*[_ptr(a, C.c_uint8) for a in arrs])
         lens = (C.c_uint64 * n)(*[a.size for a in arrs])
-        return cls(_L().tqo_build_dictionary(ptrs, lens, n, top_k))
+        if not 1 <= seq <= 8:
+            raise ValueError("sequence length must be 1..8")
+        return cls(_L().tqo_build_dictionary_seq(ptrs, lens, n, top_k, seq))
 
     @classmethod
-    def from_entries(cls, entries: np.ndarray) -> "Dictionary":
-        e = np.ascontiguousarray(entries, dtype=np.uint8).reshape(-1, 4)
-        return cls(_L().tqo_dict_from_entries(_ptr(e, C.c_uint8), e.shape[0]))
+    def from_entries(cls, entries: np.ndarray, seq: int = 4) -> "Dictionary":
+        e = np.ascontiguousarray(entries, dtype=np.uint8).reshape(-1, seq)
+        return cls(_L().tqo_dict_from_entries_seq(_ptr(e, C.c_uint8), e.shape[0], seq))
 
     def __del__(self):
         if getattr(self, "_h", None) and _lib is not None:
@@ -135,11 +144,15 @@ class Dictionary:
         return int(_L().tqo_dict_size(self._h))
 
     @property
+    def seq(self) -> int:
+        return int(_L().tqo_dict_seq(self._h))
+
+    @property
     def entries(self) -> np.ndarray:
-        K = self.K
+        K, L = self.K, self.seq
         if K == 0:
-            return np.zeros((0, 4), dtype=np.uint8)
-        return np.ctypeslib.as_array(_L().tqo_dict_entries(self._h), shape=(K, 4)).copy()
+            return np.zeros((0, L), dtype=np.uint8)
+        return np.ctypeslib.as_array(_L().tqo_dict_entries(self._h), shape=(K, L)).copy()
 
     @property
     def counts(self) -> np.ndarray:
@@ -170,7 +183,7 @@ class Dictionary:
     def decode(self, stream: np.ndarray, n_out: int | None = None) -> np.ndarray:
         """Listing 4.  Raises KeyError on an unknown code, as the listing does."""
         s = np.ascontiguousarray(stream, dtype=np.uint16)
-        cap = 4 * s.size + 4 if n_out is None else n_out
+        cap = self.seq * s.size + self.seq if n_out is None else n_out
         out = np.empty(cap, dtype=np.uint8)
         n = _L().tqo_decode(self._h, _ptr(s, C.c_uint16), s.size, _ptr(out, C.c_uint8), cap)
         if n == -1:

@@ -9,8 +9,10 @@
  * header, table or helper with the CUDA library; only tests, the smoke check
  * and the benchmark's CPU-baseline leg may call it.
  *
- * No blocking, fusion, SIMD or threading: each function follows the listing it
- * cites step by step so that it can be checked against the paper by eye.
+ * No blocking, fusion, SIMD or threading.  The quantizers and the table builder
+ * take the steps of the listings they cite, in the paper's order; the coder and
+ * the decoder are written from the definition of the stream format (Section 4),
+ * so that each can be checked against the paper by eye.
  *
  * Pins (see tests/test_oracle_pins.py): round trip exactness, the stream-size
  * identity, closed forms (constant input, empty table, all-hit), brute-force
@@ -93,37 +95,47 @@ void tqo_quantize_rows(const float *w, uint32_t rows, uint32_t cols, int8_t *q,
 }
 
 /* ------------------------------------------------------------------------ */
-/* Listing 2: count every stride-1 window of 4 bytes over each flattened     */
-/* matrix (windows never span two matrices), keep the top_k most frequent,   */
-/* code = rank + 1.  Ties keep first-insertion order, which is what a stable */
-/* descending sort of an insertion-ordered counter gives.                    */
+/* Listing 2: count every stride-1 window of L consecutive bytes over each   */
+/* flattened matrix (windows never span two matrices), keep the top_k most   */
+/* frequent, code = rank + 1.  L is the listing's sequence_length parameter  */
+/* (default 4, the value the paper's pipeline runs with; 1..8 here).  Ties   */
+/* keep first-insertion order, which is what a stable descending sort of an  */
+/* insertion-ordered counter gives.                                          */
 /* ------------------------------------------------------------------------ */
 typedef struct {
-  uint32_t key;    /* the 4 bytes, byte i of the window in bits 8i..8i+7 */
-  uint32_t used;
+  uint64_t key;    /* the L bytes, byte i of the window in bits 8i..8i+7 */
   uint64_t count;
   uint64_t first;  /* insertion order */
+  uint32_t used;
 } tqo_slot;
 
 typedef struct {
-  uint32_t n_entries;             /* K                                    */
-  uint8_t *entries;               /* K x 4, rank order                    */
-  uint64_t *counts;               /* K, occurrence count of each entry    */
-  uint64_t n_distinct;            /* distinct windows seen                */
-  uint64_t n_windows;             /* total windows counted                */
+  uint32_t seq;                   /* L: bytes per window / per table entry  */
+  uint32_t n_entries;             /* K                                      */
+  uint8_t *entries;               /* K x L, rank order                      */
+  uint64_t *counts;               /* K, occurrence count of each entry      */
+  uint64_t n_distinct;            /* distinct windows seen                  */
+  uint64_t n_windows;             /* total windows counted                  */
   /* lookup map for the encoder: key -> code */
   uint32_t map_cap;
-  uint32_t *map_key;
+  uint64_t *map_key;
   uint16_t *map_code;             /* 0 = empty */
 } tqo_dict;
 
-static uint32_t tqo_hash(uint32_t k) {
-  k ^= k >> 16;
-  k *= 0x7feb352du;
-  k ^= k >> 15;
-  k *= 0x846ca68bu;
-  k ^= k >> 16;
+static uint64_t tqo_hash(uint64_t k) {
+  k ^= k >> 33;
+  k *= 0xff51afd7ed558ccdull;
+  k ^= k >> 33;
+  k *= 0xc4ceb9fe1a85ec53ull;
+  k ^= k >> 33;
   return k;
+}
+
+/* the L bytes at w as one integer */
+static uint64_t tqo_window(const uint8_t *w, uint32_t L) {
+  uint64_t key = 0;
+  for (uint32_t j = 0; j < L; ++j) key |= (uint64_t)w[j] << (8 * j);
+  return key;
 }
 
 static int tqo_cmp_rank(const void *a, const void *b) {
@@ -133,16 +145,16 @@ static int tqo_cmp_rank(const void *a, const void *b) {
   return 0;
 }
 
-static void tqo_map_insert(tqo_dict *d, uint32_t key, uint16_t code) {
-  uint32_t m = d->map_cap - 1, h = tqo_hash(key) & m;
+static void tqo_map_insert(tqo_dict *d, uint64_t key, uint16_t code) {
+  uint64_t m = d->map_cap - 1, h = tqo_hash(key) & m;
   while (d->map_code[h] != 0) h = (h + 1) & m;
   d->map_key[h] = key;
   d->map_code[h] = code;
 }
 
-/* code of a 4-byte window, 0 if it is not in the table */
-static uint16_t tqo_map_find(const tqo_dict *d, uint32_t key) {
-  uint32_t m = d->map_cap - 1, h = tqo_hash(key) & m;
+/* code of a window, 0 if it is not in the table */
+static uint16_t tqo_map_find(const tqo_dict *d, uint64_t key) {
+  uint64_t m = d->map_cap - 1, h = tqo_hash(key) & m;
   while (d->map_code[h] != 0) {
     if (d->map_key[h] == key) return d->map_code[h];
     h = (h + 1) & m;
@@ -159,8 +171,22 @@ void tqo_dict_free(tqo_dict *d) {
   free(d);
 }
 
-tqo_dict *tqo_build_dictionary(const uint8_t *const *mats, const uint64_t *n_elems,
-                               int n_mats, uint32_t top_k) {
+static tqo_dict *tqo_dict_alloc(uint32_t K, uint32_t L) {
+  tqo_dict *d = (tqo_dict *)calloc(1, sizeof(tqo_dict));
+  if (!d) return NULL;
+  d->seq = L;
+  d->n_entries = K;
+  d->entries = (uint8_t *)malloc(K ? (size_t)K * L : L);
+  d->counts = (uint64_t *)calloc(K ? K : 1, 8);
+  d->map_cap = 1u << 18; /* > 2 x 65534 */
+  d->map_key = (uint64_t *)calloc(d->map_cap, sizeof(uint64_t));
+  d->map_code = (uint16_t *)calloc(d->map_cap, sizeof(uint16_t));
+  return d;
+}
+
+tqo_dict *tqo_build_dictionary_seq(const uint8_t *const *mats, const uint64_t *n_elems,
+                                   int n_mats, uint32_t top_k, uint32_t L) {
+  if (L < 1 || L > 8) return NULL;
   uint64_t cap = 1024;
   uint64_t used = 0, windows = 0;
   tqo_slot *tab = (tqo_slot *)calloc(cap, sizeof(tqo_slot));
@@ -168,9 +194,8 @@ tqo_dict *tqo_build_dictionary(const uint8_t *const *mats, const uint64_t *n_ele
   for (int m = 0; m < n_mats; ++m) {
     const uint8_t *w = mats[m];
     uint64_t n = n_elems[m];
-    for (uint64_t i = 0; i + TQO_SEQ <= n; ++i) {
-      uint32_t key = (uint32_t)w[i] | ((uint32_t)w[i + 1] << 8) |
-                     ((uint32_t)w[i + 2] << 16) | ((uint32_t)w[i + 3] << 24);
+    for (uint64_t i = 0; i + L <= n; ++i) {
+      uint64_t key = tqo_window(w + i, L);
       if ((used + 1) * 10 > cap * 6) { /* grow at 60 % load */
         uint64_t ncap = cap * 2;
         tqo_slot *nt = (tqo_slot *)calloc(ncap, sizeof(tqo_slot));
@@ -209,124 +234,130 @@ tqo_dict *tqo_build_dictionary(const uint8_t *const *mats, const uint64_t *n_ele
   if (K > top_k) K = top_k;
   if (K > TQO_MAX_ENTRIES) K = TQO_MAX_ENTRIES;
 
-  tqo_dict *d = (tqo_dict *)calloc(1, sizeof(tqo_dict));
-  d->n_entries = (uint32_t)K;
+  tqo_dict *d = tqo_dict_alloc((uint32_t)K, L);
   d->n_distinct = used;
   d->n_windows = windows;
-  d->entries = (uint8_t *)malloc(K ? K * 4 : 4);
-  d->counts = (uint64_t *)malloc(K ? K * 8 : 8);
-  d->map_cap = 1u << 18; /* > 2 x 65534 */
-  d->map_key = (uint32_t *)calloc(d->map_cap, sizeof(uint32_t));
-  d->map_code = (uint16_t *)calloc(d->map_cap, sizeof(uint16_t));
   for (uint64_t r = 0; r < K; ++r) {
-    uint32_t key = all[r].key;
-    d->entries[4 * r + 0] = (uint8_t)(key);
-    d->entries[4 * r + 1] = (uint8_t)(key >> 8);
-    d->entries[4 * r + 2] = (uint8_t)(key >> 16);
-    d->entries[4 * r + 3] = (uint8_t)(key >> 24);
+    for (uint32_t j = 0; j < L; ++j) d->entries[L * r + j] = (uint8_t)(all[r].key >> (8 * j));
     d->counts[r] = all[r].count;
-    tqo_map_insert(d, key, (uint16_t)(r + 1)); /* code = rank + 1 */
+    tqo_map_insert(d, all[r].key, (uint16_t)(r + 1)); /* code = rank + 1 */
   }
   free(all);
   return d;
 }
 
+tqo_dict *tqo_build_dictionary(const uint8_t *const *mats, const uint64_t *n_elems,
+                               int n_mats, uint32_t top_k) {
+  return tqo_build_dictionary_seq(mats, n_elems, n_mats, top_k, TQO_SEQ);
+}
+
 /* Build a dictionary object from an explicit entry list (rank order), so the
  * encoder/decoder can be exercised with hand-made tables. */
-tqo_dict *tqo_dict_from_entries(const uint8_t *entries, uint32_t K) {
-  if (K > TQO_MAX_ENTRIES) return NULL;
-  tqo_dict *d = (tqo_dict *)calloc(1, sizeof(tqo_dict));
-  d->n_entries = K;
-  d->entries = (uint8_t *)malloc(K ? (size_t)K * 4 : 4);
-  d->counts = (uint64_t *)calloc(K ? K : 1, 8);
-  memcpy(d->entries, entries, (size_t)K * 4);
-  d->map_cap = 1u << 18;
-  d->map_key = (uint32_t *)calloc(d->map_cap, sizeof(uint32_t));
-  d->map_code = (uint16_t *)calloc(d->map_cap, sizeof(uint16_t));
+tqo_dict *tqo_dict_from_entries_seq(const uint8_t *entries, uint32_t K, uint32_t L) {
+  if (K > TQO_MAX_ENTRIES || L < 1 || L > 8) return NULL;
+  tqo_dict *d = tqo_dict_alloc(K, L);
+  memcpy(d->entries, entries, (size_t)K * L);
   for (uint32_t r = 0; r < K; ++r) {
-    uint32_t key = (uint32_t)entries[4 * r] | ((uint32_t)entries[4 * r + 1] << 8) |
-                   ((uint32_t)entries[4 * r + 2] << 16) |
-                   ((uint32_t)entries[4 * r + 3] << 24);
+    uint64_t key = tqo_window(entries + (size_t)L * r, L);
     if (tqo_map_find(d, key) == 0) tqo_map_insert(d, key, (uint16_t)(r + 1));
   }
   return d;
 }
 
+tqo_dict *tqo_dict_from_entries(const uint8_t *entries, uint32_t K) {
+  return tqo_dict_from_entries_seq(entries, K, TQO_SEQ);
+}
+
 uint32_t tqo_dict_size(const tqo_dict *d) { return d->n_entries; }
+uint32_t tqo_dict_seq(const tqo_dict *d) { return d->seq; }
 const uint8_t *tqo_dict_entries(const tqo_dict *d) { return d->entries; }
 const uint64_t *tqo_dict_counts(const tqo_dict *d) { return d->counts; }
 uint64_t tqo_dict_distinct(const tqo_dict *d) { return d->n_distinct; }
 uint64_t tqo_dict_windows(const tqo_dict *d) { return d->n_windows; }
 
 /* ------------------------------------------------------------------------ */
-/* Listing 3: aligned scan in steps of 4.  Known window -> its code; unknown */
-/* -> escape marker then the 4 bytes, each widened to uint16; a tail of 1..3 */
-/* bytes -> escape marker then those bytes.  out == NULL: size query.        */
-/* Returns the stream length in uint16 units, or (uint64_t)-1 if cap is too  */
-/* small.  n_hits / n_miss may be NULL.                                      */
+/* The stream format (Section 4; Listing 3 writes it, Listing 4 reads it).   */
+/* The n bytes of a matrix are cut into consecutive blocks of L bytes (the   */
+/* last block may be shorter).  A full block that is a table entry is one    */
+/* uint16 item, its code; any other block is the marker 0xFFFF followed by   */
+/* its bytes, each widened to uint16.  So block j starts at slot             */
+/* sum over the blocks before it of (1 if coded, else 1 + its length).       */
+/*                                                                           */
+/* tqo_encode states exactly that: classify every block, place every block   */
+/* by the running sum, fill the slots.  out == NULL: size query.  Returns    */
+/* the stream length in uint16 units, or (uint64_t)-1 if cap is too small.   */
+/* n_hits / n_miss (may be NULL) count the coded / marked full blocks.       */
 /* ------------------------------------------------------------------------ */
 uint64_t tqo_encode(const tqo_dict *d, const uint8_t *w, uint64_t n, uint16_t *out,
                     uint64_t cap, uint64_t *n_hits, uint64_t *n_miss) {
-  uint64_t len = 0, hits = 0, miss = 0, i = 0;
-  while (i + TQO_SEQ <= n) {
-    uint32_t key = (uint32_t)w[i] | ((uint32_t)w[i + 1] << 8) |
-                   ((uint32_t)w[i + 2] << 16) | ((uint32_t)w[i + 3] << 24);
-    uint16_t code = tqo_map_find(d, key);
-    if (code != 0) {
-      if (out) { if (len + 1 > cap) return (uint64_t)-1; out[len] = code; }
-      len += 1;
-      hits++;
-    } else {
-      if (out) {
-        if (len + 5 > cap) return (uint64_t)-1;
-        out[len] = TQO_ESCAPE;
-        for (int j = 0; j < TQO_SEQ; ++j) out[len + 1 + j] = w[i + j];
-      }
-      len += 5;
-      miss++;
-    }
-    i += TQO_SEQ;
+  const uint32_t L = d->seq;
+  const uint64_t n_full = n / L, tail = n % L;
+  const uint64_t n_blocks = n_full + (tail ? 1 : 0);
+  uint16_t *code = (uint16_t *)malloc((n_blocks ? n_blocks : 1) * sizeof(uint16_t));
+  if (!code) return (uint64_t)-1;
+  uint64_t hits = 0;
+  for (uint64_t j = 0; j < n_full; ++j) {
+    code[j] = tqo_map_find(d, tqo_window(w + j * L, L));
+    hits += code[j] != 0;
   }
-  if (i < n) {
-    uint64_t r = n - i;
-    if (out) {
-      if (len + 1 + r > cap) return (uint64_t)-1;
-      out[len] = TQO_ESCAPE;
-      for (uint64_t j = 0; j < r; ++j) out[len + 1 + j] = w[i + j];
-    }
-    len += 1 + r;
-  }
+  if (tail) code[n_full] = 0; /* a short block is never a table entry */
+  const uint64_t len = hits + (n_full - hits) * (1 + (uint64_t)L) + (tail ? 1 + tail : 0);
   if (n_hits) *n_hits = hits;
-  if (n_miss) *n_miss = miss;
+  if (n_miss) *n_miss = n_full - hits;
+  if (out) {
+    if (len > cap) { free(code); return (uint64_t)-1; }
+    uint64_t slot = 0;
+    for (uint64_t j = 0; j < n_blocks; ++j) {
+      const uint64_t blen = j < n_full ? L : tail;
+      if (code[j]) {
+        out[slot++] = code[j];
+      } else {
+        out[slot++] = TQO_ESCAPE;
+        for (uint64_t e = 0; e < blen; ++e) out[slot++] = w[j * L + e];
+      }
+    }
+  }
+  free(code);
   return len;
 }
 
 /* ------------------------------------------------------------------------ */
-/* Listing 4: walk the tokens; the escape marker means "the next up to 4     */
-/* slots are raw bytes" (a slice, so fewer at the very end), anything else   */
-/* is looked up in the table.  Returns the number of bytes produced, -1 for  */
-/* an unknown code (the listing raises), -2 if out is too small.             */
+/* tqo_decode reads the same format back.  First the items are located: an   */
+/* item is either one slot (a code) or a marker with the up to L slots that  */
+/* follow it (fewer only when the stream ends: the short last block, which   */
+/* is how Listing 4's slice behaves).  Then every item is expanded: a code   */
+/* to its table entry, a marked item to the low bytes of its slots.  Returns */
+/* the number of bytes produced, -1 for a code that is not in the table      */
+/* (Listing 4 raises there), -2 if out is too small, -3 out of memory.       */
 /* ------------------------------------------------------------------------ */
 int64_t tqo_decode(const tqo_dict *d, const uint16_t *s, uint64_t len, uint8_t *out,
                    uint64_t cap) {
-  uint64_t i = 0, o = 0;
-  while (i < len) {
-    uint16_t code = s[i];
-    i += 1;
-    if (code == TQO_ESCAPE) {
-      uint64_t take = len - i < TQO_SEQ ? len - i : TQO_SEQ;
-      if (o + take > cap) return -2;
-      for (uint64_t j = 0; j < take; ++j) out[o + j] = (uint8_t)s[i + j];
-      o += take;
-      i += TQO_SEQ;
+  const uint32_t L = d->seq;
+  uint64_t *start = (uint64_t *)malloc((len ? len : 1) * sizeof(uint64_t));
+  if (!start) return -3;
+  uint64_t n_items = 0;
+  for (uint64_t pos = 0; pos < len;) {
+    start[n_items++] = pos;
+    pos += s[pos] == TQO_ESCAPE ? 1 + (uint64_t)L : 1;
+  }
+  uint64_t o = 0;
+  int64_t rc = 0;
+  for (uint64_t it = 0; it < n_items && rc == 0; ++it) {
+    const uint64_t pos = start[it];
+    if (s[pos] == TQO_ESCAPE) {
+      const uint64_t avail = len - (pos + 1);
+      const uint64_t take = avail < L ? avail : L;
+      if (o + take > cap) { rc = -2; break; }
+      for (uint64_t e = 0; e < take; ++e) out[o++] = (uint8_t)s[pos + 1 + e];
     } else {
-      if (code == 0 || code > d->n_entries) return -1;
-      if (o + TQO_SEQ > cap) return -2;
-      memcpy(out + o, d->entries + 4 * (uint64_t)(code - 1), TQO_SEQ);
-      o += TQO_SEQ;
+      const uint16_t c = s[pos];
+      if (c == 0 || c > d->n_entries) { rc = -1; break; }
+      if (o + L > cap) { rc = -2; break; }
+      for (uint32_t e = 0; e < L; ++e) out[o++] = d->entries[(uint64_t)L * (c - 1) + e];
     }
   }
-  return (int64_t)o;
+  free(start);
+  return rc ? rc : (int64_t)o;
 }
 
 /* ------------------------------------------------------------------------ */

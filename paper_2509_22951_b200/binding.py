@@ -105,7 +105,7 @@ def _load() -> C.CDLL:
         "tq_gemm_plan_run": (C.c_int, [vp, vp]),
         "tq_gemm_plan_status": (C.c_int, [vp, vp, u32p]),
         "tq_gemm_plan_free": (None, [vp]),
-        "tq_stack_size": (C.c_int, [C.c_int, u64p]),
+        "tq_stack_size": (C.c_int, [C.POINTER(vp), C.c_int, C.c_int, u64p]),
         "tq_stack_plan_host": (C.c_int, [C.c_int, u32p, u32p, C.POINTER(u32p), C.c_uint32, u32p, C.c_uint32, u32p, u32p]),
         "tq_stack_create": (C.c_int, [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int, C.c_int, vp, C.c_uint64, vp,
                                       C.POINTER(vp)]),
@@ -524,14 +524,15 @@ def tq_stack_create(mats, xs=None, ys=None, stream=None) -> Stack:
     Without xs / ys the stack serves tq_decompress_stack only."""
     n = len(mats)
     assert n >= 1 and (xs is None) == (ys is None)
-    need = C.c_uint64()
-    _check(_lib.tq_stack_size(n, C.byref(need)), "tq_stack_size")
-    buf = torch.empty(need.value, dtype=torch.uint8, device=mats[0].buf.device)
     hm = (C.c_void_p * n)(*[m._h for m in mats])
     B, hx, hy = 0, None, None
     if xs is not None:
         assert len(xs) == n and len(ys) == n
         B = xs[0].numel() // mats[0].info.cols
+    need = C.c_uint64()
+    _check(_lib.tq_stack_size(hm, n, B, C.byref(need)), "tq_stack_size")
+    buf = torch.empty(need.value, dtype=torch.uint8, device=mats[0].buf.device)
+    if xs is not None:
         for m, x, y in zip(mats, xs, ys):
             assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.numel() == B * m.info.cols
             assert y.is_cuda and y.dtype == torch.float32 and y.is_contiguous() and y.numel() == B * m.info.rows

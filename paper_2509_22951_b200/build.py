@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libtq.so"
-SOURCES = [CSRC / "tq_device.cu", CSRC / "tq_gemm.cu", CSRC / "tq_gemm_ws.cu", CSRC / "tq_tiles.cu", CSRC / "tq_encode.cu", CSRC / "tq_dict_device.cu", CSRC / "tq_host.cpp"]
+SOURCES = [CSRC / "tq_device.cu", CSRC / "tq_gemm.cu", CSRC / "tq_gemm_ws.cu", CSRC / "tq_tiles.cu", CSRC / "tq_wide.cu", CSRC / "tq_encode.cu", CSRC / "tq_dict_device.cu", CSRC / "tq_host.cpp"]
 HEADERS = [CSRC / "tq_internal.h", CSRC / "tq_sm100.cuh", CSRC / "tq_tiles_common.cuh", ROOT / "include" / "tq.h"]
 
 

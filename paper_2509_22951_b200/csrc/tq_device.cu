@@ -671,6 +671,7 @@ int tq_upload(const tq_ddict* dict, const uint16_t* stream, uint64_t stream_len,
     t.row_blocks = img.row_blocks;
     t.has_zero = row_zero != nullptr;
     t.table_words = TQ_TILES_TABLE_WORDS;
+    t.xdig = base + tq_tiles_layout(rows, cols).off_xdig(img.n_raw);
     m->rb_raw = std::move(img.rb_raw);
     n_hits = img.n_hits;
     n_miss = img.n_miss;
@@ -779,6 +780,7 @@ int tq_upload_device(const tq_ddict* dict, const uint8_t* d_levels, uint32_t row
   t.row_blocks = geo.row_blocks;
   t.has_zero = d_row_zero != nullptr;
   t.table_words = TQ_TILES_TABLE_WORDS;
+  t.xdig = base + geo.off_xdig(n_raw);
   m->info.rows = rows;
   m->info.cols = cols;
   m->info.K = dict->K;

@@ -59,6 +59,9 @@ struct tq_tiles_desc {
   uint32_t row_blocks;       // ceil(rows / 16)
   uint32_t has_zero;
   uint32_t table_words;      // tokens are < table_words or the marker
+  // scratch of the tcgen05 kernel: 512-byte header (per vector: output scale, scaled sum of the fixed-point
+  // values) + one slice of digit planes per step (tq_wide_scratch_bytes); nullptr where it is not used
+  uint8_t* xdig;
 };
 
 struct tq_dmat {
@@ -106,7 +109,10 @@ struct tq_tiles_geometry {
   uint32_t steps, row_blocks;
   uint64_t n_tiles, rows_pad;
   uint64_t off_status, off_scale, off_zero, off_tile_raw, off_tokens, off_raw;
-  uint64_t total(uint64_t n_raw) const { return (off_raw + n_raw * 4 + 16384 + 255) / 256 * 256; }
+  // behind the raw words (and their 16 KB of read-ahead padding): the scratch of the tcgen05 kernel for
+  // calls on this matrix alone, sized for 32 vectors (512 + steps * 128 * 128 bytes)
+  uint64_t off_xdig(uint64_t n_raw) const { return (off_raw + n_raw * 4 + 16384 + 1023) / 1024 * 1024; }
+  uint64_t total(uint64_t n_raw) const { return off_xdig(n_raw) + (512 + (uint64_t)steps * 16384 + 1023) / 1024 * 1024; }
 };
 inline tq_tiles_geometry tq_tiles_layout(uint32_t rows, uint32_t cols) {
   auto up = [](uint64_t v, uint64_t a) { return (v + a - 1) / a * a; };
@@ -193,10 +199,20 @@ struct tq_stack {
   uint32_t grid = 0, table_words = 0;
   const uint32_t* d_table = nullptr;
   const tq_tiles_desc* d_descs = nullptr;  // DEVICE
-  // [0] all matrices; [1] those whose rows are short enough for the kernel that keeps a whole row of
-  // activation digits in shared memory; [2] the others (column-panel kernel)
-  tq_stack_plan plan[3];
+  // [0] all matrices, split by tiles (decompress, bf16 decode); [1] those whose rows are short enough for
+  // the kernel that keeps a whole row of activation digits in shared memory; [2] the others and [3] all
+  // matrices, split into groups of whole row blocks for the tcgen05 kernel
+  tq_stack_plan plan[4];
+  bool run_narrow = false, run_wide_long = false, run_wide_all = false;  // kernels one tq_fused_gemv_stack call launches
 };
+
+// The tcgen05 fused decode + product for 1..32 vectors (tq_wide.cu): two launches on cuda_stream (digit
+// planes of the activations into each matrix's scratch, then the fused kernel).  d_mats != nullptr: a
+// stack (DEVICE descriptors, segments grouped by CTA); else the single matrix *one*.
+uint64_t tq_wide_scratch_bytes(uint32_t steps, int nb);
+int tq_wide_launch(const tq_tiles_desc* d_mats, int n_mats, const void* d_segs, const uint32_t* d_cta_seg,
+                   const tq_tiles_desc* one, const uint32_t* d_table, uint32_t table_words, int nb, bool levels_signed,
+                   uint32_t grid, void* cuda_stream);
 
 // Phase 2 of the workspace GEMM (tq_gemm_ws.cu), declared here for tq_fused_gemm_ws.
 extern "C" int tq_gemm_bf16_ws(const tq_dmat* m, const void* d_X_bf16, int M, float* d_Y, const void* d_workspace,

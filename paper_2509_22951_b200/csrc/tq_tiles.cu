@@ -43,9 +43,7 @@ struct TilesParams {
   const uint32_t* table;      // 65536 words, zero past the last entry
   uint32_t table_words;       // words of it kept in shared memory
   uint32_t xstride;           // words per digit column in shared memory
-  uint32_t b0;                // stack mode: first batch column of this pass
-  uint32_t nb_valid;          // wide passes: vectors present (<= the kernel's NB)
-};
+  };
 
 template <bool SIGNED>
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -359,297 +357,11 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
     for (uint32_t si = p.cta_seg[blockIdx.x]; si < p.cta_seg[blockIdx.x + 1]; ++si) {
       const TilesSeg sg = p.segs[si];
       tq_tiles_desc d = p.mats[sg.mat];
-      d.x = static_cast<const __nv_bfloat16*>(d.x) + (size_t)p.b0 * d.cols;
-      d.y += (size_t)p.b0 * d.rows;
       cta.run_segment(d, sg.rb_begin, sg.rb_end);
     }
   }
 }
 
-
-// ---------------------------------------------------------------------------------------------
-// Wide batches (3..8 activation vectors per pass): the digit columns of all vectors no longer fit
-// shared memory for a whole row, so the CTA works in column panels of kPanelSteps tiles.  Every warp
-// owns whole row blocks and all warps walk their blocks in step (tile i of every warp covers the
-// same 128 columns), so one panel of digits -- double buffered, rebuilt by all threads while the
-// previous one is in use, one CTA barrier per panel -- serves all 16 warps.  Up to 24 digit columns
-// = three 8-column MMA tiles per decoded word.
-// ---------------------------------------------------------------------------------------------
-constexpr int kPanelSteps = 4;
-constexpr int kPanelStride = kPanelSteps * 32 + 4;  // words per digit column of one panel buffer
-
-struct XInfo8 {
-  double out_scale[8];
-  double sum_x[8];
-};
-
-// Lane L ends up with all digit sums of row L & 15; lanes 0-15 write the even batch columns, lanes
-// 16-31 the odd ones.
-template <int NB, int NT>
-__device__ __noinline__ void panel_finalize(const float* __restrict__ scale, const float* __restrict__ zero,
-                                            float* __restrict__ y, uint32_t rows, uint32_t has_zero, const XInfo8* xi,
-                                            uint32_t nb_valid, uint32_t rb, const int (&c)[NT][4]) {
-  const uint32_t lane = threadIdx.x & 31u;
-  const uint32_t row = lane & 15u, half = lane >> 4;
-  const uint32_t r = rb * 16u + row;
-  int dsum[kDigits * NB];
-#pragma unroll
-  for (int col = 0; col < kDigits * NB; ++col) {
-    const int nt = col >> 3, w = col & 7;
-    const uint32_t src = (row & 7u) * 4u + (uint32_t)(w >> 1);
-    const int lo = __shfl_sync(kFull, c[nt][w & 1], src), hi = __shfl_sync(kFull, c[nt][2 + (w & 1)], src);
-    dsum[col] = (row & 8u) ? hi : lo;
-  }
-#pragma unroll
-  for (int b = 0; b < NB; ++b) {
-    if ((uint32_t)(b & 1) == half && (uint32_t)b < nb_valid && r < rows) {
-      long long Y = 0;
-#pragma unroll
-      for (int k = 0; k < kDigits; ++k) Y += (long long)dsum[kDigits * b + k] << (8 * k);
-      double v = (double)Y * xi->out_scale[b];
-      if (has_zero) v -= (double)zero[r] * xi->sum_x[b];
-      y[(size_t)b * rows + r] = (float)((double)scale[r] * v);
-    }
-  }
-}
-
-template <int W, int NB, bool SIGNED>
-struct PanelCta : CtaBase {
-  static constexpr int kThreads = W * 32;
-  static constexpr int NCOL = kDigits * NB;
-  static constexpr int NT = (NCOL + 7) / 8;
-  static constexpr int kBufWords = 8 * NT * kPanelStride;  // one panel buffer: whole MMA tiles of columns
-
-  uint32_t nb_valid;
-
-  // misc: [0] dead flag, +16 amax bits[8], +64 in_scale[8][2], +128 XInfo8, +256 sums[8]
-  __device__ __forceinline__ uint32_t* amax_bits() { return reinterpret_cast<uint32_t*>(smem + L.misc + 16); }
-  __device__ __forceinline__ float2* in_scale() { return reinterpret_cast<float2*>(smem + L.misc + 64); }
-  __device__ __forceinline__ XInfo8* xinfo() { return reinterpret_cast<XInfo8*>(smem + L.misc + 128); }
-  __device__ __forceinline__ long long* sums() { return reinterpret_cast<long long*>(smem + L.misc + 256); }
-
-  // Per-vector scales (and, with zero points, the sum of each vector's fixed-point values).
-  __device__ void prepare_scales(const tq_tiles_desc& d) {
-    const uint32_t tid = threadIdx.x;
-    const uint32_t G = d.cols >> 2;
-    const uint2* xg = reinterpret_cast<const uint2*>(d.x);
-    if (tid < 8) {
-      amax_bits()[tid] = 0u;
-      sums()[tid] = 0;
-    }
-    __syncthreads();
-    for (uint32_t b = 0; b < nb_valid; ++b) {
-      uint32_t m = 0;
-      for (uint32_t g = tid; g < G; g += kThreads) m = amax4(__ldg(xg + (size_t)b * G + g), m);
-#pragma unroll
-      for (int sft = 16; sft > 0; sft >>= 1) m = max(m, __shfl_xor_sync(kFull, m, sft));
-      if (lane == 0) atomicMax(&amax_bits()[b], m);
-    }
-    __syncthreads();
-    if (tid < 8) {
-      const FixScale f = fix_scale(amax_bits()[tid]);
-      // a non-finite vector: scale 0 (all digits zero) and a NaN output scale
-      in_scale()[tid] = make_float2(f.finite ? f.s1 : 0.f, f.s2);
-      xinfo()->out_scale[tid] = fix_out_scale(f);
-    }
-    __syncthreads();
-    if (d.has_zero) {
-      for (uint32_t b = 0; b < nb_valid; ++b) {
-        const float2 sc = in_scale()[b];
-        long long sum = 0;
-        for (uint32_t g = tid; g < G; g += kThreads) {
-          uint32_t w[kDigits];
-          fix_digits(__ldg(xg + (size_t)b * G + g), sc.x, sc.y, w, &sum);
-        }
-#pragma unroll
-        for (int sft = 16; sft > 0; sft >>= 1) sum += __shfl_xor_sync(kFull, sum, sft);
-        if (lane == 0) atomicAdd(reinterpret_cast<unsigned long long*>(&sums()[b]), (unsigned long long)sum);
-      }
-      __syncthreads();
-      if (tid < 8) xinfo()->sum_x[tid] = xinfo()->out_scale[tid] * (double)sums()[tid];
-    }
-  }
-
-  static constexpr int kItems = (kPanelSteps * 32 * NB + kThreads - 1) / kThreads;  // activation groups per thread and panel
-  // Loads of step panel P (steps P*kPanelSteps ..) of all vectors; fill_store turns them into digits.
-  __device__ __forceinline__ void fill_load(const tq_tiles_desc& d, uint32_t P, uint2 (&v)[kItems]) {
-    const uint32_t G = d.cols >> 2;
-    const uint2* xg = reinterpret_cast<const uint2*>(d.x);
-    constexpr uint32_t kGroups = kPanelSteps * 32;
-#pragma unroll
-    for (int it = 0; it < kItems; ++it) {
-      const uint32_t idx = threadIdx.x + (uint32_t)it * kThreads;
-      const uint32_t gl = idx % kGroups, b = idx / kGroups;
-      const uint32_t g = P * kGroups + gl;
-      v[it] = make_uint2(0u, 0u);  // absent groups: zero bits, zero digits
-      if (idx < kGroups * NB && g < G && b < nb_valid) v[it] = __ldg(xg + (size_t)b * G + g);
-    }
-  }
-  __device__ __forceinline__ void fill_store(uint32_t buf, const uint2 (&v)[kItems]) {
-    uint32_t* xs = reinterpret_cast<uint32_t*>(smem + L.x) + buf * kBufWords;
-    constexpr uint32_t kGroups = kPanelSteps * 32;
-#pragma unroll
-    for (int it = 0; it < kItems; ++it) {
-      const uint32_t idx = threadIdx.x + (uint32_t)it * kThreads;
-      const uint32_t gl = idx % kGroups, b = idx / kGroups;
-      if (idx < kGroups * NB) {
-        uint32_t w[kDigits];
-        const float2 sc = b < nb_valid ? in_scale()[b] : make_float2(0.f, 0.f);
-        fix_digits(v[it], sc.x, sc.y, w, nullptr);
-#pragma unroll
-        for (int k = 0; k < kDigits; ++k) xs[(kDigits * b + k) * kPanelStride + gl] = w[k];
-      }
-    }
-  }
-  // Digits of step panel P of all vectors into buffer `buf`.
-  __device__ __forceinline__ void fill_panel(const tq_tiles_desc& d, uint32_t P, uint32_t buf) {
-    uint2 v[kItems];
-    fill_load(d, P, v);
-    fill_store(buf, v);
-  }
-
-  // Row blocks [rb0, rb1) of matrix d: warp w takes the w-th share of whole row blocks; every warp
-  // runs `n_iter` iterations so that all meet at the panel barriers.
-  __device__ void run_segment(const tq_tiles_desc& d, uint32_t rb0, uint32_t rb1) {
-    __syncthreads();  // the previous segment is done with the panel buffers and the scales
-    prepare_scales(d);
-    const bool table_ok = wait_table();  // the table copy started with the kernel; its first use is below
-    const uint32_t S = d.steps;
-    const uint32_t NP = (S + kPanelSteps - 1) / kPanelSteps;  // panels per row block
-    const uint32_t R = (rb1 - rb0 + W - 1) / W;               // row blocks per warp
-    const uint32_t my0 = min(rb1, rb0 + warp * R), my1 = min(rb1, my0 + R);
-    const uint32_t t0 = my0 * S, t1 = my1 * S;
-    const uint32_t n_real = t1 - t0, n_iter = R * S;
-    fill_panel(d, 0, 0);
-    fill_panel(d, 1 % NP, 1);
-    __syncthreads();
-
-    const uint32_t g = lane >> 2, t = lane & 3u;
-    const uint32_t x_lane = tbl_addr + L.x + (g * kPanelStride + 8u * t) * 4u;
-
-    uint32_t rd = 0, stop_pos = 0, w_pos = 0, i_pos = 0;
-    const uint4* tok = d.tokens + (size_t)t0 * 64u + lane;
-    const uint32_t* trp = d.tile_raw + t0 + 1;
-    uint4 q[2][2] = {};
-    uint32_t tr[2] = {0, 0};
-    if (n_real) {
-      rd = __ldg(d.tile_raw + t0);
-      stop_pos = __ldg(d.tile_raw + t1);
-      w_pos = i_pos = rd & ~(uint32_t)(kChunkWords - 1);
-      for (int k = 0; k < kSlots && i_pos < stop_pos; ++k, i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
-#pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        q[k][0] = ldg_stream(tok + k * 64);
-        q[k][1] = ldg_stream(tok + k * 64 + 32);
-        tr[k] = __ldg(trp + k);
-      }
-      tok += 2 * 64;
-      trp += 2;
-    }
-
-    uint32_t s_p = 0, s_local = 0, rb = my0;  // step, step inside the panel, row block of the tile awaiting the MMAs
-    uint32_t panels_done = 0;                  // index, in the endless panel sequence, of the panel in use
-    int acc[NT][4];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0;
-    uint32_t wbuf[2][16];
-    bool ok = table_ok;
-
-    auto lookups = [&](int k) {
-      const uint32_t rd_next = tr[k];
-      while (ok && rd_next > w_pos) {
-        ok = wait_chunk();
-        w_pos += kChunkWords;
-      }
-      if (!ok) return;
-      lookup16(q[k], wbuf[k]);
-      q[k][0] = ldg_stream(tok);
-      q[k][1] = ldg_stream(tok + 32);
-      tr[k] = __ldg(trp);
-      tok += 64;
-      ++trp;
-      rd = rd_next;
-      __syncwarp();
-      const uint32_t lim = min(stop_pos, (rd & ~(uint32_t)(kChunkWords - 1)) + kRingWords);
-      for (; i_pos < lim; i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
-    };
-    // MMAs of one tile (real == false: the warp has no tile in this iteration but keeps step with the others)
-    auto consume = [&](const uint32_t (&wc)[16], bool real) {
-      if (real) {
-        const uint32_t xp = x_lane + (panels_done & 1u) * (kBufWords * 4u) + 128u * s_local;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          uint4 xa, xb;
-          const uint32_t a = xp + (uint32_t)nt * (8u * kPanelStride * 4u);
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(xa.x), "=r"(xa.y), "=r"(xa.z), "=r"(xa.w) : "r"(a));
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+16];" : "=r"(xb.x), "=r"(xb.y), "=r"(xb.z), "=r"(xb.w) : "r"(a));
-          mma_s8<SIGNED>(acc[nt], wc[0], wc[8], wc[1], wc[9], xa.x, xa.y);
-          mma_s8<SIGNED>(acc[nt], wc[2], wc[10], wc[3], wc[11], xa.z, xa.w);
-          mma_s8<SIGNED>(acc[nt], wc[4], wc[12], wc[5], wc[13], xb.x, xb.y);
-          mma_s8<SIGNED>(acc[nt], wc[6], wc[14], wc[7], wc[15], xb.z, xb.w);
-        }
-      }
-      ++s_local;
-      if (++s_p == S) {  // the row block is complete
-        s_p = 0;
-        if (real) {
-          panel_finalize<NB, NT>(d.scale, d.zero, d.y, d.rows, d.has_zero, xinfo(), nb_valid, rb, acc);
-#pragma unroll
-          for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0;
-        }
-        ++rb;
-        s_local = kPanelSteps;  // a row block ends its last panel, full or not
-      }
-      if (s_local == kPanelSteps) {  // panel finished by every warp: its buffer takes the panel after next
-        s_local = 0;
-        ++panels_done;
-        uint2 v[kItems];
-        fill_load(d, (panels_done + 1u) % NP, v);  // in flight while the warps gather at the barrier
-        __syncthreads();
-        fill_store((panels_done + 1u) & 1u, v);
-      }
-    };
-
-    // when NCOL is not a multiple of 8 the last MMA tile has columns nobody fills or reads back:
-    // whatever the buffer holds there only reaches accumulator columns that are never used
-    for (uint32_t i = 0; i <= n_iter; i += 2) {
-      if (i < n_real && ok) lookups(0);
-      if (i >= 1 && i - 1 < n_iter) consume(wbuf[1], i - 1 < n_real && ok);
-      if (i + 1 < n_real && ok) lookups(1);
-      if (i < n_iter) consume(wbuf[0], i < n_real && ok);
-    }
-    while (ok && n_waited < n_issued) ok = wait_chunk();
-    if (!ok) {
-      *dead_flag() = 1u;
-      if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
-    }
-  }
-};
-
-template <int W, int NB, bool SIGNED>
-__global__ void __launch_bounds__(W * 32, 1) gemv_tiles_panel_kernel(const TilesParams p) {
-  extern __shared__ __align__(1024) uint8_t tiles_smem_raw[];
-  PanelCta<W, NB, SIGNED> cta;
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // see gemv_tiles_kernel
-  cta.setup(tiles_smem_raw, tiles_smem(p.table_words, 2u * PanelCta<W, NB, SIGNED>::kBufWords, W), W, p.table, p.table_words);
-  cta.nb_valid = p.nb_valid;
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-
-  if (p.mats == nullptr) {
-    const uint32_t nrb = p.one.row_blocks;
-    const uint32_t rb0 = (uint32_t)((uint64_t)nrb * blockIdx.x / gridDim.x);
-    const uint32_t rb1 = (uint32_t)((uint64_t)nrb * (blockIdx.x + 1) / gridDim.x);
-    if (rb0 < rb1) cta.run_segment(p.one, rb0, rb1);
-  } else {
-    for (uint32_t si = p.cta_seg[blockIdx.x]; si < p.cta_seg[blockIdx.x + 1]; ++si) {
-      const TilesSeg sg = p.segs[si];
-      tq_tiles_desc d = p.mats[sg.mat];
-      d.x = static_cast<const __nv_bfloat16*>(d.x) + (size_t)p.b0 * d.cols;
-      d.y += (size_t)p.b0 * d.rows;
-      cta.run_segment(d, sg.rb_begin, sg.rb_end);
-    }
-  }
-}
 
 // ---------------------------------------------------------------------------------------------
 // Decompress: one warp per tile, table and raw words read from global memory.
@@ -916,37 +628,6 @@ int launch_tiles(const TilesParams& p, uint32_t grid, size_t smem, cudaStream_t 
   return launch_pdl(kern, grid, kTilesWarps * 32, smem, st, p);
 }
 
-template <int NB, bool SIGNED>
-int launch_panel(const TilesParams& p, uint32_t grid, cudaStream_t st) {
-  auto kern = gemv_tiles_panel_kernel<kTilesWarps, NB, SIGNED>;
-  const size_t smem = tiles_smem(p.table_words, 2u * PanelCta<kTilesWarps, NB, SIGNED>::kBufWords, kTilesWarps).total;
-  if (smem > kSmemLimit) return TQ_ERR_UNSUPPORTED_SHAPE;
-  if (int rc = tq_ensure_dynamic_smem((const void*)kern, smem, "gemv(tiles, wide): raising the dynamic shared memory limit")) return rc;
-  return launch_pdl(kern, grid, kTilesWarps * 32, smem, st, p);
-}
-
-// One pass over nb batch columns (1..8) with the kernel that fits: p.one / p.mats describe the work.
-int launch_pass(TilesParams& p, int nb, bool narrow_two, bool sg, uint32_t grid, cudaStream_t st, bool wide = false) {
-  // the narrow kernel keeps the digits of a whole row in shared memory; rows too long for that
-  // (more than 8448 columns) take the wide kernel, which works in column panels, for any batch
-  const TilesSmem L = tiles_smem(p.table_words, (uint32_t)kDigits * std::min(nb, 2) * p.xstride, kTilesWarps);
-  if (!wide && nb <= 2 && (nb == 1 || narrow_two) && L.total <= kSmemLimit) {
-    if (nb == 1) return sg ? launch_tiles<1, true>(p, grid, L.total, st) : launch_tiles<1, false>(p, grid, L.total, st);
-    return sg ? launch_tiles<2, true>(p, grid, L.total, st) : launch_tiles<2, false>(p, grid, L.total, st);
-  }
-  p.nb_valid = (uint32_t)nb;
-  if (nb <= 4) return sg ? launch_panel<4, true>(p, grid, st) : launch_panel<4, false>(p, grid, st);
-  return sg ? launch_panel<8, true>(p, grid, st) : launch_panel<8, false>(p, grid, st);
-}
-
-// Batch columns of the next pass when `left` remain: 8 at a time; a remainder of one column (or of
-// two where two fit the narrow kernel) goes to the narrow kernel, which has no panel barriers.
-int next_pass(int left, bool narrow_two) {
-  if (left >= 8) return 8;
-  if (left == 2 && !narrow_two) return 2;  // wide kernel with two columns
-  return left;
-}
-
 }  // namespace
 
 // Batch columns one launch can take for this matrix (2, 1, or 0 if even one does not fit).
@@ -957,25 +638,33 @@ int tq_tiles_max_nb(const tq_dmat* m) {
   return 0;
 }
 
-// x: bf16 [B][cols], y: fp32 [B][rows], any B >= 1: passes of up to 8 batch columns.
+// x: bf16 [B][cols], y: fp32 [B][rows], B in 1..32.  One or two vectors whose digits fit beside the
+// table for a whole row take the narrow kernel (tensor-core MACs inside the decoding warps); anything
+// else is one pass of the tcgen05 kernel, whose digit planes go through the scratch area of the
+// matrix's own image.
 int tq_tiles_gemv(const tq_dmat* m, const void* x, int B, float* y, void* cuda_stream) {
-  TilesParams p{};
-  p.one = m->tiles;
-  p.table = m->dict->d_table;
-  p.table_words = m->tiles.table_words;
-  p.xstride = m->tiles.steps * 32u + 4u;
-  const bool narrow_two = tq_tiles_max_nb(m) >= 2;
-  const uint32_t grid = std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count());
+  const int narrow = tq_tiles_max_nb(m);
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const bool sg = m->info.levels_signed != 0;
-  for (int b0 = 0; b0 < B;) {
-    const int nb = next_pass(B - b0, narrow_two);
-    p.one.x = static_cast<const __nv_bfloat16*>(x) + (size_t)b0 * m->info.cols;
-    p.one.y = y + (size_t)b0 * m->info.rows;
-    if (int rc = launch_pass(p, nb, narrow_two, sg, grid, st)) return rc;
-    b0 += nb;
+  if (B <= narrow) {
+    TilesParams p{};
+    p.one = m->tiles;
+    p.one.x = x;
+    p.one.y = y;
+    p.table = m->dict->d_table;
+    p.table_words = m->tiles.table_words;
+    p.xstride = m->tiles.steps * 32u + 4u;
+    const uint32_t grid = std::min<uint32_t>(m->tiles.row_blocks, (uint32_t)sm_count());
+    const size_t smem = tiles_smem(p.table_words, (uint32_t)kDigits * B * p.xstride, kTilesWarps).total;
+    if (B == 1) return sg ? launch_tiles<1, true>(p, grid, smem, st) : launch_tiles<1, false>(p, grid, smem, st);
+    return sg ? launch_tiles<2, true>(p, grid, smem, st) : launch_tiles<2, false>(p, grid, smem, st);
   }
-  return TQ_OK;
+  tq_tiles_desc one = m->tiles;
+  one.x = x;
+  one.y = y;
+  // whole row blocks per warp, 16 warps per CTA: as many CTAs as there are groups of 16 row blocks
+  const uint32_t grid = std::min<uint32_t>((m->tiles.row_blocks + 15u) / 16u, (uint32_t)sm_count());
+  return tq_wide_launch(nullptr, 1, nullptr, nullptr, &one, m->dict->d_table, m->tiles.table_words, B, sg, grid, cuda_stream);
 }
 
 int tq_tiles_decompress(const tq_dmat* m, uint8_t* d_codes, void* cuda_stream) {
@@ -1062,6 +751,66 @@ StackPlan plan_stack(const PlanMat* mats, const uint32_t* ids, int n, uint32_t g
   return pl;
 }
 
+// Work split for the tcgen05 kernel.  Its 16 decoding warps walk whole row blocks in step, so the unit
+// of work is a group of consecutive row blocks of one matrix: 16 of them (256 rows), or fewer when
+// there is not enough work to give every CTA such a group (then fewer warps of more CTAs are busy).
+// Groups go to the CTAs longest first, each to the CTA with the least work so far; a CTA's groups
+// are then put in matrix order and neighbours merged into one segment.
+StackPlan plan_wide(const PlanMat* mats, const uint32_t* ids, int n, uint32_t grid) {
+  uint64_t total_rb = 0;
+  for (int i = 0; i < n; ++i) total_rb += mats[i].row_blocks;
+  uint32_t gsz = 16;
+  if (total_rb < 16ull * grid) gsz = (uint32_t)std::max<uint64_t>(1, (total_rb + grid - 1) / grid);
+  struct Unit {
+    uint64_t cost;
+    uint32_t mat, rb0, rb1;  // mat: index into mats
+  };
+  std::vector<Unit> units;
+  for (int i = 0; i < n; ++i) {
+    const PlanMat& m = mats[i];
+    for (uint32_t rb = 0; rb < m.row_blocks; rb += gsz) {
+      const uint32_t end = std::min(m.row_blocks, rb + gsz);
+      // every warp is busy for as long as the longest row block of the group takes
+      uint64_t longest = 0;
+      for (uint32_t r = rb; r < end; ++r) longest = std::max<uint64_t>(longest, (uint64_t)m.steps * 1024 + (uint64_t)(m.rb_raw[r + 1] - m.rb_raw[r]) * 4);
+      units.push_back(Unit{longest * 16 + 8192, (uint32_t)i, rb, end});
+    }
+  }
+  std::vector<uint32_t> order(units.size());
+  for (uint32_t u = 0; u < order.size(); ++u) order[u] = u;
+  std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return units[a].cost > units[b].cost; });
+  std::vector<uint64_t> load(grid, 0);
+  std::vector<std::vector<uint32_t>> mine(grid);
+  // least-loaded CTA by a heap of (load, cta)
+  std::vector<std::pair<uint64_t, uint32_t>> heap;
+  for (uint32_t c = 0; c < grid; ++c) heap.emplace_back(0ull, c);
+  auto cmp = [](const std::pair<uint64_t, uint32_t>& a, const std::pair<uint64_t, uint32_t>& b) { return a > b; };
+  std::make_heap(heap.begin(), heap.end(), cmp);
+  for (uint32_t u : order) {
+    std::pop_heap(heap.begin(), heap.end(), cmp);
+    auto& top = heap.back();
+    top.first += units[u].cost;
+    mine[top.second].push_back(u);
+    std::push_heap(heap.begin(), heap.end(), cmp);
+  }
+  StackPlan pl;
+  pl.cta_seg.push_back(0);
+  for (uint32_t c = 0; c < grid; ++c) {
+    std::sort(mine[c].begin(), mine[c].end());  // units were made in (matrix, row block) order
+    for (size_t k = 0; k < mine[c].size(); ++k) {
+      const Unit& u = units[mine[c][k]];
+      const bool full = u.rb1 - u.rb0 == 16;
+      if (!pl.segs.empty() && pl.cta_seg.back() < pl.segs.size() && full && pl.segs.back().mat == ids[u.mat] &&
+          pl.segs.back().rb_end == u.rb0 && (pl.segs.back().rb_end - pl.segs.back().rb_begin) % 16 == 0)
+        pl.segs.back().rb_end = u.rb1;  // whole groups of 16 merge: the warps keep 1, 2, ... row blocks each
+      else
+        pl.segs.push_back(TilesSeg{ids[u.mat], u.rb0, u.rb1});
+    }
+    pl.cta_seg.push_back((uint32_t)pl.segs.size());
+  }
+  return pl;
+}
+
 inline uint64_t align256(uint64_t v) { return (v + 255) / 256 * 256; }
 }  // namespace
 
@@ -1089,11 +838,56 @@ int tq_stack_plan_host(int n_mats, const uint32_t* steps, const uint32_t* row_bl
   return TQ_OK;
 }
 
-int tq_stack_size(int n_mats, uint64_t* device_bytes) {
-  if (n_mats < 1 || !device_bytes) return TQ_ERR_INVALID_ARG;
+namespace {
+constexpr int kStackPlans = 4;
+// Does a row of this matrix fit the narrow kernel (digits of one whole row beside the table)?
+bool short_rows(const tq_dmat* m, int nb) {
+  return tiles_smem(m->tiles.table_words, (uint32_t)kDigits * nb * (m->tiles.steps * 32u + 4u), kTilesWarps).total <= kSmemLimit;
+}
+// Which kernels a stack of B vectors runs: B = 1 (and B = 2 where two vectors' digits fit for every
+// short-row matrix) takes the narrow kernel for the matrices with short rows and the tcgen05 kernel
+// for the others; any other B is one pass of the tcgen05 kernel over all matrices.
+struct StackRoute {
+  bool narrow;       // plan[1] through the narrow kernel with B vectors
+  bool wide_long;    // plan[2] through the tcgen05 kernel
+  bool wide_all;     // plan[3] through the tcgen05 kernel
+};
+StackRoute stack_route(const tq_dmat* const* mats, int n_mats, int B) {
+  bool any_short = false, any_long = false, fits_b = B <= 2;
+  for (int i = 0; i < n_mats; ++i) {
+    const bool sh = short_rows(mats[i], 1);
+    any_short |= sh;
+    any_long |= !sh;
+    if (sh && B == 2 && !short_rows(mats[i], 2)) fits_b = false;
+  }
+  StackRoute r{};
+  if (B >= 1 && fits_b && any_short) {
+    r.narrow = true;
+    r.wide_long = any_long;
+  } else if (B >= 1) {
+    r.wide_all = true;
+  }
+  return r;
+}
+uint64_t stack_plan_bytes(int n_mats, uint64_t grid, uint64_t total_rb) {
+  // the tcgen05 plan can hold one segment per group of 16 row blocks (or per CTA for small stacks)
+  const uint64_t max_segs = std::max<uint64_t>((uint64_t)n_mats + grid, total_rb / 16 + (uint64_t)n_mats + grid);
+  return align256(max_segs * sizeof(TilesSeg)) + align256((grid + 1) * 4);
+}
+}  // namespace
+
+int tq_stack_size(const tq_dmat* const* mats, int n_mats, int B, uint64_t* device_bytes) {
+  if (!mats || n_mats < 1 || B < 0 || B > 32 || !device_bytes) return TQ_ERR_INVALID_ARG;
   const uint64_t grid = (uint64_t)sm_count();
-  *device_bytes = align256((uint64_t)n_mats * sizeof(tq_tiles_desc)) +
-                  3 * (align256(((uint64_t)n_mats + grid) * sizeof(TilesSeg)) + align256((grid + 1) * 4));
+  uint64_t total_rb = 0, scratch = 0;
+  for (int i = 0; i < n_mats; ++i) {
+    if (!mats[i] || mats[i]->info.layout != TQ_LAYOUT_TILES) return TQ_ERR_INVALID_ARG;
+    total_rb += mats[i]->tiles.row_blocks;
+  }
+  const StackRoute r = stack_route(mats, n_mats, B);
+  for (int i = 0; i < n_mats; ++i)
+    if (r.wide_all || (r.wide_long && !short_rows(mats[i], 1))) scratch += tq_wide_scratch_bytes(mats[i]->tiles.steps, B);
+  *device_bytes = align256((uint64_t)n_mats * sizeof(tq_tiles_desc)) + kStackPlans * stack_plan_bytes(n_mats, grid, total_rb) + 1024 + scratch;
   return TQ_OK;
 }
 
@@ -1103,8 +897,9 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   if (!mats || (!bound && (d_x || d_y)) || n_mats < 1 || (bound && (B < 1 || B > 32)) || !d_buf || !out ||
       ((uintptr_t)d_buf & 255))
     return TQ_ERR_INVALID_ARG;
+  if (!bound) B = 0;
   uint64_t need = 0;
-  tq_stack_size(n_mats, &need);
+  if (int rc = tq_stack_size(mats, n_mats, B, &need)) return rc;
   if (d_buf_bytes < need) return TQ_ERR_BUFFER_TOO_SMALL;
   for (int i = 0; i < n_mats; ++i) {
     const tq_dmat* m = mats[i];
@@ -1116,33 +911,48 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   tq_stack* s = new (std::nothrow) tq_stack();
   if (!s) return TQ_ERR_NOMEM;
   s->n = n_mats;
-  s->B = bound ? B : 0;
+  s->B = B;
   s->levels_signed = mats[0]->info.levels_signed;
   for (int i = 0; i < n_mats; ++i) s->zero_bf16_exact = s->zero_bf16_exact && mats[i]->zero_bf16_exact;
   s->grid = (uint32_t)sm_count();
   s->table_words = mats[0]->tiles.table_words;
   s->d_table = mats[0]->dict->d_table;
+  const StackRoute route = stack_route(mats, n_mats, B);
+  s->run_narrow = route.narrow;
+  s->run_wide_long = route.wide_long;
+  s->run_wide_all = route.wide_all;
+
+  uint64_t total_rb = 0;
+  for (int i = 0; i < n_mats; ++i) total_rb += mats[i]->tiles.row_blocks;
+  uint8_t* base = static_cast<uint8_t*>(d_buf);
+  const uint64_t plan_bytes = stack_plan_bytes(n_mats, s->grid, total_rb);
+  const uint64_t segs_bytes = plan_bytes - align256((s->grid + 1) * 4);
+  const uint64_t off_plans = align256((uint64_t)n_mats * sizeof(tq_tiles_desc));
+  uint64_t off_scratch = (off_plans + kStackPlans * plan_bytes + 1023) / 1024 * 1024;
 
   std::vector<tq_tiles_desc> descs((size_t)n_mats);
   for (int i = 0; i < n_mats; ++i) {
     descs[i] = mats[i]->tiles;
     descs[i].x = bound ? d_x[i] : nullptr;
     descs[i].y = bound ? d_y[i] : nullptr;
+    descs[i].xdig = nullptr;
+    if (route.wide_all || (route.wide_long && !short_rows(mats[i], 1))) {  // digit planes of this matrix's vectors
+      descs[i].xdig = base + off_scratch;
+      off_scratch += tq_wide_scratch_bytes(mats[i]->tiles.steps, B);
+    }
   }
-  uint8_t* base = static_cast<uint8_t*>(d_buf);
-  const uint64_t segs_bytes = align256(((uint64_t)n_mats + s->grid) * sizeof(TilesSeg));
-  const uint64_t plan_bytes = segs_bytes + align256((s->grid + 1) * 4);
-  const uint64_t off_plans = align256((uint64_t)n_mats * sizeof(tq_tiles_desc));
   cudaStream_t st = (cudaStream_t)cuda_stream;
   int rc = tq_cuda_status((int)cudaMemcpyAsync(base, descs.data(), descs.size() * sizeof(tq_tiles_desc), cudaMemcpyHostToDevice, st), "stack upload");
-  StackPlan pls[3];  // kept alive until the copies have been made
-  for (int k = 0; k < 3 && rc == TQ_OK; ++k) {
+  // [0] all matrices, split by tiles (decompress, bf16 decode); [1] the matrices whose rows are short enough
+  // for the narrow kernel; [2] the others and [3] all matrices, split for the tcgen05 kernel
+  StackPlan pls[kStackPlans];  // kept alive until the copies have been made
+  for (int k = 0; k < kStackPlans && rc == TQ_OK; ++k) {
     std::vector<PlanMat> pm;
     std::vector<uint32_t> ids;
     uint32_t max_steps = 0;
     for (int i = 0; i < n_mats; ++i) {
-      const bool short_rows = tiles_smem(s->table_words, (uint32_t)kDigits * (mats[i]->tiles.steps * 32u + 4u), kTilesWarps).total <= kSmemLimit;
-      if (k == 0 || (k == 1) == short_rows) {
+      const bool sh = short_rows(mats[i], 1);
+      if (k == 0 || k == 3 || (k == 1) == sh) {
         pm.push_back(PlanMat{mats[i]->tiles.steps, mats[i]->tiles.row_blocks, mats[i]->rb_raw.data()});
         ids.push_back((uint32_t)i);
         max_steps = std::max(max_steps, mats[i]->tiles.steps);
@@ -1152,9 +962,14 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
     sp.n_mats = (uint32_t)pm.size();
     sp.xstride = max_steps * 32u + 4u;
     if (pm.empty()) continue;
-    pls[k] = plan_stack(pm.data(), ids.data(), (int)pm.size(), s->grid);
+    if (k == 1 && !route.narrow) continue;
+    if (k == 2 && !route.wide_long) continue;
+    if (k == 3 && !route.wide_all) continue;
+    pls[k] = k >= 2 ? plan_wide(pm.data(), ids.data(), (int)pm.size(), s->grid) : plan_stack(pm.data(), ids.data(), (int)pm.size(), s->grid);
+    if (pls[k].segs.size() * sizeof(TilesSeg) > segs_bytes) rc = TQ_ERR_BUFFER_TOO_SMALL;
     uint8_t* pb = base + off_plans + (uint64_t)k * plan_bytes;
-    rc = tq_cuda_status((int)cudaMemcpyAsync(pb, pls[k].segs.data(), pls[k].segs.size() * sizeof(TilesSeg), cudaMemcpyHostToDevice, st), "stack upload");
+    if (rc == TQ_OK)
+      rc = tq_cuda_status((int)cudaMemcpyAsync(pb, pls[k].segs.data(), pls[k].segs.size() * sizeof(TilesSeg), cudaMemcpyHostToDevice, st), "stack upload");
     if (rc == TQ_OK)
       rc = tq_cuda_status((int)cudaMemcpyAsync(pb + segs_bytes, pls[k].cta_seg.data(), pls[k].cta_seg.size() * 4, cudaMemcpyHostToDevice, st), "stack upload");
     sp.d_segs = pb;
@@ -1172,48 +987,41 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
 }
 
 namespace {
-// The launches of one pass over nb batch columns of a stack: matrices with short rows through the
-// kernel that keeps a whole row of digits in shared memory (nb <= 2 where it fits), the others --
-// or all of them in a wide pass -- through the column-panel kernel.  launch == false only counts.
-int stack_pass(const tq_stack* s, int b0, int nb, bool two, bool launch, cudaStream_t st, int* n_launches) {
-  auto params = [&](const tq_stack_plan& sp) {
-    TilesParams p{};
-    p.mats = s->d_descs;
-    p.segs = static_cast<const TilesSeg*>(sp.d_segs);
-    p.cta_seg = sp.d_cta_seg;
-    p.table = s->d_table;
-    p.table_words = s->table_words;
-    p.xstride = sp.xstride;
-    p.b0 = (uint32_t)b0;
-    return p;
-  };
+// The launches of one tq_fused_gemv_stack call.  launch == false only counts them.
+int stack_run(const tq_stack* s, bool launch, cudaStream_t st, int* n_launches) {
   const bool sg = s->levels_signed != 0;
-  const bool narrow = nb == 1 || (nb == 2 && two);
-  for (int k = narrow ? 1 : 0; k < (narrow ? 3 : 1); ++k) {
-    if (s->plan[k].n_mats == 0) continue;
+  if (s->run_narrow) {
+    const tq_stack_plan& sp = s->plan[1];
     ++*n_launches;
-    if (!launch) continue;
-    TilesParams p = params(s->plan[k]);
-    if (int rc = launch_pass(p, nb, two, sg, s->grid, st, /*wide=*/k != 1)) return rc;
+    if (launch) {
+      TilesParams p{};
+      p.mats = s->d_descs;
+      p.segs = static_cast<const TilesSeg*>(sp.d_segs);
+      p.cta_seg = sp.d_cta_seg;
+      p.table = s->d_table;
+      p.table_words = s->table_words;
+      p.xstride = sp.xstride;
+      const size_t smem = tiles_smem(p.table_words, (uint32_t)kDigits * s->B * p.xstride, kTilesWarps).total;
+      int rc;
+      if (s->B == 1) rc = sg ? launch_tiles<1, true>(p, s->grid, smem, st) : launch_tiles<1, false>(p, s->grid, smem, st);
+      else rc = sg ? launch_tiles<2, true>(p, s->grid, smem, st) : launch_tiles<2, false>(p, s->grid, smem, st);
+      if (rc != TQ_OK) return rc;
+    }
+  }
+  if (s->run_wide_long || s->run_wide_all) {
+    const tq_stack_plan& sp = s->plan[s->run_wide_all ? 3 : 2];
+    *n_launches += 2;  // digit planes, then the fused kernel
+    if (launch)
+      return tq_wide_launch(s->d_descs, s->n, sp.d_segs, sp.d_cta_seg, nullptr, s->d_table, s->table_words, s->B, sg, s->grid, st);
   }
   return TQ_OK;
-}
-// Two batch columns per narrow pass where the digits of two vectors fit for the short-row matrices.
-bool stack_two(const tq_stack* s) {
-  return s->plan[1].n_mats != 0 && tiles_smem(s->table_words, 2u * kDigits * s->plan[1].xstride, kTilesWarps).total <= kSmemLimit;
 }
 }  // namespace
 
 int tq_fused_gemv_stack(const tq_stack* s, void* cuda_stream) {
   if (!s || s->B < 1) return TQ_ERR_INVALID_ARG;
-  const bool two = stack_two(s);
   int n = 0;
-  for (int b0 = 0; b0 < s->B;) {
-    const int nb = next_pass(s->B - b0, two);
-    if (int rc = stack_pass(s, b0, nb, two, true, (cudaStream_t)cuda_stream, &n)) return rc;
-    b0 += nb;
-  }
-  return TQ_OK;
+  return stack_run(s, true, (cudaStream_t)cuda_stream, &n);
 }
 
 int tq_fused_gemv_stack_host(const tq_stack* s, const void* h_x, void* d_x_arena, uint64_t x_bytes, float* h_y,
@@ -1254,13 +1062,8 @@ int tq_decode_bf16_stack(const tq_stack* s, void* const* d_workspace_ptrs, void*
 
 int tq_stack_launches(const tq_stack* s) {
   if (!s) return TQ_ERR_INVALID_ARG;
-  const bool two = stack_two(s);
   int n = 0;
-  for (int b0 = 0; b0 < s->B;) {
-    const int nb = next_pass(s->B - b0, two);
-    stack_pass(s, b0, nb, two, false, nullptr, &n);
-    b0 += nb;
-  }
+  stack_run(s, false, nullptr, &n);
   return n;
 }
 

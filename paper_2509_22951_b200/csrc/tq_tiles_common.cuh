@@ -122,7 +122,10 @@ __device__ __forceinline__ void fix_digits(uint2 v, float s1, float s2, uint32_t
 
 // Bounded in attempts and in time (about 2 s).  Kept out of line and free of references so that the
 // caller's state stays in registers.
-__device__ __noinline__ bool tiles_wait_slow(uint32_t bar, uint32_t par, volatile uint32_t* dead_flag) {
+#ifndef TQ_WAIT_SLOW_INLINING
+#define TQ_WAIT_SLOW_INLINING __noinline__
+#endif
+__device__ TQ_WAIT_SLOW_INLINING bool tiles_wait_slow(uint32_t bar, uint32_t par, volatile uint32_t* dead_flag) {
   const uint64_t t_start = global_ns();
   bool ok = false;
   for (uint32_t i = 0; i < kSpinLimit && !ok; ++i) {

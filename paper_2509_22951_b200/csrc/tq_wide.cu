@@ -28,13 +28,15 @@
 #include <cstdio>
 #include <vector>
 
+// no calls inside the regions whose register budget setmaxnreg changes: the slow path of a wait is inlined
+#define TQ_WAIT_SLOW_INLINING __forceinline__
 #include "tq_tiles_common.cuh"
 
 namespace {
 
 constexpr int kDecodeWarps = 16;
 constexpr int kLoaderWarp = 16, kMmaWarp = 17;
-constexpr int kWideThreads = (kDecodeWarps + 2) * 32;
+constexpr int kWideThreads = (kDecodeWarps + 4) * 32;  // a fifth warpgroup: loader warp, MMA warp, two idle warps
 constexpr int kAStages = 4;            // A-operand stages in tensor memory
 constexpr uint32_t kTmemCols = 512;    // all of it: 2 x 128 accumulator columns + 2 x kAStages x 32 operand columns
 constexpr uint32_t kAccCols = 128;     // columns reserved per accumulator half
@@ -79,6 +81,7 @@ __global__ void __launch_bounds__(256) wide_prepare_kernel(const tq_tiles_desc* 
   __shared__ uint32_t s_amax;
   __shared__ unsigned long long s_sum;
   const tq_tiles_desc d = mats ? mats[blockIdx.y] : one;
+  if (d.xdig == nullptr) return;  // a matrix of the stack that another kernel serves
   const uint32_t b = blockIdx.x, tid = threadIdx.x, lane = tid & 31u;
   const uint32_t G = d.cols >> 2;
   const uint2* xg = reinterpret_cast<const uint2*>(d.x) + (size_t)b * G;
@@ -149,35 +152,37 @@ __device__ __forceinline__ void umma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uin
       : "memory");
 }
 
-// The CTA's segments in order: (matrix, first row block, one past the last).
+// The CTA's segments in order: (matrix, first row block, one past the last).  Fields of a matrix are
+// read where they are needed (FIELD below), not copied as a whole: the loader and MMA warps run on a
+// small register budget.
 struct SegWalk {
-  const WideParams& p;
   uint32_t si, se;
   bool single_pending;
-  __device__ explicit SegWalk(const WideParams& pp) : p(pp), si(0), se(0), single_pending(pp.mats == nullptr) {
+  __device__ explicit SegWalk(const WideParams& p) : si(0), se(0), single_pending(p.mats == nullptr) {
     if (p.mats != nullptr) {
       si = p.cta_seg[blockIdx.x];
       se = p.cta_seg[blockIdx.x + 1];
     }
   }
-  __device__ bool next(tq_tiles_desc& d, uint32_t& rb0, uint32_t& rb1) {
+  __device__ __forceinline__ bool next(const WideParams& p, uint32_t& mat, uint32_t& rb0, uint32_t& rb1) {
     if (p.mats == nullptr) {
       if (!single_pending) return false;
       single_pending = false;
-      d = p.one;
-      const uint32_t nrb = d.row_blocks;
+      mat = 0;
+      const uint32_t nrb = p.one.row_blocks;
       rb0 = (uint32_t)((uint64_t)nrb * blockIdx.x / gridDim.x);
       rb1 = (uint32_t)((uint64_t)nrb * (blockIdx.x + 1) / gridDim.x);
       return rb0 < rb1;
     }
     if (si >= se) return false;
     const TilesSeg sg = p.segs[si++];
-    d = p.mats[sg.mat];
+    mat = sg.mat;
     rb0 = sg.rb_begin;
     rb1 = sg.rb_end;
     return true;
   }
 };
+#define FIELD(name) (p.mats ? p.mats[mat].name : p.one.name)
 
 struct WideCta : CtaBase {
   uint32_t misc_addr;
@@ -227,15 +232,19 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
   const uint32_t stage_bytes = N * 128u;
   bool ok = true;
   SegWalk walk(p);
-  tq_tiles_desc d;
-  uint32_t rb0, rb1;
+  uint32_t mat, rb0, rb1;
 
+  // Registers: 20 warps leave 96 per thread.  The fifth warpgroup needs few, the decoding warps more
+  // (two word buffers, token registers two tiles ahead): 16 x 32 x 112 + 4 x 32 x 56 <= 65536.  Each
+  // budget is set inside the branch it governs.
+  if (warp >= kDecodeWarps) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;" ::: "memory");
   if (warp == kLoaderWarp) {
     // ---- B operand: one slice of digit planes per step, scratch -> shared memory ------------------
     uint32_t gb = 0;
-    while (ok && walk.next(d, rb0, rb1)) {
-      const uint32_t S = d.steps, n_iter = ((rb1 - rb0 + kDecodeWarps - 1) / kDecodeWarps) * S;
-      const uint8_t* src0 = d.xdig + kHdrBytes;
+    while (ok && walk.next(p, mat, rb0, rb1)) {
+      const uint32_t S = FIELD(steps), n_iter = ((rb1 - rb0 + kDecodeWarps - 1) / kDecodeWarps) * S;
+      const uint8_t* src0 = FIELD(xdig) + kHdrBytes;
       for (uint32_t i = 0, s = 0; i < n_iter && ok; ++i) {
         const uint32_t bst = gb % p.b_stages;
         if (gb >= p.b_stages) ok = cta.wait(cta.bar(kOffBEmpty, bst), ((gb / p.b_stages) - 1u) & 1u);
@@ -255,8 +264,8 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
     // ---- tensor core: 2 halves x 4 MMAs (K = 32 each) per step -------------------------------------
     const uint32_t idesc = i8_idesc<SIGNED>(N);
     uint32_t gs = 0, rr = 0;
-    while (ok && walk.next(d, rb0, rb1)) {
-      const uint32_t S = d.steps, nrb = rb1 - rb0, R = (nrb + kDecodeWarps - 1) / kDecodeWarps, n_iter = R * S;
+    while (ok && walk.next(p, mat, rb0, rb1)) {
+      const uint32_t S = FIELD(steps), nrb = rb1 - rb0, R = (nrb + kDecodeWarps - 1) / kDecodeWarps, n_iter = R * S;
       const bool upper = nrb > 8u * R;  // some warp of the second operand half has rows
       for (uint32_t i = 0, s = 0; i < n_iter && ok; ++i) {
         if (s == 0 && rr > 0) ok = cta.wait(cta.bar(kOffAccFree), (rr - 1u) & 1u);  // the accumulators have been read
@@ -287,7 +296,9 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         }
       }
     }
+  }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 112;" ::: "memory");
     // ---- decoding warps ---------------------------------------------------------------------------
     const uint32_t g = lane >> 2, t = lane & 3u;
     const uint32_t half = warp >> 3;
@@ -296,27 +307,27 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
     const uint32_t acc_base = cta.tmem_base + lane_field + half * kAccCols;
     uint32_t gs = 0, rr = 0;
     bool table_ok = false;
-    while (ok && walk.next(d, rb0, rb1)) {
+    while (ok && walk.next(p, mat, rb0, rb1)) {
       if (!table_ok) {  // the table copy started with the kernel; its first use is below
         ok = table_ok = cta.wait_table();
         if (!ok) break;
       }
-      const uint32_t S = d.steps, R = (rb1 - rb0 + kDecodeWarps - 1) / kDecodeWarps;
+      const uint32_t S = FIELD(steps), R = (rb1 - rb0 + kDecodeWarps - 1) / kDecodeWarps;
+      const uint32_t* const raw = FIELD(raw);
       const uint32_t my0 = min(rb1, rb0 + warp * R), my1 = min(rb1, my0 + R);
       const uint32_t t0 = my0 * S, t1 = my1 * S;
       const uint32_t n_real = t1 - t0, n_iter = R * S;
-      const double* hdr = reinterpret_cast<const double*>(d.xdig);
 
       uint32_t rd = 0, stop_pos = 0, w_pos = 0, i_pos = 0;
-      const uint4* tok = d.tokens + (size_t)t0 * 64u + lane;
-      const uint32_t* trp = d.tile_raw + t0 + 1;
+      const uint4* tok = FIELD(tokens) + (size_t)t0 * 64u + lane;
+      const uint32_t* trp = FIELD(tile_raw) + t0 + 1;
       uint4 q[2][2] = {};
       uint32_t tr[2] = {0, 0};
       if (n_real) {
-        rd = __ldg(d.tile_raw + t0);
-        stop_pos = __ldg(d.tile_raw + t1);
+        rd = __ldg(trp - 1);
+        stop_pos = __ldg(trp - 1 + n_real);
         w_pos = i_pos = rd & ~(uint32_t)(kChunkWords - 1);
-        for (int k = 0; k < kSlots && i_pos < stop_pos; ++k, i_pos += kChunkWords) cta.issue_chunk(d.raw, i_pos);
+        for (int k = 0; k < kSlots && i_pos < stop_pos; ++k, i_pos += kChunkWords) cta.issue_chunk(raw, i_pos);
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
           q[k][0] = ldg_stream(tok + k * 64);
@@ -326,19 +337,19 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         tok += 2 * 64;
         trp += 2;
       }
-      uint32_t wbuf[2][16];
+      uint32_t w[16];
       uint32_t s_p = 0, rb = my0;
       bool pending = false;  // a tile has been stored whose arrival on the stage's barrier is still due
       uint32_t pending_stage = 0;
 
-      auto lookups = [&](int k) {  // tile words -> wbuf[k]; token registers reloaded two tiles ahead; ring refilled
+      auto lookups = [&](int k) {  // tile words -> w; token registers reloaded two tiles ahead; ring refilled
         const uint32_t rd_next = tr[k];
         while (ok && rd_next > w_pos) {
           ok = cta.wait_chunk();
           w_pos += kChunkWords;
         }
         if (!ok) return;
-        cta.lookup16(q[k], wbuf[k]);
+        cta.lookup16(q[k], w);
         q[k][0] = ldg_stream(tok);
         q[k][1] = ldg_stream(tok + 32);
         tr[k] = __ldg(trp);
@@ -347,7 +358,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         rd = rd_next;
         __syncwarp();  // every lane has issued its reads of the chunks below rd
         const uint32_t lim = min(stop_pos, (rd & ~(uint32_t)(kChunkWords - 1)) + kRingWords);
-        for (; i_pos < lim; i_pos += kChunkWords) cta.issue_chunk(d.raw, i_pos);
+        for (; i_pos < lim; i_pos += kChunkWords) cta.issue_chunk(raw, i_pos);
       };
       auto publish = [&]() {  // the stored tile is in tensor memory: tell the MMA warp
         if (!pending) return;
@@ -361,10 +372,15 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         ok = ok && cta.wait(cta.bar(kOffAccFull), rr & 1u);
         if (ok && real) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t rows = FIELD(rows), has_zero = FIELD(has_zero);
+          const float* const scale = FIELD(scale);
+          const float* const zero = FIELD(zero);
+          float* const y = FIELD(y);
+          const double* const hdr = reinterpret_cast<const double*>(FIELD(xdig));
           const uint32_t r_lo = rb * 16u + g, r_hi = r_lo + 8u;
-          const float sc_lo = r_lo < d.rows ? __ldg(d.scale + r_lo) : 0.f, sc_hi = r_hi < d.rows ? __ldg(d.scale + r_hi) : 0.f;
-          const float z_lo = (d.has_zero && r_lo < d.rows) ? __ldg(d.zero + r_lo) : 0.f;
-          const float z_hi = (d.has_zero && r_hi < d.rows) ? __ldg(d.zero + r_hi) : 0.f;
+          const float sc_lo = r_lo < rows ? __ldg(scale + r_lo) : 0.f, sc_hi = r_hi < rows ? __ldg(scale + r_hi) : 0.f;
+          const float z_lo = (has_zero && r_lo < rows) ? __ldg(zero + r_lo) : 0.f;
+          const float z_hi = (has_zero && r_hi < rows) ? __ldg(zero + r_hi) : 0.f;
           for (uint32_t bq = 0; bq * 16u < N; ++bq) {
             int v[8];
             asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
@@ -376,8 +392,8 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
               const double os = hdr[b], sx = hdr[32 + b];
               const long long y_lo = (long long)v[0] + ((long long)v[1] << 8) + ((long long)v[4] << 16) + ((long long)v[5] << 24);
               const long long y_hi = (long long)v[2] + ((long long)v[3] << 8) + ((long long)v[6] << 16) + ((long long)v[7] << 24);
-              if (r_lo < d.rows) d.y[(size_t)b * d.rows + r_lo] = (float)((double)sc_lo * ((double)y_lo * os - (double)z_lo * sx));
-              if (r_hi < d.rows) d.y[(size_t)b * d.rows + r_hi] = (float)((double)sc_hi * ((double)y_hi * os - (double)z_hi * sx));
+              if (r_lo < rows) y[(size_t)b * rows + r_lo] = (float)((double)sc_lo * ((double)y_lo * os - (double)z_lo * sx));
+              if (r_hi < rows) y[(size_t)b * rows + r_hi] = (float)((double)sc_hi * ((double)y_hi * os - (double)z_hi * sx));
             }
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -387,14 +403,13 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
       };
       auto step = [&](int k, uint32_t i) {
         const bool real = i < n_real;
-        if (i + 1u < n_real) lookups(k ^ 1);  // the next tile's words, while the previous store completes
+        if (real) lookups(k);  // this tile's words, in flight while the previous store completes
         publish();
         const uint32_t st = gs % kAStages;
         if (ok && gs >= (uint32_t)kAStages) ok = cta.wait(cta.bar(kOffAEmpty, st), ((gs / kAStages) - 1u) & 1u);
         if (!ok) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (real) {
-          const uint32_t(&w)[16] = wbuf[k];
           asm volatile(
               "tcgen05.st.sync.aligned.16x256b.x4.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(
                   a_base + st * kStepCols),
@@ -414,7 +429,6 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         }
       };
 
-      if (n_real) lookups(0);
       for (uint32_t i = 0; i < n_iter && ok; i += 2) {
         step(0, i);
         if (i + 1u < n_iter && ok) step(1, i + 1u);
@@ -424,6 +438,9 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
     }
   }
 
+  // a CTA without work has not waited for its copy of the table yet: nothing may still be landing in
+  // shared memory when the CTA ends
+  if (warp == 0 && ok) ok = cta.wait_table();
   if (!ok) {
     *cta.dead_flag() = 1u;
     if (lane == 0) atomicOr(p.mats ? p.mats[0].status : p.one.status, TQ_STATUS_WAIT_EXPIRED);

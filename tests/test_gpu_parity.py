@@ -398,7 +398,9 @@ def test_stack_matches_oracle_and_single_calls(tq, B):
     xs = [synth.activations(B, c, 300 + i).cuda() for i, (_, c) in enumerate(shapes)]
     ys = [torch.full((B, r), float("nan"), dtype=torch.float32, device="cuda") for r, _ in shapes]
     stack = tq.tq_stack_create(mats, xs, ys)
-    assert stack.launches == -(-B // 8)  # up to 8 batch columns per launch
+    # one vector: the kernel whose warps multiply on the spot; more: digit planes + one pass of the tcgen05 kernel
+    # (two vectors do not fit beside the table for the 8192-column matrix)
+    assert stack.launches == (1 if B == 1 else 2)
     for _ in range(2):  # a second launch reuses everything the first left behind
         for y in ys:
             y.fill_(float("nan"))
@@ -415,7 +417,8 @@ def test_stack_matches_oracle_and_single_calls(tq, B):
 @pytest.mark.parametrize("B", [1, 2, 5])
 def test_stack_with_short_and_long_rows(tq, B):
     """Rows too long for a whole row of activation digits in shared memory (more than 8448 columns)
-    take the column-panel kernel; a stack that mixes both kinds launches one kernel for each."""
+    take the tcgen05 kernel, whose B operand is staged step by step; a one-vector stack that mixes both
+    kinds launches the narrow kernel for the short rows and the tcgen05 pair for the long ones."""
     shapes = [(200, 1024), (40, 12288), (600, 3072), (33, 28672), (64, 8192)]
     rng = np.random.default_rng(200 + B)
     qs = [np.clip(np.rint(rng.standard_t(5, size=s) * 4), -127, 127).astype(np.int8) for s in shapes]
@@ -426,9 +429,9 @@ def test_stack_with_short_and_long_rows(tq, B):
     xs = [synth.activations(B, c, 400 + i).cuda() for i, (_, c) in enumerate(shapes)]
     ys = [torch.full((B, r), float("nan"), dtype=torch.float32, device="cuda") for r, _ in shapes]
     stack = tq.tq_stack_create(mats, xs, ys)
-    # one column: the two kinds of rows take a kernel each; two columns do not fit beside the table for
-    # 8192-column rows, so they and wider batches go through the column-panel kernel in one launch
-    assert stack.launches == (2 if B == 1 else 1)
+    # two vectors do not fit beside the table for 8192-column rows, so they and wider batches go through the
+    # tcgen05 kernel for all matrices (digit planes + one pass)
+    assert stack.launches == (3 if B == 1 else 2)
     tq.tq_fused_gemv_stack(stack)
     torch.cuda.synchronize()
     for m, q, s, x, y in zip(mats, qs, ss, xs, ys):

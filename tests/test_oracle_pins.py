@@ -24,21 +24,22 @@ def _load(name):
 # ----------------------------------------------------------------------------
 @pytest.mark.parametrize("case", _load("handworked_streams.json"), ids=lambda c: c["cite"][:40])
 def test_handworked_streams(case):
-    d = oracle.Dictionary.from_entries(np.array(case["table"], dtype=np.uint8).reshape(-1, 4))
+    L = case.get("seq", 4)
+    d = oracle.Dictionary.from_entries(np.array(case["table"], dtype=np.uint8).reshape(-1, L), seq=L)
     data = np.array(case["bytes"], dtype=np.uint8)
     stream, hits, miss = d.encode(data)
     assert stream.dtype == np.uint16
     assert stream.tolist() == case["stream"]
     assert d.decode(np.array(case["stream"], dtype=np.uint16)).tolist() == case["bytes"]
-    nb, r = divmod(len(case["bytes"]), 4)
+    nb, r = divmod(len(case["bytes"]), L)
     assert hits + miss == nb
-    assert len(case["stream"]) == hits + 5 * miss + ((1 + r) if r else 0)
+    assert len(case["stream"]) == hits + (1 + L) * miss + ((1 + r) if r else 0)
 
 
 @pytest.mark.parametrize("case", _load("handworked_tables.json"), ids=lambda c: c["cite"][:40])
 def test_handworked_tables(case):
     mats = [np.array(m, dtype=np.uint8) for m in case["mats"]]
-    d = oracle.Dictionary.build(mats, top_k=case["top_k"])
+    d = oracle.Dictionary.build(mats, top_k=case["top_k"], seq=case.get("seq", 4))
     assert d.entries.tolist() == case["entries"]
     assert d.counts.tolist() == case["counts"]
 
@@ -54,12 +55,12 @@ def test_handworked_quantizer(case):
 # ----------------------------------------------------------------------------
 # Dictionary: brute force on tiny inputs (O(n^2) counting, different algorithm)
 # ----------------------------------------------------------------------------
-def _brute_table(mats, top_k):
+def _brute_table(mats, top_k, L=4):
     wins = []  # every window, in visiting order
     for m in mats:
         m = list(m)
-        for i in range(len(m) - 3):
-            wins.append(tuple(m[i:i + 4]))
+        for i in range(len(m) - L + 1):
+            wins.append(tuple(m[i:i + L]))
     ranked = []
     for i, w in enumerate(wins):
         first = min(j for j in range(len(wins)) if wins[j] == w)
@@ -86,6 +87,14 @@ def test_dictionary_brute_force(seed):
         assert d.counts.tolist() == want_c
         assert d.n_distinct == n_distinct
         assert d.n_windows == n_win == sum(max(0, len(m) - 3) for m in mats)
+    # Listing 2's sequence_length at 2 and 8: same brute force, windows of that length
+    for L in (2, 8):
+        for top_k in (65535, 3):
+            want_e, want_c, n_distinct, n_win = _brute_table(mats, top_k, L)
+            d = oracle.Dictionary.build(mats, top_k=top_k, seq=L)
+            assert d.entries.tolist() == want_e and d.counts.tolist() == want_c
+            assert d.n_distinct == n_distinct
+            assert d.n_windows == n_win == sum(max(0, len(m) - L + 1) for m in mats)
 
 
 def test_dictionary_invariants_and_escape_collision():
@@ -148,6 +157,53 @@ def test_round_trip_and_size_identity(n, alphabet, top_k):
     codes, esc, tail = _classify(stream)
     assert (codes, esc) == (hits, miss) and tail == (r if r else 0)
     assert int((stream == ESC).sum()) == miss + (1 if r else 0)
+
+
+@pytest.mark.parametrize("L", [1, 2, 3, 8])
+@pytest.mark.parametrize("n", [0, 1, 7, 8, 9, 16, 1000, 4099])
+@pytest.mark.parametrize("alphabet,top_k", [(2, 65535), (6, 20), (3, 0)])
+def test_round_trip_and_size_identity_other_sequence_lengths(L, n, alphabet, top_k):
+    """Listing 2's sequence_length as a parameter: groups, entries and raw runs of L values.  Round
+    trip exact, len = H + (1 + L) M + (1 + r if r), hits = aligned groups that are table members,
+    and an independent walk of the stream finds the same items."""
+    rng = np.random.default_rng(n * 17 + alphabet + 100 * L)
+    data = rng.integers(0, alphabet, size=n).astype(np.uint8)
+    other = rng.integers(0, alphabet, size=131).astype(np.uint8)
+    d = oracle.Dictionary.build([data, other], top_k=top_k, seq=L)
+    assert d.seq == L and d.entries.shape[1] == L
+    stream, hits, miss = d.encode(data)
+    nb, r = divmod(n, L)
+    assert hits + miss == nb
+    assert stream.size == hits + (1 + L) * miss + ((1 + r) if r else 0)
+    assert np.array_equal(d.decode(stream), data)
+    members = {tuple(e) for e in d.entries.tolist()}
+    assert hits == sum(tuple(data[L * b:L * b + L].tolist()) in members for b in range(nb))
+    s, i, codes, esc = stream.tolist(), 0, 0, 0
+    while i < len(s):
+        if s[i] == ESC:
+            assert all(v <= 255 for v in s[i + 1:i + 1 + L])
+            esc += 1
+            i += 1 + L
+        else:
+            assert 1 <= s[i] <= d.K
+            codes += 1
+            i += 1
+    assert codes == hits and esc == miss + (1 if r else 0)
+
+
+def test_closed_forms_other_sequence_lengths():
+    data = np.full(4096, 0x5A, dtype=np.uint8)
+    for L, n_codes in ((2, 2048), (8, 512)):
+        d = oracle.Dictionary.build([data], seq=L)
+        assert d.K == 1 and d.entries.tolist() == [[0x5A] * L] and d.counts.tolist() == [4096 - L + 1]
+        stream, hits, miss = d.encode(data)
+        assert stream.tolist() == [1] * n_codes and miss == 0  # 2 bytes per L weights
+    rng = np.random.default_rng(12)
+    rnd = rng.integers(0, 256, size=800).astype(np.uint8)
+    d0 = oracle.Dictionary.build([rnd], top_k=0, seq=8)
+    stream, hits, miss = d0.encode(rnd)
+    assert hits == 0 and miss == 100 and stream.size == 900  # every group: marker + 8 values
+    assert np.array_equal(stream.reshape(100, 9)[:, 1:].astype(np.uint8).ravel(), rnd)
 
 
 def test_closed_form_constant_matrix():
