@@ -1,11 +1,14 @@
 #!/usr/bin/env python
 """Benchmark of the fused dictionary-decode + GEMV path (one JSON line on stdout).
 
-A step is one pass over every linear layer of one LLaMA-3.2-3B decode step at batch 1 (197 fused
-decode+GEMV launches, replayed as one CUDA graph).  Weights are seeded synthetic Student-t values,
-quantized per row to int8 on the GPU, dictionary-coded with one table for the whole model by the
-host library, and resident in HBM before the timed region starts.  `value` is the effective
-bandwidth on algorithmic bytes (token stream + per-row index and scales + x + y) per second.
+A step is one pass over every linear layer of one LLaMA-3.2-3B decode step at batch 1: 197 products in
+ONE persistent launch (tq_fused_gemv_stack), replayed as a CUDA graph.  Weights are seeded synthetic
+Student-t values, quantized per row to int8, dictionary-coded with one table for the whole model and
+tiled on the GPU, resident in HBM before the timed region starts.  `value` is the effective bandwidth
+on algorithmic bytes (tokens and raw words of the layout + tile index + row scales + x + y) per second.
+Extra keys time the same model at 8 and 32 vectors, launched as a decoder must launch it (layers that
+feed one another in separate launches), the 1B stack, tq_decompress of the whole set and the prefill
+product at 2048 tokens; `cpu_baseline` is the CPU oracle on the host's cores.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--model 3b|1b] [--batch B] [--layers L]
   python bench.py --impl reference ...     # the CPU oracle on a bounded sample of the workload
@@ -198,26 +201,79 @@ def algorithmic_bytes(info, batch):
     return tokens + index + 4 * info.rows + 2 * batch * info.cols + 4 * batch * info.rows
 
 
-def oracle_sample_run(hd_entries, q_host, scales, shapes, batch, sample_idx, reps=1):
+def oracle_sample_run(hd_entries, q_host, scales, shapes, batch, sample_idx, reps=1, workers=1, decode_only=False):
     """The CPU oracle on a bounded sample: Listing 4 decode + fp64 layer product per matrix.
-    Streams are produced beforehand by the oracle's own encoder (untimed).  Returns
-    (algorithmic bytes of the sample, [seconds per repetition])."""
+    Streams are produced beforehand by the oracle's own encoder (untimed).  The oracle itself is
+    single-threaded plain C; with workers > 1 the matrices of the sample are dealt to that many
+    Python threads (the ctypes calls release the interpreter lock), each running the unchanged
+    oracle on its share.  Returns (algorithmic bytes of the sample, [wall seconds per repetition],
+    [wall seconds of the decode alone per repetition])."""
+    from concurrent.futures import ThreadPoolExecutor
     from oracle import oracle
     od = oracle.Dictionary.from_entries(hd_entries)
-    times = [0.0] * reps
-    total = 0
-    for i in sample_idx:
-        name, rows, cols = shapes[i]
-        stream, h, m = od.encode(q_host[i])
-        x = synth.activations(batch, cols, 7000 + i).double().numpy()
-        total += 2 * (h + 5 * m) + rows * 12 + 2 * batch * cols + 4 * batch * rows
-        for r in range(reps):
+    workers = max(1, min(workers, len(sample_idx)))
+    order = sorted(sample_idx, key=lambda i: -shapes[i][1] * shapes[i][2])
+    shares = [[] for _ in range(workers)]
+    load = [0] * workers
+    for i in order:  # largest first, each to the least loaded worker
+        w = load.index(min(load))
+        shares[w].append(i)
+        load[w] += shapes[i][1] * shapes[i][2]
+    pool = ThreadPoolExecutor(workers)
+
+    def encode_share(share):
+        return {i: od.encode(q_host[i]) for i in share}
+    enc = {}
+    for part in pool.map(encode_share, shares):
+        enc.update(part)
+    xs = {i: synth.activations(batch, shapes[i][2], 7000 + i).double().numpy() for i in sample_idx}
+    total = sum(2 * (enc[i][1] + 5 * enc[i][2]) + shapes[i][1] * 12 + 2 * batch * shapes[i][2] + 4 * batch * shapes[i][1]
+                for i in sample_idx)
+
+    def run_share(args):
+        share, with_product = args
+        for i in share:
+            _, rows, cols = shapes[i]
+            codes = od.decode(enc[i][0], rows * cols).reshape(rows, cols).view(np.int8)
+            if with_product:
+                oracle.layer_forward(codes, scales[i], xs[i])
+    times, dec_times = [], []
+    for r in range(reps):
+        t0 = time.perf_counter()
+        list(pool.map(run_share, [(sh, True) for sh in shares]))
+        times.append(time.perf_counter() - t0)
+        if decode_only:
             t0 = time.perf_counter()
-            codes = od.decode(stream, rows * cols).reshape(rows, cols).view(np.int8)
-            oracle.layer_forward(codes, scales[i], x)
-            times[r] += time.perf_counter() - t0
-        del stream
-    return total, times
+            list(pool.map(run_share, [(sh, False) for sh in shares]))
+            dec_times.append(time.perf_counter() - t0)
+    pool.shutdown()
+    return total, times, dec_times
+
+
+def time_stack(tq, stack, stream, reps, warmup=3):
+    """ms per tq_fused_gemv_stack call, replayed as a CUDA graph, CUDA events on the launching stream."""
+    with torch.cuda.stream(stream):
+        tq.tq_fused_gemv_stack(stack)  # kernel attributes are set outside the capture
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            tq.tq_fused_gemv_stack(stack)
+        for _ in range(warmup):
+            g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def batch_operands(shapes, batch, device):
+    xs = [synth.activations(batch, cols, 7000 + i, device=device) for i, (_, rows, cols) in enumerate(shapes)]
+    ys = [torch.zeros((batch, rows), dtype=torch.float32, device=device) for _, rows, cols in shapes]
+    return xs, ys
 
 
 def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
@@ -297,6 +353,30 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
                                      "frac_of_measured_hbm": alg / (ms * 1e-3) / 1e9 / measured_peaks()[0],
                                      "grouping": "{q,k,v} {o} {gate,up} {down} per decoder layer, then the output head"}
         del dep_stacks, g
+    if args.layout == "tiles" and not args.per_layer and not args.shapes and "xs" in extra and args.batch == 1 and args.model == "3b":
+        # the other batch sizes of the same workload (one pass of the tcgen05 kernel over all 197 matrices) ...
+        peak = measured_peaks()[0]
+        for b in (8, 32):
+            xs_b, ys_b = batch_operands(shapes, b, device)
+            st_b = tq.tq_stack_create(mats, xs_b, ys_b)
+            ms_b = time_stack(tq, st_b, stream, 100)
+            alg_b = sum(algorithmic_bytes(i, b) for i in infos)
+            out["batch%d" % b] = {"workload": f"llama3.2-3b linear stack ({len(mats)} matrices), batch {b}", "ms": ms_b,
+                                  "launches": st_b.launches, "GB_per_s": alg_b / (ms_b * 1e-3) / 1e9,
+                                  "frac_of_measured_hbm": alg_b / (ms_b * 1e-3) / 1e9 / peak,
+                                  "us_per_token": ms_b * 1e3 / b, "kernel": "wide_prepare_kernel + gemv_wide_kernel"}
+            del st_b, xs_b, ys_b
+        # ... and the 1B stack (BASELINE config 3) at batch 1, with its own table
+        shapes1 = synth.llama32_linear_shapes("1b")
+        m1, xs1, ys1, hd1, _, _, _, _, _, _ = build_model(tq, shapes1, 1, device, 0, None, layout=2)
+        st1 = tq.tq_stack_create(m1, xs1, ys1)
+        ms1 = time_stack(tq, st1, stream, 300)
+        alg1 = sum(algorithmic_bytes(m.info, 1) for m in m1)
+        out["llama1b_batch1"] = {"workload": f"llama3.2-1b linear stack ({len(m1)} matrices), batch 1", "ms": ms1, "us_per_token": ms1 * 1e3,
+                                 "launches": st1.launches, "algorithmic_bytes": alg1, "GB_per_s": alg1 / (ms1 * 1e-3) / 1e9,
+                                 "frac_of_measured_hbm": alg1 / (ms1 * 1e-3) / 1e9 / peak, "K": hd1.K}
+        del st1, m1, xs1, ys1, hd1
+        torch.cuda.empty_cache()
     if args.layout != "stream":
         M = args.prefill_tokens
         max_rows = max(i.rows for i in infos)
@@ -344,10 +424,15 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
                     tq.tq_fused_gemm(m, Xs[m.info.cols], Y[: M * m.info.rows].view(M, m.info.rows))
 
         ms = timed(run_gemm, 3)
+        reps = max(3, int(1100.0 / ms) + 1)  # at least a second of timed work: the power cap has acted, the sustained peak is the denominator
+        ms = timed(run_gemm, reps)
         flops = 2.0 * M * n_weights
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
         pk = float(peaks.get("bf16_tflops_sustained", 1400.0))
-        out["prefill"] = {"tokens": M, "ms": ms,
+        pk_burst = float(peaks.get("bf16_tflops", 1590.0))
+        ws_bytes = sum(sum(b for b in slot_bytes) for _ in range(2)) if args.layout == "tiles" else 0
+        out["prefill"] = {"tokens": M, "ms": ms, "reps": reps, "timed_region_ms": ms * reps, "workspace_bytes": ws_bytes,
+                          "frac_of_measured_bf16_burst": flops / (ms * 1e-3) / 1e12 / pk_burst,
                           "call": ("tq_decode_bf16_stack + tq_gemm_plan_run (TMA-fed tcgen05 GEMM over all products of the group) per %d decoder layer(s)" % max(1, args.prefill_layers_per_launch)) if args.layout == "tiles"
                           else "tq_fused_gemm (decode inside the GEMM)", "TFLOP_per_s": flops / (ms * 1e-3) / 1e12,
                           "frac_of_measured_bf16_sustained": flops / (ms * 1e-3) / 1e12 / pk, "peak_TFLOP_per_s": pk}
@@ -392,6 +477,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the tq_decompress / tq_fused_gemm timings")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "rows"],
+                    help="N > 1 GPUs: replicas = every rank runs the whole model (weak scaling, no collective); rows = every "
+                         "matrix split by output rows over the ranks, one all-gather of the outputs per step (strong scaling)")
     ap.add_argument("--prefill-tokens", type=int, default=2048)
     ap.add_argument("--prefill-layers-per-launch", type=int, default=14, help="decoder layers per decode + GEMM launch pair of the prefill leg")
     args = ap.parse_args()
@@ -458,6 +546,10 @@ def main():
     log(f"[rank {rank}] built {len(mats)} matrices, {n_weights/1e9:.3f} G weights, hit rate {hits/(hits+miss):.4f}, "
         f"stream {stream_bytes/1e9:.3f} GB, setup {stats}")
 
+    if args.shard == "rows" and world > 1:
+        run_row_sharded(tq, args, shapes, workload, device, rank, world, local_rank, dd, mats, scales, xs, alg_bytes, stats)
+        return
+
     stream = torch.cuda.Stream(device)
     use_stack = args.layout == "tiles" and not args.per_layer
     hit_rate_device = 1.0 - sum(i.n_raw_words for i in infos) / (hits + miss)
@@ -468,8 +560,8 @@ def main():
         def step_plain():
             tq.tq_fused_gemv_stack(stack)
     else:
-        per_pass = 4 if args.layout != "tiles" else 2
-        launches_per_step = len(mats) * (-(-args.batch // per_pass))
+        per_pass = 4 if args.layout != "tiles" else 32
+        launches_per_step = len(mats) * (-(-args.batch // per_pass)) * (2 if args.layout == "tiles" and args.batch > 2 else 1)
 
         def step_plain():
             for m, x, y in zip(mats, xs, ys):
@@ -619,7 +711,7 @@ def main():
                           "the flush a step takes %.5f ms (%.1f MB served from L2)"
                           % (2 * L2_BYTES >> 20, ms_unflushed, payload_bytes / 1e6)),
                    "multi_gpu": "independent replicas, no data-path collective" if world > 1 else "single GPU"},
-        "us_per_token": ms_step * 1e3 / args.batch,
+        "us_per_independent_pass": ms_step * 1e3 / args.batch,
         "bytes_per_step": {"algorithmic": alg_bytes, "paper_stream": stream_bytes, "device_payload": payload_bytes,
                            "int8_equivalent": n_weights},
         "pct_of_8TBs_nominal": 100.0 * per_gpu / 8000.0,
@@ -627,34 +719,122 @@ def main():
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
                      "traffic": (TRAFFIC_RATIO["tiles_stack"] * alg_bytes / launches_per_step
-                                 if use_stack and args.batch <= 2 else TRAFFIC.get(args.layout)),
-                     "traffic_note": ("dram bytes per launch, scaled from the ncu capture of a 14-matrix stack "
-                                      "(profiles/gemv_tiles_stack_llama3b_b1.md)" if use_stack and args.batch <= 2 else None),
-                     "kernel": {"stream": "gemv_kernel", "planes": "gemv_planes_kernel", "tiles": "gemv_tiles_kernel"}[args.layout],
+                                 if use_stack and args.batch == 1 else TRAFFIC.get(args.layout)),
+                     "traffic_note": ("not a counter of this run: profile constant %.3f (dram bytes / algorithmic bytes in the ncu capture of a "
+                                      "14-matrix stack of this kernel, profiles/gemv_tiles_stack_llama3b_b1.md) x the algorithmic bytes of the launch"
+                                      % TRAFFIC_RATIO["tiles_stack"] if use_stack and args.batch == 1 else None),
+                     "kernel": {"stream": "gemv_kernel", "planes": "gemv_planes_kernel", "tiles": "gemv_tiles_kernel" if args.batch == 1 else "gemv_wide_kernel"}[args.layout],
                      "peak_source": peak_src,
                      "note": "achieved = algorithmic bytes of the %d launch(es) of a step / step time (launch gaps included)" % launches_per_step},
         "setup_s": stats,
     }
     out.update(extras)
+    # A decoder's layers feed one another: its per-token time is that of the dependency-respecting launch sequence
+    # where it was measured, else (custom workloads) that of the independent pass.
+    dep = extras.get("dependent_launches")
+    out["us_per_token"] = (dep["ms"] * 1e3 if dep else ms_step * 1e3) / args.batch
+    out["us_per_token_source"] = ("dependent_launches leg (layers that feed one another launched one group after the other)" if dep
+                                  else "independent pass (no dependency-respecting leg for this workload)")
     if e2e:
         out["e2e"] = {"value": world * alg_bytes / (e2e["ms_per_step"] * 1e-3) / 1e9, "unit": UNIT,
                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                       "ms_per_step": e2e["ms_per_step"], "steps": e2e["steps"]}
 
     if not args.no_cpu_baseline and args.quantizer == "rows":
-        sample = pick_sample(shapes, 3_300_000_000)  # ~13 s of single-thread oracle work for the 3B stack
-        total, times = oracle_sample_run(hd.entries, q_host, scales, shapes, args.batch, sample, reps=1)
-        best = min(times)
-        out["cpu_baseline"] = {"value": total / best / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-                               "sample": f"first {len(sample)} matrices of the workload "
-                                         f"({sum(shapes[i][1]*shapes[i][2] for i in sample)/1e6:.1f} M weights), "
-                                         f"Listing-4 decode + fp64 product, one pass, {best:.2f} s",
-                               "host_cores_available": ncores}
+        sample = pick_sample(shapes, 3_300_000_000)  # ~6-13 s of single-thread oracle work for the 3B stack
+        nw = sum(shapes[i][1] * shapes[i][2] for i in sample)
+        desc = f"first {len(sample)} matrices of the workload ({nw/1e6:.1f} M weights), Listing-4 decode + fp64 product, one pass"
+        total, t_all, d_all = oracle_sample_run(hd.entries, q_host, scales, shapes, args.batch, sample, reps=1, workers=ncores, decode_only=True)
+        total1, t_one, d_one = oracle_sample_run(hd.entries, q_host, scales, shapes, args.batch, sample, reps=1, workers=1, decode_only=True)
+        used = min(ncores, len(sample))
+        out["cpu_baseline"] = {
+            "value": total / min(t_all) / 1e9, "unit": UNIT, "cores": used, "kind": "oracle",
+            "sample": desc + f", {min(t_all):.2f} s; the single-threaded oracle on {used} worker threads, matrices dealt largest first",
+            "one_core": {"value": total1 / min(t_one) / 1e9, "unit": UNIT, "cores": 1, "seconds": min(t_one)},
+            "decode_only": {"note": "Listing-4 decode alone (no product), same sample; GB/s on the same algorithmic bytes",
+                            "all_cores": {"value": total / min(d_all) / 1e9, "seconds": min(d_all), "cores": used},
+                            "one_core": {"value": total1 / min(d_one) / 1e9, "seconds": min(d_one), "cores": 1}},
+            "host_cores_available": ncores}
     print(json.dumps(out), flush=True)
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_row_sharded(tq, args, shapes, workload, device, rank, world, local_rank, dd, full_mats, scales, xs, alg_bytes, stats):
+    """N GPUs, one model: every matrix split by output rows in whole 16-row blocks (paper_2509_22951_b200/sharding.py),
+    the table and the activations replicated.  A step is this rank's tq_fused_gemv_stack launch over its shards
+    followed by ONE NCCL all-gather of the output arenas; no kernel reads another GPU's memory.  The shards are cut
+    out of the matrices the replica path builds (each rank decompresses its rows again and re-encodes them as
+    matrices of their own), so both modes run on the same weights."""
+    import torch.distributed as dist
+    from paper_2509_22951_b200 import sharding
+    assert args.layout == "tiles" and args.quantizer == "rows"
+    so = sharding.ShardedOutputs(shapes, args.batch, world)
+    shard_mats, keep = [], []
+    for i, m in enumerate(full_mats):
+        r0, r1 = so.ranges[rank][i]
+        if r1 > r0:
+            q = tq.tq_decompress(m).view(torch.int8).view(m.info.rows, m.info.cols)
+            shard_mats.append(tq.tq_upload_device_rows(dd, q, r0, r1, torch.from_numpy(scales[i]).to(device)))
+            keep.append(i)
+            del q
+    del full_mats
+    torch.cuda.empty_cache()
+    arena = torch.zeros(so.arena_len, dtype=torch.float32, device=device)
+    gathered = torch.empty(world * so.arena_len, dtype=torch.float32, device=device)
+    views = so.local_views(arena, rank)
+    stack = tq.tq_stack_create(shard_mats, [xs[i] for i in keep], [views[i] for i in keep])
+    stream = torch.cuda.Stream(device)
+
+    def step():
+        tq.tq_fused_gemv_stack(stack, stream=stream)
+        with torch.cuda.stream(stream):
+            so.all_gather(arena, gathered)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    stream.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    sampler.wait_first()
+    dist.barrier()
+    torch.cuda.synchronize()
+    t_start = time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize()
+    dist.barrier()
+    clocks = sampler.stop(t_start, time.time())
+    t = torch.tensor([e0.elapsed_time(e1) / args.steps], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t[0].item())
+    status = 0
+    for m in shard_mats:
+        status |= tq.tq_device_status(m)
+    assert status == 0, f"device status {status}"
+    if rank == 0:
+        peak, peak_src = measured_peaks()
+        value = alg_bytes / (ms_step * 1e-3) / 1e9  # the bytes of ONE model, streamed once per step by all ranks together
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": DTYPE[args.layout],
+            "data": "synthetic",
+            "config": {"workload": workload, "multi_gpu": "rows of every matrix split over %d GPUs in whole 16-row blocks, table and "
+                       "activations replicated, one NCCL all-gather of %d bytes per rank per step" % (world, 4 * so.arena_len),
+                       "l2": "inputs larger than L2: each rank streams %.2f GB per step" % (alg_bytes / world / 1e9)},
+            "us_per_independent_pass": ms_step * 1e3 / args.batch, "gpu_launches": stack.launches * args.steps, "clocks": clocks,
+            "roofline": {"bound": "hbm", "achieved": value / world, "peak": peak, "unit": "GB/s", "frac": value / world / peak,
+                         "traffic": None, "kernel": "gemv_tiles_kernel" if args.batch == 1 else "gemv_wide_kernel", "peak_source": peak_src,
+                         "note": "per GPU: its share of the algorithmic bytes / step time, the all-gather included"},
+            "setup_s": stats}), flush=True)
+    dist.barrier()
+    dist.destroy_process_group()
 
 
 def run_reference(args, shapes, workload):
@@ -669,8 +849,8 @@ def run_reference(args, shapes, workload):
         q_host[i], scales[i] = oracle.quantize_rows(w)
     od = oracle.Dictionary.build([q_host[i] for i in sample])  # the oracle's own table over the sample
     log(f"reference setup {time.time()-t0:.1f} s, sample {sample}")
-    total, times = oracle_sample_run(od.entries, q_host, scales, shapes, args.batch, sample,
-                                     reps=max(args.warmup, 1) + args.steps)
+    total, times, _ = oracle_sample_run(od.entries, q_host, scales, shapes, args.batch, sample,
+                                        reps=max(args.warmup, 1) + args.steps)
     times = times[max(args.warmup, 1):]
     ms = 1e3 * sum(times) / len(times)
     v = total / (ms * 1e-3) / 1e9

@@ -202,6 +202,20 @@ int tq_upload_device(const tq_ddict* dict, const uint8_t* d_levels, uint32_t row
                      const float* d_row_scale, const float* d_row_zero, int levels_signed, void* d_buf,
                      uint64_t d_buf_bytes, void* cuda_stream, tq_dmat** out);
 
+/* Row shard (for a model split by output rows over several GPUs, one process each: every GPU holds
+ * the whole table and the whole activation, decodes and multiplies its own rows, and the outputs are
+ * concatenated; the product needs no reduction because a row's sum never leaves its GPU).  Rows
+ * row_begin .. row_end-1 of the rows x cols matrix at d_levels become a compressed matrix of their
+ * own, exactly as tq_upload_device would make it from those rows alone: Listing 3 takes its decision
+ * per aligned group, and with cols % 4 == 0 no group spans two rows, so the shard's tokens are the
+ * tokens those rows have in the unsharded stream.  d_row_scale / d_row_zero: the full [rows] arrays.
+ * The first row of the shard must start on a 16-byte boundary (TQ_ERR_INVALID_ARG otherwise).
+ * d_buf: tq_upload_device_size(row_end - row_begin, cols) bytes. */
+int tq_upload_device_rows(const tq_ddict* dict, const uint8_t* d_levels, uint32_t rows, uint32_t cols,
+                          uint32_t row_begin, uint32_t row_end, const float* d_row_scale,
+                          const float* d_row_zero, int levels_signed, void* d_buf, uint64_t d_buf_bytes,
+                          void* cuda_stream, tq_dmat** out);
+
 typedef struct tq_dmat_info {
   uint32_t rows, cols, K;
   int32_t layout, levels_signed;

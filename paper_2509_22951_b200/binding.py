@@ -35,7 +35,7 @@ EXPORTS = [
     "tq_strerror", "tq_last_cuda_error", "tq_set_num_threads", "tq_quantize_tensor", "tq_quantize_tensor_bits", "tq_quantize_rows",
     "tq_quantize_rows_device", "tq_build_dictionary", "tq_build_dictionary_device_size", "tq_build_dictionary_device", "tq_dict_from_entries", "tq_dict_entries",
     "tq_encode", "tq_dict_free", "tq_dict_upload_size", "tq_dict_upload", "tq_ddict_free",
-    "tq_upload_size", "tq_upload", "tq_upload_device_size", "tq_upload_device", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
+    "tq_upload_size", "tq_upload", "tq_upload_device_size", "tq_upload_device", "tq_upload_device_rows", "tq_tiles_image_host", "tq_dmat_get_info", "tq_decompress", "tq_fused_gemv",
     "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_gemm_workspace_size",
     "tq_fused_gemm_ws", "tq_decode_bf16", "tq_gemm_bf16_ws", "tq_decode_bf16_stack", "tq_gemm_plan_size", "tq_gemm_plan_create", "tq_gemm_plan_run",
     "tq_gemm_plan_status", "tq_gemm_plan_free", "tq_stack_size", "tq_stack_plan_host", "tq_stack_create",
@@ -86,6 +86,8 @@ def _load() -> C.CDLL:
                                 C.c_int, vp, C.c_uint64, vp, C.POINTER(vp)]),
         "tq_upload_device_size": (C.c_int, [C.c_uint32, C.c_uint32, u64p]),
         "tq_upload_device": (C.c_int, [vp, vp, C.c_uint32, C.c_uint32, vp, vp, C.c_int, vp, C.c_uint64, vp, C.POINTER(vp)]),
+        "tq_upload_device_rows": (C.c_int, [vp, vp, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, vp, vp, C.c_int, vp, C.c_uint64, vp,
+                                            C.POINTER(vp)]),
         "tq_tiles_image_host": (C.c_int, [vp, u16p, C.c_uint64, C.c_uint32, C.c_uint32, f32p, f32p, u8p,
                                           C.c_uint64, u64p, u64p, u32p]),
         "tq_dmat_get_info": (C.c_int, [vp, C.POINTER(_Info)]),
@@ -365,6 +367,26 @@ def tq_upload_device(ddict: DeviceDict, levels: torch.Tensor, row_scale: torch.T
         _check(_lib.tq_upload_device(ddict._h, levels.data_ptr(), rows, cols, row_scale.data_ptr(),
                                      row_zero.data_ptr() if row_zero is not None else None, int(levels_signed),
                                      buf.data_ptr(), buf.numel(), _stream_ptr(cuda_stream), C.byref(out)), "tq_upload_device")
+    return DeviceMatrix(out.value, buf, ddict)
+
+
+def tq_upload_device_rows(ddict: DeviceDict, levels: torch.Tensor, row_begin: int, row_end: int, row_scale: torch.Tensor,
+                          row_zero: torch.Tensor | None = None, levels_signed: bool = True, cuda_stream=None) -> DeviceMatrix:
+    """Rows row_begin .. row_end-1 of `levels` (CUDA int8/uint8 [rows][cols]) as a compressed matrix of their
+    own; row_scale / row_zero are the full [rows] arrays."""
+    assert levels.is_cuda and levels.is_contiguous() and levels.element_size() == 1 and levels.dim() == 2
+    rows, cols = levels.shape
+    assert row_scale.is_cuda and row_scale.dtype == torch.float32 and row_scale.is_contiguous() and row_scale.numel() == rows
+    if row_zero is not None:
+        assert row_zero.is_cuda and row_zero.dtype == torch.float32 and row_zero.is_contiguous() and row_zero.numel() == rows
+    need = C.c_uint64()
+    _check(_lib.tq_upload_device_size(max(row_end - row_begin, 1), cols, C.byref(need)), "tq_upload_device_size")
+    buf = torch.empty(need.value, dtype=torch.uint8, device=levels.device)
+    out = C.c_void_p()
+    with torch.cuda.device(buf.device):
+        _check(_lib.tq_upload_device_rows(ddict._h, levels.data_ptr(), rows, cols, row_begin, row_end, row_scale.data_ptr(),
+                                          row_zero.data_ptr() if row_zero is not None else None, int(levels_signed),
+                                          buf.data_ptr(), buf.numel(), _stream_ptr(cuda_stream), C.byref(out)), "tq_upload_device_rows")
     return DeviceMatrix(out.value, buf, ddict)
 
 

@@ -796,6 +796,17 @@ int tq_upload_device(const tq_ddict* dict, const uint8_t* d_levels, uint32_t row
   return TQ_OK;
 }
 
+int tq_upload_device_rows(const tq_ddict* dict, const uint8_t* d_levels, uint32_t rows, uint32_t cols, uint32_t row_begin,
+                          uint32_t row_end, const float* d_row_scale, const float* d_row_zero, int levels_signed,
+                          void* d_buf, uint64_t d_buf_bytes, void* cuda_stream, tq_dmat** out) {
+  if (!d_levels || !d_row_scale || row_begin >= row_end || row_end > rows || cols == 0) return TQ_ERR_INVALID_ARG;
+  // a row range of a row-major matrix is a matrix of its own: same table, its own image
+  const uint8_t* first = d_levels + (uint64_t)row_begin * cols;
+  if ((uintptr_t)first & 15) return TQ_ERR_INVALID_ARG;
+  return tq_upload_device(dict, first, row_end - row_begin, cols, d_row_scale + row_begin,
+                          d_row_zero ? d_row_zero + row_begin : nullptr, levels_signed, d_buf, d_buf_bytes, cuda_stream, out);
+}
+
 int tq_dmat_get_info(const tq_dmat* m, tq_dmat_info* info) {
   if (!m || !info) return TQ_ERR_INVALID_ARG;
   *info = m->info;

@@ -61,8 +61,7 @@ __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, ui
 
 // Per-CTA values of the activation vectors of the current segment.
 struct XInfo {
-  double out_scale[2];  // 2^(e-22), NaN for a vector with a non-finite element
-  double sum_x[2];      // out_scale * sum_c X[c]
+  double out_scale[2];  // 2^(e-30), NaN for a vector with a non-finite element
 };
 
 // Turns the 16 x 8 accumulator tile (MMA fragment layout: lane 4g+t holds rows g, g+8 and columns
@@ -71,7 +70,8 @@ struct XInfo {
 template <int NB>
 __device__ __noinline__ void tiles_finalize(const float* __restrict__ scale, const float* __restrict__ zero,
                                             float* __restrict__ y, uint32_t rows, uint32_t has_zero, const XInfo* xi,
-                                            uint32_t rb, int c0, int c1, int c2, int c3) {
+                                            const long long* warp_sums, int n_warps, uint32_t rb, int c0, int c1, int c2,
+                                            int c3) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t row = lane & 15u, b = lane >> 4;
   long long Y = 0;
@@ -87,7 +87,11 @@ __device__ __noinline__ void tiles_finalize(const float* __restrict__ scale, con
   const uint32_t r = rb * 16u + row;
   if (b < (uint32_t)NB && r < rows) {
     double v = (double)Y * xi->out_scale[b];
-    if (has_zero) v -= (double)zero[r] * xi->sum_x[b];
+    if (has_zero) {  // zero_r * sum_c x[c] on the same grid: the warps' sums of the fixed-point values
+      long long sx = 0;
+      for (int w = 0; w < n_warps; ++w) sx += warp_sums[b * n_warps + w];
+      v -= (double)zero[r] * (xi->out_scale[b] * (double)sx);
+    }
     y[(size_t)b * rows + r] = (float)((double)scale[r] * v);
   }
 }
@@ -101,58 +105,71 @@ struct TilesCta : CtaBase {
   bool dead = false;
 
   __device__ __forceinline__ uint32_t* misc_u32() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
-  // misc: [0] dead flag, [1..2] amax bits per vector, [4..4+2W) partial ids, then 8-byte aligned XInfo and
-  // reduction scratch
+  // misc (1 KB): [0] dead flag; +16 partial ids [2W]; +192 XInfo; +224 per-warp maxima [NB][W]; +400 table
+  // barrier; +512 per-warp sums of the fixed-point values [NB][W] (64-bit)
   __device__ __forceinline__ uint32_t* part_ids() { return misc_u32() + 4; }
   __device__ __forceinline__ XInfo* xinfo() { return reinterpret_cast<XInfo*>(smem + L.misc + 192); }
-  __device__ __forceinline__ long long* sum_scratch() { return reinterpret_cast<long long*>(smem + L.misc + 256); }
+  __device__ __forceinline__ uint32_t* warp_max() { return reinterpret_cast<uint32_t*>(smem + L.misc + 224); }
+  __device__ __forceinline__ long long* warp_sum() { return reinterpret_cast<long long*>(smem + L.misc + 512); }
 
   // ---- activation vectors -> digit columns in shared memory --------------------------------
+  // Every thread keeps its groups of x in registers between the search for the largest magnitude and
+  // the conversion, so x is read once; one CTA barrier in the middle (per-warp maxima), the caller's
+  // barrier at the end.  Rows of up to kMaxItems * kThreads groups (10240 columns) fit; longer rows
+  // do not come here (their digits would not fit beside the table either).
+  static constexpr int kMaxItems = 5;
   __device__ void prepare_x(const tq_tiles_desc& d) {
     const uint32_t tid = threadIdx.x;
     const uint32_t G = d.cols >> 2;
     uint32_t* xs = reinterpret_cast<uint32_t*>(smem + L.x);
     const uint2* xg = reinterpret_cast<const uint2*>(d.x);
-    if (tid < 2) misc_u32()[1 + tid] = 0u;
-    if (tid < 2 * NB) sum_scratch()[tid] = 0;
-    __syncthreads();
-    // largest magnitude per vector
+    uint2 v[NB][kMaxItems];
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
       uint32_t m = 0;
-      for (uint32_t g = tid; g < G; g += kThreads) m = amax4(__ldg(xg + (size_t)b * G + g), m);
+#pragma unroll
+      for (int it = 0; it < kMaxItems; ++it) {
+        const uint32_t g = tid + (uint32_t)it * kThreads;
+        v[b][it] = g < G ? __ldg(xg + (size_t)b * G + g) : make_uint2(0u, 0u);
+        m = amax4(v[b][it], m);
+      }
 #pragma unroll
       for (int s = 16; s > 0; s >>= 1) m = max(m, __shfl_xor_sync(kFull, m, s));
-      if (lane == 0) atomicMax(&misc_u32()[1 + b], m);
+      if (lane == 0) warp_max()[b * W + warp] = m;
     }
     __syncthreads();
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-      const FixScale f = fix_scale(misc_u32()[1 + b]);
+      uint32_t mb = 0;
+#pragma unroll
+      for (int w = 0; w < W; ++w) mb = max(mb, warp_max()[b * W + w]);
+      const FixScale f = fix_scale(mb);
       const float s1 = f.finite ? f.s1 : 0.f;  // a non-finite vector: all digits zero, NaN output scale
       long long sum = 0;
-      for (uint32_t g = tid; g < G; g += kThreads) {
-        uint32_t w[kDigits];
-        fix_digits(__ldg(xg + (size_t)b * G + g), s1, f.s2, w, &sum);
 #pragma unroll
-        for (int k = 0; k < kDigits; ++k) xs[(kDigits * b + k) * xstride + g] = w[k];
+      for (int it = 0; it < kMaxItems; ++it) {
+        const uint32_t g = tid + (uint32_t)it * kThreads;
+        if (g < G) {
+          uint32_t w[kDigits];
+          fix_digits(v[b][it], s1, f.s2, w, &sum);
+#pragma unroll
+          for (int k = 0; k < kDigits; ++k) xs[(kDigits * b + k) * xstride + g] = w[k];
+        }
       }
       if (d.has_zero) {
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) sum += __shfl_xor_sync(kFull, sum, s);
-        if (lane == 0) atomicAdd(reinterpret_cast<unsigned long long*>(&sum_scratch()[b]), (unsigned long long)sum);
+        if (lane == 0) warp_sum()[b * W + warp] = sum;
       }
       if (tid == 0) xinfo()->out_scale[b] = fix_out_scale(f);
     }
-    __syncthreads();
-    if (tid < NB) xinfo()->sum_x[tid] = xinfo()->out_scale[tid] * (double)sum_scratch()[tid];
     // digit words of the groups between G and the end of the last tile are never initialised: they
     // only ever multiply the zero bytes that token 0 decodes to, and integers have no NaN.
   }
 
   // ---- results ----------------------------------------------------------------------------
   __device__ __forceinline__ void finalize(const tq_tiles_desc& d, uint32_t rb, int c0, int c1, int c2, int c3) {
-    tiles_finalize<NB>(d.scale, d.zero, d.y, d.rows, d.has_zero, xinfo(), rb, c0, c1, c2, c3);
+    tiles_finalize<NB>(d.scale, d.zero, d.y, d.rows, d.has_zero, xinfo(), warp_sum(), W, rb, c0, c1, c2, c3);
   }
 
   // Partial sums of a row block shared with a neighbouring warp; parked in the warp's own ring,
@@ -344,6 +361,20 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
   // while its predecessor was still running.  Nothing above reads or writes what a predecessor
   // produces (the table and the weights are constant); the activations are first read below.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // The CTA's first segment is read before the set-up: the work split and the matrix descriptors are
+  // constant data, so these three dependent loads overlap the barrier set-up and the start of the
+  // table copy instead of following them.
+  uint32_t si = 0, se = 0;
+  TilesSeg sg{};
+  tq_tiles_desc d{};
+  if (p.mats != nullptr) {
+    si = p.cta_seg[blockIdx.x];
+    se = p.cta_seg[blockIdx.x + 1];
+    if (si < se) {
+      sg = p.segs[si];
+      d = p.mats[sg.mat];
+    }
+  }
   cta.setup(tiles_smem_raw, tiles_smem(p.table_words, (uint32_t)kDigits * NB * p.xstride, W), W, p.table, p.table_words);
   cta.xstride = p.xstride;
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -354,12 +385,17 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
     const uint32_t rb1 = (uint32_t)((uint64_t)nrb * (blockIdx.x + 1) / gridDim.x);
     if (rb0 < rb1) cta.run_segment(p.one, rb0, rb1);
   } else {
-    for (uint32_t si = p.cta_seg[blockIdx.x]; si < p.cta_seg[blockIdx.x + 1]; ++si) {
-      const TilesSeg sg = p.segs[si];
-      tq_tiles_desc d = p.mats[sg.mat];
+    while (si < se) {
       cta.run_segment(d, sg.rb_begin, sg.rb_end);
+      if (++si < se) {
+        sg = p.segs[si];
+        d = p.mats[sg.mat];
+      }
     }
   }
+  // a CTA without work has not waited for its copy of the table: nothing may still be landing in
+  // shared memory when the CTA ends
+  if (cta.warp == 0 && !cta.dead) cta.wait_table();
 }
 
 
@@ -881,7 +917,8 @@ int tq_stack_size(const tq_dmat* const* mats, int n_mats, int B, uint64_t* devic
   const uint64_t grid = (uint64_t)sm_count();
   uint64_t total_rb = 0, scratch = 0;
   for (int i = 0; i < n_mats; ++i) {
-    if (!mats[i] || mats[i]->info.layout != TQ_LAYOUT_TILES) return TQ_ERR_INVALID_ARG;
+    if (!mats[i]) return TQ_ERR_INVALID_ARG;
+    if (mats[i]->info.layout != TQ_LAYOUT_TILES) return TQ_ERR_UNSUPPORTED_SHAPE;
     total_rb += mats[i]->tiles.row_blocks;
   }
   const StackRoute r = stack_route(mats, n_mats, B);

@@ -39,7 +39,7 @@ __host__ __device__ inline TilesSmem tiles_smem(uint32_t table_words, uint32_t x
   L.x = L.ring + (uint32_t)warps * kRingWords * 4u;
   L.bar = align_up_u32(L.x + x_words * 4u, 16u);
   L.misc = L.bar + (uint32_t)warps * kSlots * 8u;
-  L.total = L.misc + 512u;
+  L.total = L.misc + 1024u;
   return L;
 }
 

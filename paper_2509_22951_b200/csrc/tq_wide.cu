@@ -28,7 +28,7 @@
 #include <cstdio>
 #include <vector>
 
-// no calls inside the regions whose register budget setmaxnreg changes: the slow path of a wait is inlined
+// the slow path of a wait inlined: a call there makes the compiler spill around every wait of the roles below
 #define TQ_WAIT_SLOW_INLINING __forceinline__
 #include "tq_tiles_common.cuh"
 
@@ -36,7 +36,7 @@ namespace {
 
 constexpr int kDecodeWarps = 16;
 constexpr int kLoaderWarp = 16, kMmaWarp = 17;
-constexpr int kWideThreads = (kDecodeWarps + 4) * 32;  // a fifth warpgroup: loader warp, MMA warp, two idle warps
+constexpr int kWideThreads = (kDecodeWarps + 2) * 32;  // + loader warp + MMA warp
 constexpr int kAStages = 4;            // A-operand stages in tensor memory
 constexpr uint32_t kTmemCols = 512;    // all of it: 2 x 128 accumulator columns + 2 x kAStages x 32 operand columns
 constexpr uint32_t kAccCols = 128;     // columns reserved per accumulator half
@@ -234,11 +234,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
   SegWalk walk(p);
   uint32_t mat, rb0, rb1;
 
-  // Registers: 20 warps leave 96 per thread.  The fifth warpgroup needs few, the decoding warps more
-  // (two word buffers, token registers two tiles ahead): 16 x 32 x 112 + 4 x 32 x 56 <= 65536.  Each
-  // budget is set inside the branch it governs.
-  if (warp >= kDecodeWarps) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;" ::: "memory");
+  // (18 warps leave 96 registers per thread, which the decoding warps fit without spilling.)
   if (warp == kLoaderWarp) {
     // ---- B operand: one slice of digit planes per step, scratch -> shared memory ------------------
     uint32_t gb = 0;
@@ -296,9 +292,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         }
       }
     }
-  }
-  } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 112;" ::: "memory");
+  } else if (warp < kDecodeWarps) {
     // ---- decoding warps ---------------------------------------------------------------------------
     const uint32_t g = lane >> 2, t = lane & 3u;
     const uint32_t half = warp >> 3;

@@ -597,3 +597,58 @@ def test_full_3b_prefill_group_at_2048_tokens(tq, model3b):
         y = plan.Ys[k][torch.from_numpy(tsel).to(device)][:, torch.from_numpy(rsel).to(device)].cpu().numpy().astype(np.float64)
         assert _rel_err(y, yref) <= GEMM_TIGHT, name
         assert tq.tq_device_status(mats[i]) == 0
+
+
+# ------------------------------------------------------------------ row shards (the multi-GPU split, on one GPU)
+@pytest.mark.parametrize("B", [1, 8])
+@pytest.mark.parametrize("world", [2, 3])
+def test_row_shards_reproduce_the_unsharded_product(tq, B, world):
+    """The split a multi-GPU run makes (output rows in whole blocks of 16 per rank, same table), run
+    here one shard after the other on one GPU: shard outputs concatenated must equal the unsharded
+    call bit for bit (the sums are exact integers, so no split can change them), decoded levels of the
+    shards must be the matrix's rows, and the one-arena-per-rank layout must reassemble the stack."""
+    from paper_2509_22951_b200 import sharding
+
+    shapes = [("a", 1000, 3072), ("b", 300, 1024), ("c", 16, 128), ("d", 130, 8192)]
+    rng = np.random.default_rng(500 + B + world)
+    qs = [np.clip(np.rint(rng.standard_t(5, size=(r, c)) * 5), -127, 127).astype(np.int8) for _, r, c in shapes]
+    ss = [(rng.random(r) + 0.5).astype(np.float32) for _, r, _ in shapes]
+    d, _ = _oracle_pack(qs)
+    dd = tq.tq_dict_upload(tq.tq_dict_from_entries(d.entries))
+    qd = [torch.from_numpy(q).cuda() for q in qs]
+    sd = [torch.from_numpy(s).cuda() for s in ss]
+    xs = [synth.activations(B, c, 600 + i).cuda() for i, (_, _, c) in enumerate(shapes)]
+    whole = [tq.tq_upload_device(dd, q, s) for q, s in zip(qd, sd)]
+    y_whole = [tq.tq_fused_gemv(m, x) for m, x in zip(whole, xs)]
+    so = sharding.ShardedOutputs(shapes, B, world)
+    arenas = []
+    for rank in range(world):
+        mats = sharding.upload_row_shards(tq, dd, qd, sd, rank, world)
+        arena = torch.full((so.arena_len,), float("nan"), dtype=torch.float32, device="cuda")
+        views = so.local_views(arena, rank)
+        have = [i for i, m in enumerate(mats) if m is not None]
+        if have:
+            tq.tq_fused_gemv_stack(tq.tq_stack_create([mats[i] for i in have], [xs[i] for i in have], [views[i] for i in have]))
+        torch.cuda.synchronize()
+        for i in have:
+            r0, r1 = so.ranges[rank][i]
+            assert np.array_equal(tq.tq_decompress(mats[i]).cpu().numpy().view(np.int8), qs[i][r0:r1])
+            assert tq.tq_device_status(mats[i]) == 0
+        arenas.append(arena)
+    gathered = torch.cat(arenas)  # what one all-gather leaves on every rank
+    for i, (_, rows, cols) in enumerate(shapes):
+        y = so.full_output(gathered, i)
+        assert torch.equal(y, y_whole[i])
+        yref = oracle.layer_forward(qs[i], ss[i], xs[i].cpu().double().numpy())
+        assert _rel_err(y.cpu().numpy().astype(np.float64), yref) <= TIGHT
+
+
+def test_row_shard_rejects_unaligned_start(tq):
+    q = torch.zeros((40, 12), dtype=torch.int8, device="cuda")  # 12-byte rows: row 1 starts on byte 12
+    s = torch.ones(40, dtype=torch.float32, device="cuda")
+    dd = tq.tq_dict_upload(tq.tq_dict_from_entries(np.zeros((1, 4), dtype=np.uint8)))
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_upload_device_rows(dd, q, 1, 17, s)
+    assert e.value.status == tq.TQ_ERR_INVALID_ARG
+    m = tq.tq_upload_device_rows(dd, q, 4, 20, s)  # row 4 starts on byte 48
+    assert m.info.rows == 16 and m.info.cols == 12

@@ -168,7 +168,9 @@ def test_upload_size_accepts_valid_and_rejects_corrupt(layout):
 
 def test_row_partition_helper_two_ranks_gloo():
     """Row sharding for several GPUs is a plain split of the rows: check with 2 gloo ranks that the
-    shards tile the matrix and that concatenating per-rank oracle outputs gives the full output."""
+    shards tile the matrix in whole blocks of 16 rows, that concatenating per-rank oracle outputs
+    gives the full output, and that the one-collective-per-stack arena layout reassembles every
+    matrix of a stack."""
     import torch.multiprocessing as mp
     mp.spawn(_rank_main, args=(2,), nprocs=2, join=True)
 
@@ -181,19 +183,34 @@ def _rank_main(rank, world):
     os.environ.setdefault("MASTER_PORT", "29531")
     dist.init_process_group("gloo", rank=rank, world_size=world)
     try:
-        rows, cols = 37, 16
         rng = np.random.default_rng(7)
-        q = rng.integers(-127, 128, size=(rows, cols)).astype(np.int8)
-        s = (rng.random(rows) + 0.5).astype(np.float32)
-        x = rng.standard_normal((2, cols))
+        shapes = [("a", 37, 16), ("b", 64, 8), ("c", 5, 12), ("d", 100, 4)]
+        B = 3
+        qs = [rng.integers(-127, 128, size=(r, c)).astype(np.int8) for _, r, c in shapes]
+        ss = [(rng.random(r) + 0.5).astype(np.float32) for _, r, _ in shapes]
+        xs = [rng.standard_normal((B, c)) for _, _, c in shapes]
+        # single matrix
+        rows = shapes[0][1]
         r0, r1 = sharding.row_range(rows, rank, world)
-        y_local = torch.from_numpy(oracle.layer_forward(q[r0:r1], s[r0:r1], x))
+        y_local = torch.from_numpy(oracle.layer_forward(qs[0][r0:r1], ss[0][r0:r1], xs[0]))
         parts = sharding.all_gather_rows(y_local, rows, rank, world)
-        full = torch.from_numpy(oracle.layer_forward(q, s, x))
-        assert torch.equal(parts, full)
-        # shards tile [0, rows)
-        cover = sorted(sharding.row_range(rows, r, world) for r in range(world))
-        assert cover[0][0] == 0 and cover[-1][1] == rows and all(a[1] == b[0] for a, b in zip(cover, cover[1:]))
+        assert torch.equal(parts, torch.from_numpy(oracle.layer_forward(qs[0], ss[0], xs[0])))
+        # shards tile [0, rows) in whole blocks of 16 rows; 5 rows over 2 ranks leave one rank empty
+        for _, rows, _ in shapes:
+            cover = [sharding.row_range(rows, r, world) for r in range(world)]
+            assert cover[0][0] == 0 and cover[-1][1] == rows and all(a[1] == b[0] for a, b in zip(cover, cover[1:]))
+            assert all(a % 16 == 0 for a, _ in cover)
+        assert sharding.row_range(5, 0, 2) == (0, 0) and sharding.row_range(5, 1, 2) == (0, 5)
+        # a stack: every rank writes its slices into its arena, one all-gather, every matrix reassembled
+        so = sharding.ShardedOutputs(shapes, B, world)
+        arena = torch.zeros(so.arena_len, dtype=torch.float64)
+        for i, view in enumerate(so.local_views(arena, rank)):
+            a, b = so.ranges[rank][i]
+            if b > a:
+                view.copy_(torch.from_numpy(oracle.layer_forward(qs[i][a:b], ss[i][a:b], xs[i])))
+        gathered = so.all_gather(arena)
+        for i in range(len(shapes)):
+            assert torch.equal(so.full_output(gathered, i), torch.from_numpy(oracle.layer_forward(qs[i], ss[i], xs[i])))
     finally:
         dist.destroy_process_group()
 
