@@ -372,6 +372,13 @@ int tq_gemm_plan_status(const tq_gemm_plan* plan, void* cuda_stream, uint32_t* s
 void tq_gemm_plan_free(tq_gemm_plan* plan); /* host handle only */
 void tq_stack_free(tq_stack* s);
 
+/* Test hook for the bounded waits inside the kernels (no counterpart in the paper).  While on, the
+ * one- and two-vector TQ_LAYOUT_TILES GEMV kernel is launched expecting one chunk of the table that is
+ * never copied: every wait for the table runs into its limit (about 2 s), the warps give up, the
+ * kernel ends normally with undefined y and TQ_STATUS_WAIT_EXPIRED in the matrix's status word, and
+ * the context stays usable.  Nothing faults, traps or waits without bound.  Off by default. */
+void tq_test_withhold_table_chunk(int on);
+
 /* Read and clear the matrix's device status word (TQ_STATUS_* bits); synchronises cuda_stream. */
 int tq_device_status(const tq_dmat* m, void* cuda_stream, uint32_t* status);
 

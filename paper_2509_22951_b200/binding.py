@@ -39,7 +39,7 @@ EXPORTS = [
     "tq_fused_gemv_host", "tq_fused_gemv_host_static", "tq_fused_gemm", "tq_gemm_workspace_size",
     "tq_fused_gemm_ws", "tq_decode_bf16", "tq_gemm_bf16_ws", "tq_decode_bf16_stack", "tq_gemm_plan_size", "tq_gemm_plan_create", "tq_gemm_plan_run",
     "tq_gemm_plan_status", "tq_gemm_plan_free", "tq_stack_size", "tq_stack_plan_host", "tq_stack_create",
-    "tq_fused_gemv_stack", "tq_fused_gemv_stack_host", "tq_stack_launches", "tq_decompress_stack", "tq_stack_free", "tq_device_status", "tq_dmat_free",
+    "tq_fused_gemv_stack", "tq_fused_gemv_stack_host", "tq_stack_launches", "tq_test_withhold_table_chunk", "tq_decompress_stack", "tq_stack_free", "tq_device_status", "tq_dmat_free",
 ]
 
 
@@ -114,6 +114,7 @@ def _load() -> C.CDLL:
         "tq_fused_gemv_stack": (C.c_int, [vp, vp]),
         "tq_fused_gemv_stack_host": (C.c_int, [vp, vp, vp, C.c_uint64, vp, vp, C.c_uint64, vp]),
         "tq_stack_launches": (C.c_int, [vp]),
+        "tq_test_withhold_table_chunk": (None, [C.c_int]),
         "tq_decompress_stack": (C.c_int, [vp, vp, vp]),
         "tq_stack_free": (None, [vp]),
         "tq_device_status": (C.c_int, [vp, vp, u32p]),
@@ -539,6 +540,11 @@ class Stack:
         if getattr(self, "_h", None) and _lib is not None:
             _lib.tq_stack_free(self._h)
             self._h = None
+
+
+def tq_test_withhold_table_chunk(on: bool) -> None:
+    """Test hook: see tq.h."""
+    _lib.tq_test_withhold_table_chunk(int(bool(on)))
 
 
 def tq_stack_create(mats, xs=None, ys=None, stream=None) -> Stack:

@@ -27,6 +27,12 @@ def is_stale() -> bool:
 
 
 def build_library(force: bool = False, verbose: bool = False) -> Path:
+    # a prebuilt library elsewhere (deployments without nvcc): TQ_LIBTQ=/path/to/libtq.so
+    prebuilt = os.environ.get("TQ_LIBTQ")
+    if prebuilt and not force:
+        if not os.path.exists(prebuilt):
+            raise RuntimeError(f"TQ_LIBTQ={prebuilt} does not exist")
+        return Path(prebuilt)
     if not force and not is_stale():
         return LIB
     nvcc = _nvcc()

@@ -27,6 +27,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 #include <new>
 #include <vector>
@@ -43,6 +44,7 @@ struct TilesParams {
   const uint32_t* table;      // 65536 words, zero past the last entry
   uint32_t table_words;       // words of it kept in shared memory
   uint32_t xstride;           // words per digit column in shared memory
+  uint32_t test_withhold;     // test hook (tq_test_withhold_table_chunk): expect a table chunk that is never copied
   };
 
 template <bool SIGNED>
@@ -63,6 +65,18 @@ __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, ui
 struct XInfo {
   double out_scale[2];  // 2^(e-30), NaN for a vector with a non-finite element
 };
+// Places inside the misc area of the shared-memory plan (TilesCta): XInfo at +192, the warps' sums of the
+// fixed-point values at +512.
+// The CTA's first segment, fetched by one thread during the set-up (gemv_tiles_kernel): at +768.
+struct FirstSegment {
+  uint32_t begin, end;
+  TilesSeg seg;
+  tq_tiles_desc desc;
+};
+constexpr uint32_t kFirstSegmentOffset = 768u;
+static_assert(kFirstSegmentOffset + sizeof(FirstSegment) <= 1024u, "misc area of the shared-memory plan");
+constexpr int kTilesWarpsC = 16;
+constexpr uint32_t kXInfoOffset = 192u, kWarpSumsOffset = 512u, kWarpSumsFromXInfo = kWarpSumsOffset - kXInfoOffset;
 
 // Turns the 16 x 8 accumulator tile (MMA fragment layout: lane 4g+t holds rows g, g+8 and columns
 // 2t, 2t+1) of row block rb into y.  Lane L gathers the four digit sums of row L & 15, batch
@@ -70,8 +84,7 @@ struct XInfo {
 template <int NB>
 __device__ __noinline__ void tiles_finalize(const float* __restrict__ scale, const float* __restrict__ zero,
                                             float* __restrict__ y, uint32_t rows, uint32_t has_zero, const XInfo* xi,
-                                            const long long* warp_sums, int n_warps, uint32_t rb, int c0, int c1, int c2,
-                                            int c3) {
+                                            uint32_t rb, int c0, int c1, int c2, int c3) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t row = lane & 15u, b = lane >> 4;
   long long Y = 0;
@@ -88,8 +101,9 @@ __device__ __noinline__ void tiles_finalize(const float* __restrict__ scale, con
   if (b < (uint32_t)NB && r < rows) {
     double v = (double)Y * xi->out_scale[b];
     if (has_zero) {  // zero_r * sum_c x[c] on the same grid: the warps' sums of the fixed-point values
+      const long long* warp_sums = reinterpret_cast<const long long*>(reinterpret_cast<const uint8_t*>(xi) + kWarpSumsFromXInfo);
       long long sx = 0;
-      for (int w = 0; w < n_warps; ++w) sx += warp_sums[b * n_warps + w];
+      for (int w = 0; w < kTilesWarpsC; ++w) sx += warp_sums[b * kTilesWarpsC + w];
       v -= (double)zero[r] * (xi->out_scale[b] * (double)sx);
     }
     y[(size_t)b * rows + r] = (float)((double)scale[r] * v);
@@ -100,6 +114,7 @@ template <int W, int NB, bool SIGNED>
 struct TilesCta : CtaBase {
   static constexpr int kThreads = W * 32;
   static constexpr int NCOL = kDigits * NB;
+  static_assert(W == kTilesWarpsC, "tiles_finalize sums the per-warp values of kTilesWarpsC warps");
 
   uint32_t xstride;
   bool dead = false;
@@ -108,9 +123,9 @@ struct TilesCta : CtaBase {
   // misc (1 KB): [0] dead flag; +16 partial ids [2W]; +192 XInfo; +224 per-warp maxima [NB][W]; +400 table
   // barrier; +512 per-warp sums of the fixed-point values [NB][W] (64-bit)
   __device__ __forceinline__ uint32_t* part_ids() { return misc_u32() + 4; }
-  __device__ __forceinline__ XInfo* xinfo() { return reinterpret_cast<XInfo*>(smem + L.misc + 192); }
+  __device__ __forceinline__ XInfo* xinfo() { return reinterpret_cast<XInfo*>(smem + L.misc + kXInfoOffset); }
   __device__ __forceinline__ uint32_t* warp_max() { return reinterpret_cast<uint32_t*>(smem + L.misc + 224); }
-  __device__ __forceinline__ long long* warp_sum() { return reinterpret_cast<long long*>(smem + L.misc + 512); }
+  __device__ __forceinline__ long long* warp_sum() { return reinterpret_cast<long long*>(smem + L.misc + kWarpSumsOffset); }
 
   // ---- activation vectors -> digit columns in shared memory --------------------------------
   // Every thread keeps its groups of x in registers between the search for the largest magnitude and
@@ -169,7 +184,7 @@ struct TilesCta : CtaBase {
 
   // ---- results ----------------------------------------------------------------------------
   __device__ __forceinline__ void finalize(const tq_tiles_desc& d, uint32_t rb, int c0, int c1, int c2, int c3) {
-    tiles_finalize<NB>(d.scale, d.zero, d.y, d.rows, d.has_zero, xinfo(), warp_sum(), W, rb, c0, c1, c2, c3);
+    tiles_finalize<NB>(d.scale, d.zero, d.y, d.rows, d.has_zero, xinfo(), rb, c0, c1, c2, c3);
   }
 
   // Partial sums of a row block shared with a neighbouring warp; parked in the warp's own ring,
@@ -188,6 +203,7 @@ struct TilesCta : CtaBase {
   __device__ void run_tiles(const tq_tiles_desc& d, uint32_t t0, uint32_t t1) {
     if (!wait_table()) {  // the table copy started with the kernel; its first use is here
       dead = true;
+      *dead_flag() = 1u;
       if (lane == 0) atomicOr(d.status, TQ_STATUS_WAIT_EXPIRED);
       return;
     }
@@ -320,13 +336,13 @@ struct TilesCta : CtaBase {
 
   // ---- one segment: row blocks [rb0, rb1) of matrix d, all warps ----------------------------
   __device__ void run_segment(const tq_tiles_desc& d, uint32_t rb0, uint32_t rb1) {
+    const uint64_t T = (uint64_t)(rb1 - rb0) * d.steps;
+    const uint32_t t0 = rb0 * d.steps + (uint32_t)(T * warp / W);
+    const uint32_t t1 = rb0 * d.steps + (uint32_t)(T * (warp + 1) / W);
     __syncthreads();  // the previous segment is done with x and with the partials in the rings
     prepare_x(d);
     if (lane < 2) part_ids()[2 * warp + lane] = kNoBlock;
     __syncthreads();
-    const uint64_t T = (uint64_t)(rb1 - rb0) * d.steps;
-    const uint32_t t0 = rb0 * d.steps + (uint32_t)(T * warp / W);
-    const uint32_t t1 = rb0 * d.steps + (uint32_t)(T * (warp + 1) / W);
     if (t0 < t1 && !dead && !*dead_flag()) run_tiles(d, t0, t1);
     __syncthreads();
     // partial row blocks: entries of the same block are adjacent (warp order = tile order)
@@ -361,21 +377,21 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
   // while its predecessor was still running.  Nothing above reads or writes what a predecessor
   // produces (the table and the weights are constant); the activations are first read below.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // The CTA's first segment is read before the set-up: the work split and the matrix descriptors are
-  // constant data, so these three dependent loads overlap the barrier set-up and the start of the
-  // table copy instead of following them.
-  uint32_t si = 0, se = 0;
-  TilesSeg sg{};
-  tq_tiles_desc d{};
-  if (p.mats != nullptr) {
-    si = p.cta_seg[blockIdx.x];
-    se = p.cta_seg[blockIdx.x + 1];
-    if (si < se) {
-      sg = p.segs[si];
-      d = p.mats[sg.mat];
+  // The CTA's first segment is fetched before the set-up by one thread and parked in shared memory: the work
+  // split and the matrix descriptors are constant data, so the three dependent loads that find the work
+  // overlap the barrier set-up and the start of the table copy instead of following them, and no register
+  // holds them meanwhile (registers are short in the tile loop).
+  const TilesSmem plan = tiles_smem(p.table_words, (uint32_t)kDigits * NB * p.xstride, W);
+  FirstSegment* first = reinterpret_cast<FirstSegment*>(tiles_smem_raw + plan.misc + kFirstSegmentOffset);
+  if (p.mats != nullptr && threadIdx.x == 32) {
+    first->begin = p.cta_seg[blockIdx.x];
+    first->end = p.cta_seg[blockIdx.x + 1];
+    if (first->begin < first->end) {
+      first->seg = p.segs[first->begin];
+      first->desc = p.mats[first->seg.mat];
     }
   }
-  cta.setup(tiles_smem_raw, tiles_smem(p.table_words, (uint32_t)kDigits * NB * p.xstride, W), W, p.table, p.table_words);
+  cta.setup(tiles_smem_raw, plan, W, p.table, p.table_words, p.test_withhold != 0u);  // ends with a CTA barrier
   cta.xstride = p.xstride;
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -384,18 +400,21 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
     const uint32_t rb0 = (uint32_t)((uint64_t)nrb * blockIdx.x / gridDim.x);
     const uint32_t rb1 = (uint32_t)((uint64_t)nrb * (blockIdx.x + 1) / gridDim.x);
     if (rb0 < rb1) cta.run_segment(p.one, rb0, rb1);
+    else if (cta.warp == 0) cta.wait_table();  // nothing may still be landing in shared memory when the CTA ends
   } else {
-    while (si < se) {
+    uint32_t si = first->begin;
+    TilesSeg sg = first->seg;
+    tq_tiles_desc d = first->desc;
+    if (si >= p.cta_seg[blockIdx.x + 1] && cta.warp == 0) cta.wait_table();  // a CTA without work: as above
+    while (si < p.cta_seg[blockIdx.x + 1]) {  // the bound is read again rather than kept across a segment
       cta.run_segment(d, sg.rb_begin, sg.rb_end);
-      if (++si < se) {
+      if (++si < p.cta_seg[blockIdx.x + 1]) {
         sg = p.segs[si];
         d = p.mats[sg.mat];
       }
     }
   }
-  // a CTA without work has not waited for its copy of the table: nothing may still be landing in
-  // shared memory when the CTA ends
-  if (cta.warp == 0 && !cta.dead) cta.wait_table();
+  cta.linger_after_failure();
 }
 
 
@@ -630,6 +649,7 @@ __global__ void __launch_bounds__(W * 32, 1) decompress_tiles_smem_kernel(const 
       cta.run_segment(d, p.outs[sg.mat], sg.rb_begin, sg.rb_end);
     }
   }
+  cta.linger_after_failure();
 }
 
 template <bool BF16>
@@ -657,8 +677,11 @@ int launch_pdl(Kern kern, uint32_t grid, uint32_t threads, size_t smem, cudaStre
   return tq_cuda_status((int)cudaLaunchKernelEx(&cfg, kern, p), "gemv(tiles) launch");
 }
 
+std::atomic<int> g_test_withhold{0};
+
 template <int NB, bool SIGNED>
-int launch_tiles(const TilesParams& p, uint32_t grid, size_t smem, cudaStream_t st) {
+int launch_tiles(TilesParams p, uint32_t grid, size_t smem, cudaStream_t st) {
+  p.test_withhold = (uint32_t)g_test_withhold.load();
   auto kern = gemv_tiles_kernel<kTilesWarps, NB, SIGNED>;
   if (int rc = tq_ensure_dynamic_smem((const void*)kern, smem, "gemv(tiles): raising the dynamic shared memory limit")) return rc;
   return launch_pdl(kern, grid, kTilesWarps * 32, smem, st, p);
@@ -851,6 +874,8 @@ inline uint64_t align256(uint64_t v) { return (v + 255) / 256 * 256; }
 }  // namespace
 
 extern "C" {
+
+void tq_test_withhold_table_chunk(int on) { g_test_withhold.store(on ? 1 : 0); }
 
 int tq_stack_plan_host(int n_mats, const uint32_t* steps, const uint32_t* row_blocks, const uint32_t* const* rb_raw,
                        uint32_t n_ctas, uint32_t* segs, uint32_t segs_cap, uint32_t* n_segs, uint32_t* cta_seg) {

@@ -63,11 +63,16 @@ __device__ __forceinline__ uint64_t global_ns() {
 // The table into shared memory with bulk copies (one thread issues them; nothing waits until the
 // first lookup, so the activation set-up and the first loads of the streams overlap the copy).
 constexpr uint32_t kTableBarOffset = 400u;  // inside the misc area of the shared-memory plan
-__device__ __forceinline__ void table_load_async(uint32_t tbl_addr, uint32_t bar, const uint32_t* table, uint32_t words) {
+// withhold_last (test hook): the barrier is told to expect the whole table but the last copy is not made, so
+// the barrier never completes and every wait for the table runs into its limit.
+__device__ __forceinline__ void table_load_async(uint32_t tbl_addr, uint32_t bar, const uint32_t* table, uint32_t words,
+                                                 bool withhold_last = false) {
   const uint32_t bytes = words * 4u;
   mbar_expect_tx(bar, bytes);
-  for (uint32_t off = 0; off < bytes; off += 8192u)
+  for (uint32_t off = 0; off < bytes; off += 8192u) {
+    if (withhold_last && off + 8192u >= bytes) break;
     bulk_g2s(tbl_addr + off, reinterpret_cast<const uint8_t*>(table) + off, min(8192u, bytes - off), bar);
+  }
 }
 
 // ---- activations as block fixed point ------------------------------------------------------
@@ -155,7 +160,7 @@ struct CtaBase {
 
   // Barriers, table copy (asynchronous: wait_table() before the first lookup), one CTA barrier.
   __device__ __forceinline__ void setup(uint8_t* smem_raw, const TilesSmem& plan, int warps, const uint32_t* table,
-                                        uint32_t table_words) {
+                                        uint32_t table_words, bool withhold_last_table_chunk = false) {
     smem = smem_raw;
     L = plan;
     tbl_addr = smem_u32(smem_raw);
@@ -170,8 +175,15 @@ struct CtaBase {
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    if (threadIdx.x == 0) table_load_async(tbl_addr, tbl_addr + L.misc + kTableBarOffset, table, table_words);
+    if (threadIdx.x == 0)
+      table_load_async(tbl_addr, tbl_addr + L.misc + kTableBarOffset, table, table_words, withhold_last_table_chunk);
     __syncthreads();
+  }
+  // After a wait has run out: copies that were issued may still be landing in this CTA's shared memory, so
+  // the CTA stays a little (2 ms) before it ends.
+  __device__ __forceinline__ void linger_after_failure() {
+    if (*dead_flag())
+      for (int i = 0; i < 2000; ++i) __nanosleep(1000);
   }
   // False if the bounded wait ran out.
   __device__ __forceinline__ bool wait_table() {

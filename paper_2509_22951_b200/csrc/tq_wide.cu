@@ -37,19 +37,16 @@ namespace {
 constexpr int kDecodeWarps = 16;
 constexpr int kLoaderWarp = 16, kMmaWarp = 17;
 constexpr int kWideThreads = (kDecodeWarps + 2) * 32;  // + loader warp + MMA warp
-constexpr int kAStages = 4;            // A-operand stages in tensor memory
-constexpr uint32_t kTmemCols = 512;    // all of it: 2 x 128 accumulator columns + 2 x kAStages x 32 operand columns
-constexpr uint32_t kAccCols = 128;     // columns reserved per accumulator half
-constexpr uint32_t kAColBase = 2 * kAccCols;
+constexpr uint32_t kTmemCols = 512;    // all of it: 2 x N accumulator columns, then 2 x a_stages x 32 operand columns
 constexpr uint32_t kStepCols = 32;     // 128 bytes of a row = 32 columns of tensor memory
+constexpr uint32_t kMaxAStages = 8;    // A-operand stages in tensor memory: as many as fit, at most this
 constexpr uint32_t kSmemLimit = 232448u;
 constexpr uint32_t kHdrBytes = 512u;   // scratch header: out_scale[32], sum_x[32] (doubles)
-static_assert(kAColBase + 2 * kAStages * kStepCols <= kTmemCols, "tensor memory plan");
 static_assert((TQ_TILES_TABLE_WORDS * 4u) % 1024u == 0, "the B-operand stages behind the table and the rings must be 1024-byte aligned");
 
 // misc area of the shared-memory plan: [0] dead flag, [8] tensor-memory base, barriers from 16 on
-constexpr uint32_t kOffTmem = 8, kOffAFull = 16, kOffAEmpty = 48, kOffBFull = 80, kOffBEmpty = 112, kOffAccFull = 144,
-                   kOffAccFree = 152;
+constexpr uint32_t kOffTmem = 8, kOffAFull = 16, kOffAEmpty = 80, kOffBFull = 144, kOffBEmpty = 176, kOffAccFull = 208,
+                   kOffAccFree = 216;
 
 struct WideParams {
   const tq_tiles_desc* mats;  // stack mode: DEVICE array; nullptr in single-matrix mode
@@ -60,7 +57,8 @@ struct WideParams {
   uint32_t table_words;
   uint32_t nb;                // vectors, 1..32
   uint32_t n_cols;            // N: digit rows of the B operand, 4 * nb rounded up to a multiple of 16
-  uint32_t b_stages;          // B-operand stages in shared memory
+  uint32_t b_stages;          // B-operand stages in shared memory (2..4)
+  uint32_t a_stages;          // A-operand stages in tensor memory (4..8): (512 - 2 N) / 64, at most kMaxAStages
 };
 
 // Row of the B operand (= accumulator column) that holds digit k of vector b: the two digits a
@@ -205,9 +203,11 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
   const uint32_t smem0 = smem_u32(tiles_smem_raw);
   cta.misc_addr = smem0 + plan.misc;
   if (threadIdx.x == 64) {
-    for (int i = 0; i < 4; ++i) {
+    for (uint32_t i = 0; i < kMaxAStages; ++i) {
       mbar_init(cta.bar(kOffAFull, i), kDecodeWarps);
       mbar_init(cta.bar(kOffAEmpty, i), 1u);
+    }
+    for (uint32_t i = 0; i < 4; ++i) {
       mbar_init(cta.bar(kOffBFull, i), 1u);
       mbar_init(cta.bar(kOffBEmpty, i), 1u);
     }
@@ -230,6 +230,8 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
   const uint32_t warp = cta.warp, lane = cta.lane;
   const uint32_t N = p.n_cols;
   const uint32_t stage_bytes = N * 128u;
+  const uint32_t nst = p.a_stages;
+  const uint32_t a_col0 = 2u * N;  // tensor-memory columns: accumulator halves at 0 and N, then the A stages
   bool ok = true;
   SegWalk walk(p);
   uint32_t mat, rb0, rb1;
@@ -260,14 +262,15 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
     // ---- tensor core: 2 halves x 4 MMAs (K = 32 each) per step -------------------------------------
     const uint32_t idesc = i8_idesc<SIGNED>(N);
     uint32_t gs = 0, rr = 0;
+    uint32_t st = 0, st_wraps = 0;  // A stage of step gs and how often the stages have wrapped: gs = st_wraps * nst + st
     while (ok && walk.next(p, mat, rb0, rb1)) {
       const uint32_t S = FIELD(steps), nrb = rb1 - rb0, R = (nrb + kDecodeWarps - 1) / kDecodeWarps, n_iter = R * S;
       const bool upper = nrb > 8u * R;  // some warp of the second operand half has rows
       for (uint32_t i = 0, s = 0; i < n_iter && ok; ++i) {
         if (s == 0 && rr > 0) ok = cta.wait(cta.bar(kOffAccFree), (rr - 1u) & 1u);  // the accumulators have been read
-        const uint32_t bst = gs % p.b_stages, st = gs % kAStages;
+        const uint32_t bst = gs % p.b_stages;
         if (ok) ok = cta.wait(cta.bar(kOffBFull, bst), (gs / p.b_stages) & 1u);
-        if (ok) ok = cta.wait(cta.bar(kOffAFull, st), (gs / kAStages) & 1u);
+        if (ok) ok = cta.wait(cta.bar(kOffAFull, st), st_wraps & 1u);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (lane == 0) {
@@ -275,10 +278,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
 #pragma unroll
           for (uint32_t h = 0; h < 2; ++h) {
             if (h == 1 && !upper) break;
-            const uint32_t a = cta.tmem_base + kAColBase + (h * kAStages + st) * kStepCols;
+            const uint32_t a = cta.tmem_base + a_col0 + (h * nst + st) * kStepCols;
 #pragma unroll
             for (uint32_t k = 0; k < 4; ++k)
-              umma_i8_ts(cta.tmem_base + h * kAccCols, a + 8u * k, umma_desc(b_tile + k * 32u), idesc, (s | k) != 0u);
+              umma_i8_ts(cta.tmem_base + h * N, a + 8u * k, umma_desc(b_tile + k * 32u), idesc, (s | k) != 0u);
           }
           umma_commit(cta.bar(kOffAEmpty, st));
           umma_commit(cta.bar(kOffBEmpty, bst));
@@ -286,6 +289,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         }
         __syncwarp();
         ++gs;
+        if (++st == nst) {
+          st = 0;
+          ++st_wraps;
+        }
         if (++s == S) {
           s = 0;
           ++rr;
@@ -297,9 +304,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
     const uint32_t g = lane >> 2, t = lane & 3u;
     const uint32_t half = warp >> 3;
     const uint32_t lane_field = (32u * (warp & 3u) + 16u * ((warp >> 2) & 1u)) << 16;
-    const uint32_t a_base = cta.tmem_base + lane_field + kAColBase + half * kAStages * kStepCols;
-    const uint32_t acc_base = cta.tmem_base + lane_field + half * kAccCols;
-    uint32_t gs = 0, rr = 0;
+    const uint32_t a_base = cta.tmem_base + lane_field + a_col0 + half * nst * kStepCols;
+    const uint32_t acc_base = cta.tmem_base + lane_field + half * N;
+    uint32_t rr = 0;
+    uint32_t st = 0, st_wraps = 0;  // A stage of the next step and how often the stages have wrapped
     bool table_ok = false;
     while (ok && walk.next(p, mat, rb0, rb1)) {
       if (!table_ok) {  // the table copy started with the kernel; its first use is below
@@ -335,6 +343,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
       uint32_t s_p = 0, rb = my0;
       bool pending = false;  // a tile has been stored whose arrival on the stage's barrier is still due
       uint32_t pending_stage = 0;
+      // (Reading a finished row block's accumulators back a few tiles into the next row block, and prefetching the
+      // token tiles into L2 as the one-vector kernel does, were both measured slower: +6 % each at 8 vectors.)
+      bool drain_due = false, drain_real = false;
+      uint32_t drain_rb = 0;
 
       auto lookups = [&](int k) {  // tile words -> w; token registers reloaded two tiles ahead; ring refilled
         const uint32_t rd_next = tr[k];
@@ -361,8 +373,12 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         if (lane == 0) mbar_arrive_one(cta.bar(kOffAFull, pending_stage));
         pending = false;
       };
-      // the accumulators of row block `rb` (rows of this warp) -> y
-      auto drain = [&](bool real) {
+      // the accumulators of row block drain_rb (rows of this warp, round rr) -> y
+      auto drain = [&]() {
+        if (!drain_due) return;
+        drain_due = false;
+        const bool real = drain_real;
+        const uint32_t rb = drain_rb;
         ok = ok && cta.wait(cta.bar(kOffAccFull), rr & 1u);
         if (ok && real) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -394,13 +410,13 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         }
         __syncwarp();
         if (lane == 0) mbar_arrive_one(cta.bar(kOffAccFree));
+        ++rr;
       };
       auto step = [&](int k, uint32_t i) {
         const bool real = i < n_real;
         if (real) lookups(k);  // this tile's words, in flight while the previous store completes
         publish();
-        const uint32_t st = gs % kAStages;
-        if (ok && gs >= (uint32_t)kAStages) ok = cta.wait(cta.bar(kOffAEmpty, st), ((gs / kAStages) - 1u) & 1u);
+        if (ok && st_wraps != 0u) ok = cta.wait(cta.bar(kOffAEmpty, st), (st_wraps - 1u) & 1u);
         if (!ok) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (real) {
@@ -413,12 +429,17 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         }
         pending = true;
         pending_stage = st;
-        ++gs;
-        if (++s_p == S) {  // the row block is complete
+        if (++st == nst) {
+          st = 0;
+          ++st_wraps;
+        }
+        if (++s_p == S) {  // the row block is complete: all warps read their rows of the accumulators back
           s_p = 0;
           publish();
-          drain(real);
-          ++rr;
+          drain_due = true;
+          drain_real = real;
+          drain_rb = rb;
+          drain();
           ++rb;
         }
       };
@@ -492,6 +513,7 @@ int tq_wide_launch(const tq_tiles_desc* d_mats, int n_mats, const void* d_segs, 
   uint32_t stages = 4;
   while (stages > 2 && tiles_smem(table_words, stages * p.n_cols * 32u, kDecodeWarps).total > kSmemLimit) --stages;
   p.b_stages = stages;
+  p.a_stages = std::min<uint32_t>(kMaxAStages, (kTmemCols - 2u * p.n_cols) / (2u * kStepCols));
   const size_t smem = tiles_smem(table_words, stages * p.n_cols * 32u, kDecodeWarps).total;
   if (smem > kSmemLimit) return TQ_ERR_UNSUPPORTED_SHAPE;
   cudaStream_t st = (cudaStream_t)cuda_stream;

@@ -652,3 +652,27 @@ def test_row_shard_rejects_unaligned_start(tq):
     assert e.value.status == tq.TQ_ERR_INVALID_ARG
     m = tq.tq_upload_device_rows(dd, q, 4, 20, s)  # row 4 starts on byte 48
     assert m.info.rows == 16 and m.info.cols == 12
+
+
+# ------------------------------------------------------------------ bounded waits
+def test_expired_wait_is_reported_and_the_context_survives(tq):
+    """The waits inside the kernels are bounded.  With the library's test hook on, the one-vector kernel
+    expects a chunk of the table that is never copied: the waits run out (about 2 s), the kernel ends by
+    itself, the status word says so, and the next, ordinary call on the same matrix is correct."""
+    rng = np.random.default_rng(321)
+    q = np.clip(np.rint(rng.standard_t(5, size=(64, 1024)) * 4), -127, 127).astype(np.int8)
+    s = (rng.random(64) + 0.5).astype(np.float32)
+    d, (stream,) = _oracle_pack([q])
+    m = _upload_from_oracle(tq, d, stream, 64, 1024, s, layout=tq.TQ_LAYOUT_TILES)
+    x = synth.activations(1, 1024, 3)
+    yref = oracle.layer_forward(q, s, x.double().numpy())
+    tq.tq_test_withhold_table_chunk(True)
+    try:
+        tq.tq_fused_gemv(m, x.cuda())
+        torch.cuda.synchronize()
+    finally:
+        tq.tq_test_withhold_table_chunk(False)
+    assert tq.tq_device_status(m) == tq.TQ_STATUS_WAIT_EXPIRED
+    y = tq.tq_fused_gemv(m, x.cuda()).cpu().numpy().astype(np.float64)
+    assert _rel_err(y, yref) <= TIGHT
+    assert tq.tq_device_status(m) == 0
