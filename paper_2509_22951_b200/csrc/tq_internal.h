@@ -210,6 +210,7 @@ struct tq_stack {
 // planes of the activations into each matrix's scratch, then the fused kernel).  d_mats != nullptr: a
 // stack (DEVICE descriptors, segments grouped by CTA); else the single matrix *one*.
 uint64_t tq_wide_scratch_bytes(uint32_t steps, int nb);
+constexpr uint32_t kWideGroupRowBlocks = 16;  // row blocks the tcgen05 kernel's CTA works on at a time: one per decoding warp
 int tq_wide_launch(const tq_tiles_desc* d_mats, int n_mats, const void* d_segs, const uint32_t* d_cta_seg,
                    const tq_tiles_desc* one, const uint32_t* d_table, uint32_t table_words, int nb, bool levels_signed,
                    uint32_t grid, void* cuda_stream);

@@ -721,8 +721,8 @@ int tq_tiles_gemv(const tq_dmat* m, const void* x, int B, float* y, void* cuda_s
   tq_tiles_desc one = m->tiles;
   one.x = x;
   one.y = y;
-  // whole row blocks per warp, 16 warps per CTA: as many CTAs as there are groups of 16 row blocks
-  const uint32_t grid = std::min<uint32_t>((m->tiles.row_blocks + 15u) / 16u, (uint32_t)sm_count());
+  // whole row blocks per warp, 16 decoding warps per CTA: as many CTAs as there are groups of 16 row blocks
+  const uint32_t grid = std::min<uint32_t>((m->tiles.row_blocks + kWideGroupRowBlocks - 1u) / kWideGroupRowBlocks, (uint32_t)sm_count());
   return tq_wide_launch(nullptr, 1, nullptr, nullptr, &one, m->dict->d_table, m->tiles.table_words, B, sg, grid, cuda_stream);
 }
 
@@ -818,8 +818,9 @@ StackPlan plan_stack(const PlanMat* mats, const uint32_t* ids, int n, uint32_t g
 StackPlan plan_wide(const PlanMat* mats, const uint32_t* ids, int n, uint32_t grid) {
   uint64_t total_rb = 0;
   for (int i = 0; i < n; ++i) total_rb += mats[i].row_blocks;
-  uint32_t gsz = 16;
-  if (total_rb < 16ull * grid) gsz = (uint32_t)std::max<uint64_t>(1, (total_rb + grid - 1) / grid);
+  const uint32_t G = kWideGroupRowBlocks;
+  uint32_t gsz = G;
+  if (total_rb < (uint64_t)G * grid) gsz = (uint32_t)std::max<uint64_t>(1, (total_rb + grid - 1) / grid);
   struct Unit {
     uint64_t cost;
     uint32_t mat, rb0, rb1;  // mat: index into mats
@@ -832,7 +833,7 @@ StackPlan plan_wide(const PlanMat* mats, const uint32_t* ids, int n, uint32_t gr
       // every warp is busy for as long as the longest row block of the group takes
       uint64_t longest = 0;
       for (uint32_t r = rb; r < end; ++r) longest = std::max<uint64_t>(longest, (uint64_t)m.steps * 1024 + (uint64_t)(m.rb_raw[r + 1] - m.rb_raw[r]) * 4);
-      units.push_back(Unit{longest * 16 + 8192, (uint32_t)i, rb, end});
+      units.push_back(Unit{longest * G + 8192, (uint32_t)i, rb, end});
     }
   }
   std::vector<uint32_t> order(units.size());
@@ -858,10 +859,10 @@ StackPlan plan_wide(const PlanMat* mats, const uint32_t* ids, int n, uint32_t gr
     std::sort(mine[c].begin(), mine[c].end());  // units were made in (matrix, row block) order
     for (size_t k = 0; k < mine[c].size(); ++k) {
       const Unit& u = units[mine[c][k]];
-      const bool full = u.rb1 - u.rb0 == 16;
+      const bool full = u.rb1 - u.rb0 == G;
       if (!pl.segs.empty() && pl.cta_seg.back() < pl.segs.size() && full && pl.segs.back().mat == ids[u.mat] &&
-          pl.segs.back().rb_end == u.rb0 && (pl.segs.back().rb_end - pl.segs.back().rb_begin) % 16 == 0)
-        pl.segs.back().rb_end = u.rb1;  // whole groups of 16 merge: the warps keep 1, 2, ... row blocks each
+          pl.segs.back().rb_end == u.rb0 && (pl.segs.back().rb_end - pl.segs.back().rb_begin) % G == 0)
+        pl.segs.back().rb_end = u.rb1;  // whole groups merge: the warps keep 1, 2, ... row blocks each
       else
         pl.segs.push_back(TilesSeg{ids[u.mat], u.rb0, u.rb1});
     }
@@ -931,8 +932,8 @@ StackRoute stack_route(const tq_dmat* const* mats, int n_mats, int B) {
   return r;
 }
 uint64_t stack_plan_bytes(int n_mats, uint64_t grid, uint64_t total_rb) {
-  // the tcgen05 plan can hold one segment per group of 16 row blocks (or per CTA for small stacks)
-  const uint64_t max_segs = std::max<uint64_t>((uint64_t)n_mats + grid, total_rb / 16 + (uint64_t)n_mats + grid);
+  // the tcgen05 plan can hold one segment per group of row blocks (or per CTA for small stacks)
+  const uint64_t max_segs = std::max<uint64_t>((uint64_t)n_mats + grid, total_rb / kWideGroupRowBlocks + (uint64_t)n_mats + grid);
   return align256(max_segs * sizeof(TilesSeg)) + align256((grid + 1) * 4);
 }
 }  // namespace
