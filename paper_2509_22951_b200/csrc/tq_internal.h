@@ -190,6 +190,11 @@ struct tq_stack_plan {
   const uint32_t* d_cta_seg = nullptr;  // DEVICE: grid + 1 offsets into the segments
   uint32_t n_segs = 0, n_mats = 0;
   uint32_t xstride = 0;                 // words per digit column a whole row of its longest matrix needs
+  // the split of the narrow kernel only: one 128-byte record per segment (segment + matrix descriptor) and
+  // per CTA the record of its first segment; CTAs grid_used.. have no segment and are not launched
+  const void* d_recs = nullptr;
+  const void* d_firsts = nullptr;
+  uint32_t grid_used = 0;
 };
 
 struct tq_stack {

@@ -36,10 +36,20 @@
 
 namespace {
 
+// One segment with everything a CTA needs to run it, in one 128-byte line: [begin, end) are the segments
+// of the CTA the record belongs to, seg and desc this segment and its matrix.
+struct SegRecord {
+  uint32_t begin, end;
+  TilesSeg seg;
+  uint32_t pad0;
+  tq_tiles_desc desc;
+  uint32_t pad1[2];
+};
+static_assert(sizeof(SegRecord) == 128, "one record = one 128-byte line, fetched by one warp");
+
 struct TilesParams {
-  const tq_tiles_desc* mats;  // stack mode: DEVICE array; nullptr in single-matrix mode
-  const TilesSeg* segs;       // stack mode: segments, grouped by CTA
-  const uint32_t* cta_seg;    // stack mode: gridDim.x + 1 offsets into segs
+  const SegRecord* firsts;    // stack mode: DEVICE, per CTA the record of its first segment; nullptr in single-matrix mode
+  const SegRecord* recs;      // stack mode: DEVICE, one record per segment, grouped by CTA
   tq_tiles_desc one;          // single-matrix mode
   const uint32_t* table;      // 65536 words, zero past the last entry
   uint32_t table_words;       // words of it kept in shared memory
@@ -67,14 +77,9 @@ struct XInfo {
 };
 // Places inside the misc area of the shared-memory plan (TilesCta): XInfo at +192, the warps' sums of the
 // fixed-point values at +512.
-// The CTA's first segment, fetched by one thread during the set-up (gemv_tiles_kernel): at +768.
-struct FirstSegment {
-  uint32_t begin, end;
-  TilesSeg seg;
-  tq_tiles_desc desc;
-};
+// The record of the CTA's first segment, fetched by one warp during the set-up (gemv_tiles_kernel): at +768.
 constexpr uint32_t kFirstSegmentOffset = 768u;
-static_assert(kFirstSegmentOffset + sizeof(FirstSegment) <= 1024u, "misc area of the shared-memory plan");
+static_assert(kFirstSegmentOffset + sizeof(SegRecord) <= 1024u, "misc area of the shared-memory plan");
 constexpr int kTilesWarpsC = 16;
 constexpr uint32_t kXInfoOffset = 192u, kWarpSumsOffset = 512u, kWarpSumsFromXInfo = kWarpSumsOffset - kXInfoOffset;
 
@@ -117,7 +122,7 @@ struct TilesCta : CtaBase {
   static_assert(W == kTilesWarpsC, "tiles_finalize sums the per-warp values of kTilesWarpsC warps");
 
   uint32_t xstride;
-  bool dead = false;
+  bool dead = false, waited = false;
 
   __device__ __forceinline__ uint32_t* misc_u32() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
   // misc (1 KB): [0] dead flag; +16 partial ids [2W]; +192 XInfo; +224 per-warp maxima [NB][W]; +400 table
@@ -133,7 +138,8 @@ struct TilesCta : CtaBase {
   // barrier at the end.  Rows of up to kMaxItems * kThreads groups (10240 columns) fit; longer rows
   // do not come here (their digits would not fit beside the table either).
   static constexpr int kMaxItems = 5;
-  __device__ void prepare_x(const tq_tiles_desc& d) {
+  template <class Mid>
+  __device__ __forceinline__ void prepare_x(const tq_tiles_desc& d, Mid&& between) {
     const uint32_t tid = threadIdx.x;
     const uint32_t G = d.cols >> 2;
     uint32_t* xs = reinterpret_cast<uint32_t*>(smem + L.x);
@@ -153,6 +159,7 @@ struct TilesCta : CtaBase {
       if (lane == 0) warp_max()[b * W + warp] = m;
     }
     __syncthreads();
+    between();  // work that needs the rings free and does not need x: placed behind the loads of x
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
       uint32_t mb = 0;
@@ -195,12 +202,49 @@ struct TilesCta : CtaBase {
     if (lane == 0) part_ids()[2 * warp + slot] = rb;
   }
 
+  // ---- the start of a warp's run, fetched before the activations are prepared ----------------
+  // The tile index and the tokens are constant data, so their loads are issued at the very start of a
+  // segment (for a CTA's first segment: before the wait for the preceding kernel) and their latency
+  // passes under the set-up of the activations; the first raw chunks follow as soon as the rings are free.
+  // The values travel as plain variables: gathered in a struct the same code was measured 3 % slower in
+  // the tile loop (the compiler then recomputes loop constants in every iteration).
+  __device__ __forceinline__ void load_head(const tq_tiles_desc& d, uint32_t t0, uint32_t t1, uint32_t& h_rd,
+                                            uint32_t& h_stop_pos, uint4 (&h_q)[2][2], uint32_t (&h_tr)[2]) {
+    h_rd = __ldg(d.tile_raw + t0);
+    h_stop_pos = __ldg(d.tile_raw + t1);  // raw words of the run end here
+    const uint4* tok = d.tokens + (size_t)t0 * 64u + lane;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      h_q[k][0] = ldg_stream(tok + k * 64);
+      h_q[k][1] = ldg_stream(tok + k * 64 + 32);
+      h_tr[k] = __ldg(d.tile_raw + t0 + 1 + k);
+    }
+    // the row scales of the row blocks this run shares with its neighbours are wanted by whoever merges
+    // the partial sums at the end of the segment: brought near now
+    const uint32_t S = d.steps;
+    if (lane < 4u) {
+      const uint32_t t = (lane & 1u) ? t1 : t0;
+      const float* a = ((lane & 2u) ? d.zero : d.scale) + (size_t)(t / S) * 16u;
+      if (t % S != 0u && ((lane & 2u) == 0u || d.has_zero)) asm volatile("prefetch.global.L1 [%0];" ::"l"(a));
+    }
+  }
+  __device__ __forceinline__ void first_chunks(const tq_tiles_desc& d, uint32_t h_rd, uint32_t h_stop_pos,
+                                               uint32_t& h_w_pos, uint32_t& h_i_pos) {
+    h_w_pos = h_rd & ~(uint32_t)(kChunkWords - 1);  // first word of the next chunk to wait for
+    h_i_pos = h_w_pos;                              // first word of the next chunk to issue
+    for (int k = 0; k < kSlots && h_i_pos < h_stop_pos; ++k, h_i_pos += kChunkWords) issue_chunk(d.raw, h_i_pos);
+  }
+
   // ---- one warp, tiles [t0, t1) of matrix d -------------------------------------------------
   // Tile i of the run uses token registers q[i & 1] and word buffer i & 1; its words are consumed
   // by the MMAs while tile i + 1 is being looked up, and its token registers are reloaded (two
   // tiles ahead) only after the last use, so no register is copied while a load into it is in
   // flight.
-  __device__ void run_tiles(const tq_tiles_desc& d, uint32_t t0, uint32_t t1) {
+  // rd, stop_pos, q, tr: what load_head fetched; w_pos, i_pos: where first_chunks left the raw stream
+  // (q[k], tr[k]: tokens of tile t0 + k and the index of the first raw word behind it).
+  __device__ __forceinline__ void run_tiles(const tq_tiles_desc& d, uint32_t t0, uint32_t t1, uint32_t rd,
+                                            const uint32_t stop_pos, uint32_t w_pos, uint32_t i_pos, uint4 (&q)[2][2],
+                                            uint32_t (&tr)[2]) {
     if (!wait_table()) {  // the table copy started with the kernel; its first use is here
       dead = true;
       *dead_flag() = 1u;
@@ -213,25 +257,10 @@ struct TilesCta : CtaBase {
     // reaches accumulator columns nobody reads
     const uint32_t x_lane = tbl_addr + L.x + (min(g, (uint32_t)NCOL - 1u) * xstride + 8u * t) * 4u;
 
-    uint32_t rd = __ldg(d.tile_raw + t0);
-    const uint32_t stop_pos = __ldg(d.tile_raw + t1);          // raw words of the run end here
-    uint32_t w_pos = rd & ~(uint32_t)(kChunkWords - 1);        // first word of the next chunk to wait for
-    uint32_t i_pos = w_pos;                                    // first word of the next chunk to issue
-    for (int k = 0; k < kSlots && i_pos < stop_pos; ++k, i_pos += kChunkWords) issue_chunk(d.raw, i_pos);
 
-    const uint4* tok = d.tokens + (size_t)t0 * 64u + lane;
+    const uint4* tok = d.tokens + (size_t)t0 * 64u + lane + 2 * 64;
     const uint4* tok_end = d.tokens + (size_t)t1 * 64u;  // lane 0's view of the end of the run
-    const uint32_t* trp = d.tile_raw + t0 + 1;
-    uint4 q[2][2];
-    uint32_t tr[2];  // tile_raw[tile + 1]: where the tile's raw words end
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      q[k][0] = ldg_stream(tok + k * 64);
-      q[k][1] = ldg_stream(tok + k * 64 + 32);
-      tr[k] = __ldg(trp + k);
-    }
-    tok += 2 * 64;
-    trp += 2;
+    const uint32_t* trp = d.tile_raw + t0 + 1 + 2;
 
     uint32_t s_p = t0 % S, rb = t0 / S;  // step and row block of the tile whose words await the MMAs
     bool from_start = s_p == 0;
@@ -336,34 +365,50 @@ struct TilesCta : CtaBase {
 
   // ---- one segment: row blocks [rb0, rb1) of matrix d, all warps ----------------------------
   __device__ void run_segment(const tq_tiles_desc& d, uint32_t rb0, uint32_t rb1) {
+    static_assert(2 * W == 32, "the merge below looks at the 2 W partial-sum slots with one lane each");
     const uint64_t T = (uint64_t)(rb1 - rb0) * d.steps;
     const uint32_t t0 = rb0 * d.steps + (uint32_t)(T * warp / W);
     const uint32_t t1 = rb0 * d.steps + (uint32_t)(T * (warp + 1) / W);
+    const bool has_tiles = t0 < t1 && !dead;
+    uint32_t h_rd = 0, h_stop = 0, h_w = 0, h_i = 0, h_tr[2];
+    uint4 h_q[2][2];
+    if (has_tiles) load_head(d, t0, t1, h_rd, h_stop, h_q, h_tr);
+    if (!waited) {  // x is the first thing read that a preceding kernel may have written
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      waited = true;
+    }
     __syncthreads();  // the previous segment is done with x and with the partials in the rings
-    prepare_x(d);
+    prepare_x(d, [&] {
+      if (has_tiles) first_chunks(d, h_rd, h_stop, h_w, h_i);
+    });
     if (lane < 2) part_ids()[2 * warp + lane] = kNoBlock;
     __syncthreads();
-    if (t0 < t1 && !dead && !*dead_flag()) run_tiles(d, t0, t1);
+    if (has_tiles && !*dead_flag()) run_tiles(d, t0, t1, h_rd, h_stop, h_w, h_i, h_q, h_tr);
     __syncthreads();
-    // partial row blocks: entries of the same block are adjacent (warp order = tile order)
-    if (warp == 0 && !*dead_flag()) {
-      uint32_t cur = kNoBlock;
-      int sum[4] = {0, 0, 0, 0};
-      for (uint32_t e = 0; e < 2u * W; ++e) {
-        const uint32_t id = part_ids()[e];
-        if (id == kNoBlock) continue;
-        if (id != cur) {
-          if (cur != kNoBlock) finalize(d, cur, sum[0], sum[1], sum[2], sum[3]);
-          cur = id;
-          sum[0] = sum[1] = sum[2] = sum[3] = 0;
+    // Partial row blocks: the slots of one block are adjacent (warp order = tile order).  The k-th
+    // block that has partial sums is summed and finished by warp k mod W.
+    if (!*dead_flag()) {
+      const uint32_t id = part_ids()[lane];
+      const uint32_t used = __ballot_sync(kFull, id != kNoBlock);
+      const uint32_t below = used & ((1u << lane) - 1u);
+      const uint32_t prev = __shfl_sync(kFull, id, below ? 31 - __clz(below) : 0);
+      uint32_t firsts = __ballot_sync(kFull, id != kNoBlock && (below == 0u || prev != id));
+      for (uint32_t k = 0; firsts != 0u; ++k) {
+        const uint32_t e0 = __ffs(firsts) - 1u;
+        firsts &= firsts - 1u;
+        const uint32_t e1 = firsts ? __ffs(firsts) - 1u : 32u;
+        if (k % W != warp) continue;
+        int sum[4] = {0, 0, 0, 0};
+        for (uint32_t e = e0; e < e1; ++e) {
+          if (!((used >> e) & 1u)) continue;
+          const int4 v = reinterpret_cast<const int4*>(smem + L.ring + (e >> 1) * (kRingWords * 4u) + (e & 1u) * 512u)[lane];
+          sum[0] += v.x;
+          sum[1] += v.y;
+          sum[2] += v.z;
+          sum[3] += v.w;
         }
-        const int4 v = reinterpret_cast<const int4*>(smem + L.ring + (e >> 1) * (kRingWords * 4u) + (e & 1u) * 512u)[lane];
-        sum[0] += v.x;
-        sum[1] += v.y;
-        sum[2] += v.z;
-        sum[3] += v.w;
+        finalize(d, __shfl_sync(kFull, id, e0), sum[0], sum[1], sum[2], sum[3]);
       }
-      if (cur != kNoBlock) finalize(d, cur, sum[0], sum[1], sum[2], sum[3]);
     }
   }
 };
@@ -377,25 +422,20 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
   // while its predecessor was still running.  Nothing above reads or writes what a predecessor
   // produces (the table and the weights are constant); the activations are first read below.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // The CTA's first segment is fetched before the set-up by one thread and parked in shared memory: the work
-  // split and the matrix descriptors are constant data, so the three dependent loads that find the work
-  // overlap the barrier set-up and the start of the table copy instead of following them, and no register
-  // holds them meanwhile (registers are short in the tile loop).
+  // The record of the CTA's first segment (work split and matrix descriptor: constant data) is fetched by
+  // warp 1 with one load before the set-up and parked in shared memory, so that its latency overlaps the
+  // barrier set-up and the start of the table copy, and no register holds it meanwhile (registers are
+  // short in the tile loop).
   const TilesSmem plan = tiles_smem(p.table_words, (uint32_t)kDigits * NB * p.xstride, W);
-  FirstSegment* first = reinterpret_cast<FirstSegment*>(tiles_smem_raw + plan.misc + kFirstSegmentOffset);
-  if (p.mats != nullptr && threadIdx.x == 32) {
-    first->begin = p.cta_seg[blockIdx.x];
-    first->end = p.cta_seg[blockIdx.x + 1];
-    if (first->begin < first->end) {
-      first->seg = p.segs[first->begin];
-      first->desc = p.mats[first->seg.mat];
-    }
-  }
+  SegRecord* first = reinterpret_cast<SegRecord*>(tiles_smem_raw + plan.misc + kFirstSegmentOffset);
+  if (p.firsts != nullptr && (threadIdx.x >> 5) == 1u)
+    reinterpret_cast<uint32_t*>(first)[threadIdx.x & 31u] =
+        __ldg(reinterpret_cast<const uint32_t*>(p.firsts + blockIdx.x) + (threadIdx.x & 31u));
   cta.setup(tiles_smem_raw, plan, W, p.table, p.table_words, p.test_withhold != 0u);  // ends with a CTA barrier
   cta.xstride = p.xstride;
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // griddepcontrol.wait: in run_segment, behind the loads of constant data that open a segment
 
-  if (p.mats == nullptr) {
+  if (p.firsts == nullptr) {
     const uint32_t nrb = p.one.row_blocks;
     const uint32_t rb0 = (uint32_t)((uint64_t)nrb * blockIdx.x / gridDim.x);
     const uint32_t rb1 = (uint32_t)((uint64_t)nrb * (blockIdx.x + 1) / gridDim.x);
@@ -405,15 +445,18 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
     uint32_t si = first->begin;
     TilesSeg sg = first->seg;
     tq_tiles_desc d = first->desc;
-    if (si >= p.cta_seg[blockIdx.x + 1] && cta.warp == 0) cta.wait_table();  // a CTA without work: as above
-    while (si < p.cta_seg[blockIdx.x + 1]) {  // the bound is read again rather than kept across a segment
+    if (si >= first->end && cta.warp == 0) cta.wait_table();  // a CTA without work: as above
+    while (si < first->end) {  // the bound is read again rather than kept across a segment
+      // the next record comes near while this segment runs
+      if (threadIdx.x == 0 && si + 1 < first->end) asm volatile("prefetch.global.L1 [%0];" ::"l"(p.recs + si + 1));
       cta.run_segment(d, sg.rb_begin, sg.rb_end);
-      if (++si < p.cta_seg[blockIdx.x + 1]) {
-        sg = p.segs[si];
-        d = p.mats[sg.mat];
+      if (++si < first->end) {
+        sg = p.recs[si].seg;
+        d = p.recs[si].desc;
       }
     }
   }
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // a CTA without work completes after its predecessors too
   cta.linger_after_failure();
 }
 
@@ -931,6 +974,9 @@ StackRoute stack_route(const tq_dmat* const* mats, int n_mats, int B) {
   }
   return r;
 }
+// Records of the narrow kernel's split: at most n_mats + grid segments (every matrix starts one, every CTA
+// boundary splits at most one), and one record per CTA.
+uint64_t stack_record_bytes(int n_mats, uint64_t grid) { return align256(((uint64_t)n_mats + 2 * grid) * sizeof(SegRecord)); }
 uint64_t stack_plan_bytes(int n_mats, uint64_t grid, uint64_t total_rb) {
   // the tcgen05 plan can hold one segment per group of row blocks (or per CTA for small stacks)
   const uint64_t max_segs = std::max<uint64_t>((uint64_t)n_mats + grid, total_rb / kWideGroupRowBlocks + (uint64_t)n_mats + grid);
@@ -950,7 +996,8 @@ int tq_stack_size(const tq_dmat* const* mats, int n_mats, int B, uint64_t* devic
   const StackRoute r = stack_route(mats, n_mats, B);
   for (int i = 0; i < n_mats; ++i)
     if (r.wide_all || (r.wide_long && !short_rows(mats[i], 1))) scratch += tq_wide_scratch_bytes(mats[i]->tiles.steps, B);
-  *device_bytes = align256((uint64_t)n_mats * sizeof(tq_tiles_desc)) + kStackPlans * stack_plan_bytes(n_mats, grid, total_rb) + 1024 + scratch;
+  *device_bytes = align256((uint64_t)n_mats * sizeof(tq_tiles_desc)) + kStackPlans * stack_plan_bytes(n_mats, grid, total_rb) +
+                  stack_record_bytes(n_mats, grid) + 1024 + scratch;
   return TQ_OK;
 }
 
@@ -991,7 +1038,8 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   const uint64_t plan_bytes = stack_plan_bytes(n_mats, s->grid, total_rb);
   const uint64_t segs_bytes = plan_bytes - align256((s->grid + 1) * 4);
   const uint64_t off_plans = align256((uint64_t)n_mats * sizeof(tq_tiles_desc));
-  uint64_t off_scratch = (off_plans + kStackPlans * plan_bytes + 1023) / 1024 * 1024;
+  const uint64_t off_records = off_plans + kStackPlans * plan_bytes;
+  uint64_t off_scratch = (off_records + stack_record_bytes(n_mats, s->grid) + 1023) / 1024 * 1024;
 
   std::vector<tq_tiles_desc> descs((size_t)n_mats);
   for (int i = 0; i < n_mats; ++i) {
@@ -1009,6 +1057,7 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
   // [0] all matrices, split by tiles (decompress, bf16 decode); [1] the matrices whose rows are short enough
   // for the narrow kernel; [2] the others and [3] all matrices, split for the tcgen05 kernel
   StackPlan pls[kStackPlans];  // kept alive until the copies have been made
+  std::vector<SegRecord> records;
   for (int k = 0; k < kStackPlans && rc == TQ_OK; ++k) {
     std::vector<PlanMat> pm;
     std::vector<uint32_t> ids;
@@ -1038,6 +1087,29 @@ int tq_stack_create(const tq_dmat* const* mats, const void* const* d_x, float* c
     sp.d_segs = pb;
     sp.d_cta_seg = reinterpret_cast<const uint32_t*>(pb + segs_bytes);
     sp.n_segs = (uint32_t)pls[k].segs.size();
+    if (k == 1 && rc == TQ_OK) {  // the narrow kernel's records: per segment, then per CTA
+      const StackPlan& pl = pls[k];
+      const size_t n_segs = pl.segs.size();
+      if ((n_segs + s->grid) * sizeof(SegRecord) > stack_record_bytes(n_mats, s->grid)) rc = TQ_ERR_BUFFER_TOO_SMALL;
+      records.assign(n_segs + s->grid, SegRecord{});
+      for (uint32_t c = 0; c < s->grid && rc == TQ_OK; ++c) {
+        const uint32_t b = pl.cta_seg[c], e = pl.cta_seg[c + 1];
+        for (uint32_t i = b; i < e; ++i) {
+          records[i].begin = b;
+          records[i].end = e;
+          records[i].seg = pl.segs[i];
+          records[i].desc = descs[pl.segs[i].mat];
+        }
+        if (b < e) {
+          records[n_segs + c] = records[b];
+          sp.grid_used = c + 1;
+        }
+      }
+      if (rc == TQ_OK)
+        rc = tq_cuda_status((int)cudaMemcpyAsync(base + off_records, records.data(), records.size() * sizeof(SegRecord), cudaMemcpyHostToDevice, st), "stack upload");
+      sp.d_recs = base + off_records;
+      sp.d_firsts = base + off_records + n_segs * sizeof(SegRecord);
+    }
   }
   if (rc == TQ_OK) rc = tq_cuda_status((int)cudaStreamSynchronize(st), "stack upload");
   if (rc != TQ_OK) {
@@ -1058,16 +1130,16 @@ int stack_run(const tq_stack* s, bool launch, cudaStream_t st, int* n_launches) 
     ++*n_launches;
     if (launch) {
       TilesParams p{};
-      p.mats = s->d_descs;
-      p.segs = static_cast<const TilesSeg*>(sp.d_segs);
-      p.cta_seg = sp.d_cta_seg;
+      p.firsts = static_cast<const SegRecord*>(sp.d_firsts);
+      p.recs = static_cast<const SegRecord*>(sp.d_recs);
       p.table = s->d_table;
       p.table_words = s->table_words;
       p.xstride = sp.xstride;
       const size_t smem = tiles_smem(p.table_words, (uint32_t)kDigits * s->B * p.xstride, kTilesWarps).total;
+      const uint32_t grid = sp.grid_used;  // the split fills the CTAs in order: the rest would only copy the table
       int rc;
-      if (s->B == 1) rc = sg ? launch_tiles<1, true>(p, s->grid, smem, st) : launch_tiles<1, false>(p, s->grid, smem, st);
-      else rc = sg ? launch_tiles<2, true>(p, s->grid, smem, st) : launch_tiles<2, false>(p, s->grid, smem, st);
+      if (s->B == 1) rc = sg ? launch_tiles<1, true>(p, grid, smem, st) : launch_tiles<1, false>(p, grid, smem, st);
+      else rc = sg ? launch_tiles<2, true>(p, grid, smem, st) : launch_tiles<2, false>(p, grid, smem, st);
       if (rc != TQ_OK) return rc;
     }
   }
