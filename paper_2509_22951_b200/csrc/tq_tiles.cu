@@ -78,6 +78,8 @@ struct XInfo {
 // Places inside the misc area of the shared-memory plan (TilesCta): XInfo at +192, the warps' sums of the
 // fixed-point values at +512.
 // The record of the CTA's first segment, fetched by one warp during the set-up (gemv_tiles_kernel): at +768.
+// Barrier "the digits of this segment's activations are in shared memory" (one arrival per warp): at +416.
+constexpr uint32_t kXReadyBarOffset = 416u;
 constexpr uint32_t kFirstSegmentOffset = 768u;
 static_assert(kFirstSegmentOffset + sizeof(SegRecord) <= 1024u, "misc area of the shared-memory plan");
 constexpr int kTilesWarpsC = 16;
@@ -122,11 +124,13 @@ struct TilesCta : CtaBase {
   static_assert(W == kTilesWarpsC, "tiles_finalize sums the per-warp values of kTilesWarpsC warps");
 
   uint32_t xstride;
+  uint32_t x_phase = 0;  // segments run so far: the phase the x-ready barrier completes next
   bool dead = false, waited = false;
 
   __device__ __forceinline__ uint32_t* misc_u32() { return reinterpret_cast<uint32_t*>(smem + L.misc); }
   // misc (1 KB): [0] dead flag; +16 partial ids [2W]; +192 XInfo; +224 per-warp maxima [NB][W]; +400 table
-  // barrier; +512 per-warp sums of the fixed-point values [NB][W] (64-bit)
+  // barrier; +416 x-ready barrier; +512 per-warp sums of the fixed-point values [NB][W] (64-bit); +768 the
+  // record of the CTA's first segment
   __device__ __forceinline__ uint32_t* part_ids() { return misc_u32() + 4; }
   __device__ __forceinline__ XInfo* xinfo() { return reinterpret_cast<XInfo*>(smem + L.misc + kXInfoOffset); }
   __device__ __forceinline__ uint32_t* warp_max() { return reinterpret_cast<uint32_t*>(smem + L.misc + 224); }
@@ -134,8 +138,8 @@ struct TilesCta : CtaBase {
 
   // ---- activation vectors -> digit columns in shared memory --------------------------------
   // Every thread keeps its groups of x in registers between the search for the largest magnitude and
-  // the conversion, so x is read once; one CTA barrier in the middle (per-warp maxima), the caller's
-  // barrier at the end.  Rows of up to kMaxItems * kThreads groups (10240 columns) fit; longer rows
+  // the conversion, so x is read once; one CTA barrier in the middle (per-warp maxima); the caller tells
+  // the x-ready barrier when this warp's share is written.  Rows of up to kMaxItems * kThreads groups (10240 columns) fit; longer rows
   // do not come here (their digits would not fit beside the table either).
   static constexpr int kMaxItems = 5;
   template <class Mid>
@@ -325,6 +329,11 @@ struct TilesCta : CtaBase {
     const uint32_t n = t1 - t0;
     bool ok = lookups(0);
     if (ok) refill(true);
+    // the first tile has been looked up while other warps were still converting activations; the MMAs need them
+    if (ok) {
+      const uint32_t xbar = tbl_addr + L.misc + kXReadyBarOffset, par = (x_phase - 1u) & 1u;
+      ok = __all_sync(kFull, mbar_try(xbar, par)) || tiles_wait_slow(xbar, par, dead_flag());
+    }
     uint32_t i = 1;
     for (; ok && i + 1 < n; i += 2) {
       ok = lookups(1);
@@ -382,7 +391,11 @@ struct TilesCta : CtaBase {
       if (has_tiles) first_chunks(d, h_rd, h_stop, h_w, h_i);
     });
     if (lane < 2) part_ids()[2 * warp + lane] = kNoBlock;
-    __syncthreads();
+    // no CTA barrier here: a warp tells the x-ready barrier that its share of the digits is written and goes on
+    // to its first lookups; it waits for the other warps' shares before its first MMA (run_tiles)
+    __syncwarp();
+    if (lane == 0) mbar_arrive(tbl_addr + L.misc + kXReadyBarOffset);
+    ++x_phase;
     if (has_tiles && !*dead_flag()) run_tiles(d, t0, t1, h_rd, h_stop, h_w, h_i, h_q, h_tr);
     __syncthreads();
     // Partial row blocks: the slots of one block are adjacent (warp order = tile order).  The k-th
@@ -399,13 +412,22 @@ struct TilesCta : CtaBase {
         const uint32_t e1 = firsts ? __ffs(firsts) - 1u : 32u;
         if (k % W != warp) continue;
         int sum[4] = {0, 0, 0, 0};
-        for (uint32_t e = e0; e < e1; ++e) {
-          if (!((used >> e) & 1u)) continue;
-          const int4 v = reinterpret_cast<const int4*>(smem + L.ring + (e >> 1) * (kRingWords * 4u) + (e & 1u) * 512u)[lane];
-          sum[0] += v.x;
-          sum[1] += v.y;
-          sum[2] += v.z;
-          sum[3] += v.w;
+        for (uint32_t c = e0 & ~7u; c < e1; c += 8u) {  // eight loads in flight at a time
+          int4 v[8];
+#pragma unroll
+          for (uint32_t i = 0; i < 8u; ++i) {
+            const uint32_t e = c + i;
+            const bool on = e >= e0 && e < e1 && ((used >> e) & 1u);
+            v[i] = on ? reinterpret_cast<const int4*>(smem + L.ring + (e >> 1) * (kRingWords * 4u) + (e & 1u) * 512u)[lane]
+                      : make_int4(0, 0, 0, 0);
+          }
+#pragma unroll
+          for (uint32_t i = 0; i < 8u; ++i) {
+            sum[0] += v[i].x;
+            sum[1] += v[i].y;
+            sum[2] += v[i].z;
+            sum[3] += v[i].w;
+          }
         }
         finalize(d, __shfl_sync(kFull, id, e0), sum[0], sum[1], sum[2], sum[3]);
       }
@@ -431,7 +453,8 @@ __global__ void __launch_bounds__(W * 32, 1) gemv_tiles_kernel(const TilesParams
   if (p.firsts != nullptr && (threadIdx.x >> 5) == 1u)
     reinterpret_cast<uint32_t*>(first)[threadIdx.x & 31u] =
         __ldg(reinterpret_cast<const uint32_t*>(p.firsts + blockIdx.x) + (threadIdx.x & 31u));
-  cta.setup(tiles_smem_raw, plan, W, p.table, p.table_words, p.test_withhold != 0u);  // ends with a CTA barrier
+  if (threadIdx.x == 0) mbar_init(smem_u32(tiles_smem_raw) + plan.misc + kXReadyBarOffset, (uint32_t)W);
+  cta.setup(tiles_smem_raw, plan, W, p.table, p.table_words, p.test_withhold != 0u);  // fence, ends with a CTA barrier
   cta.xstride = p.xstride;
   // griddepcontrol.wait: in run_segment, behind the loads of constant data that open a segment
 
