@@ -111,6 +111,7 @@ class ClockSampler:
 # tiles_stack: 219.9 MB read + 6.7 MB written for 207.7 MB of algorithmic bytes on a 14-matrix stack (2 decoder
 # layers), i.e. 1.091 x; traffic grows with the bytes streamed, so the 3B launch (3.36 GB) is scaled by that ratio.
 L2_BYTES = 126 << 20
+E2E_GROUPS = 4  # host-buffer calls per step of the pipelined end-to-end leg
 TRAFFIC_RATIO = {"tiles_stack": 1.091}
 TRAFFIC = {}
 # the arithmetic each layout's product kernel computes in
@@ -476,6 +477,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-groups", type=int, default=E2E_GROUPS, help="host-buffer calls per step of the pipelined end-to-end leg")
     ap.add_argument("--no-extras", action="store_true", help="skip the tq_decompress / tq_fused_gemm timings")
     ap.add_argument("--shard", default="replicas", choices=["replicas", "rows"],
                     help="N > 1 GPUs: replicas = every rank runs the whole model (weak scaling, no collective); rows = every "
@@ -650,23 +652,65 @@ def main():
                     for m, a, b, dx, dy in zip(mats, hx, hy, xs, ys):
                         tq.tq_fused_gemv_host(m, a, b, dx, dy)
 
-            for _ in range(3):
-                step_e2e()
-            stream.synchronize()
-            barrier()
-            t0 = time.perf_counter()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            for _ in range(e_steps):
-                step_e2e()
-                stream.synchronize()  # the step's result is on the host
-            e1.record(stream)
-            stream.synchronize()
-            wall = time.perf_counter() - t0
-            e2e_ms = max(e0.elapsed_time(e1), wall * 1e3) / e_steps
+            def time_e2e(step_fn):
+                for _ in range(3):
+                    step_fn()
+                stream.synchronize()
+                barrier()
+                t0 = time.perf_counter()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(e_steps):
+                    step_fn()
+                    stream.synchronize()  # the step's result is on the host
+                e1.record(stream)
+                stream.synchronize()
+                wall = time.perf_counter() - t0
+                return max(e0.elapsed_time(e1), wall * 1e3) / e_steps
+
+            e2e_ms = time_e2e(step_e2e)
             e2e = {"ms_per_step": e2e_ms, "steps": e_steps,
                    "h2d": sum(2 * args.batch * i.cols for i in infos),
-                   "d2h": sum(4 * args.batch * i.rows for i in infos)}
+                   "d2h": sum(4 * args.batch * i.rows for i in infos),
+                   "calls": "one tq_fused_gemv_stack_host call per step" if use_stack else "one tq_fused_gemv_host call per matrix"}
+            if use_stack and len(mats) >= 8:
+                # The same step as --e2e-groups host-buffer calls on two streams: consecutive matrices grouped by bytes,
+                # each call copies its slice of x, runs its matrices and copies its slice of y back, so the copies of
+                # one group pass under the kernel of the next.  Same bytes in and out, same public call.
+                ab = [algorithmic_bytes(i, args.batch) for i in infos]
+                cuts, acc, tot = [0], 0, sum(ab)
+                for i, v in enumerate(ab):
+                    acc += v
+                    if acc >= tot * len(cuts) / args.e2e_groups and len(cuts) < args.e2e_groups and i + 1 < len(ab):
+                        cuts.append(i + 1)
+                cuts.append(len(mats))
+                x0, y0 = x_arena.data_ptr(), y_arena.data_ptr()
+                xo = [(x.data_ptr() - x0) // 2 for x in xs] + [x_arena.numel()]
+                yo = [(y.data_ptr() - y0) // 4 for y in ys] + [y_arena.numel()]
+                side = [torch.cuda.Stream(), torch.cuda.Stream()]
+                groups = []
+                for a_, b_ in zip(cuts[:-1], cuts[1:]):
+                    st_ = tq.tq_stack_create(mats[a_:b_], xs[a_:b_], ys[a_:b_])
+                    groups.append((st_, hxa[xo[a_]:xo[b_]], x_arena[xo[a_]:xo[b_]], hya[yo[a_]:yo[b_]], y_arena[yo[a_]:yo[b_]]))
+                done = [torch.cuda.Event() for _ in side]
+
+                def step_pipelined():
+                    for sd in side:
+                        sd.wait_stream(stream)
+                    for k, (st_, hx_, dx_, hy_, dy_) in enumerate(groups):
+                        tq.tq_fused_gemv_stack_host(st_, hx_, dx_, hy_, dy_, stream=side[k % 2])
+                    for sd, ev in zip(side, done):
+                        ev.record(sd)
+                        stream.wait_event(ev)
+
+                p_ms = time_e2e(step_pipelined)
+                e2e["single_call_ms_per_step"] = e2e_ms
+                e2e["pipelined_ms_per_step"] = p_ms
+                if p_ms < e2e_ms:
+                    e2e["ms_per_step"] = p_ms
+                    e2e["calls"] = ("%d tq_fused_gemv_stack_host calls per step (consecutive matrices grouped by bytes) on two "
+                                    "streams: the copies of one group pass under the kernel of the next" % len(groups))
+                del groups
 
         # ---- the other device calls on the same resident model (single GPU only) ----
         extras = {}
@@ -738,7 +782,8 @@ def main():
     if e2e:
         out["e2e"] = {"value": world * alg_bytes / (e2e["ms_per_step"] * 1e-3) / 1e9, "unit": UNIT,
                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                      "ms_per_step": e2e["ms_per_step"], "steps": e2e["steps"]}
+                      "ms_per_step": e2e["ms_per_step"], "steps": e2e["steps"],
+                      **{k: e2e[k] for k in ("calls", "single_call_ms_per_step", "pipelined_ms_per_step") if k in e2e}}
 
     if not args.no_cpu_baseline and args.quantizer == "rows":
         sample = pick_sample(shapes, 3_300_000_000)  # ~6-13 s of single-thread oracle work for the 3B stack
