@@ -8,7 +8,8 @@ tiled on the GPU, resident in HBM before the timed region starts.  `value` is th
 on algorithmic bytes (tokens and raw words of the layout + tile index + row scales + x + y) per second.
 Extra keys time the same model at 8 and 32 vectors, launched as a decoder must launch it (layers that
 feed one another in separate launches), the 1B stack, tq_decompress of the whole set and the prefill
-product at 2048 tokens; `cpu_baseline` is the CPU oracle on the host's cores.
+product at 2048 tokens; `e2e` is the same step through the host-buffer call (x from pinned host memory, y back
+to it, every step: as one call and as a few calls on two streams); `cpu_baseline` is the CPU oracle on the host's cores.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--model 3b|1b] [--batch B] [--layers L]
   python bench.py --impl reference ...     # the CPU oracle on a bounded sample of the workload
