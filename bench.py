@@ -464,7 +464,7 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="tq", choices=["tq", "reference"])
-    ap.add_argument("--model", default="3b", choices=["1b", "3b", "11b"])
+    ap.add_argument("--model", default="3b", choices=["1b", "3b", "11b", "90b"])
     ap.add_argument("--bits", type=int, default=8, help="bit count of the per-tensor quantizer (--quantizer paper)")
     ap.add_argument("--quantizer", default="rows", choices=["rows", "paper"],
                     help="rows: per-row symmetric int8 (the workload definition); paper: Listing 1, per tensor, unsigned levels "

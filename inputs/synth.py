@@ -131,6 +131,8 @@ def llama32_linear_shapes(model: str, n_layers: int | None = None, lm_head: bool
         "3b": dict(h=3072, kv=1024, ffn=8192, layers=28, vocab=128256),
         # text decoder of LLaMA-3.2-11B-Vision (its self-attention layers): a second workload with long rows
         "11b": dict(h=4096, kv=1024, ffn=14336, layers=32, vocab=128256),
+        # text decoder of LLaMA-3.2-90B-Vision (self-attention layers): the longest rows of the family
+        "90b": dict(h=8192, kv=1024, ffn=28672, layers=80, vocab=128256),
     }[model.lower()]
     L = cfg["layers"] if n_layers is None else n_layers
     out = []
