@@ -379,18 +379,19 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
         drain_due = false;
         const bool real = drain_real;
         const uint32_t rb = drain_rb;
+        // the row scales are asked for before the wait for the last MMAs of the row block, not after it
+        const uint32_t rows = FIELD(rows), has_zero = FIELD(has_zero);
+        const float* const scale = FIELD(scale);
+        const float* const zero = FIELD(zero);
+        const uint32_t r_lo = rb * 16u + g, r_hi = r_lo + 8u;
+        const float sc_lo = (real && r_lo < rows) ? __ldg(scale + r_lo) : 0.f, sc_hi = (real && r_hi < rows) ? __ldg(scale + r_hi) : 0.f;
+        const float z_lo = (real && has_zero && r_lo < rows) ? __ldg(zero + r_lo) : 0.f;
+        const float z_hi = (real && has_zero && r_hi < rows) ? __ldg(zero + r_hi) : 0.f;
         ok = ok && cta.wait(cta.bar(kOffAccFull), rr & 1u);
         if (ok && real) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t rows = FIELD(rows), has_zero = FIELD(has_zero);
-          const float* const scale = FIELD(scale);
-          const float* const zero = FIELD(zero);
           float* const y = FIELD(y);
           const double* const hdr = reinterpret_cast<const double*>(FIELD(xdig));
-          const uint32_t r_lo = rb * 16u + g, r_hi = r_lo + 8u;
-          const float sc_lo = r_lo < rows ? __ldg(scale + r_lo) : 0.f, sc_hi = r_hi < rows ? __ldg(scale + r_hi) : 0.f;
-          const float z_lo = (has_zero && r_lo < rows) ? __ldg(zero + r_lo) : 0.f;
-          const float z_hi = (has_zero && r_hi < rows) ? __ldg(zero + r_hi) : 0.f;
           for (uint32_t bq = 0; bq * 16u < N; ++bq) {
             int v[8];
             asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
