@@ -328,16 +328,16 @@ __global__ void __launch_bounds__(kWideThreads, 1) gemv_wide_kernel(const WidePa
       if (n_real) {
         rd = __ldg(trp - 1);
         stop_pos = __ldg(trp - 1 + n_real);
-        w_pos = i_pos = rd & ~(uint32_t)(kChunkWords - 1);
-        for (int k = 0; k < kSlots && i_pos < stop_pos; ++k, i_pos += kChunkWords) cta.issue_chunk(raw, i_pos);
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {
+        for (int k = 0; k < 2; ++k) {  // the tokens do not wait for the tile index: asked for before its first use
           q[k][0] = ldg_stream(tok + k * 64);
           q[k][1] = ldg_stream(tok + k * 64 + 32);
           tr[k] = __ldg(trp + k);
         }
         tok += 2 * 64;
         trp += 2;
+        w_pos = i_pos = rd & ~(uint32_t)(kChunkWords - 1);
+        for (int k = 0; k < kSlots && i_pos < stop_pos; ++k, i_pos += kChunkWords) cta.issue_chunk(raw, i_pos);
       }
       uint32_t w[16];
       uint32_t s_p = 0, rb = my0;
