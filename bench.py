@@ -368,7 +368,7 @@ def time_extras(tq, mats, infos, shapes, args, device, stream, extra):
                                   "frac_of_measured_hbm": alg_b / (ms_b * 1e-3) / 1e9 / peak,
                                   "us_per_token": ms_b * 1e3 / b, "kernel": "wide_prepare_kernel + gemv_wide_kernel"}
             del st_b, xs_b, ys_b
-        # ... and the 1B stack (BASELINE config 3) at batch 1, with its own table
+        # ... and the LLaMA-3.2-1B stack at batch 1, with its own table
         shapes1 = synth.llama32_linear_shapes("1b")
         m1, xs1, ys1, hd1, _, _, _, _, _, _ = build_model(tq, shapes1, 1, device, 0, None, layout=2)
         st1 = tq.tq_stack_create(m1, xs1, ys1)
