@@ -414,6 +414,38 @@ def test_stack_matches_oracle_and_single_calls(tq, B):
             assert tq.tq_device_status(m) == 0
 
 
+@pytest.mark.parametrize("B", [1, 2])
+@pytest.mark.parametrize("n_mats,max_rows", [(3, 40), (60, 200), (400, 48)])
+def test_stack_of_many_small_matrices(tq, B, n_mats, max_rows):
+    """Few small matrices leave most CTAs without a segment (they are not launched); hundreds of them
+    give every CTA several segments of different matrices, each fetched as one record.  Unsigned levels
+    with zero points, so the per-warp sums of x are used too.  Results: bit-equal to single calls, and
+    within the tolerance of the oracle."""
+    rng = np.random.default_rng(7000 + 10 * n_mats + B)
+    shapes = [(int(rng.integers(1, max_rows + 1)), 4 * int(rng.integers(1, 300))) for _ in range(n_mats)]
+    qs = [rng.integers(100, 140, size=s).astype(np.uint8) for s in shapes]
+    ss = [(rng.random(r) + 0.5).astype(np.float32) for r, _ in shapes]
+    zs = [rng.integers(110, 130, size=r).astype(np.float32) for r, _ in shapes]
+    d, streams = _oracle_pack(qs, top_k=3000)
+    dd = tq.tq_dict_upload(tq.tq_dict_from_entries(d.entries))
+    mats = [tq.tq_upload(dd, st, r, c, s, z, levels_signed=False, layout=tq.TQ_LAYOUT_TILES)
+            for st, (r, c), s, z in zip(streams, shapes, ss, zs)]
+    xs = [synth.activations(B, c, 900 + i).cuda() for i, (_, c) in enumerate(shapes)]
+    ys = [torch.full((B, r), float("nan"), dtype=torch.float32, device="cuda") for r, _ in shapes]
+    stack = tq.tq_stack_create(mats, xs, ys)
+    assert stack.launches == 1
+    for _ in range(2):
+        for y in ys:
+            y.fill_(float("nan"))
+        tq.tq_fused_gemv_stack(stack)
+        torch.cuda.synchronize()
+        for m, q, s, z, x, y in zip(mats, qs, ss, zs, xs, ys):
+            assert torch.equal(tq.tq_fused_gemv(m, x), y)
+            yref = oracle.layer_forward(q, s, x.cpu().double().numpy(), zero=z)
+            assert _rel_err(y.cpu().numpy().astype(np.float64), yref) <= TIGHT
+            assert tq.tq_device_status(m) == 0
+
+
 @pytest.mark.parametrize("B", [1, 2, 5])
 def test_stack_with_short_and_long_rows(tq, B):
     """Rows too long for a whole row of activation digits in shared memory (more than 8448 columns)
