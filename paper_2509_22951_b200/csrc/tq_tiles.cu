@@ -323,6 +323,9 @@ struct TilesCta : CtaBase {
         for (int i = 0; i < 4; ++i) acc[i] = acc2[i] = 0;
         from_start = true;
         ++rb;
+        // the row scales of the block that starts now are wanted when it ends: asked for a whole row block ahead
+        // (behind the last row block this is the start of the zero points, inside the same image)
+        if (lane == 0) asm volatile("prefetch.global.L1 [%0];" ::"l"(d.scale + (size_t)rb * 16u));
       }
     };
 
